@@ -1,0 +1,237 @@
+/*
+ * cocodc.h - C ABI of the CoCoDC outer synchronisation step for NVIDIA B200 (sm_100a).
+ *
+ * The library implements what CoCoDC ("Cross-region Model Training with
+ * Communication-Computation Overlapping and Delay Compensation") does to
+ * parameter memory when the synchronisation of a model fragment completes, and
+ * the decision which fragments to synchronise next:
+ *
+ *   S0  record theta^m_{p,t_p} when a sync is initiated           (Algorithm 1, input)
+ *   S1  per-worker pseudo-gradient  theta^m_{p,t_p} - theta^g_{p,t_p-H}   (Section 2.1)
+ *   S2  their mean over the M workers                              (Eq. 1)
+ *   S3  outer optimizer: SGD with Nesterov momentum                (Eq. 2)
+ *   S4  Taylor-expansion delay compensation                        (Eq. 4-7, Algorithm 1)
+ *   S5  merge into every worker's local parameters                 (Eq. 7 / Eq. 3)
+ *   S6  per-fragment change-rate score R_p = ||Delta theta^g_p|| / I_p   (Eq. 10)
+ *   S7  fragment selection under a budget                          (Algorithm 2, Eq. 11)
+ *   S8  schedule sizing N, h                                       (Eq. 8-9)
+ *
+ * The M workers are M stacked replicas in one GPU's memory; the mean over
+ * workers is a reduction along that axis, not a collective.
+ *
+ * Conventions
+ *   - "dev" pointers are device-memory addresses, "host" pointers host addresses.
+ *     All parameter data is fp32.  Streams are passed as void* (a cudaStream_t;
+ *     NULL is the default stream).
+ *   - The caller owns every buffer it passes.  The library owns only the context
+ *     (a copy of the fragment table, a few KB of launch scratch, a status word),
+ *     allocated by cocodc_create and released by cocodc_destroy.
+ *   - Device entry points are asynchronous on the given stream and allocate
+ *     nothing.  Their return value reports host-side validation and launch
+ *     errors; conditions found on the device (a non-finite norm, an invalid id
+ *     list, a NaN score) are recorded in the context's status word, read with
+ *     cocodc_poll_status.  Nothing aborts, traps or prints.
+ *   - Base pointers of parameter buffers must be 16-byte aligned and row strides
+ *     multiples of 4 elements (COCODC_ERR_ALIGNMENT otherwise).  Segment offsets
+ *     and lengths are arbitrary; ragged edges are handled inside the kernels.
+ *   - Offsets, strides and sizes are int64 (element counts): M*N exceeds 2^32 for
+ *     billion-parameter models.
+ *   - A context serialises its own launches on one stream at a time: calls that
+ *     share a context must not overlap on the GPU.
+ */
+#ifndef COCODC_H
+#define COCODC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  COCODC_OK = 0,
+  COCODC_ERR_INVALID_ARG = 1,
+  COCODC_ERR_ALIGNMENT = 2,
+  COCODC_ERR_ALIAS = 3,
+  COCODC_ERR_NONFINITE = 4,   /* device: a fragment norm or a score was NaN/Inf where not allowed */
+  COCODC_ERR_TIMEOUT = 5,     /* device: a bounded wait ran out */
+  COCODC_ERR_CUDA = 6,
+  COCODC_ERR_NOMEM = 7
+} cocodc_status;
+
+/* How the merged local parameters are formed (S4-S5). */
+typedef enum {
+  COCODC_COMP_NONE = 0,    /* no compensation: blend the new global state, Eq. 3 (Streaming DiLoCo, DiLoCo) */
+  COCODC_COMP_TAYLOR = 1   /* Eq. 4-7 */
+} cocodc_comp_mode;
+
+/*
+ * Eq. 4 as printed takes theta_{t_p} - theta_{t_l} while the text calls it the
+ * change rate over the overlap and Eq. 7 adds it; the three consistent readings
+ * are all available.  With d = a - b (a = theta^m_{t_l}, b = theta^m_{t_p}),
+ * D = G - b, G = theta^g_{p,t_p}, c = lambda/(tau*H):
+ *   FORWARD : target = G + d + c*d*d*D   (rate taken forward in time; default)
+ *   PRINTED : target = G - d + c*d*d*D   (Eq. 4, 6, 7 literally)
+ *   DESCENT : target = G + d - c*d*d*D   (Eq. 4-6 literally, Eq. 7 subtracting)
+ */
+typedef enum {
+  COCODC_SIGN_FORWARD = 0,
+  COCODC_SIGN_PRINTED = 1,
+  COCODC_SIGN_DESCENT = 2
+} cocodc_sign_mode;
+
+typedef enum { COCODC_BUDGET_COUNT = 0, COCODC_BUDGET_PARAMS = 1 } cocodc_budget_kind;
+
+/* Stages of cocodc_outer_step. */
+#define COCODC_STAGE_OUTER 1u   /* S1-S3: update theta_g and momentum (required) */
+#define COCODC_STAGE_MERGE 2u   /* S4-S5: update w_now */
+#define COCODC_STAGE_SCORE 4u   /* S6: norms, scores, last_sync of the processed fragments */
+#define COCODC_STAGE_ALL   7u
+
+/*
+ * Fragment partition (Section 2.1: the model is cut into K disjoint fragments).
+ * CSR over segments: fragment p owns segments frag_seg_ptr[p] .. frag_seg_ptr[p+1]-1,
+ * each a run of seg_len[s] elements starting at element seg_offset[s] of every
+ * N-sized buffer.  A strided shard (Section 4.1) is a fragment with several
+ * segments.  Segments must not overlap and must lie inside [0, N).  All three
+ * arrays are host memory and are copied by cocodc_create.
+ */
+typedef struct {
+  int64_t N;
+  int32_t K;
+  int32_t n_segments;
+  const int32_t* frag_seg_ptr;  /* host, K+1 */
+  const int64_t* seg_offset;    /* host, n_segments */
+  const int64_t* seg_len;       /* host, n_segments */
+} cocodc_partition;
+
+/* Hyper-parameters of one completion (paper symbols in brackets). */
+typedef struct {
+  int32_t M;          /* worker replicas [M], 1..64 */
+  int32_t comp_mode;  /* cocodc_comp_mode */
+  int32_t sign_mode;  /* cocodc_sign_mode */
+  int32_t reserved;
+  int64_t H;          /* local steps between syncs of a fragment [H], > 0 */
+  int64_t tau;        /* overlap depth [tau], >= 0; 0 only with COMP_NONE or w_snap == w_now */
+  float outer_lr;     /* outer learning rate (Eq. 2) */
+  float momentum;     /* outer Nesterov momentum (Eq. 2) */
+  float lambda;       /* compensation strength [lambda] (Eq. 6) */
+  float alpha;        /* mixing factor [alpha] (Eq. 3); 1 assigns the target (Eq. 7) */
+} cocodc_hyper;
+
+typedef struct cocodc_ctx cocodc_ctx;
+
+/*
+ * Create a context for one partition on one device.  max_M bounds hyper.M of
+ * later calls.  Allocates device scratch (cudaMalloc) and copies the fragment
+ * table.  Errors: INVALID_ARG (NULLs, K < 1, K > 1024, overlapping or
+ * out-of-range segments, empty fragments, max_M outside 1..64), NOMEM, CUDA.
+ */
+cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* partition,
+                            int32_t max_M, int32_t device);
+cocodc_status cocodc_destroy(cocodc_ctx* ctx);
+
+/*
+ * S8, host only.  Eq. 8: N = max(K, floor(gamma*H*Tc/Ts)); Eq. 9: h = floor(H/N),
+ * raised to 1 when N > H.  Tc, Ts: seconds per local step / per fragment sync.
+ * INVALID_ARG unless K >= 1, H >= 1, 0 < gamma <= 1, Tc > 0, Ts > 0.
+ */
+cocodc_status cocodc_sync_budget(int32_t K, int64_t H, double gamma, double Tc, double Ts,
+                                 int64_t* N_out, int64_t* h_out);
+
+/*
+ * S6 stand-alone (Eq. 10): norms[p] = ||delta_g restricted to fragment p||_2 and
+ * scores[p] = norms[p] / max(1, interval[p]) for all K fragments.
+ *   delta_g  dev fp32[N]   the received mean pseudo-gradients
+ *   interval dev int64[K]  I_p = t_p - t_{p,b}; NULL means 1
+ *   norms, scores dev fp32[K], written
+ * Sums of squares are accumulated in double in a fixed order (run-to-run
+ * reproducible).  A non-finite norm sets COCODC_ERR_NONFINITE in the status word.
+ */
+cocodc_status cocodc_fragment_scores(cocodc_ctx* ctx, const float* delta_g, const int64_t* interval,
+                                     float* norms, float* scores, void* stream);
+
+/*
+ * S7 (Algorithm 2, Eq. 11, extended to a budget).  Priority order: eligible
+ * fragments with t_now - last_sync[p] >= H by ascending index (Algorithm 2's
+ * loop), then the other eligible fragments by score, largest first, ties to the
+ * lower index; +Inf is a legal score (never-synced fragments).  The head of the
+ * order is always taken; each later fragment is taken iff its cost (1 for
+ * COUNT, its size for PARAMS) still fits what is left of the budget.  budget = 1
+ * (COUNT) is exactly Algorithm 2.
+ *   scores dev fp32[K]; last_sync dev int64[K]; ineligible dev uint8[K] or NULL
+ *   mask dev uint8[K] (1 = selected); ids dev int32[K] (first n_sel entries, admission
+ *   order; the rest set to -1); n_sel dev int32[1]
+ * A NaN score selects nothing and sets COCODC_ERR_NONFINITE.
+ */
+cocodc_status cocodc_select_fragments(cocodc_ctx* ctx, const float* scores, const int64_t* last_sync,
+                                      const uint8_t* ineligible, int64_t t_now, int64_t H,
+                                      int32_t budget_kind, int64_t budget,
+                                      uint8_t* mask, int32_t* ids, int32_t* n_sel, void* stream);
+
+/*
+ * S1-S6 fused, at completion time t_l, for the fragments listed on the device
+ * (typically the ids that cocodc_select_fragments wrote tau steps earlier).
+ * Per element i of each listed fragment, in fp32:
+ *   Delta = (sum_m (w_snap[m][i] - theta_g[i])) / M                        (Eq. 1)
+ *   u'    = momentum*u + Delta ; G = theta_g + outer_lr*(Delta + momentum*u')   (Eq. 2)
+ *   target_m = per sign_mode above, or G for COMP_NONE                     (Eq. 4-7)
+ *   w_now[m][i] = (1-alpha)*w_now[m][i] + alpha*target_m                   (Eq. 3 / Eq. 7)
+ * and theta_g[i] = G, momentum[i] = u', delta_g_out[i] = Delta (if not NULL).
+ * With STAGE_SCORE, for each listed p: norms[p] = ||Delta||_2 over the fragment,
+ * scores[p] = norms[p] / max(1, t_p - last_sync[p]), then last_sync[p] = t_l.
+ * Fragments not listed are not touched.
+ *
+ *   w_now   dev fp32, worker m's element i at w_now[m*now_stride + i]   (theta^m_{.,t_l}, in/out)
+ *   w_snap  dev fp32, theta^m_{p,t_p}: at w_snap[m*snap_stride + i] if snap_offset is NULL,
+ *           else fragment p packed (segments back to back) from w_snap[m*snap_stride + snap_offset[p]]
+ *           w_snap == w_now (same stride, snap_offset NULL) is legal: zero delay, blocking sync
+ *   snap_offset dev int64[K] or NULL
+ *   theta_g, momentum dev fp32[N] in/out; delta_g_out dev fp32[N] or NULL
+ *   ids dev int32[<=K] distinct fragment ids; n_ids dev int32[1]
+ *   last_sync dev int64[K]; norms, scores dev fp32[K] (needed with STAGE_SCORE)
+ * Errors: INVALID_ARG, ALIGNMENT, ALIAS (buffers overlapping other than w_snap == w_now), CUDA.
+ * Device-side: an id outside [0,K) or listed twice processes nothing and sets INVALID_ARG.
+ */
+cocodc_status cocodc_outer_step(cocodc_ctx* ctx, const cocodc_hyper* hyper,
+                                float* w_now, const float* w_snap,
+                                int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                float* theta_g, float* momentum, float* delta_g_out,
+                                const int32_t* ids, const int32_t* n_ids,
+                                int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                float* norms, float* scores, uint32_t stages, void* stream);
+
+/*
+ * S4-S5 alone (Algorithm 1, or Eq. 3 for COMP_NONE), given the new global state:
+ * w_now[m][i] = (1-alpha)*w_now[m][i] + alpha*target_m with G = theta_g_new[i].
+ * Together with cocodc_outer_step(stages without MERGE) this is the unfused path.
+ */
+cocodc_status cocodc_merge(cocodc_ctx* ctx, const cocodc_hyper* hyper,
+                           float* w_now, const float* w_snap,
+                           int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                           const float* theta_g_new, const int32_t* ids, const int32_t* n_ids,
+                           void* stream);
+
+/*
+ * S0: copy the listed fragments of every worker from w_now into w_snap (same
+ * layout rules as above) when their synchronisation is initiated at t_p.
+ */
+cocodc_status cocodc_snapshot(cocodc_ctx* ctx, const float* w_now, float* w_snap,
+                              int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                              int32_t M, const int32_t* ids, const int32_t* n_ids, void* stream);
+
+/*
+ * Waits for the stream, then returns and clears the device status word
+ * (COCODC_OK if nothing was recorded since the last poll).
+ */
+cocodc_status cocodc_poll_status(cocodc_ctx* ctx, void* stream);
+
+/* Number of kernels the library has launched through this context so far. */
+int64_t cocodc_launch_count(const cocodc_ctx* ctx);
+
+const char* cocodc_status_string(cocodc_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COCODC_H */

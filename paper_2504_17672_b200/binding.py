@@ -1,0 +1,196 @@
+"""ctypes binding of libcocodc.so with the same names as the C ABI (include/cocodc.h).
+
+Argument marshalling only.  Tensors are torch CUDA tensors used as plain device
+memory: the binding passes their addresses and the current CUDA stream.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_NONFINITE, ERR_TIMEOUT, ERR_CUDA, ERR_NOMEM = range(8)
+COMP_NONE, COMP_TAYLOR = 0, 1
+SIGN_FORWARD, SIGN_PRINTED, SIGN_DESCENT = 0, 1, 2
+BUDGET_COUNT, BUDGET_PARAMS = 0, 1
+STAGE_OUTER, STAGE_MERGE, STAGE_SCORE, STAGE_ALL = 1, 2, 4, 7
+
+EXPORTS = (
+    "cocodc_create", "cocodc_destroy", "cocodc_sync_budget", "cocodc_fragment_scores",
+    "cocodc_select_fragments", "cocodc_outer_step", "cocodc_merge", "cocodc_snapshot",
+    "cocodc_poll_status", "cocodc_launch_count", "cocodc_status_string",
+)
+
+
+class CocodcError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = int(code)
+        super().__init__(f"{where}: {status_string(code)} (status {int(code)})")
+
+
+class _Partition(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int64), ("K", ctypes.c_int32), ("n_segments", ctypes.c_int32),
+                ("frag_seg_ptr", ctypes.POINTER(ctypes.c_int32)),
+                ("seg_offset", ctypes.POINTER(ctypes.c_int64)),
+                ("seg_len", ctypes.POINTER(ctypes.c_int64))]
+
+
+class _Hyper(ctypes.Structure):
+    _fields_ = [("M", ctypes.c_int32), ("comp_mode", ctypes.c_int32), ("sign_mode", ctypes.c_int32),
+                ("reserved", ctypes.c_int32), ("H", ctypes.c_int64), ("tau", ctypes.c_int64),
+                ("outer_lr", ctypes.c_float), ("momentum", ctypes.c_float),
+                ("lam", ctypes.c_float), ("alpha", ctypes.c_float)]
+
+
+@dataclass
+class Hyper:
+    """Hyper-parameters of one completion, in the paper's symbols."""
+    M: int
+    H: int = 100
+    tau: int = 1
+    outer_lr: float = 0.7
+    momentum: float = 0.9
+    lam: float = 0.5
+    alpha: float = 1.0
+    comp_mode: int = COMP_TAYLOR
+    sign_mode: int = SIGN_FORWARD
+
+    def _c(self) -> _Hyper:
+        return _Hyper(self.M, self.comp_mode, self.sign_mode, 0, self.H, self.tau,
+                      self.outer_lr, self.momentum, self.lam, self.alpha)
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIBRARY
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build the CUDA library first "
+            "(python -m paper_2504_17672_b200.build, or __graft_entry__.build()); there is no fallback path")
+    lib = ctypes.CDLL(path)
+    vp, i32, i64, u32, f64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_double
+    lib.cocodc_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(_Partition), i32, i32]
+    lib.cocodc_destroy.argtypes = [vp]
+    lib.cocodc_sync_budget.argtypes = [i32, i64, f64, f64, f64, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.cocodc_fragment_scores.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.cocodc_select_fragments.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp]
+    lib.cocodc_outer_step.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, vp,
+                                      i64, i64, vp, vp, vp, u32, vp]
+    lib.cocodc_merge.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp]
+    lib.cocodc_snapshot.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp]
+    lib.cocodc_poll_status.argtypes = [vp, vp]
+    lib.cocodc_launch_count.argtypes = [vp]
+    lib.cocodc_launch_count.restype = i64
+    lib.cocodc_status_string.argtypes = [ctypes.c_int]
+    lib.cocodc_status_string.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name not in ("cocodc_launch_count", "cocodc_status_string"):
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+_lib = _load()
+
+
+def library() -> ctypes.CDLL:
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return _lib.cocodc_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise CocodcError(code, where)
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def cocodc_sync_budget(K: int, H: int, gamma: float, Tc: float, Ts: float):
+    """Eq. 8-9 on the host: returns (N, h)."""
+    N, h = ctypes.c_int64(), ctypes.c_int64()
+    _check(_lib.cocodc_sync_budget(K, H, gamma, Tc, Ts, ctypes.byref(N), ctypes.byref(h)), "cocodc_sync_budget")
+    return N.value, h.value
+
+
+class Context:
+    """Owns a cocodc_ctx for one fragment partition on one device."""
+
+    def __init__(self, N: int, frag_seg_ptr: Sequence[int], seg_offset: Sequence[int],
+                 seg_len: Sequence[int], max_M: int, device: int = 0):
+        self._h = ctypes.c_void_p()
+        ptr = np.ascontiguousarray(frag_seg_ptr, dtype=np.int32)
+        off = np.ascontiguousarray(seg_offset, dtype=np.int64)
+        ln = np.ascontiguousarray(seg_len, dtype=np.int64)
+        part = _Partition(int(N), len(ptr) - 1, len(off),
+                          ptr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                          off.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)),
+                          ln.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)))
+        self.N, self.K, self.device = int(N), len(ptr) - 1, int(device)
+        _check(_lib.cocodc_create(ctypes.byref(self._h), ctypes.byref(part), int(max_M), int(device)), "cocodc_create")
+
+    def close(self) -> None:
+        if self._h:
+            _lib.cocodc_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def launch_count(self) -> int:
+        return int(_lib.cocodc_launch_count(self._h))
+
+    def cocodc_fragment_scores(self, delta_g, interval, norms, scores, stream=None) -> None:
+        _check(_lib.cocodc_fragment_scores(self._h, _p(delta_g), _p(interval), _p(norms), _p(scores),
+                                           _stream(stream)), "cocodc_fragment_scores")
+
+    def cocodc_select_fragments(self, scores, last_sync, ineligible, t_now: int, H: int, budget_kind: int,
+                                budget: int, mask, ids, n_sel, stream=None) -> None:
+        _check(_lib.cocodc_select_fragments(self._h, _p(scores), _p(last_sync), _p(ineligible), int(t_now), int(H),
+                                            int(budget_kind), int(budget), _p(mask), _p(ids), _p(n_sel),
+                                            _stream(stream)), "cocodc_select_fragments")
+
+    def cocodc_outer_step(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
+                          theta_g, momentum, delta_g_out, ids, n_ids, t_p: int, t_l: int, last_sync,
+                          norms, scores, stages: int = STAGE_ALL, stream=None) -> None:
+        h = hyper._c()
+        _check(_lib.cocodc_outer_step(self._h, ctypes.byref(h), _p(w_now), _p(w_snap), int(now_stride),
+                                      int(snap_stride), _p(snap_offset), _p(theta_g), _p(momentum),
+                                      _p(delta_g_out), _p(ids), _p(n_ids), int(t_p), int(t_l), _p(last_sync),
+                                      _p(norms), _p(scores), int(stages), _stream(stream)), "cocodc_outer_step")
+
+    def cocodc_merge(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
+                     theta_g_new, ids, n_ids, stream=None) -> None:
+        h = hyper._c()
+        _check(_lib.cocodc_merge(self._h, ctypes.byref(h), _p(w_now), _p(w_snap), int(now_stride), int(snap_stride),
+                                 _p(snap_offset), _p(theta_g_new), _p(ids), _p(n_ids), _stream(stream)),
+               "cocodc_merge")
+
+    def cocodc_snapshot(self, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset, M: int,
+                        ids, n_ids, stream=None) -> None:
+        _check(_lib.cocodc_snapshot(self._h, _p(w_now), _p(w_snap), int(now_stride), int(snap_stride),
+                                    _p(snap_offset), int(M), _p(ids), _p(n_ids), _stream(stream)),
+               "cocodc_snapshot")
+
+    def cocodc_poll_status(self, stream=None) -> int:
+        """Waits for the stream; returns and clears the device status word."""
+        return int(_lib.cocodc_poll_status(self._h, _stream(stream)))

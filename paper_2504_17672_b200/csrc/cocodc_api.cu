@@ -1,0 +1,438 @@
+// Host side of the C ABI declared in include/cocodc.h: argument validation,
+// the context, and kernel launches.  Every arithmetic step runs in the kernels
+// of outer.cuh / select.cuh / plan.cuh; nothing here computes on parameter data.
+
+#include "../../include/cocodc.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <new>
+#include <utility>
+#include <vector>
+
+#include "outer.cuh"
+#include "plan.cuh"
+#include "select.cuh"
+
+using namespace cocodc;
+
+struct cocodc_ctx {
+  int device = 0;
+  int sm_count = 0;
+  int K = 0;
+  int n_segments = 0;
+  long long N = 0;
+  int max_M = 0;
+  int max_grid = 0;
+  // device copies of the fragment table
+  int* d_frag_seg_ptr = nullptr;
+  long long* d_seg_off = nullptr;
+  long long* d_seg_len = nullptr;
+  long long* d_frag_size = nullptr;
+  // launch scratch
+  SegPlan* d_plan = nullptr;
+  PlanHeader* d_hdr = nullptr;
+  double* d_partial = nullptr;
+  int* d_status = nullptr;
+  long long launches = 0;
+  std::vector<std::pair<const void*, int>> occupancy;  // kernel -> resident CTAs per SM
+};
+
+namespace {
+
+struct DeviceGuard {
+  int prev = -1;
+  bool switched = false;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) switched = (cudaSetDevice(dev) == cudaSuccess);
+  }
+  ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Range { uintptr_t lo, hi; };
+inline Range range_of(const void* p, long long elems) {
+  uintptr_t b = reinterpret_cast<uintptr_t>(p);
+  return Range{b, b + (uintptr_t)elems * sizeof(float)};
+}
+inline bool overlap(Range a, Range b) { return a.lo < b.hi && b.lo < a.hi; }
+
+int grid_for(cocodc_ctx* c, const void* kernel) {
+  for (auto& kv : c->occupancy) if (kv.first == kernel) return kv.second * c->sm_count;
+  int per_sm = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, 0) != cudaSuccess || per_sm < 1)
+    per_sm = 1;
+  per_sm = std::min(per_sm, 8);
+  c->occupancy.emplace_back(kernel, per_sm);
+  return per_sm * c->sm_count;
+}
+
+cocodc_status launch_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_ids,
+                          const int64_t* snap_offset, int lanes_per_tile, cudaStream_t st) {
+  k_plan<<<1, kPlanThreads, 0, st>>>(ids, n_ids, c->K, c->d_frag_seg_ptr, c->d_seg_off, c->d_seg_len,
+                                     reinterpret_cast<const long long*>(snap_offset), lanes_per_tile,
+                                     c->n_segments, c->d_plan, c->d_hdr, c->d_status,
+                                     (int)COCODC_ERR_INVALID_ARG);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+// Lanes per thread and tile for each instantiated worker count.
+template <int M> struct Unroll { static constexpr int U = (M >= 8) ? 1 : 2; };
+template <> struct Unroll<0> { static constexpr int U = 2; };
+
+template <int M, int MODE, bool SAME>
+cocodc_status launch_outer_variant(cocodc_ctx* c, const OuterArgs& A, const int32_t* ids, const int32_t* n_ids,
+                                   const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
+  constexpr int U = Unroll<M>::U;
+  auto kernel = k_outer<M, U, MODE, SAME>;
+  const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads * U, st);
+  if (s != COCODC_OK) return s;
+  kernel<<<grid, kThreads, 0, st>>>(A);
+  c->launches++;
+  *grid_out = grid;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+template <int MODE, bool SAME>
+cocodc_status launch_outer_m(cocodc_ctx* c, const OuterArgs& A, const int32_t* ids, const int32_t* n_ids,
+                             const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
+  switch (A.M) {
+    case 1: return launch_outer_variant<1, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
+    case 2: return launch_outer_variant<2, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
+    case 3: return launch_outer_variant<3, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
+    case 4: return launch_outer_variant<4, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
+    case 8: return launch_outer_variant<8, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
+    default: return launch_outer_variant<0, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
+  }
+}
+
+// Shared checks of the three entry points that stream worker buffers.
+cocodc_status check_hyper(const cocodc_ctx* c, const cocodc_hyper* h) {
+  if (!c || !h) return COCODC_ERR_INVALID_ARG;
+  if (h->M < 1 || h->M > c->max_M) return COCODC_ERR_INVALID_ARG;
+  if (h->H < 1 || h->tau < 0) return COCODC_ERR_INVALID_ARG;
+  if (h->comp_mode != COCODC_COMP_NONE && h->comp_mode != COCODC_COMP_TAYLOR) return COCODC_ERR_INVALID_ARG;
+  if (h->sign_mode < COCODC_SIGN_FORWARD || h->sign_mode > COCODC_SIGN_DESCENT) return COCODC_ERR_INVALID_ARG;
+  if (!std::isfinite(h->outer_lr) || !std::isfinite(h->momentum) || !std::isfinite(h->lambda) ||
+      !std::isfinite(h->alpha))
+    return COCODC_ERR_INVALID_ARG;
+  return COCODC_OK;
+}
+
+// Eq. 6-7 folded into two scalars (computed in double, rounded once).
+void fold_coefficients(const cocodc_hyper* h, bool zero_delay, OuterArgs* A) {
+  double c1 = 0.0, c2 = 0.0;
+  if (h->comp_mode == COCODC_COMP_TAYLOR && h->tau > 0 && !zero_delay) {
+    const double c = (double)h->lambda / ((double)h->tau * (double)h->H);
+    switch (h->sign_mode) {
+      case COCODC_SIGN_FORWARD: c1 = 1.0; c2 = c; break;
+      case COCODC_SIGN_PRINTED: c1 = -1.0; c2 = c; break;
+      default: c1 = 1.0; c2 = -c; break;
+    }
+  }
+  A->c1 = (float)c1;
+  A->c2 = (float)c2;
+  A->alpha = h->alpha;
+  A->one_minus_alpha = (float)(1.0 - (double)h->alpha);
+  A->eta = h->outer_lr;
+  A->mu = h->momentum;
+  A->M = h->M;
+  A->Mf = (float)h->M;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* cocodc_status_string(cocodc_status s) {
+  switch (s) {
+    case COCODC_OK: return "ok";
+    case COCODC_ERR_INVALID_ARG: return "invalid argument";
+    case COCODC_ERR_ALIGNMENT: return "buffer not 16-byte aligned or stride not a multiple of 4 elements";
+    case COCODC_ERR_ALIAS: return "buffers overlap";
+    case COCODC_ERR_NONFINITE: return "non-finite value";
+    case COCODC_ERR_TIMEOUT: return "bounded wait ran out";
+    case COCODC_ERR_CUDA: return "CUDA error";
+    case COCODC_ERR_NOMEM: return "out of memory";
+  }
+  return "unknown status";
+}
+
+cocodc_status cocodc_sync_budget(int32_t K, int64_t H, double gamma, double Tc, double Ts,
+                                 int64_t* N_out, int64_t* h_out) {
+  if (!N_out || !h_out || K < 1 || H < 1) return COCODC_ERR_INVALID_ARG;
+  if (!(gamma > 0.0 && gamma <= 1.0) || !(Tc > 0.0) || !(Ts > 0.0)) return COCODC_ERR_INVALID_ARG;
+  const double cap = std::floor(gamma * (double)H * Tc / Ts);
+  if (!std::isfinite(cap)) return COCODC_ERR_INVALID_ARG;
+  int64_t N = (cap >= 9.0e18) ? INT64_MAX : (int64_t)cap;   // Eq. 8
+  if (N < K) N = K;
+  int64_t h = H / N;                                         // Eq. 9
+  if (h < 1) h = 1;
+  *N_out = N;
+  *h_out = h;
+  return COCODC_OK;
+}
+
+cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, int32_t max_M, int32_t device) {
+  if (!ctx_out) return COCODC_ERR_INVALID_ARG;
+  *ctx_out = nullptr;
+  if (!part || !part->frag_seg_ptr || !part->seg_offset || !part->seg_len) return COCODC_ERR_INVALID_ARG;
+  if (part->K < 1 || part->K > kMaxK || part->n_segments < part->K || part->N < 1) return COCODC_ERR_INVALID_ARG;
+  if (max_M < 1 || max_M > 64) return COCODC_ERR_INVALID_ARG;
+  const int K = part->K, S = part->n_segments;
+  if (part->frag_seg_ptr[0] != 0 || part->frag_seg_ptr[K] != S) return COCODC_ERR_INVALID_ARG;
+  std::vector<long long> frag_size(K, 0);
+  std::vector<std::pair<long long, long long>> segs;
+  segs.reserve(S);
+  for (int p = 0; p < K; ++p) {
+    if (part->frag_seg_ptr[p + 1] <= part->frag_seg_ptr[p]) return COCODC_ERR_INVALID_ARG;  // empty fragment
+    for (int s = part->frag_seg_ptr[p]; s < part->frag_seg_ptr[p + 1]; ++s) {
+      const long long o = part->seg_offset[s], l = part->seg_len[s];
+      if (o < 0 || l < 1 || o > part->N - l) return COCODC_ERR_INVALID_ARG;
+      frag_size[p] += l;
+      segs.emplace_back(o, l);
+    }
+  }
+  std::sort(segs.begin(), segs.end());
+  for (size_t i = 1; i < segs.size(); ++i)
+    if (segs[i].first < segs[i - 1].first + segs[i - 1].second) return COCODC_ERR_INVALID_ARG;  // overlap
+
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess) return COCODC_ERR_CUDA;
+  if (device < 0 || device >= n_dev) return COCODC_ERR_INVALID_ARG;
+  DeviceGuard guard(device);
+  cocodc_ctx* c = new (std::nothrow) cocodc_ctx();
+  if (!c) return COCODC_ERR_NOMEM;
+  c->device = device;
+  c->K = K;
+  c->n_segments = S;
+  c->N = part->N;
+  c->max_M = max_M;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete c; return COCODC_ERR_CUDA; }
+  c->sm_count = prop.multiProcessorCount;
+  c->max_grid = c->sm_count * 8;
+
+  std::vector<long long> off(S), len(S);
+  for (int s = 0; s < S; ++s) { off[s] = part->seg_offset[s]; len[s] = part->seg_len[s]; }
+  const size_t partial_elems = (size_t)K * c->max_grid * (kThreads / 32);
+  bool ok = true;
+  ok = ok && cudaMalloc(&c->d_frag_seg_ptr, sizeof(int) * (K + 1)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_seg_off, sizeof(long long) * S) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_seg_len, sizeof(long long) * S) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_frag_size, sizeof(long long) * K) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_plan, sizeof(SegPlan) * S) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_hdr, sizeof(PlanHeader)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_partial, sizeof(double) * partial_elems) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); cocodc_destroy(c); return COCODC_ERR_NOMEM; }
+  ok = ok && cudaMemcpy(c->d_frag_seg_ptr, part->frag_seg_ptr, sizeof(int) * (K + 1), cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->d_seg_off, off.data(), sizeof(long long) * S, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->d_seg_len, len.data(), sizeof(long long) * S, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemcpy(c->d_frag_size, frag_size.data(), sizeof(long long) * K, cudaMemcpyHostToDevice) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_hdr, 0, sizeof(PlanHeader)) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); cocodc_destroy(c); return COCODC_ERR_CUDA; }
+  *ctx_out = c;
+  return COCODC_OK;
+}
+
+cocodc_status cocodc_destroy(cocodc_ctx* c) {
+  if (!c) return COCODC_OK;
+  DeviceGuard guard(c->device);
+  cudaFree(c->d_frag_seg_ptr);
+  cudaFree(c->d_seg_off);
+  cudaFree(c->d_seg_len);
+  cudaFree(c->d_frag_size);
+  cudaFree(c->d_plan);
+  cudaFree(c->d_hdr);
+  cudaFree(c->d_partial);
+  cudaFree(c->d_status);
+  delete c;
+  return COCODC_OK;
+}
+
+int64_t cocodc_launch_count(const cocodc_ctx* c) { return c ? c->launches : 0; }
+
+cocodc_status cocodc_poll_status(cocodc_ctx* c, void* stream) {
+  if (!c) return COCODC_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int word = 0;
+  if (cudaMemcpyAsync(&word, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return COCODC_ERR_CUDA;
+  if (cudaMemsetAsync(c->d_status, 0, sizeof(int), st) != cudaSuccess) return COCODC_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return COCODC_ERR_CUDA;
+  return static_cast<cocodc_status>(word);
+}
+
+cocodc_status cocodc_fragment_scores(cocodc_ctx* c, const float* delta_g, const int64_t* interval,
+                                     float* norms, float* scores, void* stream) {
+  if (!c || !delta_g || !norms || !scores) return COCODC_ERR_INVALID_ARG;
+  if (!aligned16(delta_g)) return COCODC_ERR_ALIGNMENT;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  constexpr int U = 4;
+  auto kernel = k_sumsq<U>;
+  const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
+  cocodc_status s = launch_plan(c, nullptr, nullptr, nullptr, kThreads * U, st);
+  if (s != COCODC_OK) return s;
+  kernel<<<grid, kThreads, 0, st>>>(delta_g, c->d_plan, c->d_hdr, c->d_partial);
+  c->launches++;
+  k_finalize_scores<<<c->K, kFinalizeThreads, 0, st>>>(
+      c->d_hdr, nullptr, c->d_partial, grid * (kThreads / 32), 1, 0, 0,
+      reinterpret_cast<const long long*>(interval), nullptr, norms, scores, c->d_status,
+      (int)COCODC_ERR_NONFINITE);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
+                                      const uint8_t* ineligible, int64_t t_now, int64_t H,
+                                      int32_t budget_kind, int64_t budget,
+                                      uint8_t* mask, int32_t* ids, int32_t* n_sel, void* stream) {
+  if (!c || !scores || !last_sync || !mask || !ids || !n_sel) return COCODC_ERR_INVALID_ARG;
+  if (H < 1 || budget < 0) return COCODC_ERR_INVALID_ARG;
+  if (budget_kind != COCODC_BUDGET_COUNT && budget_kind != COCODC_BUDGET_PARAMS) return COCODC_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  k_select<<<1, kSelectThreads, 0, st>>>(c->K, scores, reinterpret_cast<const long long*>(last_sync), ineligible,
+                                         c->d_frag_size, t_now, H, budget_kind, budget, mask, ids, n_sel,
+                                         c->d_status, (int)COCODC_ERR_NONFINITE);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
+                                float* w_now, const float* w_snap,
+                                int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                float* theta_g, float* momentum, float* delta_g_out,
+                                const int32_t* ids, const int32_t* n_ids,
+                                int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                float* norms, float* scores, uint32_t stages, void* stream) {
+  cocodc_status s = check_hyper(c, h);
+  if (s != COCODC_OK) return s;
+  if (!(stages & COCODC_STAGE_OUTER) || (stages & ~COCODC_STAGE_ALL)) return COCODC_ERR_INVALID_ARG;
+  const bool do_merge = (stages & COCODC_STAGE_MERGE) != 0;
+  const bool do_score = (stages & COCODC_STAGE_SCORE) != 0;
+  if (!w_snap || !theta_g || !momentum || !ids || !n_ids) return COCODC_ERR_INVALID_ARG;
+  if (do_merge && !w_now) return COCODC_ERR_INVALID_ARG;
+  if (do_score && (!last_sync || !norms || !scores)) return COCODC_ERR_INVALID_ARG;
+  if (t_l < t_p) return COCODC_ERR_INVALID_ARG;
+  const long long N = c->N;
+  if (snap_stride < (snap_offset ? 1 : N) || (do_merge && now_stride < N)) return COCODC_ERR_INVALID_ARG;
+  const bool same = do_merge && (w_snap == w_now) && (snap_stride == now_stride) && (snap_offset == nullptr);
+  if (h->tau == 0 && h->comp_mode == COCODC_COMP_TAYLOR && do_merge && !same) return COCODC_ERR_INVALID_ARG;
+  if (!aligned16(w_snap) || !aligned16(theta_g) || !aligned16(momentum) || (snap_stride & 3)) return COCODC_ERR_ALIGNMENT;
+  if (do_merge && (!aligned16(w_now) || (now_stride & 3))) return COCODC_ERR_ALIGNMENT;
+  if (delta_g_out && !aligned16(delta_g_out)) return COCODC_ERR_ALIGNMENT;
+  // aliasing: every output range must be disjoint from every other buffer
+  {
+    const int M = h->M;
+    std::vector<Range> r;
+    r.push_back(range_of(theta_g, N));
+    r.push_back(range_of(momentum, N));
+    if (delta_g_out) r.push_back(range_of(delta_g_out, N));
+    if (do_merge) r.push_back(range_of(w_now, (long long)(M - 1) * now_stride + N));
+    for (size_t i = 0; i < r.size(); ++i)
+      for (size_t j = i + 1; j < r.size(); ++j)
+        if (overlap(r[i], r[j])) return COCODC_ERR_ALIAS;
+    if (!same) {
+      const Range rs = range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N));
+      for (const Range& x : r) if (overlap(rs, x)) return COCODC_ERR_ALIAS;
+    }
+  }
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  OuterArgs A{};
+  A.w_now = w_now;
+  A.w_snap = w_snap;
+  A.now_stride = now_stride;
+  A.snap_stride = snap_stride;
+  A.theta_g = theta_g;
+  A.momentum = momentum;
+  A.delta_out = delta_g_out;
+  A.plan = c->d_plan;
+  A.hdr = c->d_hdr;
+  A.partial = do_score ? c->d_partial : nullptr;
+  fold_coefficients(h, same, &A);
+  int grid = 0;
+  if (!do_merge) s = launch_outer_m<MODE_OUTER_ONLY, false>(c, A, ids, n_ids, snap_offset, st, &grid);
+  else if (same) s = launch_outer_m<MODE_FUSED, true>(c, A, ids, n_ids, snap_offset, st, &grid);
+  else s = launch_outer_m<MODE_FUSED, false>(c, A, ids, n_ids, snap_offset, st, &grid);
+  if (s != COCODC_OK) return s;
+  if (do_score) {
+    k_finalize_scores<<<c->K, kFinalizeThreads, 0, st>>>(
+        c->d_hdr, ids, c->d_partial, grid * (kThreads / 32), 0, t_p, t_l, nullptr,
+        reinterpret_cast<long long*>(last_sync), norms, scores, c->d_status, (int)COCODC_ERR_NONFINITE);
+    c->launches++;
+    if (cudaGetLastError() != cudaSuccess) return COCODC_ERR_CUDA;
+  }
+  return COCODC_OK;
+}
+
+cocodc_status cocodc_merge(cocodc_ctx* c, const cocodc_hyper* h,
+                           float* w_now, const float* w_snap,
+                           int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                           const float* theta_g_new, const int32_t* ids, const int32_t* n_ids, void* stream) {
+  cocodc_status s = check_hyper(c, h);
+  if (s != COCODC_OK) return s;
+  if (!w_now || !w_snap || !theta_g_new || !ids || !n_ids) return COCODC_ERR_INVALID_ARG;
+  const long long N = c->N;
+  if (now_stride < N || snap_stride < (snap_offset ? 1 : N)) return COCODC_ERR_INVALID_ARG;
+  const bool same = (w_snap == w_now) && (snap_stride == now_stride) && (snap_offset == nullptr);
+  if (h->tau == 0 && h->comp_mode == COCODC_COMP_TAYLOR && !same) return COCODC_ERR_INVALID_ARG;
+  if (!aligned16(w_now) || !aligned16(w_snap) || !aligned16(theta_g_new) || (now_stride & 3) || (snap_stride & 3))
+    return COCODC_ERR_ALIGNMENT;
+  {
+    const int M = h->M;
+    const Range rn = range_of(w_now, (long long)(M - 1) * now_stride + N);
+    if (overlap(rn, range_of(theta_g_new, N))) return COCODC_ERR_ALIAS;
+    if (!same && overlap(rn, range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N))))
+      return COCODC_ERR_ALIAS;
+  }
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  OuterArgs A{};
+  A.w_now = w_now;
+  A.w_snap = w_snap;
+  A.now_stride = now_stride;
+  A.snap_stride = snap_stride;
+  A.theta_g = const_cast<float*>(theta_g_new);  // read only in this mode
+  A.plan = c->d_plan;
+  A.hdr = c->d_hdr;
+  fold_coefficients(h, same, &A);
+  int grid = 0;
+  if (same) return launch_outer_m<MODE_MERGE_ONLY, true>(c, A, ids, n_ids, snap_offset, st, &grid);
+  return launch_outer_m<MODE_MERGE_ONLY, false>(c, A, ids, n_ids, snap_offset, st, &grid);
+}
+
+cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
+                              int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                              int32_t M, const int32_t* ids, const int32_t* n_ids, void* stream) {
+  if (!c || !w_now || !w_snap || !ids || !n_ids) return COCODC_ERR_INVALID_ARG;
+  if (M < 1 || M > c->max_M) return COCODC_ERR_INVALID_ARG;
+  const long long N = c->N;
+  if (now_stride < N || snap_stride < (snap_offset ? 1 : N)) return COCODC_ERR_INVALID_ARG;
+  if (!aligned16(w_now) || !aligned16(w_snap) || (now_stride & 3) || (snap_stride & 3)) return COCODC_ERR_ALIGNMENT;
+  if (overlap(range_of(w_now, (long long)(M - 1) * now_stride + N),
+              range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N))))
+    return COCODC_ERR_ALIAS;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  constexpr int U = 4;
+  auto kernel = k_snapshot<U>;
+  const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads * U, st);
+  if (s != COCODC_OK) return s;
+  kernel<<<grid, kThreads, 0, st>>>(w_now, w_snap, now_stride, snap_stride, M, c->d_plan, c->d_hdr);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+}  // extern "C"

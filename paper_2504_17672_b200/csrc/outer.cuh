@@ -1,0 +1,307 @@
+// The streaming kernels of the outer synchronisation step.
+//
+// k_outer<M, U, MODE, SAME> makes one pass over the listed fragments.  Per
+// element it reads every worker's recorded and current value, the global state
+// and the momentum once, keeps pseudo-gradient, mean, Nesterov update, delay
+// compensation and merge in registers, and writes each output once (Eq. 1-7,
+// Eq. 3).  The sum of squares of the mean pseudo-gradient (Eq. 10) is collected
+// on the way.  Nothing here is a contraction: the kernel is bound by HBM
+// bandwidth, so the design is about keeping enough 16-byte loads in flight per
+// SM and touching every byte once.
+//
+// Work decomposition: a persistent grid; CTA c handles tiles c, c+grid, ...  A
+// tile is THREADS*U lanes of four elements of one segment; a thread issues all
+// of its U lanes' loads (U * (2M+2) 16-byte loads) before the first use.
+#pragma once
+
+#include "plan.cuh"
+
+namespace cocodc {
+
+constexpr int kThreads = 256;
+
+enum : int { MODE_FUSED = 0, MODE_OUTER_ONLY = 1, MODE_MERGE_ONLY = 2 };
+
+struct OuterArgs {
+  float* w_now;             // [M][now_stride]
+  const float* w_snap;      // [M][snap_stride]
+  long long now_stride;
+  long long snap_stride;
+  float* theta_g;           // in/out (MODE_MERGE_ONLY: read only, the new global state)
+  float* momentum;          // in/out
+  float* delta_out;         // optional
+  const SegPlan* plan;
+  const PlanHeader* hdr;
+  double* partial;          // nullptr: no score accumulation
+  int M;                    // runtime worker count (used by the generic M = 0 instantiation)
+  float eta, mu;            // outer learning rate, Nesterov momentum
+  float c1, c2;             // target = G + c1*d + c2*d*d*D
+  float alpha, one_minus_alpha;
+  float Mf;                 // (float)M
+};
+
+// ---- memory access helpers -------------------------------------------------
+// Every byte is used exactly once per launch, so loads and stores are marked
+// streaming (evict-first) to keep them from displacing each other in L2.
+__device__ __forceinline__ float4 ld4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ void st4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+__device__ __forceinline__ float ld1(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ void st1(float* p, float v) { __stcs(p, v); }
+
+// ---- the arithmetic of one element -----------------------------------------
+// S1-S3.  Differences first, summed in worker order, then divided by M (Eq. 1);
+// u' = mu*u + Delta, G = thg + eta*(Delta + mu*u') (Eq. 2, Nesterov).
+__device__ __forceinline__ void outer_update(float sum, float thg, float u, const OuterArgs& A,
+                                             float& Delta, float& u_new, float& G) {
+  Delta = __fdiv_rn(sum, A.Mf);
+  u_new = __fmaf_rn(A.mu, u, Delta);
+  const float t = __fmaf_rn(A.mu, u_new, Delta);
+  G = __fmaf_rn(A.eta, t, thg);
+}
+
+// S4-S5.  d = a - b is the local change over the overlap (tau times Eq. 4's
+// rate), D = G - b the divergence of Eq. 5; Eq. 6-7 collapse to
+// target = G + c1*d + c2*d*d*D with c2 = +-lambda/(tau*H); then Eq. 3's blend.
+__device__ __forceinline__ float merged(float a, float b, float G, const OuterArgs& A) {
+  const float d = __fsub_rn(a, b);
+  const float D = __fsub_rn(G, b);
+  const float lin = __fmaf_rn(A.c1, d, G);
+  const float target = __fmaf_rn(__fmul_rn(__fmul_rn(A.c2, d), d), D, lin);
+  return __fmaf_rn(A.alpha, target, __fmul_rn(A.one_minus_alpha, a));
+}
+
+__device__ __forceinline__ float& comp(float4& v, int k) { return reinterpret_cast<float*>(&v)[k]; }
+__device__ __forceinline__ float comp(const float4& v, int k) { return reinterpret_cast<const float*>(&v)[k]; }
+
+// One scalar element, any M (used on ragged edges, unaligned snapshot layouts and M not instantiated).
+template <int MODE, bool SAME>
+__device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, long long snap_e, double& acc) {
+  const int M = A.M;
+  const float thg = ld1(A.theta_g + e);
+  float G;
+  if (MODE == MODE_MERGE_ONLY) {
+    G = thg;
+  } else {
+    float sum = 0.f;
+    for (int m = 0; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(ld1(A.w_snap + m * A.snap_stride + snap_e), thg));
+    float Delta, u_new;
+    outer_update(sum, thg, ld1(A.momentum + e), A, Delta, u_new, G);
+    acc += (double)__fmul_rn(Delta, Delta);
+    st1(A.theta_g + e, G);
+    st1(A.momentum + e, u_new);
+    if (A.delta_out) st1(A.delta_out + e, Delta);
+  }
+  if (MODE != MODE_OUTER_ONLY) {
+    for (int m = 0; m < M; ++m) {
+      const float b = ld1(A.w_snap + m * A.snap_stride + snap_e);
+      const float a = SAME ? b : ld1(A.w_now + m * A.now_stride + e);
+      st1(A.w_now + m * A.now_stride + e, merged(a, b, G, A));
+    }
+  }
+}
+
+// Registers of one 16-byte lane.
+template <int M, int MODE, bool SAME>
+struct Lane {
+  float4 b[M];
+  float4 a[(MODE != MODE_OUTER_ONLY && !SAME) ? M : 1];
+  float4 thg;
+  float4 u;
+
+  __device__ __forceinline__ void load(const OuterArgs& A, long long e, long long snap_e) {
+    thg = ld4(A.theta_g + e);
+    if (MODE != MODE_MERGE_ONLY) u = ld4(A.momentum + e);
+#pragma unroll
+    for (int m = 0; m < M; ++m) b[m] = ld4(A.w_snap + m * A.snap_stride + snap_e);
+    if (MODE != MODE_OUTER_ONLY && !SAME) {
+#pragma unroll
+      for (int m = 0; m < M; ++m) a[m] = ld4(A.w_now + m * A.now_stride + e);
+    }
+  }
+
+  __device__ __forceinline__ void compute_store(const OuterArgs& A, long long e, double& acc) {
+    float4 G4;
+    if (MODE == MODE_MERGE_ONLY) {
+      G4 = thg;
+    } else {
+      float4 D4, U4;
+      float sq = 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float t = comp(thg, k);
+        float sum = __fsub_rn(comp(b[0], k), t);
+#pragma unroll
+        for (int m = 1; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(comp(b[m], k), t));
+        float Delta, u_new, G;
+        outer_update(sum, t, comp(u, k), A, Delta, u_new, G);
+        comp(D4, k) = Delta; comp(U4, k) = u_new; comp(G4, k) = G;
+        sq = __fmaf_rn(Delta, Delta, sq);
+      }
+      acc += (double)sq;
+      st4(A.theta_g + e, G4);
+      st4(A.momentum + e, U4);
+      if (A.delta_out) st4(A.delta_out + e, D4);
+    }
+    if (MODE != MODE_OUTER_ONLY) {
+#pragma unroll
+      for (int m = 0; m < M; ++m) {
+        float4 o;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float bb = comp(b[m], k);
+          const float aa = SAME ? bb : comp(a[m], k);
+          comp(o, k) = merged(aa, bb, comp(G4, k), A);
+        }
+        st4(A.w_now + m * A.now_stride + e, o);
+      }
+    }
+  }
+};
+
+// M = 0 instantiates the generic path: every lane goes element by element with the runtime M.
+template <int M, int U, int MODE, bool SAME>
+__global__ void __launch_bounds__(kThreads)
+k_outer(const OuterArgs A) {
+  const PlanHeader h = *A.hdr;
+  constexpr int LPT = kThreads * U;  // lanes per tile
+  SlotAccumulator sa;
+  int seg = 0;
+  int seg_loaded = -1;
+  SegPlan sp;
+  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+    while (seg + 1 < h.n_seg && tile >= A.plan[seg + 1].first_tile) ++seg;
+    if (seg != seg_loaded) {
+      sp = A.plan[seg];
+      seg_loaded = seg;
+      if (A.partial) sa.advance(sp.slot, A.partial);
+    }
+    const long long lane0 = (long long)(tile - sp.first_tile) * LPT;
+    const long long e_tile = sp.abase + 4 * lane0;          // first element of the tile (aligned)
+    const long long seg_end = sp.off + sp.len;
+    const long long snap_shift = sp.snap_off - sp.off;       // snap index = native index + shift
+    const bool interior = (M > 0) && sp.vec_ok && e_tile >= sp.off && e_tile + 4LL * LPT <= seg_end;
+    if (interior) {
+      if constexpr (M > 0) {
+        Lane<M, MODE, SAME> L[U];
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+          const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
+          L[j].load(A, e, e + snap_shift);
+        }
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+          const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
+          L[j].compute_store(A, e, sa.acc);
+        }
+      }
+    } else {
+      for (int j = 0; j < U; ++j) {
+        const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
+        if (e >= seg_end) break;
+        bool done = false;
+        if constexpr (M > 0) {
+          if (sp.vec_ok && e >= sp.off && e + 4 <= seg_end) {
+            Lane<M, MODE, SAME> L1;
+            L1.load(A, e, e + snap_shift);
+            L1.compute_store(A, e, sa.acc);
+            done = true;
+          }
+        }
+        if (!done) {
+          for (int k = 0; k < 4; ++k) {
+            const long long ee = e + k;
+            if (ee >= sp.off && ee < seg_end) scalar_element<MODE, SAME>(A, ee, ee + snap_shift, sa.acc);
+          }
+        }
+      }
+    }
+  }
+  if (A.partial) sa.finish(h.n_ids, A.partial);
+}
+
+// ---------------------------------------------------------------------------
+// S6 stand-alone: sums of squares of an N-sized vector over the planned tiles.
+// ---------------------------------------------------------------------------
+template <int U>
+__global__ void __launch_bounds__(kThreads)
+k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ plan,
+        const PlanHeader* __restrict__ hdr, double* __restrict__ partial) {
+  const PlanHeader h = *hdr;
+  constexpr int LPT = kThreads * U;
+  SlotAccumulator sa;
+  int seg = 0, seg_loaded = -1;
+  SegPlan sp;
+  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+    while (seg + 1 < h.n_seg && tile >= plan[seg + 1].first_tile) ++seg;
+    if (seg != seg_loaded) { sp = plan[seg]; seg_loaded = seg; sa.advance(sp.slot, partial); }
+    const long long e_tile = sp.abase + 4LL * (long long)(tile - sp.first_tile) * LPT;
+    const long long seg_end = sp.off + sp.len;
+    if (e_tile >= sp.off && e_tile + 4LL * LPT <= seg_end) {
+      float4 v[U];
+#pragma unroll
+      for (int j = 0; j < U; ++j) v[j] = ld4(x + e_tile + 4LL * (j * kThreads + threadIdx.x));
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+        float sq = __fmul_rn(v[j].x, v[j].x);
+        sq = __fmaf_rn(v[j].y, v[j].y, sq);
+        sq = __fmaf_rn(v[j].z, v[j].z, sq);
+        sq = __fmaf_rn(v[j].w, v[j].w, sq);
+        sa.acc += (double)sq;
+      }
+    } else {
+      for (int j = 0; j < U; ++j) {
+        const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
+        if (e >= seg_end) break;
+        for (int k = 0; k < 4; ++k) {
+          const long long ee = e + k;
+          if (ee >= sp.off && ee < seg_end) { const float t = ld1(x + ee); sa.acc += (double)__fmul_rn(t, t); }
+        }
+      }
+    }
+  }
+  sa.finish(h.n_ids, partial);
+}
+
+// ---------------------------------------------------------------------------
+// S0: copy the listed fragments of every worker from w_now into w_snap.
+// ---------------------------------------------------------------------------
+template <int U>
+__global__ void __launch_bounds__(kThreads)
+k_snapshot(const float* __restrict__ w_now, float* __restrict__ w_snap, long long now_stride,
+           long long snap_stride, int M, const SegPlan* __restrict__ plan,
+           const PlanHeader* __restrict__ hdr) {
+  const PlanHeader h = *hdr;
+  constexpr int LPT = kThreads * U;
+  int seg = 0, seg_loaded = -1;
+  SegPlan sp;
+  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+    while (seg + 1 < h.n_seg && tile >= plan[seg + 1].first_tile) ++seg;
+    if (seg != seg_loaded) { sp = plan[seg]; seg_loaded = seg; }
+    const long long e_tile = sp.abase + 4LL * (long long)(tile - sp.first_tile) * LPT;
+    const long long seg_end = sp.off + sp.len;
+    const long long shift = sp.snap_off - sp.off;
+    if (sp.vec_ok && e_tile >= sp.off && e_tile + 4LL * LPT <= seg_end) {
+      for (int m = 0; m < M; ++m) {
+        float4 v[U];
+#pragma unroll
+        for (int j = 0; j < U; ++j)
+          v[j] = ld4(w_now + m * now_stride + e_tile + 4LL * (j * kThreads + threadIdx.x));
+#pragma unroll
+        for (int j = 0; j < U; ++j)
+          st4(w_snap + m * snap_stride + shift + e_tile + 4LL * (j * kThreads + threadIdx.x), v[j]);
+      }
+    } else {
+      for (int j = 0; j < U; ++j) {
+        const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
+        if (e >= seg_end) break;
+        for (int k = 0; k < 4; ++k) {
+          const long long ee = e + k;
+          if (ee >= sp.off && ee < seg_end)
+            for (int m = 0; m < M; ++m) st1(w_snap + m * snap_stride + shift + ee, ld1(w_now + m * now_stride + ee));
+        }
+      }
+    }
+  }
+}
+
+}  // namespace cocodc

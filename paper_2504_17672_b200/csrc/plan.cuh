@@ -1,0 +1,198 @@
+// Launch plan: which tiles of which segments one call processes.
+//
+// A call works on a list of fragment ids that lives in device memory (it is
+// usually written by the selection kernel, and the host never reads it).  A
+// one-block kernel expands that list into a table of segments with a running
+// tile count; the streaming kernels then map a tile index to (segment, lane
+// range) without any host round-trip.
+//
+// Geometry.  Every segment [off, off+len) is covered by 16-byte "lanes" of four
+// elements that start at abase = off rounded down to a multiple of 4, so lane
+// addresses are aligned in every N-sized buffer whose base is aligned.  A tile
+// is `lanes_per_tile` consecutive lanes of one segment.  Only the first and the
+// last lane of a segment can be partial; partial lanes take a scalar path.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cocodc {
+
+struct SegPlan {
+  long long off;       // element offset of the segment in every N-sized buffer
+  long long len;       // elements
+  long long snap_off;  // element offset of the segment inside a row of w_snap
+  long long abase;     // off & ~3
+  int first_tile;      // index of the segment's first tile in this launch
+  int slot;            // position of the owning fragment in the id list
+  int frag;            // fragment id
+  int vec_ok;          // 1 if w_snap lanes are 16-byte aligned together with the native lanes
+};
+
+struct PlanHeader {
+  int total_tiles;
+  int n_seg;
+  int n_ids;
+  int pad;
+};
+
+// Status word helper: keep the first error recorded since the last poll.
+__device__ __forceinline__ void record_status(int* status, int code) {
+  atomicCAS(status, 0, code);
+}
+
+constexpr int kPlanThreads = 256;
+constexpr int kMaxK = 1024;
+
+// ids == nullptr means "all K fragments in index order" (stand-alone scoring).
+__global__ void __launch_bounds__(kPlanThreads)
+k_plan(const int* __restrict__ ids, const int* __restrict__ n_ids_p, int K,
+       const int* __restrict__ frag_seg_ptr, const long long* __restrict__ seg_off,
+       const long long* __restrict__ seg_len, const long long* __restrict__ snap_offset,
+       int lanes_per_tile, int plan_capacity, SegPlan* __restrict__ plan,
+       PlanHeader* __restrict__ hdr, int* __restrict__ status, int err_invalid) {
+  __shared__ int seen[kMaxK];
+  __shared__ int bad;
+  const int tid = threadIdx.x;
+  int n = (ids == nullptr) ? K : *n_ids_p;
+  if (tid == 0) bad = (n < 0 || n > K) ? 1 : 0;
+  for (int i = tid; i < K; i += blockDim.x) seen[i] = 0;
+  __syncthreads();
+  if (!bad && ids != nullptr) {
+    for (int i = tid; i < n; i += blockDim.x) {
+      int p = ids[i];
+      if (p < 0 || p >= K) {
+        bad = 1;
+      } else if (atomicAdd(&seen[p], 1) != 0) {
+        bad = 1;
+      } else if (snap_offset != nullptr && snap_offset[p] < 0) {
+        bad = 1;  // the fragment has no slot in the snapshot pool
+      }
+    }
+  }
+  __syncthreads();
+  if (tid != 0) return;
+  if (bad) {
+    hdr->total_tiles = 0; hdr->n_seg = 0; hdr->n_ids = 0; hdr->pad = 0;
+    record_status(status, err_invalid);
+    return;
+  }
+  long long tiles = 0;
+  int ns = 0;
+  bool overflow = false;
+  for (int j = 0; j < n && !overflow; ++j) {
+    const int p = (ids == nullptr) ? j : ids[j];
+    long long pos = 0;  // elements of the fragment placed so far (packed snapshot layout)
+    for (int s = frag_seg_ptr[p]; s < frag_seg_ptr[p + 1]; ++s) {
+      if (ns >= plan_capacity) { overflow = true; break; }
+      SegPlan sp;
+      sp.off = seg_off[s];
+      sp.len = seg_len[s];
+      sp.snap_off = (snap_offset != nullptr) ? snap_offset[p] + pos : sp.off;
+      sp.abase = sp.off & ~3LL;
+      sp.first_tile = (int)tiles;
+      sp.slot = j;
+      sp.frag = p;
+      sp.vec_ok = (((sp.snap_off - sp.off) & 3LL) == 0) ? 1 : 0;
+      plan[ns++] = sp;
+      const long long lanes = (sp.off - sp.abase + sp.len + 3) >> 2;
+      tiles += (lanes + lanes_per_tile - 1) / lanes_per_tile;
+      pos += sp.len;
+      if (tiles > 0x7fffffffLL) { overflow = true; break; }
+    }
+  }
+  if (overflow) {
+    hdr->total_tiles = 0; hdr->n_seg = 0; hdr->n_ids = 0; hdr->pad = 0;
+    record_status(status, err_invalid);
+    return;
+  }
+  hdr->total_tiles = (int)tiles;
+  hdr->n_seg = ns;
+  hdr->n_ids = n;
+  hdr->pad = 0;
+}
+
+// ---------------------------------------------------------------------------
+// Per-CTA accumulation of sums of squares, one slot per listed fragment.
+//
+// A persistent CTA walks its tiles in increasing order, so the fragment slot it
+// works on never decreases.  Every thread keeps a double accumulator for the
+// current slot; when the slot changes the warp reduces it and lane 0 writes
+// partial[(slot*gridDim.x + blockIdx.x)*warps + warp].  Slots a CTA never
+// touched get an explicit zero, so the finalize kernel can sum every entry
+// without the buffer being cleared first.  The tile-to-CTA map is static,
+// hence the summation order - and the rounded result - is the same every run.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+struct SlotAccumulator {
+  double acc = 0.0;
+  int slot = 0;
+
+  __device__ __forceinline__ void flush_to(int new_slot, double* __restrict__ partial) {
+    const int warps = blockDim.x >> 5;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    double v = warp_sum(acc);
+    if (lane == 0) {
+      partial[((size_t)slot * gridDim.x + blockIdx.x) * warps + warp] = v;
+      for (int s = slot + 1; s < new_slot; ++s)
+        partial[((size_t)s * gridDim.x + blockIdx.x) * warps + warp] = 0.0;
+    }
+    acc = 0.0;
+    slot = new_slot;
+  }
+  __device__ __forceinline__ void advance(int new_slot, double* __restrict__ partial) {
+    if (new_slot != slot) flush_to(new_slot, partial);
+  }
+  // after the last tile: write the current slot and zero the rest up to n_ids
+  __device__ __forceinline__ void finish(int n_ids, double* __restrict__ partial) {
+    if (slot < n_ids) flush_to(n_ids, partial);
+  }
+};
+
+constexpr int kFinalizeThreads = 256;
+
+// One block per listed fragment: sum its partials in a fixed order, take the
+// square root, form the score of Eq. 10 and (for a completion) stamp last_sync.
+//   mode 0: completion - I_p = max(1, t_p - last_sync[p]); last_sync[p] = t_l
+//   mode 1: stand-alone scoring - I_p = max(1, interval[p]) or 1; last_sync untouched
+__global__ void __launch_bounds__(kFinalizeThreads)
+k_finalize_scores(const PlanHeader* __restrict__ hdr, const int* __restrict__ ids,
+                  const double* __restrict__ partial, int entries_per_slot,
+                  int mode, long long t_p, long long t_l, const long long* __restrict__ interval,
+                  long long* __restrict__ last_sync, float* __restrict__ norms,
+                  float* __restrict__ scores, int* __restrict__ status, int err_nonfinite) {
+  __shared__ double red[kFinalizeThreads];
+  const int j = blockIdx.x;
+  if (j >= hdr->n_ids) return;
+  const double* src = partial + (size_t)j * entries_per_slot;
+  double s = 0.0;
+  for (int i = threadIdx.x; i < entries_per_slot; i += kFinalizeThreads) s += src[i];
+  red[threadIdx.x] = s;
+  __syncthreads();
+#pragma unroll
+  for (int w = kFinalizeThreads / 2; w > 0; w >>= 1) {
+    if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x != 0) return;
+  const int p = (ids == nullptr) ? j : ids[j];
+  const double norm = sqrt(red[0]);
+  long long I = 1;
+  if (mode == 0) {
+    I = t_p - last_sync[p];
+    last_sync[p] = t_l;
+  } else if (interval != nullptr) {
+    I = interval[p];
+  }
+  if (I < 1) I = 1;
+  norms[p] = (float)norm;
+  scores[p] = (float)(norm / (double)I);
+  if (!isfinite(norm)) record_status(status, err_nonfinite);
+}
+
+}  // namespace cocodc

@@ -1,0 +1,116 @@
+"""Host-only checks of the C-ABI library: it loads, exports what the header declares, and validates arguments.
+
+No kernel is launched here; these run without a GPU.
+"""
+
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2504_17672_b200 import build
+    build.build()
+    from paper_2504_17672_b200 import binding
+    return binding
+
+
+def declared_functions():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in os.listdir(inc):
+        if fn.endswith(".h"):
+            text = open(os.path.join(inc, fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(cocodc_[a-z_0-9]+)\s*\(", text))
+    return names
+
+
+def test_library_exports_every_declared_symbol(B):
+    lib = B.library()
+    names = declared_functions()
+    assert {"cocodc_fragment_scores", "cocodc_select_fragments", "cocodc_outer_step", "cocodc_merge"} <= names
+    for name in names:
+        assert hasattr(lib, name), name
+    assert names == set(B.EXPORTS)
+
+
+def rows(name):
+    out = []
+    for line in open(os.path.join(ROOT, "tests", "golden", name)):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            out.append([float(x) for x in line.split()])
+    return out
+
+
+@pytest.mark.parametrize("row", rows("schedule_sizing.txt"))
+def test_sync_budget_matches_paper_values(B, row):
+    K, H, gamma, Tc, Ts, N, h = row
+    assert B.cocodc_sync_budget(int(K), int(H), gamma, Tc, Ts) == (int(N), int(h))
+
+
+def test_sync_budget_agrees_with_oracle_and_rejects_bad_input(B):
+    from oracle import reference as orc
+    rng = np.random.default_rng(0)
+    for _ in range(200):
+        K = int(rng.integers(1, 40)); H = int(rng.integers(1, 500))
+        gamma = float(rng.uniform(0.01, 1.0)); Tc = float(rng.uniform(0.01, 3)); Ts = float(rng.uniform(0.01, 30))
+        assert B.cocodc_sync_budget(K, H, gamma, Tc, Ts) == orc.sync_budget(K, H, gamma, Tc, Ts)
+    for bad in ((0, 100, 0.4, 1, 1), (4, 0, 0.4, 1, 1), (4, 100, 0.0, 1, 1), (4, 100, 1.5, 1, 1),
+                (4, 100, 0.4, 0.0, 1), (4, 100, 0.4, 1, -1.0), (4, 100, float("nan"), 1, 1)):
+        with pytest.raises(B.CocodcError) as e:
+            B.cocodc_sync_budget(*bad)
+        assert e.value.code == B.ERR_INVALID_ARG
+
+
+def test_status_strings(B):
+    seen = {B.status_string(c) for c in range(8)}
+    assert len(seen) == 8 and "ok" in seen
+    assert "unknown" in B.status_string(99)
+
+
+def test_create_rejects_bad_partitions_before_touching_the_device(B):
+    def create(N, ptr, off, ln, max_M=4):
+        return B.Context(N, ptr, off, ln, max_M, device=0)
+
+    cases = [
+        (100, [0, 1, 2], [0, 40], [50, 50]),      # overlapping segments
+        (100, [0, 1, 2], [0, 60], [50, 50]),      # runs past N
+        (100, [0, 1, 1], [0], [50]),              # empty fragment
+        (100, [0, 1], [-4], [50]),                # negative offset
+        (100, [0, 1], [0], [0]),                  # empty segment
+        (100, [1, 2], [0, 50], [50, 50]),         # CSR does not start at 0
+    ]
+    for N, ptr, off, ln in cases:
+        with pytest.raises(B.CocodcError) as e:
+            create(N, ptr, off, ln)
+        assert e.value.code == B.ERR_INVALID_ARG, (ptr, off, ln)
+    for bad_M in (0, 65):
+        with pytest.raises(B.CocodcError) as e:
+            create(100, [0, 1], [0], [100], max_M=bad_M)
+        assert e.value.code == B.ERR_INVALID_ARG
+
+
+def test_null_context_is_rejected(B):
+    lib = B.library()
+    assert lib.cocodc_poll_status(None, None) == B.ERR_INVALID_ARG
+    assert lib.cocodc_fragment_scores(None, None, None, None, None, None) == B.ERR_INVALID_ARG
+    assert lib.cocodc_destroy(None) == B.OK
+    assert lib.cocodc_launch_count(None) == 0
+
+
+def test_missing_library_fails_loudly(tmp_path, monkeypatch):
+    """The binding has no fallback: without the built library the import raises."""
+    import importlib
+    from paper_2504_17672_b200 import build
+    monkeypatch.setattr(build, "LIBRARY", str(tmp_path / "libcocodc.so"))
+    import paper_2504_17672_b200.binding as binding
+    with pytest.raises(ImportError):
+        binding._load()

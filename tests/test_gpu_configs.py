@@ -1,0 +1,171 @@
+"""Parity on the five benchmark workloads, in the launch configuration the benchmark times.
+
+tiny and gpt2_small are compared element by element over every processed fragment.  The
+billion-parameter shapes are compared on sampled elements (edges, tile borders, random positions),
+whole-fragment norms from the oracle for two fragments, a float64 torch reduction for the rest, and
+bit-exact checksums of everything that must not change."""
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import reference as orc
+from helpers import (GpuProblem, SampledCheck, check_step_against_oracle, fragment_checksums, np_,
+                     oracle_fragment_norm, orc_hyper, TOL_NORM)
+
+pytestmark = pytest.mark.gpu
+
+
+def free_gb():
+    free, _ = torch.cuda.mem_get_info()
+    return free / 2 ** 30
+
+
+def test_tiny_three_rounds():
+    w = synth.get_workload("tiny")
+    prob = GpuProblem(w, synth.generate(w, "cuda"))
+    t = 0
+    for rnd in range(3):
+        t += 12
+        before = prob.host_state()
+        prob.select(t)
+        prob.outer_step(t, t + w.tau)
+        assert prob.poll() == 0
+        ids = np_(prob.ids)[:int(prob.n_ids.item())].tolist()
+        assert len(ids) == 2
+        check_step_against_oracle(prob, before, ids, t, t + w.tau, orc_hyper(w))
+        prob.snapshot()
+        prob.bufs.w_now.add_(torch.randn_like(prob.bufs.w_now) * 1e-3)
+
+
+def test_gpt2_small_full_parity():
+    w = synth.get_workload("gpt2_small")
+    prob = GpuProblem(w, synth.generate(w, "cuda"))
+    # round 0: complete every fragment once (the start-up round of the schedule): full element-wise parity
+    all_ids = list(range(w.K))
+    prob.set_ids(all_ids)
+    before = prob.host_state()
+    prob.outer_step(10, 10 + w.tau)
+    assert prob.poll() == 0
+    check_step_against_oracle(prob, before, all_ids, 10, 10 + w.tau, orc_hyper(w))
+    del before
+    # round 1: local training moves on, then selection under the 25 % parameter budget
+    prob.snapshot()
+    g = torch.Generator(device="cuda").manual_seed(11)
+    for m in range(w.M):
+        prob.bufs.w_now[m].add_(torch.randn(w.N, generator=g, device="cuda") * 1e-3)
+    before = prob.host_state()
+    prob.select(t_now=20)
+    n = int(prob.n_ids.item())
+    ids = np_(prob.ids)[:n].tolist()
+    emask, eids, en = orc.select_fragments(before["scores"], before["last_sync"], w.partition.frag_sizes, 20, w.H,
+                                           orc.BUDGET_PARAMS, w.budget)
+    assert ids == eids.tolist() and np.array_equal(np_(prob.mask), emask)
+    assert sum(w.partition.frag_size(p) for p in ids) <= w.budget or n == 1
+    prob.outer_step(20, 20 + w.tau)
+    assert prob.poll() == 0
+    check_step_against_oracle(prob, before, ids, 20, 20 + w.tau, orc_hyper(w))
+
+
+def _sampled_round(prob, ids, t_p, t_l, ohp, full_norm=2, same=False):
+    w = prob.w
+    ids = [int(p) for p in ids]
+    prob.set_ids(ids)
+    sc = SampledCheck(prob, ids, seed=t_p, same=same)
+    exp_norm = {p: oracle_fragment_norm(prob, p) for p in ids[:full_norm]} if not same else {}
+    # float64 reduction on the device for the remaining fragments (library cross-check at full size)
+    for p in ids[full_norm:]:
+        acc = 0.0
+        b = prob.bufs
+        pos = 0
+        for o, l in w.partition.fragments[p]:
+            if b.snap_offset is None or same:
+                s = (b.w_now if same else b.w_snap)[:, o:o + l]
+            else:
+                so = int(b.snap_offset[p].item()) + pos
+                s = b.w_snap[:, so:so + l]
+            d = (s.double() - b.theta_g[o:o + l].double()).mean(0)
+            acc += float((d * d).sum().item())
+            pos += l
+            del d
+        exp_norm[p] = float(np.sqrt(acc))
+    untouched = [p for p in range(w.K) if p not in ids]
+    cs_before = {k: fragment_checksums(w, getattr(prob.bufs, k)) for k in ("theta_g", "momentum", "w_now")}
+    last_before = np_(prob.last_sync).copy()
+    prob.outer_step(t_p, t_l, hyper=prob.hyper(**{k: getattr(ohp, k) for k in ("tau", "lam", "alpha", "comp_mode", "sign_mode")}),
+                    w_snap=prob.bufs.w_now if same else None)
+    assert prob.poll() == 0
+    worst = sc.check(t_p, t_l, ohp)
+    cs_after = {k: fragment_checksums(w, getattr(prob.bufs, k)) for k in cs_before}
+    for k in cs_before:
+        assert np.array_equal(cs_before[k][untouched], cs_after[k][untouched]), f"{k} changed outside ids"
+        assert not np.array_equal(cs_before[k][ids], cs_after[k][ids])
+    norms, scores, last = np_(prob.norms), np_(prob.scores), np_(prob.last_sync)
+    for p, en in exp_norm.items():
+        assert abs(norms[p] - en) <= TOL_NORM * en, (p, norms[p], en)
+        es = en / max(1, t_p - int(last_before[p]))
+        assert abs(scores[p] - es) <= TOL_NORM * es
+    exp_last = last_before.copy()
+    exp_last[ids] = t_l
+    assert np.array_equal(last, exp_last)
+    return worst
+
+
+def test_llama_1b_selected_by_change_norm():
+    if free_gb() < 60:
+        pytest.skip("needs 60 GB of free device memory")
+    w = synth.get_workload("llama_1b")
+    prob = GpuProblem(w, synth.generate(w, "cuda"))
+    ohp = orc_hyper(w)
+    # start-up round: every fragment completes once; this produces the change norms that drive selection
+    _sampled_round(prob, list(range(w.K)), 25, 25 + w.tau, ohp)
+    scores = np_(prob.scores).copy()
+    srt = np.sort(scores)[::-1]
+    assert np.all((srt[:-1] - srt[1:]) > 1e-4 * srt[:-1]), "scores too close for a rounding-proof order"
+    prob.snapshot()
+    g = torch.Generator(device="cuda").manual_seed(12)
+    for m in range(w.M):
+        prob.bufs.w_now[m].add_(torch.randn(w.N, generator=g, device="cuda") * 1e-3)
+    prob.select(t_now=40)
+    n = int(prob.n_ids.item())
+    ids = np_(prob.ids)[:n].tolist()
+    _, eids, en = orc.select_fragments(scores, np_(prob.last_sync), w.partition.frag_sizes, 40, w.H,
+                                       orc.BUDGET_COUNT, w.budget)
+    assert n == en == 4 and ids == eids.tolist()
+    assert ids == list(np.argsort(-scores, kind="stable")[:4])
+    _sampled_round(prob, ids, 40, 40 + w.tau, ohp)
+
+
+@pytest.mark.parametrize("tau,lam,frac", [(1, 0.0, 0.25), (2, 0.25, 0.5), (8, 1.0, 1.0), (4, 0.5, 0.5)])
+def test_sweep_1b_variants(tau, lam, frac):
+    if free_gb() < 60:
+        pytest.skip("needs 60 GB of free device memory")
+    w = synth.get_workload("sweep_1b").with_(tau=tau, lam=lam)
+    prob = GpuProblem(w, synth.generate(w, "cuda"))
+    n = int(round(frac * w.K))
+    prob.select(t_now=5, budget_kind=0, budget=n)      # all scores infinite: the first n fragments
+    ids = np_(prob.ids)[:int(prob.n_ids.item())].tolist()
+    assert ids == list(range(n))
+    _sampled_round(prob, ids, 5, 5 + tau, orc_hyper(w))
+
+
+def test_llama_3b_snapshot_pool():
+    if free_gb() < 130:
+        pytest.skip("needs 130 GB of free device memory")
+    w = synth.get_workload("llama_3b")
+    from paper_2504_17672_b200 import binding as B
+    ptr, off, ln = w.partition.csr()
+    sizes = w.partition.frag_sizes
+    # scores of an earlier round, taken as the expected change norm s_p*sqrt(n_p) of this seed
+    scores = (synth.fragment_scales(w) * np.sqrt(sizes)).astype(np.float32)
+    _, eids, en = orc.select_fragments(scores, np.zeros(w.K, dtype=np.int64), sizes, 40, w.H,
+                                       orc.BUDGET_PARAMS, w.budget)
+    assert sum(sizes[eids]) <= w.budget and en >= 2
+    bufs = synth.generate(w, "cuda", snap_layout="pool", pool_ids=eids.tolist())
+    prob = GpuProblem(w, bufs)
+    prob.scores.copy_(torch.from_numpy(scores))
+    prob.select(t_now=40)
+    ids = np_(prob.ids)[:int(prob.n_ids.item())].tolist()
+    assert ids == eids.tolist()
+    _sampled_round(prob, ids, 40, 40 + w.tau, orc_hyper(w), full_norm=1)

@@ -1,0 +1,227 @@
+"""GPU-vs-oracle parity of the outer step on small problems that still span several tiles,
+ragged edges, odd offsets, every worker count path, every mode, and both snapshot layouts."""
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import reference as orc
+from helpers import (GpuProblem, Guarded, assert_close, check_step_against_oracle, fragments_of, np_,
+                     orc_hyper, touched_mask, TOL_PARAM)
+
+pytestmark = pytest.mark.gpu
+
+# several tiles per fragment (a tile is 2048 elements at M <= 4), odd sizes, odd offsets, gaps, a strided fragment
+RAGGED = (60_000, [[(3, 9_001), (40_010, 4_097)], [(9_004, 12_345)], [(21_349, 5)], [(21_360, 18_640)],
+                   [(44_111, 15_000)]])
+
+
+def make(M, seed=0, frs=RAGGED, snap_layout="full", pool_ids=None, pool_offsets=None, **kw):
+    w = synth.small_workload(frs, M=M, seed=seed, scale_kind="loguniform", **kw)
+    bufs = synth.generate(w, "cuda", snap_layout=snap_layout, pool_ids=pool_ids, pool_offsets=pool_offsets,
+                          momentum_sigma=1e-3)
+    return GpuProblem(w, bufs)
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 8])
+def test_fused_step_all_worker_counts(M):
+    prob = make(M, seed=M)
+    ids = [3, 0, 2, 4]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    delta = torch.full((prob.w.N,), 7.0, dtype=torch.float32, device="cuda")
+    prob.outer_step(t_p=10, t_l=12, delta_out=delta)
+    assert prob.poll() == 0
+    check_step_against_oracle(prob, before, ids, 10, 12, orc_hyper(prob.w), delta_out=delta)
+    assert bool((delta[torch.from_numpy(~touched_mask(prob.w, ids)).cuda()] == 7.0).all())
+
+
+@pytest.mark.parametrize("sign", [0, 1, 2])
+@pytest.mark.parametrize("alpha", [1.0, 0.5, 0.0])
+def test_sign_modes_and_mixing(sign, alpha):
+    prob = make(4, seed=20 + sign, tau=4, lam=1.0)
+    ids = [1, 4]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    prob.outer_step(5, 9, hyper=prob.hyper(sign_mode=sign, alpha=alpha))
+    check_step_against_oracle(prob, before, ids, 5, 9, orc_hyper(prob.w, sign_mode=sign, alpha=alpha))
+
+
+def test_no_compensation_is_streaming_diloco():
+    prob = make(4, seed=30)
+    ids = [0, 1, 2, 3, 4]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    prob.outer_step(5, 7, hyper=prob.hyper(comp_mode=0, alpha=0.25))
+    check_step_against_oracle(prob, before, ids, 5, 7, orc_hyper(prob.w, comp_mode=orc.COMP_NONE, alpha=0.25))
+
+
+@pytest.mark.parametrize("M", [2, 4, 6])
+def test_zero_delay_blocking_sync(M):
+    """w_snap == w_now: the DiLoCo case; every worker leaves with the new global state."""
+    prob = make(M, seed=40)
+    ids = [4, 0]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    prob.outer_step(100, 100, hyper=prob.hyper(tau=0), w_snap=prob.bufs.w_now)
+    check_step_against_oracle(prob, before, ids, 100, 100, orc_hyper(prob.w, tau=0), same=True)
+    g = np_(prob.bufs.theta_g)
+    wn = np_(prob.bufs.w_now)
+    t = touched_mask(prob.w, ids)
+    for m in range(M):
+        assert np.array_equal(wn[m][t], g[t])
+
+
+def test_three_consecutive_steps_carry_momentum():
+    prob = make(4, seed=50)
+    rng = np.random.default_rng(0)
+    ids = [0, 1, 3]
+    for step in range(3):
+        prob.set_ids(ids)
+        before = prob.host_state()
+        prob.outer_step(10 * step + 5, 10 * step + 7)
+        check_step_against_oracle(prob, before, ids, 10 * step + 5, 10 * step + 7, orc_hyper(prob.w))
+        # local training moves on: new snapshot = current, then drift
+        prob.snapshot()
+        prob.bufs.w_now.add_(torch.randn_like(prob.bufs.w_now) * 1e-3)
+    assert prob.poll() == 0
+
+
+def test_unfused_path_equals_fused_bit_for_bit():
+    a = make(4, seed=60)
+    b = make(4, seed=60)
+    ids = [2, 1, 4]
+    for prob in (a, b):
+        prob.set_ids(ids)
+    a.outer_step(3, 5)
+    before = b.host_state()
+    b.outer_step(3, 5, stages=1 | 4)          # S1-S3 + S6
+    check_step_against_oracle(b, before, ids, 3, 5, orc_hyper(b.w), do_merge=False)
+    b.merge(b.bufs.theta_g)                    # S4-S5
+    for x, y in ((a.bufs.w_now, b.bufs.w_now), (a.bufs.theta_g, b.bufs.theta_g), (a.bufs.momentum, b.bufs.momentum),
+                 (a.scores, b.scores), (a.norms, b.norms)):
+        assert torch.equal(x, y)
+    # merge alone against the oracle
+    res = orc.merge(fragments_of(b.w), orc_hyper(b.w), before["w_now"], before["w_snap"],
+                    np_(a.bufs.theta_g), ids)
+    for p in ids:
+        got = orc.gather_fragment(fragments_of(b.w), np_(b.bufs.w_now), p)
+        assert_close(got, res[p], TOL_PARAM, f"merge[{p}]")
+
+
+@pytest.mark.parametrize("aligned", [True, False])
+def test_snapshot_pool_layouts(aligned):
+    """Snapshots packed in a pool: 16-byte-compatible offsets take the vector path, others the scalar one."""
+    pool_offsets = None if aligned else {4: 1, 0: 15_002, 1: 28_103}
+    prob = make(4, seed=70, snap_layout="pool", pool_ids=[4, 0, 1], pool_offsets=pool_offsets)
+    ids = [0, 4, 1]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    prob.outer_step(8, 11)
+    assert prob.poll() == 0
+    check_step_against_oracle(prob, before, ids, 8, 11, orc_hyper(prob.w))
+    # a fragment without a pool slot is refused on the device and nothing is touched
+    prob.set_ids([0, 2])
+    before = prob.host_state()
+    prob.outer_step(12, 13)
+    assert prob.poll() == prob.B.ERR_INVALID_ARG
+    after = prob.host_state()
+    for k in ("w_now", "theta_g", "momentum", "last_sync"):
+        assert np.array_equal(before[k], after[k])
+
+
+def test_snapshot_kernel_copies_exactly_the_listed_fragments():
+    for layout, pool_ids in (("full", None), ("pool", [1, 3, 0])):
+        prob = make(3, seed=80, snap_layout=layout, pool_ids=pool_ids)
+        ids = [3, 0]
+        prob.set_ids(ids)
+        before = prob.host_state()
+        prob.snapshot()
+        assert prob.poll() == 0
+        exp = orc.snapshot(fragments_of(prob.w), before["w_now"], ids, 3, before["snap_offset"], before["w_snap"])
+        assert np.array_equal(np_(prob.bufs.w_snap), exp)
+        assert np.array_equal(np_(prob.bufs.w_now), before["w_now"])
+
+
+def test_guard_bands_and_untouched_memory():
+    """Canary words around every buffer survive; sizes are chosen so the last tile is ragged."""
+    w = synth.small_workload([4099, 2048, 1, 6000], M=4, seed=90)
+    bufs = synth.generate(w, "cuda", momentum_sigma=1e-3)
+    g = {k: Guarded(getattr(bufs, k).shape, torch.float32, "cuda", fill=getattr(bufs, k))
+         for k in ("theta_g", "momentum", "w_now", "w_snap")}
+    for k, v in g.items():
+        setattr(bufs, k, v.t)
+    prob = GpuProblem(w, bufs)
+    gd = Guarded((w.N,), torch.float32, "cuda")
+    ids = [0, 2, 3]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    prob.outer_step(1, 2, delta_out=gd.t)
+    prob.snapshot()
+    assert prob.poll() == 0
+    assert all(v.intact() for v in g.values()) and gd.intact()
+    prob.bufs.w_snap.copy_(torch.from_numpy(before["w_snap"]).cuda())
+    check_step_against_oracle(prob, before, ids, 1, 2, orc_hyper(w), delta_out=gd.t)
+
+
+def test_device_side_id_validation():
+    prob = make(2, seed=100)
+    before = prob.host_state()
+    for bad in ([0, 0], [5], [-1], [0, 1, 2, 3, 4, 4]):
+        prob.ids.fill_(-1)
+        prob.ids[:len(bad)] = torch.tensor(bad[:prob.w.K], dtype=torch.int32, device="cuda")
+        prob.n_ids.fill_(len(bad))
+        prob.outer_step(1, 2)
+        assert prob.poll() == prob.B.ERR_INVALID_ARG, bad
+    after = prob.host_state()
+    for k in ("w_now", "theta_g", "momentum", "last_sync", "scores"):
+        assert np.array_equal(before[k], after[k], equal_nan=True)
+    # an empty list is legal and does nothing
+    prob.set_ids([])
+    prob.outer_step(1, 2)
+    assert prob.poll() == 0
+    assert np.array_equal(prob.host_state()["w_now"], before["w_now"])
+
+
+def test_host_validation_errors():
+    prob = make(2, seed=110)
+    B, b = prob.B, prob.bufs
+    prob.set_ids([0])
+
+    def call(**kw):
+        a = dict(hyper=prob.hyper(), w_now=b.w_now, w_snap=b.w_snap, now_stride=b.now_stride,
+                 snap_stride=b.snap_stride, snap_offset=None, theta_g=b.theta_g, momentum=b.momentum,
+                 delta_g_out=None, ids=prob.ids, n_ids=prob.n_ids, t_p=1, t_l=2, last_sync=prob.last_sync,
+                 norms=prob.norms, scores=prob.scores, stages=7)
+        a.update(kw)
+        prob.ctx.cocodc_outer_step(**a)
+
+    def code(**kw):
+        with pytest.raises(B.CocodcError) as e:
+            call(**kw)
+        return e.value.code
+
+    assert code(theta_g=b.momentum) == B.ERR_ALIAS
+    assert code(delta_g_out=b.w_now[1]) == B.ERR_ALIAS
+    assert code(w_snap=b.w_now[:, 4:], snap_stride=b.now_stride) in (B.ERR_ALIAS, B.ERR_INVALID_ARG)
+    assert code(theta_g=b.theta_g[1:]) == B.ERR_ALIGNMENT
+    assert code(now_stride=b.now_stride + 2) == B.ERR_ALIGNMENT
+    assert code(hyper=prob.hyper(M=3)) == B.ERR_INVALID_ARG          # beyond max_M of the context
+    assert code(hyper=prob.hyper(H=0)) == B.ERR_INVALID_ARG
+    assert code(hyper=prob.hyper(tau=0)) == B.ERR_INVALID_ARG        # Eq. 4 divides by tau
+    assert code(hyper=prob.hyper(sign_mode=3)) == B.ERR_INVALID_ARG
+    assert code(stages=2) == B.ERR_INVALID_ARG
+    assert code(ids=None) == B.ERR_INVALID_ARG
+    assert code(t_p=5, t_l=4) == B.ERR_INVALID_ARG
+    call(hyper=prob.hyper(tau=0, comp_mode=0))                        # legal: no compensation
+    assert prob.poll() == 0
+
+
+def test_nonfinite_norm_is_reported():
+    prob = make(2, seed=120)
+    prob.bufs.w_snap[0, 100] = float("inf")
+    prob.set_ids([0])
+    prob.outer_step(1, 2)
+    assert prob.poll() == prob.B.ERR_NONFINITE
+    assert prob.poll() == 0

@@ -1,0 +1,135 @@
+"""Bit-exact parity of the device-side fragment selection (Algorithm 2 under a budget) and
+parity of the stand-alone fragment scores (Eq. 10)."""
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import reference as orc
+from helpers import GpuProblem, fragments_of, np_, TOL_NORM
+
+pytestmark = pytest.mark.gpu
+
+
+def selection_problem(K, rng, sizes=None):
+    sizes = rng.integers(1, 5000, size=K) if sizes is None else sizes
+    w = synth.small_workload([int(s) for s in sizes], M=1, seed=0)
+    from paper_2504_17672_b200 import binding as B
+    ptr, off, ln = w.partition.csr()
+    return w, B.Context(w.N, ptr, off, ln, 1), B
+
+
+@pytest.mark.parametrize("K", [1, 2, 7, 13, 32, 64, 333, 1024])
+def test_selection_matches_oracle_bit_for_bit(K):
+    rng = np.random.default_rng(K)
+    w, ctx, B = selection_problem(K, rng)
+    sizes = w.partition.frag_sizes
+    dev = "cuda"
+    mask = torch.zeros(K, dtype=torch.uint8, device=dev)
+    ids = torch.zeros(K, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    for trial in range(12):
+        pool = np.array([0.0, 0.5, 1.0, 1.0, 2.5, 3.0, np.inf, np.inf], dtype=np.float32)
+        if trial % 2:
+            scores = rng.choice(pool, size=K)
+        else:
+            scores = rng.random(K).astype(np.float32)
+        H = 100
+        last = rng.integers(0, 200, size=K).astype(np.int64)
+        t_now = int(rng.integers(100, 280))
+        inel = (rng.random(K) < 0.3).astype(np.uint8) if trial % 3 else None
+        if trial == 5 and inel is not None:
+            inel[:] = 1
+        for kind, budget in ((B.BUDGET_COUNT, int(rng.integers(0, K + 2))),
+                             (B.BUDGET_PARAMS, int(rng.integers(0, sizes.sum() + 1))),
+                             (B.BUDGET_COUNT, 1)):
+            ctx.cocodc_select_fragments(torch.from_numpy(scores).to(dev), torch.from_numpy(last).to(dev),
+                                        None if inel is None else torch.from_numpy(inel).to(dev),
+                                        t_now, H, kind, budget, mask, ids, n_sel)
+            assert ctx.cocodc_poll_status() == 0
+            emask, eids, en = orc.select_fragments(scores, last, sizes, t_now, H, kind, budget, inel)
+            assert int(n_sel.item()) == en
+            assert np.array_equal(np_(mask), emask)
+            got = np_(ids)
+            assert np.array_equal(got[:en], eids) and (got[en:] == -1).all()
+
+
+def test_selection_rejects_nan_scores():
+    rng = np.random.default_rng(1)
+    w, ctx, B = selection_problem(6, rng)
+    scores = torch.tensor([1.0, float("nan"), 2.0, 0.0, 0.0, 0.0], device="cuda")
+    last = torch.zeros(6, dtype=torch.int64, device="cuda")
+    mask = torch.ones(6, dtype=torch.uint8, device="cuda")
+    ids = torch.zeros(6, dtype=torch.int32, device="cuda")
+    n_sel = torch.full((1,), 9, dtype=torch.int32, device="cuda")
+    ctx.cocodc_select_fragments(scores, last, None, 5, 100, B.BUDGET_COUNT, 2, mask, ids, n_sel)
+    assert ctx.cocodc_poll_status() == B.ERR_NONFINITE
+    assert int(n_sel.item()) == 0 and int(mask.sum().item()) == 0
+    with pytest.raises(B.CocodcError):
+        ctx.cocodc_select_fragments(scores, last, None, 5, 0, B.BUDGET_COUNT, 2, mask, ids, n_sel)
+    with pytest.raises(B.CocodcError):
+        ctx.cocodc_select_fragments(scores, last, None, 5, 100, 7, 2, mask, ids, n_sel)
+
+
+def test_selection_feeds_the_outer_step_without_a_host_round_trip():
+    """select -> snapshot -> outer_step chained on the stream; the host reads ids only afterwards to check."""
+    w = synth.get_workload("tiny")
+    prob = GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3))
+    from helpers import check_step_against_oracle, orc_hyper
+    # first round: all scores infinite -> fragments 0 and 1 (budget 2), then 2 and 3, ...
+    expected_rounds = [[0, 1], [2, 3], [4, 5], [6, 7]]
+    t = 0
+    for rnd in range(6):
+        t += 12
+        before = prob.host_state()
+        prob.select(t_now=t)
+        prob.outer_step(t_p=t, t_l=t + w.tau)
+        assert prob.poll() == 0
+        n = int(prob.n_ids.item())
+        ids = np_(prob.ids)[:n].tolist()
+        emask, eids, en = orc.select_fragments(before["scores"], before["last_sync"], w.partition.frag_sizes,
+                                               t, w.H, orc.BUDGET_COUNT, w.budget)
+        assert ids == eids.tolist()
+        if rnd < 4:
+            assert ids == expected_rounds[rnd]
+        check_step_against_oracle(prob, before, ids, t, t + w.tau, orc_hyper(w))
+        prob.snapshot()
+        prob.bufs.w_now.add_(torch.randn_like(prob.bufs.w_now) * 1e-3)
+    # after every fragment has a finite score the two largest win, unless one is overdue
+    assert np.isfinite(np_(prob.scores)).all()
+
+
+@pytest.mark.parametrize("frs", [
+    [5000, 1, 4097, 123_457],
+    (300_000, [[(1, 70_001), (200_003, 999)], [(70_002, 129_998)], [(201_002, 98_000)]]),
+])
+def test_standalone_scores(frs):
+    w = synth.small_workload(frs, M=1, seed=3)
+    from paper_2504_17672_b200 import binding as B
+    ptr, off, ln = w.partition.csr()
+    ctx = B.Context(w.N, ptr, off, ln, 1)
+    g = torch.Generator(device="cuda").manual_seed(5)
+    x = torch.randn(w.N, generator=g, device="cuda") * 1e-3
+    K = w.K
+    norms = torch.zeros(K, device="cuda")
+    scores = torch.zeros(K, device="cuda")
+    interval = torch.tensor([0, 3, 100, 7][:K], dtype=torch.int64, device="cuda")
+    for iv in (None, interval):
+        ctx.cocodc_fragment_scores(x, iv, norms, scores)
+        assert ctx.cocodc_poll_status() == 0
+        en, es = orc.fragment_scores(fragments_of(w), np_(x), None if iv is None else np_(iv))
+        assert np.all(np.abs(np_(norms) - en) <= TOL_NORM * en)
+        assert np.all(np.abs(np_(scores) - es) <= TOL_NORM * es)
+    # reproducible to the bit from run to run
+    first = norms.clone()
+    ctx.cocodc_fragment_scores(x, None, norms, scores)
+    assert torch.equal(first, norms)
+    # closed form: a constant vector
+    x.fill_(-0.25)
+    ctx.cocodc_fragment_scores(x, None, norms, scores)
+    exp = 0.25 * np.sqrt(w.partition.frag_sizes.astype(np.float64))
+    assert np.all(np.abs(np_(norms) - exp) <= 1e-6 * exp)
+    x[7] = float("nan")
+    ctx.cocodc_fragment_scores(x, None, norms, scores)
+    assert ctx.cocodc_poll_status() == B.ERR_NONFINITE
