@@ -162,12 +162,18 @@ cocodc_status cocodc_fragment_scores(cocodc_ctx* ctx, const float* delta_g, cons
  *   scores dev fp32[K]; last_sync dev int64[K]; ineligible dev uint8[K] or NULL
  *   mask dev uint8[K] (1 = selected); ids dev int32[K] (first n_sel entries, admission
  *   order; the rest set to -1); n_sel dev int32[1]
+ *   pool_offset dev int64[K] or NULL: if given, the selected fragments are assigned places in a
+ *   packed snapshot pool (the snap_offset argument of the calls below): admission order, back to
+ *   back, each start a multiple of 4 elements; -1 for fragments not selected.  A pool row of
+ *   budget + (largest fragment) elements (PARAMS), or the `budget` largest fragments (COUNT),
+ *   plus 4 per fragment for rounding, always suffices.
  * A NaN score selects nothing and sets COCODC_ERR_NONFINITE.
  */
 cocodc_status cocodc_select_fragments(cocodc_ctx* ctx, const float* scores, const int64_t* last_sync,
                                       const uint8_t* ineligible, int64_t t_now, int64_t H,
                                       int32_t budget_kind, int64_t budget,
-                                      uint8_t* mask, int32_t* ids, int32_t* n_sel, void* stream);
+                                      uint8_t* mask, int32_t* ids, int32_t* n_sel,
+                                      int64_t* pool_offset, void* stream);
 
 /*
  * S1-S6 fused, at completion time t_l, for the fragments listed on the device

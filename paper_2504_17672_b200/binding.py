@@ -79,7 +79,7 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_destroy.argtypes = [vp]
     lib.cocodc_sync_budget.argtypes = [i32, i64, f64, f64, f64, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     lib.cocodc_fragment_scores.argtypes = [vp, vp, vp, vp, vp, vp]
-    lib.cocodc_select_fragments.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp]
+    lib.cocodc_select_fragments.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp]
     lib.cocodc_outer_step.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, vp,
                                       i64, i64, vp, vp, vp, u32, vp]
     lib.cocodc_merge.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp]
@@ -164,10 +164,10 @@ class Context:
                                            _stream(stream)), "cocodc_fragment_scores")
 
     def cocodc_select_fragments(self, scores, last_sync, ineligible, t_now: int, H: int, budget_kind: int,
-                                budget: int, mask, ids, n_sel, stream=None) -> None:
+                                budget: int, mask, ids, n_sel, pool_offset=None, stream=None) -> None:
         _check(_lib.cocodc_select_fragments(self._h, _p(scores), _p(last_sync), _p(ineligible), int(t_now), int(H),
                                             int(budget_kind), int(budget), _p(mask), _p(ids), _p(n_sel),
-                                            _stream(stream)), "cocodc_select_fragments")
+                                            _p(pool_offset), _stream(stream)), "cocodc_select_fragments")
 
     def cocodc_outer_step(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                           theta_g, momentum, delta_g_out, ids, n_ids, t_p: int, t_l: int, last_sync,

@@ -295,7 +295,8 @@ cocodc_status cocodc_fragment_scores(cocodc_ctx* c, const float* delta_g, const 
 cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
                                       const uint8_t* ineligible, int64_t t_now, int64_t H,
                                       int32_t budget_kind, int64_t budget,
-                                      uint8_t* mask, int32_t* ids, int32_t* n_sel, void* stream) {
+                                      uint8_t* mask, int32_t* ids, int32_t* n_sel,
+                                      int64_t* pool_offset, void* stream) {
   if (!c || !scores || !last_sync || !mask || !ids || !n_sel) return COCODC_ERR_INVALID_ARG;
   if (H < 1 || budget < 0) return COCODC_ERR_INVALID_ARG;
   if (budget_kind != COCODC_BUDGET_COUNT && budget_kind != COCODC_BUDGET_PARAMS) return COCODC_ERR_INVALID_ARG;
@@ -303,7 +304,7 @@ cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   k_select<<<1, kSelectThreads, 0, st>>>(c->K, scores, reinterpret_cast<const long long*>(last_sync), ineligible,
                                          c->d_frag_size, t_now, H, budget_kind, budget, mask, ids, n_sel,
-                                         c->d_status, (int)COCODC_ERR_NONFINITE);
+                                         reinterpret_cast<long long*>(pool_offset), c->d_status, (int)COCODC_ERR_NONFINITE);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }

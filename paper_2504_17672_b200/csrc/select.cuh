@@ -17,7 +17,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
          const unsigned char* __restrict__ ineligible, const long long* __restrict__ frag_size,
          long long t_now, long long H, int budget_kind, long long budget,
          unsigned char* __restrict__ mask, int* __restrict__ ids, int* __restrict__ n_sel,
-         int* __restrict__ status, int err_nonfinite) {
+         long long* __restrict__ pool_offset, int* __restrict__ status, int err_nonfinite) {
   __shared__ float s_score[kMaxK];
   __shared__ unsigned char s_class[kMaxK];  // 0 = ineligible, 1 = ordinary, 2 = overdue
   __shared__ int s_order[kMaxK];
@@ -35,6 +35,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     if (r != r) s_nan = 1;
     mask[p] = 0;
     ids[p] = -1;
+    if (pool_offset) pool_offset[p] = -1;
   }
   __syncthreads();
   if (s_nan) {
@@ -63,6 +64,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   __syncthreads();
   if (p != 0) return;
   long long remaining = budget;
+  long long pool_pos = 0;   // next free element of the snapshot pool (kept a multiple of 4)
   int n = 0;
   const int n_elig = s_count;
   for (int j = 0; j < n_elig; ++j) {
@@ -72,6 +74,10 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
       mask[f] = 1;
       ids[n++] = f;
       remaining -= cost;
+      if (pool_offset) {
+        pool_offset[f] = pool_pos;
+        pool_pos = (pool_pos + frag_size[f] + 3) & ~3LL;
+      }
     }
   }
   *n_sel = n;
