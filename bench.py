@@ -1,0 +1,482 @@
+#!/usr/bin/env python
+"""Benchmark of the CoCoDC outer synchronisation step on B200.
+
+One step = one pass of the whole path over the fragments in flight:
+    cocodc_outer_step (S1-S6, fused) on the fragments whose sync completes now,
+    cocodc_select_fragments (S7) for the next set, cocodc_snapshot (S0) of that set.
+The metric is fragment parameters completed per second (whole job), with the achieved HBM rate of
+the fused kernel beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+N > 1 is launched by torch.distributed.run, one rank per GPU; every rank owns an independent
+parameter shard of the same shape (weak scaling, no data-path collective).
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import synth
+
+METRIC = "outer_step_params_per_s"
+UNIT = "params/s"
+DEFAULT_WORKLOAD = "llama_1b"
+
+
+def bytes_per_param(M: int) -> int:
+    """Algorithmic HBM bytes of the fused step per fragment parameter: reads 4M (recorded) + 4M (current)
+    + 4 (global) + 4 (momentum), writes 4M + 4 + 4."""
+    return 12 * M + 16
+
+
+# --------------------------------------------------------------------------------------------
+# helpers
+# --------------------------------------------------------------------------------------------
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples taken while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+        return self
+
+    def __exit__(self, *exc):
+        self.result = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return False
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if sm:
+            self.result = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                           "samples": len(sm)}
+        return False
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def shard_units(n_units: int, world: int, rank: int):
+    """Contiguous block of units owned by `rank` (used when a fixed list of problems is split)."""
+    base, rem = divmod(n_units, world)
+    lo = rank * base + min(rank, rem)
+    return lo, lo + base + (1 if rank < rem else 0)
+
+
+def aggregate(total_units_local: float, seconds_local: float, world: int, backend_ready: bool):
+    """Whole-job figures: units summed over ranks, time = max over ranks."""
+    if world == 1 or not backend_ready:
+        return total_units_local, seconds_local
+    import torch.distributed as dist
+    dev = torch.device("cuda", torch.cuda.current_device()) if dist.get_backend() == "nccl" else torch.device("cpu")
+    u = torch.tensor([total_units_local], dtype=torch.float64, device=dev)
+    t = torch.tensor([seconds_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(u.item()), float(t.item())
+
+
+def pool_capacity(w: synth.Workload) -> int:
+    sizes = np.sort(w.partition.frag_sizes)[::-1]
+    if w.budget_kind == "params":
+        cap = int(w.budget + sizes[0])
+    else:
+        cap = int(sizes[:max(1, w.budget)].sum())
+    return (cap + 4 * w.K + 1023) // 1024 * 1024
+
+
+# --------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------
+
+class DeviceJob:
+    """Workload resident in HBM plus its schedule state, stepped through the C-ABI binding."""
+
+    def __init__(self, w: synth.Workload, device: torch.device):
+        from paper_2504_17672_b200 import binding as B
+        self.B, self.w, self.dev = B, w, device
+        ptr, off, ln = w.partition.csr()
+        self.ctx = B.Context(w.N, ptr, off, ln, w.M, device=device.index or 0)
+        K = w.K
+        self.sizes = w.partition.frag_sizes
+        self.kind = B.BUDGET_PARAMS if w.budget_kind == "params" else B.BUDGET_COUNT
+        # scores of an earlier round: the expected change norm of this seed, s_p * sqrt(n_p)
+        scores0 = (synth.fragment_scales(w) * np.sqrt(self.sizes)).astype(np.float32)
+        self.scores = torch.from_numpy(scores0).to(device)
+        self.norms = torch.zeros(K, dtype=torch.float32, device=device)
+        self.last_sync = torch.zeros(K, dtype=torch.int64, device=device)
+        self.mask = torch.zeros(K, dtype=torch.uint8, device=device)
+        self.ids = torch.full((K,), -1, dtype=torch.int32, device=device)
+        self.n_ids = torch.zeros(1, dtype=torch.int32, device=device)
+        self.pool_off = torch.full((K,), -1, dtype=torch.int64, device=device)
+        self.t = w.tau
+        self.hyper = B.Hyper(M=w.M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam,
+                             alpha=w.alpha)
+        # first selection, then generate the buffers with the selected fragments' snapshots in the pool
+        self.select()
+        torch.cuda.synchronize(device)
+        n = int(self.n_ids.item())
+        ids0 = self.ids[:n].tolist()
+        offs = {p: int(self.pool_off[p].item()) for p in ids0}
+        self.bufs = synth.generate(w, device, snap_layout="pool", pool_ids=ids0, pool_offsets=offs,
+                                   pool_len=pool_capacity(w))
+
+    def select(self):
+        w = self.w
+        self.ctx.cocodc_select_fragments(self.scores, self.last_sync, None, self.t, w.H, self.kind, w.budget,
+                                         self.mask, self.ids, self.n_ids, self.pool_off)
+
+    def outer(self):
+        b, w = self.bufs, self.w
+        self.ctx.cocodc_outer_step(self.hyper, b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off,
+                                   b.theta_g, b.momentum, None, self.ids, self.n_ids, self.t, self.t + w.tau,
+                                   self.last_sync, self.norms, self.scores)
+
+    def snapshot(self):
+        b = self.bufs
+        self.ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off, self.w.M,
+                                 self.ids, self.n_ids)
+
+    def step(self, log_ids=None, log_n=None, ev=None):
+        """Complete the fragments in flight, choose the next set, record their snapshots."""
+        if ev is not None:
+            ev[0].record()
+        self.outer()
+        if ev is not None:
+            ev[1].record()
+        if log_ids is not None:
+            log_ids.copy_(self.ids)
+            log_n.copy_(self.n_ids)
+        self.t += self.w.tau
+        self.select()
+        self.snapshot()
+
+
+def run_ours(args):
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    backend_ready = False
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+        backend_ready = True
+    w = synth.get_workload(args.workload)
+    if world > 1:
+        w = w.with_(seed=w.seed + 1000 * rank)   # every rank owns a different shard of the same shape
+    job = DeviceJob(w, device)
+    K, W = args.steps, args.warmup
+    log_ids = torch.full((K, w.K), -1, dtype=torch.int32, device=device)
+    log_n = torch.zeros((K, 1), dtype=torch.int32, device=device)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    for _ in range(W):
+        job.step()
+    status = job.ctx.cocodc_poll_status()
+    if status != 0:
+        raise RuntimeError(f"device status after warm-up: {job.B.status_string(status)}")
+
+    def barrier():
+        torch.cuda.synchronize(device)
+        if backend_ready:
+            import torch.distributed as dist
+            dist.barrier()
+            torch.cuda.synchronize(device)
+
+    barrier()
+    launches0 = job.ctx.launch_count
+    with ClockSampler(local) as clocks:
+        t_begin.record()
+        for i in range(K):
+            job.step(log_ids[i], log_n[i], evs[i])
+        t_end.record()
+        barrier()
+    launches = job.ctx.launch_count - launches0
+    status = job.ctx.cocodc_poll_status()
+    if status != 0:
+        raise RuntimeError(f"device status after the timed region: {job.B.status_string(status)}")
+    seconds = t_begin.elapsed_time(t_end) / 1e3
+    ids_h, n_h = log_ids.cpu().numpy(), log_n.cpu().numpy().ravel()
+    per_step = [int(job.sizes[ids_h[i, :n_h[i]]].sum()) for i in range(K)]
+    params_local = float(sum(per_step))
+    outer_ms = [a.elapsed_time(b) for a, b in evs]
+    outer_seconds = sum(outer_ms) / 1e3
+    total_params, max_seconds = aggregate(params_local, seconds, world, backend_ready)
+
+    peak, peak_kind = read_peaks()
+    bpp = bytes_per_param(w.M)
+    achieved = params_local * bpp / outer_seconds / 1e9
+    traffic = read_traffic_note(w)
+    out = {
+        "metric": METRIC, "value": total_params / max_seconds, "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": max_seconds / K * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "N": w.N, "K": w.K, "M": w.M, "tau": w.tau, "H": w.H,
+                   "budget": f"{w.budget} {w.budget_kind}", "params_per_step": params_local / K,
+                   "step": "outer_step(S1-S6) + select(S7) + snapshot(S0)", "snapshot_layout": "pool",
+                   "l2": "inputs larger than L2 (every step streams GBs)", "parallelism": f"replicas x{world}"},
+        "gpu_launches": int(launches),
+        "clocks": clocks.result,
+        "roofline": {"bound": "hbm", "kernel": "k_outer (fused S1-S6)", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_of_nominal_8TBs": achieved / 8000.0, "bytes_per_param": bpp,
+                     "ms_per_launch": outer_seconds / K * 1e3, "traffic": traffic},
+        "step_gbs": (params_local * (bpp + 8 * w.M)) / seconds / 1e9,
+    }
+    if rank == 0 and not args.no_e2e:
+        out["e2e"] = run_e2e(job, args)
+    elif rank == 0:
+        out["e2e"] = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(job, per_step[-1] if per_step else 0, args)
+    if rank == 0:
+        print(json.dumps(out))
+    if backend_ready:
+        import torch.distributed as dist
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def read_traffic_note(w):
+    """DRAM bytes per launch from the committed ncu summary, if it covers the current kernel."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return d.get(w.name)
+    except (OSError, ValueError):
+        return None
+
+
+# --------------------------------------------------------------------------------------------
+# end to end: parameters in pinned host memory, through the host-buffer entry points
+# --------------------------------------------------------------------------------------------
+
+def run_e2e(job: DeviceJob, args):
+    """Same step with the trainer's state (w_now, theta_g, momentum, schedule arrays) in pinned host memory.
+
+    Per step: cocodc_outer_step_host streams the completing fragments host->device->host (snapshots were
+    put on the device at initiation); selection runs on the device from the host's schedule arrays;
+    cocodc_snapshot_host copies the next set's parameters into the device pool."""
+    w, dev, B = job.w, job.dev, job.B
+    b = job.bufs
+    torch.cuda.synchronize(dev)
+    try:
+        host = {k: torch.empty(getattr(b, k).shape, dtype=torch.float32, pin_memory=True)
+                for k in ("w_now", "theta_g", "momentum")}
+    except RuntimeError as e:
+        return {"value": None, "unit": UNIT, "error": f"pinned host allocation failed: {e}"}
+    for k, v in host.items():
+        v.copy_(getattr(b, k))
+    scores_h = job.scores.cpu()
+    norms_h = job.norms.cpu()
+    last_h = job.last_sync.cpu()
+    n = int(job.n_ids.item())
+    ids_h = job.ids.cpu()
+    pool_off_h = job.pool_off.cpu()
+    ws = torch.empty(768 * 2 ** 20 // 4, dtype=torch.float32, device=dev)
+    steps = max(1, min(args.e2e_steps, args.steps))
+    t = job.t
+    h2d = d2h = 0
+    params = 0
+    small = w.K * (4 + 8 + 4 + 4 + 8)
+
+    def one(timed):
+        nonlocal t, n, ids_h, pool_off_h, h2d, d2h, params
+        cnt = int(job.sizes[ids_h[:n].numpy()].sum())
+        job.ctx.cocodc_outer_step_host(job.hyper, host["w_now"], b.w_snap, w.N, b.snap_stride, pool_off_h,
+                                       host["theta_g"], host["momentum"], None, ids_h, n, t, t + w.tau,
+                                       last_h, norms_h, scores_h, ws, snap_on_device=True)
+        t += w.tau
+        job.scores.copy_(scores_h, non_blocking=True)
+        job.last_sync.copy_(last_h, non_blocking=True)
+        job.ctx.cocodc_select_fragments(job.scores, job.last_sync, None, t, w.H, job.kind, w.budget, job.mask,
+                                        job.ids, job.n_ids, job.pool_off)
+        ids_h = job.ids.cpu()
+        pool_off_h = job.pool_off.cpu()
+        n2 = int(job.n_ids.item())
+        cnt2 = int(job.sizes[ids_h[:n2].numpy()].sum())
+        job.ctx.cocodc_snapshot_host(host["w_now"], b.w_snap, w.N, b.snap_stride, pool_off_h, w.M, ids_h, n2)
+        torch.cuda.synchronize(dev)
+        if timed:
+            params += cnt
+            h2d += cnt * (4 * w.M + 8) + cnt2 * 4 * w.M + small
+            d2h += cnt * (4 * w.M + 8) + small
+        n = n2
+
+    one(False)                      # warm-up
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one(True)
+    torch.cuda.synchronize(dev)
+    dt = time.perf_counter() - t0
+    status = job.ctx.cocodc_poll_status()
+    res = {"value": params / dt, "unit": UNIT, "h2d_bytes_per_step": h2d // steps,
+           "d2h_bytes_per_step": d2h // steps, "steps": steps, "ms_per_step": dt / steps * 1e3,
+           "api": "cocodc_outer_step_host + cocodc_select_fragments + cocodc_snapshot_host",
+           "host_memory": "pinned", "status": int(status)}
+    del host, ws
+    return res
+
+
+# --------------------------------------------------------------------------------------------
+# CPU baseline: the oracle, as it stands, on the host cores
+# --------------------------------------------------------------------------------------------
+
+def oracle_sample_inputs(w: synth.Workload, n_elems: int, seed: int):
+    """A bounded sample of the workload for the oracle: the head of fragment 0, generated on the CPU."""
+    small = synth.small_workload([n_elems], M=w.M, seed=seed, tau=w.tau, H=w.H, outer_lr=w.outer_lr,
+                                 momentum=w.momentum, lam=w.lam, alpha=w.alpha)
+    bufs = synth.generate(small, "cpu")
+    return small, {k: getattr(bufs, k).numpy() for k in ("w_now", "w_snap", "theta_g", "momentum")}
+
+
+def oracle_runner(w: synth.Workload, n_elems: int, threads: int, seed: int = 0):
+    """Returns a callable that runs the oracle's fused step once on a prepared sample and returns seconds."""
+    from oracle import reference as orc
+    small, x = oracle_sample_inputs(w, n_elems, seed)
+    hp = orc.Hyper(M=w.M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam, alpha=w.alpha)
+
+    def run():
+        t0 = time.perf_counter()
+        orc.outer_step([[(0, n_elems)]], hp, x["w_now"], x["w_snap"], x["theta_g"], x["momentum"], [0],
+                       w.tau, 2 * w.tau, [0], threads=threads)
+        return time.perf_counter() - t0
+    return run
+
+
+def host_cores() -> int:
+    return len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+
+
+def cpu_baseline(job_or_workload, params_per_step, args):
+    w = job_or_workload.w if hasattr(job_or_workload, "w") else job_or_workload
+    cores = host_cores()
+    n = args.cpu_sample
+    run = oracle_runner(w, n, cores)
+    run()                                   # page in the sample and the library
+    total, reps = 0.0, 0
+    while total < args.cpu_seconds and reps < 1000:
+        total += run()
+        reps += 1
+    return {"value": n * reps / total, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"{reps} passes over {n} parameters (one fragment-shaped slice, M={w.M}) of {w.name}, "
+                      f"fused step S1-S6, element range split over {cores} threads; {total:.1f} s",
+            "seconds": total}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, timed on the host cores on a bounded sample per step."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    w = synth.get_workload(args.workload)
+    cores = host_cores()
+    n = args.reference_sample
+    run = oracle_runner(w, n, cores)
+    for _ in range(args.warmup):
+        run()
+    total = 0.0
+    for i in range(args.steps):
+        total += run()
+    value = n * args.steps / total
+    sample = (f"each step = {n} parameters (one fragment-shaped slice, M={w.M}) of {w.name}, fused step S1-S6 "
+              f"by the CPU oracle over {cores} threads")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "N": w.N, "K": w.K, "M": w.M, "tau": w.tau, "H": w.H,
+                   "budget": f"{w.budget} {w.budget_kind}", "sample_params_per_step": n},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", choices=list(synth.WORKLOAD_NAMES), default=DEFAULT_WORKLOAD)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="wall time spent timing the oracle")
+    ap.add_argument("--cpu-sample", type=int, default=16_000_000, help="parameters in the oracle's sample")
+    ap.add_argument("--reference-sample", type=int, default=8_000_000)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -227,6 +227,42 @@ cocodc_status cocodc_snapshot(cocodc_ctx* ctx, const float* w_now, float* w_snap
                               int32_t M, const int32_t* ids, const int32_t* n_ids, void* stream);
 
 /*
+ * S1-S6 as cocodc_outer_step (all stages), for callers whose parameters live in HOST memory.
+ * Every buffer argument here is a host pointer (pinned memory makes the copies asynchronous and
+ * fast; pageable memory works); ids is a host array of n_ids fragment ids; last_sync, norms and
+ * scores are host arrays of K entries, updated for the listed fragments.  The listed fragments
+ * are streamed through the device in chunks: host->device copies, the fused kernel and
+ * device->host copies of consecutive chunks overlap on three streams.  Results are in host
+ * memory when the call returns (it synchronises).  Host pointers need no particular alignment.
+ *   snap_on_device   0: w_snap is a host buffer like the others.  1: w_snap (and only it) is DEVICE
+ *                    memory, e.g. a snapshot pool filled by cocodc_snapshot_host at t_p, read in place
+ *                    (16-byte aligned, stride a multiple of 4); snap_offset stays a host array
+ *   workspace        dev, 16-byte aligned staging memory provided by the caller
+ *   workspace_bytes  at least 3*(2M+3)*4096*4 bytes; a few hundred MB gives full-size chunks
+ *   stream           the stream the kernels run on (two internal streams carry the copies)
+ * Sums of squares are accumulated chunk by chunk in a fixed order.
+ */
+cocodc_status cocodc_outer_step_host(cocodc_ctx* ctx, const cocodc_hyper* hyper,
+                                     float* w_now, const float* w_snap,
+                                     int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                     float* theta_g, float* momentum, float* delta_g_out,
+                                     const int32_t* ids, int32_t n_ids,
+                                     int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                     float* norms, float* scores, int32_t snap_on_device,
+                                     void* workspace, uint64_t workspace_bytes, void* stream);
+
+/*
+ * S0 for parameters that live in host memory: copy the listed fragments of every worker from the
+ * HOST buffer w_now into the DEVICE buffer w_snap (layout rules as for cocodc_snapshot; ids and
+ * snap_offset are host arrays).  Asynchronous on the stream when w_now is pinned.  The snapshot
+ * then waits on the device for the completion tau steps later (cocodc_outer_step_host with
+ * snap_on_device = 1), so it crosses the bus once.
+ */
+cocodc_status cocodc_snapshot_host(cocodc_ctx* ctx, const float* w_now, float* w_snap,
+                                   int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                   int32_t M, const int32_t* ids, int32_t n_ids, void* stream);
+
+/*
  * Waits for the stream, then returns and clears the device status word
  * (COCODC_OK if nothing was recorded since the last poll).
  */

@@ -24,7 +24,7 @@ STAGE_OUTER, STAGE_MERGE, STAGE_SCORE, STAGE_ALL = 1, 2, 4, 7
 
 EXPORTS = (
     "cocodc_create", "cocodc_destroy", "cocodc_sync_budget", "cocodc_fragment_scores",
-    "cocodc_select_fragments", "cocodc_outer_step", "cocodc_merge", "cocodc_snapshot",
+    "cocodc_select_fragments", "cocodc_outer_step", "cocodc_outer_step_host", "cocodc_merge", "cocodc_snapshot", "cocodc_snapshot_host",
     "cocodc_poll_status", "cocodc_launch_count", "cocodc_status_string",
 )
 
@@ -82,6 +82,9 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_select_fragments.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp]
     lib.cocodc_outer_step.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, vp,
                                       i64, i64, vp, vp, vp, u32, vp]
+    lib.cocodc_outer_step_host.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, i32,
+                                           i64, i64, vp, vp, vp, i32, vp, ctypes.c_uint64, vp]
+    lib.cocodc_snapshot_host.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, i32, vp]
     lib.cocodc_merge.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp]
     lib.cocodc_snapshot.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp]
     lib.cocodc_poll_status.argtypes = [vp, vp]
@@ -178,6 +181,20 @@ class Context:
                                       _p(delta_g_out), _p(ids), _p(n_ids), int(t_p), int(t_l), _p(last_sync),
                                       _p(norms), _p(scores), int(stages), _stream(stream)), "cocodc_outer_step")
 
+    def cocodc_outer_step_host(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
+                               theta_g, momentum, delta_g_out, ids, n_ids: int, t_p: int, t_l: int,
+                               last_sync, norms, scores, workspace, snap_on_device: bool = False,
+                               stream=None) -> None:
+        """Host-buffer variant: every tensor is a CPU tensor, except `workspace` (CUDA) and, with
+        snap_on_device, `w_snap` (CUDA)."""
+        h = hyper._c()
+        _check(_lib.cocodc_outer_step_host(self._h, ctypes.byref(h), _p(w_now), _p(w_snap), int(now_stride),
+                                           int(snap_stride), _p(snap_offset), _p(theta_g), _p(momentum),
+                                           _p(delta_g_out), _p(ids), int(n_ids), int(t_p), int(t_l),
+                                           _p(last_sync), _p(norms), _p(scores), 1 if snap_on_device else 0, _p(workspace),
+                                           workspace.numel() * workspace.element_size(), _stream(stream)),
+               "cocodc_outer_step_host")
+
     def cocodc_merge(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                      theta_g_new, ids, n_ids, stream=None) -> None:
         h = hyper._c()
@@ -190,6 +207,13 @@ class Context:
         _check(_lib.cocodc_snapshot(self._h, _p(w_now), _p(w_snap), int(now_stride), int(snap_stride),
                                     _p(snap_offset), int(M), _p(ids), _p(n_ids), _stream(stream)),
                "cocodc_snapshot")
+
+    def cocodc_snapshot_host(self, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset, M: int,
+                             ids, n_ids: int, stream=None) -> None:
+        """S0 from a host w_now into a device w_snap; ids and snap_offset are CPU tensors."""
+        _check(_lib.cocodc_snapshot_host(self._h, _p(w_now), _p(w_snap), int(now_stride), int(snap_stride),
+                                         _p(snap_offset), int(M), _p(ids), int(n_ids), _stream(stream)),
+               "cocodc_snapshot_host")
 
     def cocodc_poll_status(self, stream=None) -> int:
         """Waits for the stream; returns and clears the device status word."""

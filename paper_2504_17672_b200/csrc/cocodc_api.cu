@@ -39,6 +39,18 @@ struct cocodc_ctx {
   int* d_status = nullptr;
   long long launches = 0;
   std::vector<std::pair<const void*, int>> occupancy;  // kernel -> resident CTAs per SM
+  // host copy of the fragment table (host-buffer entry point walks it on the host)
+  std::vector<int> h_frag_seg_ptr;
+  std::vector<long long> h_seg_off, h_seg_len;
+  // host-buffer entry point: copy streams, pipeline events, K-sized device staging
+  static constexpr int kSlots = 3;
+  cudaStream_t s_h2d = nullptr, s_d2h = nullptr;
+  cudaEvent_t ev_h2d[kSlots] = {}, ev_comp[kSlots] = {}, ev_d2h[kSlots] = {};
+  double* d_frag_sumsq = nullptr;   // [K]
+  int* d_k_ids = nullptr;           // [K]
+  long long* d_k_last = nullptr;    // [K]
+  float* d_k_norms = nullptr;       // [K]
+  float* d_k_scores = nullptr;      // [K]
 };
 
 namespace {
@@ -85,31 +97,44 @@ cocodc_status launch_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_id
 template <int M> struct Unroll { static constexpr int U = (M >= 8) ? 1 : 2; };
 template <> struct Unroll<0> { static constexpr int U = 2; };
 
+struct Variant {
+  void (*kernel)(const OuterArgs);
+  int U;  // lanes per thread; a tile is kThreads*U lanes
+};
+
 template <int M, int MODE, bool SAME>
-cocodc_status launch_outer_variant(cocodc_ctx* c, const OuterArgs& A, const int32_t* ids, const int32_t* n_ids,
-                                   const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
-  constexpr int U = Unroll<M>::U;
-  auto kernel = k_outer<M, U, MODE, SAME>;
-  const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads * U, st);
+Variant make_variant() { return Variant{k_outer<M, Unroll<M>::U, MODE, SAME>, Unroll<M>::U}; }
+
+// Instantiated worker counts run fully in registers; any other M takes the generic element loop.
+template <int MODE, bool SAME>
+Variant pick_variant(int M) {
+  switch (M) {
+    case 1: return make_variant<1, MODE, SAME>();
+    case 2: return make_variant<2, MODE, SAME>();
+    case 3: return make_variant<3, MODE, SAME>();
+    case 4: return make_variant<4, MODE, SAME>();
+    case 8: return make_variant<8, MODE, SAME>();
+    default: return make_variant<0, MODE, SAME>();
+  }
+}
+
+Variant pick_variant(int M, int mode, bool same) {
+  if (mode == MODE_OUTER_ONLY) return pick_variant<MODE_OUTER_ONLY, false>(M);
+  if (mode == MODE_MERGE_ONLY) return same ? pick_variant<MODE_MERGE_ONLY, true>(M) : pick_variant<MODE_MERGE_ONLY, false>(M);
+  return same ? pick_variant<MODE_FUSED, true>(M) : pick_variant<MODE_FUSED, false>(M);
+}
+
+// plan + streaming kernel for a device-resident id list
+cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool same, const int32_t* ids,
+                           const int32_t* n_ids, const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
+  const Variant v = pick_variant(A.M, mode, same);
+  const int grid = grid_for(c, reinterpret_cast<const void*>(v.kernel));
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads * v.U, st);
   if (s != COCODC_OK) return s;
-  kernel<<<grid, kThreads, 0, st>>>(A);
+  v.kernel<<<grid, kThreads, 0, st>>>(A);
   c->launches++;
   *grid_out = grid;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
-}
-
-template <int MODE, bool SAME>
-cocodc_status launch_outer_m(cocodc_ctx* c, const OuterArgs& A, const int32_t* ids, const int32_t* n_ids,
-                             const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
-  switch (A.M) {
-    case 1: return launch_outer_variant<1, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
-    case 2: return launch_outer_variant<2, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
-    case 3: return launch_outer_variant<3, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
-    case 4: return launch_outer_variant<4, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
-    case 8: return launch_outer_variant<8, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
-    default: return launch_outer_variant<0, MODE, SAME>(c, A, ids, n_ids, snap_offset, st, grid_out);
-  }
 }
 
 // Shared checks of the three entry points that stream worker buffers.
@@ -231,7 +256,23 @@ cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, 
   ok = ok && cudaMalloc(&c->d_hdr, sizeof(PlanHeader)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_partial, sizeof(double) * partial_elems) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_frag_sumsq, sizeof(double) * K) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_k_ids, sizeof(int) * K) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_k_last, sizeof(long long) * K) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_k_norms, sizeof(float) * K) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_k_scores, sizeof(float) * K) == cudaSuccess;
   if (!ok) { cudaGetLastError(); cocodc_destroy(c); return COCODC_ERR_NOMEM; }
+  ok = ok && cudaStreamCreateWithFlags(&c->s_h2d, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&c->s_d2h, cudaStreamNonBlocking) == cudaSuccess;
+  for (int i = 0; i < cocodc_ctx::kSlots && ok; ++i) {
+    ok = ok && cudaEventCreateWithFlags(&c->ev_h2d[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_comp[i], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_d2h[i], cudaEventDisableTiming) == cudaSuccess;
+  }
+  if (!ok) { cudaGetLastError(); cocodc_destroy(c); return COCODC_ERR_CUDA; }
+  c->h_frag_seg_ptr.assign(part->frag_seg_ptr, part->frag_seg_ptr + K + 1);
+  c->h_seg_off = off;
+  c->h_seg_len = len;
   ok = ok && cudaMemcpy(c->d_frag_seg_ptr, part->frag_seg_ptr, sizeof(int) * (K + 1), cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->d_seg_off, off.data(), sizeof(long long) * S, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->d_seg_len, len.data(), sizeof(long long) * S, cudaMemcpyHostToDevice) == cudaSuccess;
@@ -254,6 +295,18 @@ cocodc_status cocodc_destroy(cocodc_ctx* c) {
   cudaFree(c->d_hdr);
   cudaFree(c->d_partial);
   cudaFree(c->d_status);
+  cudaFree(c->d_frag_sumsq);
+  cudaFree(c->d_k_ids);
+  cudaFree(c->d_k_last);
+  cudaFree(c->d_k_norms);
+  cudaFree(c->d_k_scores);
+  for (int i = 0; i < cocodc_ctx::kSlots; ++i) {
+    if (c->ev_h2d[i]) cudaEventDestroy(c->ev_h2d[i]);
+    if (c->ev_comp[i]) cudaEventDestroy(c->ev_comp[i]);
+    if (c->ev_d2h[i]) cudaEventDestroy(c->ev_d2h[i]);
+  }
+  if (c->s_h2d) cudaStreamDestroy(c->s_h2d);
+  if (c->s_d2h) cudaStreamDestroy(c->s_d2h);
   delete c;
   return COCODC_OK;
 }
@@ -363,9 +416,7 @@ cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
   A.partial = do_score ? c->d_partial : nullptr;
   fold_coefficients(h, same, &A);
   int grid = 0;
-  if (!do_merge) s = launch_outer_m<MODE_OUTER_ONLY, false>(c, A, ids, n_ids, snap_offset, st, &grid);
-  else if (same) s = launch_outer_m<MODE_FUSED, true>(c, A, ids, n_ids, snap_offset, st, &grid);
-  else s = launch_outer_m<MODE_FUSED, false>(c, A, ids, n_ids, snap_offset, st, &grid);
+  s = launch_outer(c, A, do_merge ? MODE_FUSED : MODE_OUTER_ONLY, same, ids, n_ids, snap_offset, st, &grid);
   if (s != COCODC_OK) return s;
   if (do_score) {
     k_finalize_scores<<<c->K, kFinalizeThreads, 0, st>>>(
@@ -409,8 +460,7 @@ cocodc_status cocodc_merge(cocodc_ctx* c, const cocodc_hyper* h,
   A.hdr = c->d_hdr;
   fold_coefficients(h, same, &A);
   int grid = 0;
-  if (same) return launch_outer_m<MODE_MERGE_ONLY, true>(c, A, ids, n_ids, snap_offset, st, &grid);
-  return launch_outer_m<MODE_MERGE_ONLY, false>(c, A, ids, n_ids, snap_offset, st, &grid);
+  return launch_outer(c, A, MODE_MERGE_ONLY, same, ids, n_ids, snap_offset, st, &grid);
 }
 
 cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
@@ -434,6 +484,176 @@ cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
   kernel<<<grid, kThreads, 0, st>>>(w_now, w_snap, now_stride, snap_stride, M, c->d_plan, c->d_hdr);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
+                                     float* w_now, const float* w_snap,
+                                     int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                     float* theta_g, float* momentum, float* delta_g_out,
+                                     const int32_t* ids, int32_t n_ids,
+                                     int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                     float* norms, float* scores, int32_t snap_on_device,
+                                     void* workspace, uint64_t workspace_bytes, void* stream) {
+  cocodc_status s = check_hyper(c, h);
+  if (s != COCODC_OK) return s;
+  if (!w_now || !w_snap || !theta_g || !momentum || !ids || !last_sync || !norms || !scores || !workspace)
+    return COCODC_ERR_INVALID_ARG;
+  if (n_ids < 0 || n_ids > c->K || t_l < t_p) return COCODC_ERR_INVALID_ARG;
+  const long long N = c->N;
+  const int M = h->M, K = c->K;
+  if (now_stride < N || snap_stride < (snap_offset ? 1 : N)) return COCODC_ERR_INVALID_ARG;
+  const bool same = !snap_on_device && (w_snap == w_now) && (snap_stride == now_stride) && (snap_offset == nullptr);
+  if (h->tau == 0 && h->comp_mode == COCODC_COMP_TAYLOR && !same) return COCODC_ERR_INVALID_ARG;
+  if (!aligned16(workspace)) return COCODC_ERR_ALIGNMENT;
+  if (snap_on_device && (!aligned16(w_snap) || (snap_stride & 3))) return COCODC_ERR_ALIGNMENT;
+  {
+    std::vector<char> seen(K, 0);
+    for (int j = 0; j < n_ids; ++j) {
+      const int p = ids[j];
+      if (p < 0 || p >= K || seen[p]) return COCODC_ERR_INVALID_ARG;
+      if (snap_offset && snap_offset[p] < 0) return COCODC_ERR_INVALID_ARG;
+      seen[p] = 1;
+    }
+    std::vector<Range> r;
+    r.push_back(range_of(theta_g, N));
+    r.push_back(range_of(momentum, N));
+    if (delta_g_out) r.push_back(range_of(delta_g_out, N));
+    r.push_back(range_of(w_now, (long long)(M - 1) * now_stride + N));
+    for (size_t i = 0; i < r.size(); ++i)
+      for (size_t j = i + 1; j < r.size(); ++j)
+        if (overlap(r[i], r[j])) return COCODC_ERR_ALIAS;
+    if (!same && !snap_on_device) {
+      const Range rs = range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N));
+      for (const Range& x : r) if (overlap(rs, x)) return COCODC_ERR_ALIAS;
+    }
+  }
+  // staging slots: [snap M][now M][theta_g][momentum][delta] chunks of C elements each
+  const long long per_elem = 2LL * M + 3;
+  long long C = (long long)(workspace_bytes / sizeof(float)) / (cocodc_ctx::kSlots * per_elem);
+  C &= ~1023LL;
+  if (C < 4096) return COCODC_ERR_INVALID_ARG;
+  if (C > (1LL << 28)) C = 1LL << 28;
+
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Variant v = pick_variant(M, MODE_FUSED, same);
+  const int grid = grid_for(c, reinterpret_cast<const void*>(v.kernel));
+  const int entries = grid * (kThreads / 32);
+  bool ok = true;
+  auto CK = [&](cudaError_t e) { ok = ok && (e == cudaSuccess); };
+  CK(cudaMemsetAsync(c->d_frag_sumsq, 0, sizeof(double) * K, st));
+  CK(cudaMemcpyAsync(c->d_k_ids, ids, sizeof(int) * n_ids, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(c->d_k_last, last_sync, sizeof(long long) * K, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(c->d_k_norms, norms, sizeof(float) * K, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(c->d_k_scores, scores, sizeof(float) * K, cudaMemcpyHostToDevice, st));
+
+  OuterArgs A{};
+  A.now_stride = C;
+  A.snap_stride = C;
+  A.plan = c->d_plan;
+  A.hdr = c->d_hdr;
+  A.partial = c->d_partial;
+  fold_coefficients(h, same, &A);
+  const size_t B4 = sizeof(float);
+  long long chunk = 0;
+  for (int j = 0; j < n_ids && ok; ++j) {
+    const int p = ids[j];
+    long long pos = 0;
+    for (int sgi = c->h_frag_seg_ptr[p]; sgi < c->h_frag_seg_ptr[p + 1] && ok; ++sgi) {
+      const long long off = c->h_seg_off[sgi], len = c->h_seg_len[sgi];
+      const long long sbase = snap_offset ? snap_offset[p] + pos : off;
+      for (long long lo = 0; lo < len && ok; lo += C, ++chunk) {
+        const long long cnt = std::min(C, len - lo);
+        const int slot = (int)(chunk % cocodc_ctx::kSlots);
+        float* base = static_cast<float*>(workspace) + (size_t)slot * per_elem * C;
+        float* d_snap = base;
+        float* d_now = base + (size_t)M * C;
+        float* d_thg = base + (size_t)2 * M * C;
+        float* d_u = d_thg + C;
+        float* d_delta = d_u + C;
+        // host -> device, once the slot's previous results have left it
+        if (chunk >= cocodc_ctx::kSlots) CK(cudaStreamWaitEvent(c->s_h2d, c->ev_d2h[slot], 0));
+        for (int m = 0; m < M; ++m) {
+          if (!same && !snap_on_device)
+            CK(cudaMemcpyAsync(d_snap + (size_t)m * C, w_snap + (size_t)m * snap_stride + sbase + lo, cnt * B4,
+                               cudaMemcpyHostToDevice, c->s_h2d));
+          CK(cudaMemcpyAsync(d_now + (size_t)m * C, w_now + (size_t)m * now_stride + off + lo, cnt * B4,
+                             cudaMemcpyHostToDevice, c->s_h2d));
+        }
+        CK(cudaMemcpyAsync(d_thg, theta_g + off + lo, cnt * B4, cudaMemcpyHostToDevice, c->s_h2d));
+        CK(cudaMemcpyAsync(d_u, momentum + off + lo, cnt * B4, cudaMemcpyHostToDevice, c->s_h2d));
+        CK(cudaEventRecord(c->ev_h2d[slot], c->s_h2d));
+        // compute on the caller's stream
+        CK(cudaStreamWaitEvent(st, c->ev_h2d[slot], 0));
+        A.w_now = d_now;
+        A.w_snap = same ? d_now : (snap_on_device ? w_snap : d_snap);
+        A.snap_stride = snap_on_device ? snap_stride : C;
+        A.theta_g = d_thg;
+        A.momentum = d_u;
+        A.delta_out = delta_g_out ? d_delta : nullptr;
+        k_plan_chunk<<<1, 1, 0, st>>>(cnt, snap_on_device ? sbase + lo : 0, kThreads * v.U, c->d_plan, c->d_hdr);
+        v.kernel<<<grid, kThreads, 0, st>>>(A);
+        k_accumulate_chunk<<<1, kFinalizeThreads, 0, st>>>(c->d_partial, entries, c->d_frag_sumsq + j);
+        c->launches += 3;
+        CK(cudaEventRecord(c->ev_comp[slot], st));
+        // device -> host
+        CK(cudaStreamWaitEvent(c->s_d2h, c->ev_comp[slot], 0));
+        for (int m = 0; m < M; ++m)
+          CK(cudaMemcpyAsync(w_now + (size_t)m * now_stride + off + lo, d_now + (size_t)m * C, cnt * B4,
+                             cudaMemcpyDeviceToHost, c->s_d2h));
+        CK(cudaMemcpyAsync(theta_g + off + lo, d_thg, cnt * B4, cudaMemcpyDeviceToHost, c->s_d2h));
+        CK(cudaMemcpyAsync(momentum + off + lo, d_u, cnt * B4, cudaMemcpyDeviceToHost, c->s_d2h));
+        if (delta_g_out)
+          CK(cudaMemcpyAsync(delta_g_out + off + lo, d_delta, cnt * B4, cudaMemcpyDeviceToHost, c->s_d2h));
+        CK(cudaEventRecord(c->ev_d2h[slot], c->s_d2h));
+      }
+      pos += len;
+    }
+  }
+  if (ok && n_ids > 0) {
+    k_finalize_from_sums<<<1, kFinalizeThreads, 0, st>>>(c->d_frag_sumsq, c->d_k_ids, n_ids, t_p, t_l, c->d_k_last,
+                                                         c->d_k_norms, c->d_k_scores, c->d_status,
+                                                         (int)COCODC_ERR_NONFINITE);
+    c->launches++;
+  }
+  CK(cudaMemcpyAsync(last_sync, c->d_k_last, sizeof(long long) * K, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(norms, c->d_k_norms, sizeof(float) * K, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(scores, c->d_k_scores, sizeof(float) * K, cudaMemcpyDeviceToHost, st));
+  // the call is synchronous: results are in host memory when it returns
+  cudaError_t e1 = cudaStreamSynchronize(c->s_h2d);
+  cudaError_t e2 = cudaStreamSynchronize(st);
+  cudaError_t e3 = cudaStreamSynchronize(c->s_d2h);
+  if (!ok || e1 != cudaSuccess || e2 != cudaSuccess || e3 != cudaSuccess || cudaGetLastError() != cudaSuccess)
+    return COCODC_ERR_CUDA;
+  return COCODC_OK;
+}
+
+cocodc_status cocodc_snapshot_host(cocodc_ctx* c, const float* w_now, float* w_snap,
+                                   int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                   int32_t M, const int32_t* ids, int32_t n_ids, void* stream) {
+  if (!c || !w_now || !w_snap || !ids) return COCODC_ERR_INVALID_ARG;
+  if (M < 1 || M > c->max_M || n_ids < 0 || n_ids > c->K) return COCODC_ERR_INVALID_ARG;
+  if (now_stride < c->N || snap_stride < (snap_offset ? 1 : c->N)) return COCODC_ERR_INVALID_ARG;
+  for (int j = 0; j < n_ids; ++j) {
+    if (ids[j] < 0 || ids[j] >= c->K) return COCODC_ERR_INVALID_ARG;
+    if (snap_offset && snap_offset[ids[j]] < 0) return COCODC_ERR_INVALID_ARG;
+  }
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bool ok = true;
+  for (int j = 0; j < n_ids; ++j) {
+    const int p = ids[j];
+    long long pos = 0;
+    for (int sgi = c->h_frag_seg_ptr[p]; sgi < c->h_frag_seg_ptr[p + 1]; ++sgi) {
+      const long long off = c->h_seg_off[sgi], len = c->h_seg_len[sgi];
+      const long long sbase = snap_offset ? snap_offset[p] + pos : off;
+      for (int m = 0; m < M; ++m)
+        ok = ok && cudaMemcpyAsync(w_snap + (size_t)m * snap_stride + sbase, w_now + (size_t)m * now_stride + off,
+                                   (size_t)len * sizeof(float), cudaMemcpyHostToDevice, st) == cudaSuccess;
+      pos += len;
+    }
+  }
+  return ok ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
 }  // extern "C"

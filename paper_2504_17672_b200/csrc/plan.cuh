@@ -195,4 +195,51 @@ k_finalize_scores(const PlanHeader* __restrict__ hdr, const int* __restrict__ id
   if (!isfinite(norm)) record_status(status, err_nonfinite);
 }
 
+// ---------------------------------------------------------------------------
+// Helpers of the host-buffer entry point, which streams a fragment through
+// device staging in chunks: each chunk is a one-segment plan, and the chunk's
+// sum of squares is added to its fragment's running total in chunk order.
+// ---------------------------------------------------------------------------
+__global__ void k_plan_chunk(long long len, long long snap_off, int lanes_per_tile,
+                             SegPlan* __restrict__ plan, PlanHeader* __restrict__ hdr) {
+  SegPlan sp;
+  sp.off = 0; sp.len = len; sp.snap_off = snap_off; sp.abase = 0;
+  sp.first_tile = 0; sp.slot = 0; sp.frag = 0; sp.vec_ok = ((snap_off & 3LL) == 0) ? 1 : 0;
+  plan[0] = sp;
+  const long long lanes = (len + 3) >> 2;
+  hdr->total_tiles = (int)((lanes + lanes_per_tile - 1) / lanes_per_tile);
+  hdr->n_seg = 1; hdr->n_ids = 1; hdr->pad = 0;
+}
+
+__global__ void __launch_bounds__(kFinalizeThreads)
+k_accumulate_chunk(const double* __restrict__ partial, int entries, double* __restrict__ total) {
+  __shared__ double red[kFinalizeThreads];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < entries; i += kFinalizeThreads) s += partial[i];
+  red[threadIdx.x] = s;
+  __syncthreads();
+#pragma unroll
+  for (int w = kFinalizeThreads / 2; w > 0; w >>= 1) {
+    if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *total += red[0];
+}
+
+__global__ void k_finalize_from_sums(const double* __restrict__ sums, const int* __restrict__ ids, int n,
+                                     long long t_p, long long t_l, long long* __restrict__ last_sync,
+                                     float* __restrict__ norms, float* __restrict__ scores,
+                                     int* __restrict__ status, int err_nonfinite) {
+  for (int j = threadIdx.x; j < n; j += blockDim.x) {
+    const int p = ids[j];
+    const double norm = sqrt(sums[j]);
+    long long I = t_p - last_sync[p];
+    if (I < 1) I = 1;
+    last_sync[p] = t_l;
+    norms[p] = (float)norm;
+    scores[p] = (float)(norm / (double)I);
+    if (!isfinite(norm)) record_status(status, err_nonfinite);
+  }
+}
+
 }  // namespace cocodc

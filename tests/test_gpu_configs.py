@@ -18,6 +18,9 @@ pytestmark = pytest.mark.gpu
 
 
 def free_gb():
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     return free / 2 ** 30
 

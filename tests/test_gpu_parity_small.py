@@ -225,3 +225,59 @@ def test_nonfinite_norm_is_reported():
     prob.outer_step(1, 2)
     assert prob.poll() == prob.B.ERR_NONFINITE
     assert prob.poll() == 0
+
+
+@pytest.mark.parametrize("same", [False, True])
+def test_host_buffer_entry_point_matches_device_path_and_oracle(same):
+    """Parameters in host memory, streamed through a small workspace (several chunks per fragment)."""
+    frs = (300_000, [[(3, 90_001), (200_010, 40_097)], [(90_004, 100_000)], [(250_000, 50_000)]])
+    w = synth.small_workload(frs, M=4, seed=130, scale_kind="loguniform")
+    bufs = synth.generate(w, "cuda", momentum_sigma=1e-3)
+    prob = GpuProblem(w, bufs)
+    ids = [2, 0]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    host = {k: torch.from_numpy(before[k].copy()).pin_memory() for k in ("w_now", "w_snap", "theta_g", "momentum")}
+    delta_h = torch.zeros(w.N).pin_memory()
+    last_h = torch.from_numpy(before["last_sync"].copy())
+    norms_h = torch.zeros(w.K)
+    scores_h = torch.full((w.K,), float("inf"))
+    ids_h = torch.tensor(ids, dtype=torch.int32)
+    ws = torch.empty(3 * 11 * 8192, dtype=torch.float32, device="cuda")       # 8192-element chunks
+    snap_h = host["w_now"] if same else host["w_snap"]
+    hp = prob.hyper(tau=0) if same else prob.hyper()
+    prob.ctx.cocodc_outer_step_host(hp, host["w_now"], snap_h, w.N, w.N, None, host["theta_g"], host["momentum"],
+                                    delta_h, ids_h, len(ids), 8, 8 if same else 10, last_h, norms_h, scores_h, ws)
+    assert prob.poll() == 0
+    # device path on the same inputs
+    delta_d = torch.zeros(w.N, device="cuda")
+    prob.outer_step(8, 8 if same else 10, hyper=hp, delta_out=delta_d, w_snap=prob.bufs.w_now if same else None)
+    assert prob.poll() == 0
+    for k in ("w_now", "theta_g", "momentum"):
+        assert torch.equal(host[k], getattr(prob.bufs, k).cpu()), k
+    assert torch.equal(delta_h, delta_d.cpu())
+    assert torch.equal(last_h, prob.last_sync.cpu())
+    assert np.allclose(norms_h.numpy(), np_(prob.norms), rtol=1e-6)
+    ohp = orc_hyper(w, tau=0) if same else orc_hyper(w)
+    check_step_against_oracle(prob, before, ids, 8, 8 if same else 10, ohp, delta_out=delta_d, same=same)
+    if not same:
+        # snapshots kept on the device: S0 from the host buffer into a device pool, then the completion
+        host2 = {k: torch.from_numpy(before[k].copy()).pin_memory() for k in ("w_now", "theta_g", "momentum")}
+        snap_src = torch.from_numpy(before["w_snap"].copy()).pin_memory()      # parameters as they were at t_p
+        pool = torch.zeros((w.M, 190_104), device="cuda")
+        pool_off = torch.tensor([50_001, -1, 0], dtype=torch.int64)             # fragment 0 lands on an odd offset
+        prob.ctx.cocodc_snapshot_host(snap_src, pool, w.N, pool.stride(0), pool_off, w.M, ids_h, len(ids))
+        last2 = torch.from_numpy(before["last_sync"].copy())
+        n2, s2 = torch.zeros(w.K), torch.full((w.K,), float("inf"))
+        prob.ctx.cocodc_outer_step_host(hp, host2["w_now"], pool, w.N, pool.stride(0), pool_off, host2["theta_g"],
+                                        host2["momentum"], None, ids_h, len(ids), 8, 10, last2, n2, s2, ws,
+                                        snap_on_device=True)
+        assert prob.poll() == 0
+        for k in ("w_now", "theta_g", "momentum"):
+            assert torch.equal(host2[k], host[k]), k
+        assert torch.equal(n2, norms_h) and torch.equal(s2, scores_h)
+    # too small a workspace is refused
+    with pytest.raises(prob.B.CocodcError):
+        prob.ctx.cocodc_outer_step_host(hp, host["w_now"], snap_h, w.N, w.N, None, host["theta_g"],
+                                        host["momentum"], None, ids_h, len(ids), 8, 10, last_h, norms_h,
+                                        scores_h, ws[:1000])
