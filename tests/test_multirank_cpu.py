@@ -1,0 +1,87 @@
+"""The N > 1 host logic of the benchmark on CPU: two gloo ranks, no GPU.
+
+Ranks own independent shards (weak scaling, no data-path collective); what crosses ranks is only the
+timing reduction: units are summed, time is the maximum."""
+
+import os
+import socket
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK=str(rank))
+    import bench
+    import synth
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        assert bench.dist_env() == (rank, world, rank)
+        # each rank reports different local figures; the job figure is (sum of units, max of seconds)
+        units, seconds = bench.aggregate(100.0 * (rank + 1), 2.0 + rank, world, True)
+        assert units == 300.0 and seconds == 3.0
+        # a fixed list of problems splits into disjoint contiguous blocks that cover it
+        lo, hi = bench.shard_units(13, world, rank)
+        spans = [None] * world
+        dist.all_gather_object(spans, (lo, hi))
+        assert spans[0][0] == 0 and spans[-1][1] == 13 and all(spans[i][1] == spans[i + 1][0] for i in range(world - 1))
+        # ranks own different shards of the same shape: same fragment table, different seeded values
+        w = synth.small_workload([1000, 2000], M=2, seed=7)
+        mine = synth.generate(w.with_(seed=w.seed + 1000 * rank), "cpu")
+        sums = [None] * world
+        dist.all_gather_object(sums, float(mine.theta_g.double().sum()))
+        assert sums[0] != sums[1]
+        # the selection decision is deterministic on every rank given the same history (Section 3.2)
+        from oracle import reference as orc
+        sel = orc.select_fragments([1.0, 2.0], [0, 0], [1000, 2000], 5, 100, 0, 1)[1].tolist()
+        allsel = [None] * world
+        dist.all_gather_object(allsel, sel)
+        assert allsel[0] == allsel[1] == [1]
+        out.put((rank, "ok"))
+    except Exception as e:  # pragma: no cover
+        out.put((rank, repr(e)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_gloo_ranks_aggregate_like_the_benchmark():
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    for p in procs:
+        p.join(timeout=120)
+    results = sorted(out.get(timeout=5) for _ in range(2))
+    assert results == [(0, "ok"), (1, "ok")], results
+
+
+def test_reference_arm_runs_only_on_rank_zero(monkeypatch, capsys):
+    import bench
+
+    class A:
+        workload = "tiny"; steps = 1; warmup = 0; reference_sample = 20_000
+
+    monkeypatch.setenv("RANK", "1")
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    bench.run_reference(A)
+    assert capsys.readouterr().out == ""
+    monkeypatch.setenv("RANK", "0")
+    bench.run_reference(A)
+    import json
+    line = json.loads(capsys.readouterr().out)
+    assert line["impl"] == "reference" and line["value"] > 0 and line["e2e"]["h2d_bytes_per_step"] == 0
