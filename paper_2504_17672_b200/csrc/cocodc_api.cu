@@ -14,6 +14,7 @@
 #include <vector>
 
 #include "outer.cuh"
+#include "outer_tma.cuh"
 #include "plan.cuh"
 #include "select.cuh"
 
@@ -93,28 +94,39 @@ cocodc_status launch_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_id
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
-// Lanes per thread and tile for each instantiated worker count.
-template <int M> struct Unroll { static constexpr int U = (M >= 8) ? 1 : 2; };
-template <> struct Unroll<0> { static constexpr int U = 2; };
-
+// One way to run the streaming step: which kernel, with how many threads and how much dynamic
+// shared memory, on how many CTAs.  Every variant uses tiles of kTileElems elements and eight
+// accumulating warps, so the plan and the finalize kernel do not depend on the choice.
 struct Variant {
   void (*kernel)(const OuterArgs);
-  int U;  // lanes per thread; a tile is kThreads*U lanes
+  int threads;
+  unsigned smem;
+  bool one_cta_per_sm;   // staged kernel: persistent, one CTA per SM; otherwise sized by occupancy
 };
 
 template <int M, int MODE, bool SAME>
-Variant make_variant() { return Variant{k_outer<M, Unroll<M>::U, MODE, SAME>, Unroll<M>::U}; }
+Variant staged_variant() {
+  using L = StageLayout<M, MODE, SAME>;
+  auto kernel = k_outer_tma<M, MODE, SAME>;
+  static bool configured = false;   // one-time opt-in to more than 48 KB of dynamic shared memory
+  if (!configured) {
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kSmemBytes);
+    configured = true;
+  }
+  return Variant{kernel, kTmaThreads, L::kSmemBytes, true};
+}
 
-// Instantiated worker counts run fully in registers; any other M takes the generic element loop.
+// Instantiated worker counts are staged through shared memory by TMA; any other M takes the
+// generic element loop.
 template <int MODE, bool SAME>
 Variant pick_variant(int M) {
   switch (M) {
-    case 1: return make_variant<1, MODE, SAME>();
-    case 2: return make_variant<2, MODE, SAME>();
-    case 3: return make_variant<3, MODE, SAME>();
-    case 4: return make_variant<4, MODE, SAME>();
-    case 8: return make_variant<8, MODE, SAME>();
-    default: return make_variant<0, MODE, SAME>();
+    case 1: return staged_variant<1, MODE, SAME>();
+    case 2: return staged_variant<2, MODE, SAME>();
+    case 3: return staged_variant<3, MODE, SAME>();
+    case 4: return staged_variant<4, MODE, SAME>();
+    case 8: return staged_variant<8, MODE, SAME>();
+    default: return Variant{k_outer_generic<MODE, SAME>, kThreads, 0u, false};
   }
 }
 
@@ -124,14 +136,18 @@ Variant pick_variant(int M, int mode, bool same) {
   return same ? pick_variant<MODE_FUSED, true>(M) : pick_variant<MODE_FUSED, false>(M);
 }
 
+int variant_grid(cocodc_ctx* c, const Variant& v) {
+  return v.one_cta_per_sm ? c->sm_count : grid_for(c, reinterpret_cast<const void*>(v.kernel));
+}
+
 // plan + streaming kernel for a device-resident id list
 cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool same, const int32_t* ids,
                            const int32_t* n_ids, const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
   const Variant v = pick_variant(A.M, mode, same);
-  const int grid = grid_for(c, reinterpret_cast<const void*>(v.kernel));
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads * v.U, st);
+  const int grid = variant_grid(c, v);
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads, st);
   if (s != COCODC_OK) return s;
-  v.kernel<<<grid, kThreads, 0, st>>>(A);
+  v.kernel<<<grid, v.threads, v.smem, st>>>(A);
   c->launches++;
   *grid_out = grid;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
@@ -169,6 +185,11 @@ void fold_coefficients(const cocodc_hyper* h, bool zero_delay, OuterArgs* A) {
   A->mu = h->momentum;
   A->M = h->M;
   A->Mf = (float)h->M;
+}
+
+void set_status_sink(const cocodc_ctx* c, OuterArgs* A) {
+  A->status = c->d_status;
+  A->err_timeout = (int)COCODC_ERR_TIMEOUT;
 }
 
 }  // namespace
@@ -415,6 +436,7 @@ cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
   A.hdr = c->d_hdr;
   A.partial = do_score ? c->d_partial : nullptr;
   fold_coefficients(h, same, &A);
+  set_status_sink(c, &A);
   int grid = 0;
   s = launch_outer(c, A, do_merge ? MODE_FUSED : MODE_OUTER_ONLY, same, ids, n_ids, snap_offset, st, &grid);
   if (s != COCODC_OK) return s;
@@ -459,6 +481,7 @@ cocodc_status cocodc_merge(cocodc_ctx* c, const cocodc_hyper* h,
   A.plan = c->d_plan;
   A.hdr = c->d_hdr;
   fold_coefficients(h, same, &A);
+  set_status_sink(c, &A);
   int grid = 0;
   return launch_outer(c, A, MODE_MERGE_ONLY, same, ids, n_ids, snap_offset, st, &grid);
 }
@@ -537,7 +560,7 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Variant v = pick_variant(M, MODE_FUSED, same);
-  const int grid = grid_for(c, reinterpret_cast<const void*>(v.kernel));
+  const int grid = variant_grid(c, v);
   const int entries = grid * (kThreads / 32);
   bool ok = true;
   auto CK = [&](cudaError_t e) { ok = ok && (e == cudaSuccess); };
@@ -554,6 +577,7 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
   A.hdr = c->d_hdr;
   A.partial = c->d_partial;
   fold_coefficients(h, same, &A);
+  set_status_sink(c, &A);
   const size_t B4 = sizeof(float);
   long long chunk = 0;
   for (int j = 0; j < n_ids && ok; ++j) {
@@ -591,8 +615,8 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
         A.theta_g = d_thg;
         A.momentum = d_u;
         A.delta_out = delta_g_out ? d_delta : nullptr;
-        k_plan_chunk<<<1, 1, 0, st>>>(cnt, snap_on_device ? sbase + lo : 0, kThreads * v.U, c->d_plan, c->d_hdr);
-        v.kernel<<<grid, kThreads, 0, st>>>(A);
+        k_plan_chunk<<<1, 1, 0, st>>>(cnt, snap_on_device ? sbase + lo : 0, kThreads, c->d_plan, c->d_hdr);
+        v.kernel<<<grid, v.threads, v.smem, st>>>(A);
         k_accumulate_chunk<<<1, kFinalizeThreads, 0, st>>>(c->d_partial, entries, c->d_frag_sumsq + j);
         c->launches += 3;
         CK(cudaEventRecord(c->ev_comp[slot], st));

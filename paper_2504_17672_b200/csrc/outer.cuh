@@ -1,24 +1,22 @@
-// The streaming kernels of the outer synchronisation step.
+// Arithmetic of the outer synchronisation step and the kernels that do not stage through
+// shared memory: the generic-M fallback, the stand-alone sum of squares and the snapshot copy.
 //
-// k_outer<M, U, MODE, SAME> makes one pass over the listed fragments.  Per
-// element it reads every worker's recorded and current value, the global state
-// and the momentum once, keeps pseudo-gradient, mean, Nesterov update, delay
-// compensation and merge in registers, and writes each output once (Eq. 1-7,
-// Eq. 3).  The sum of squares of the mean pseudo-gradient (Eq. 10) is collected
-// on the way.  Nothing here is a contraction: the kernel is bound by HBM
-// bandwidth, so the design is about keeping enough 16-byte loads in flight per
-// SM and touching every byte once.
+// Per element the step reads every worker's recorded and current value, the global state and the
+// momentum once, keeps pseudo-gradient, mean, Nesterov update, delay compensation and merge in
+// registers, and writes each output once (Eq. 1-7, Eq. 3).  The sum of squares of the mean
+// pseudo-gradient (Eq. 10) is collected on the way.  Nothing here is a contraction: every kernel
+// is bound by HBM bandwidth.
 //
-// Work decomposition: a persistent grid; CTA c handles tiles c, c+grid, ...  A
-// tile is THREADS*U lanes of four elements of one segment; a thread issues all
-// of its U lanes' loads (U * (2M+2) 16-byte loads) before the first use.
+// The main kernel for the instantiated worker counts lives in outer_tma.cuh and uses the
+// per-lane code (struct Lane, ragged_lane) defined here.
 #pragma once
 
 #include "plan.cuh"
 
 namespace cocodc {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;        // consumer threads per CTA; a tile is kThreads lanes of 16 bytes
+constexpr int kTileElems = 4 * kThreads;
 
 enum : int { MODE_FUSED = 0, MODE_OUTER_ONLY = 1, MODE_MERGE_ONLY = 2 };
 
@@ -33,7 +31,9 @@ struct OuterArgs {
   const SegPlan* plan;
   const PlanHeader* hdr;
   double* partial;          // nullptr: no score accumulation
-  int M;                    // runtime worker count (used by the generic M = 0 instantiation)
+  int* status;              // device status word
+  int err_timeout;          // code recorded when a bounded wait runs out
+  int M;                    // runtime worker count (used by the generic kernel and scalar paths)
   float eta, mu;            // outer learning rate, Nesterov momentum
   float c1, c2;             // target = G + c1*d + c2*d*d*D
   float alpha, one_minus_alpha;
@@ -41,8 +41,8 @@ struct OuterArgs {
 };
 
 // ---- memory access helpers -------------------------------------------------
-// Every byte is used exactly once per launch, so loads and stores are marked
-// streaming (evict-first) to keep them from displacing each other in L2.
+// Every byte is used exactly once per launch, so direct loads and stores are marked streaming
+// (evict-first) to keep them from displacing each other in L2.
 __device__ __forceinline__ float4 ld4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
 __device__ __forceinline__ void st4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
 __device__ __forceinline__ float ld1(const float* p) { return __ldcs(p); }
@@ -59,9 +59,9 @@ __device__ __forceinline__ void outer_update(float sum, float thg, float u, cons
   G = __fmaf_rn(A.eta, t, thg);
 }
 
-// S4-S5.  d = a - b is the local change over the overlap (tau times Eq. 4's
-// rate), D = G - b the divergence of Eq. 5; Eq. 6-7 collapse to
-// target = G + c1*d + c2*d*d*D with c2 = +-lambda/(tau*H); then Eq. 3's blend.
+// S4-S5.  d = a - b is the local change over the overlap (tau times Eq. 4's rate), D = G - b the
+// divergence of Eq. 5; Eq. 6-7 collapse to target = G + c1*d + c2*d*d*D with c2 = +-lambda/(tau*H);
+// then Eq. 3's blend.
 __device__ __forceinline__ float merged(float a, float b, float G, const OuterArgs& A) {
   const float d = __fsub_rn(a, b);
   const float D = __fsub_rn(G, b);
@@ -73,7 +73,7 @@ __device__ __forceinline__ float merged(float a, float b, float G, const OuterAr
 __device__ __forceinline__ float& comp(float4& v, int k) { return reinterpret_cast<float*>(&v)[k]; }
 __device__ __forceinline__ float comp(const float4& v, int k) { return reinterpret_cast<const float*>(&v)[k]; }
 
-// One scalar element, any M (used on ragged edges, unaligned snapshot layouts and M not instantiated).
+// One scalar element, any M (ragged edges, unaligned snapshot layouts, worker counts not instantiated).
 template <int MODE, bool SAME>
 __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, long long snap_e, double& acc) {
   const int M = A.M;
@@ -100,31 +100,36 @@ __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, 
   }
 }
 
-// Registers of one 16-byte lane.
+// Registers of one 16-byte lane (four consecutive elements) of every stream.
+// compute() works in place: afterwards thg holds G, u holds u', delta holds Delta and the merged
+// local parameters sit in out(m) (= a[m], or b[m] when the snapshot is the current state).
 template <int M, int MODE, bool SAME>
 struct Lane {
+  static constexpr bool kHasNow = (MODE != MODE_OUTER_ONLY) && !SAME;
   float4 b[M];
-  float4 a[(MODE != MODE_OUTER_ONLY && !SAME) ? M : 1];
+  float4 a[kHasNow ? M : 1];
   float4 thg;
   float4 u;
+  float4 delta;
+
+  __device__ __forceinline__ float4& out(int m) {
+    if constexpr (kHasNow) return a[m];
+    else return b[m];
+  }
 
   __device__ __forceinline__ void load(const OuterArgs& A, long long e, long long snap_e) {
     thg = ld4(A.theta_g + e);
     if (MODE != MODE_MERGE_ONLY) u = ld4(A.momentum + e);
 #pragma unroll
     for (int m = 0; m < M; ++m) b[m] = ld4(A.w_snap + m * A.snap_stride + snap_e);
-    if (MODE != MODE_OUTER_ONLY && !SAME) {
+    if (kHasNow) {
 #pragma unroll
       for (int m = 0; m < M; ++m) a[m] = ld4(A.w_now + m * A.now_stride + e);
     }
   }
 
-  __device__ __forceinline__ void compute_store(const OuterArgs& A, long long e, double& acc) {
-    float4 G4;
-    if (MODE == MODE_MERGE_ONLY) {
-      G4 = thg;
-    } else {
-      float4 D4, U4;
+  __device__ __forceinline__ void compute(const OuterArgs& A, double& acc) {
+    if (MODE != MODE_MERGE_ONLY) {
       float sq = 0.f;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -134,87 +139,96 @@ struct Lane {
         for (int m = 1; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(comp(b[m], k), t));
         float Delta, u_new, G;
         outer_update(sum, t, comp(u, k), A, Delta, u_new, G);
-        comp(D4, k) = Delta; comp(U4, k) = u_new; comp(G4, k) = G;
+        comp(delta, k) = Delta; comp(u, k) = u_new; comp(thg, k) = G;
         sq = __fmaf_rn(Delta, Delta, sq);
       }
       acc += (double)sq;
-      st4(A.theta_g + e, G4);
-      st4(A.momentum + e, U4);
-      if (A.delta_out) st4(A.delta_out + e, D4);
     }
     if (MODE != MODE_OUTER_ONLY) {
 #pragma unroll
       for (int m = 0; m < M; ++m) {
-        float4 o;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const float bb = comp(b[m], k);
-          const float aa = SAME ? bb : comp(a[m], k);
-          comp(o, k) = merged(aa, bb, comp(G4, k), A);
+          const float aa = kHasNow ? comp(a[m], k) : bb;
+          comp(out(m), k) = merged(aa, bb, comp(thg, k), A);
         }
-        st4(A.w_now + m * A.now_stride + e, o);
       }
+    }
+  }
+
+  __device__ __forceinline__ void store(const OuterArgs& A, long long e) {
+    if (MODE != MODE_MERGE_ONLY) {
+      st4(A.theta_g + e, thg);
+      st4(A.momentum + e, u);
+      if (A.delta_out) st4(A.delta_out + e, delta);
+    }
+    if (MODE != MODE_OUTER_ONLY) {
+#pragma unroll
+      for (int m = 0; m < M; ++m) st4(A.w_now + m * A.now_stride + e, out(m));
     }
   }
 };
 
-// M = 0 instantiates the generic path: every lane goes element by element with the runtime M.
-template <int M, int U, int MODE, bool SAME>
-__global__ void __launch_bounds__(kThreads)
-k_outer(const OuterArgs A) {
-  const PlanHeader h = *A.hdr;
-  constexpr int LPT = kThreads * U;  // lanes per tile
-  SlotAccumulator sa;
+// One lane at element e of a segment, straight from global memory: a full, 16-byte-compatible lane
+// goes through registers as a vector, anything else element by element.  M = 0: always by element.
+template <int M, int MODE, bool SAME>
+__device__ __forceinline__ void ragged_lane(const OuterArgs& A, const SegPlan& sp, long long e, double& acc) {
+  const long long seg_end = sp.off + sp.len;
+  const long long snap_shift = sp.snap_off - sp.off;   // snapshot index = native index + shift
+  if (e >= seg_end) return;
+  if constexpr (M > 0) {
+    if (sp.vec_ok && e >= sp.off && e + 4 <= seg_end) {
+      Lane<M, MODE, SAME> L;
+      L.load(A, e, e + snap_shift);
+      L.compute(A, acc);
+      L.store(A, e);
+      return;
+    }
+  }
+  for (int k = 0; k < 4; ++k) {
+    const long long ee = e + k;
+    if (ee >= sp.off && ee < seg_end) scalar_element<MODE, SAME>(A, ee, ee + snap_shift, acc);
+  }
+}
+
+// Walks the tiles of one CTA (tile = blockIdx.x + i*gridDim.x) and keeps the segment they fall in.
+struct TileWalker {
+  const SegPlan* plan;
+  int n_seg;
   int seg = 0;
-  int seg_loaded = -1;
+  int loaded = -1;
   SegPlan sp;
+
+  __device__ __forceinline__ TileWalker(const SegPlan* p, int n) : plan(p), n_seg(n) {}
+  // returns true if the segment changed
+  __device__ __forceinline__ bool seek(int tile) {
+    while (seg + 1 < n_seg && tile >= plan[seg + 1].first_tile) ++seg;
+    if (seg == loaded) return false;
+    sp = plan[seg];
+    loaded = seg;
+    return true;
+  }
+  __device__ __forceinline__ long long tile_start(int tile) const {   // first element (16-byte aligned)
+    return sp.abase + (long long)(tile - sp.first_tile) * kTileElems;
+  }
+  // the whole tile lies inside the segment and every stream is 16-byte aligned there
+  __device__ __forceinline__ bool interior(long long e_tile) const {
+    return sp.vec_ok && e_tile >= sp.off && e_tile + kTileElems <= sp.off + sp.len;
+  }
+};
+
+// Generic kernel: any worker count, every lane through ragged_lane<0> (element loop with runtime M;
+// the second pass over the recorded values hits in cache).
+template <int MODE, bool SAME>
+__global__ void __launch_bounds__(kThreads)
+k_outer_generic(const OuterArgs A) {
+  const PlanHeader h = *A.hdr;
+  SlotAccumulator sa(kThreads / 32);
+  TileWalker tw(A.plan, h.n_seg);
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
-    while (seg + 1 < h.n_seg && tile >= A.plan[seg + 1].first_tile) ++seg;
-    if (seg != seg_loaded) {
-      sp = A.plan[seg];
-      seg_loaded = seg;
-      if (A.partial) sa.advance(sp.slot, A.partial);
-    }
-    const long long lane0 = (long long)(tile - sp.first_tile) * LPT;
-    const long long e_tile = sp.abase + 4 * lane0;          // first element of the tile (aligned)
-    const long long seg_end = sp.off + sp.len;
-    const long long snap_shift = sp.snap_off - sp.off;       // snap index = native index + shift
-    const bool interior = (M > 0) && sp.vec_ok && e_tile >= sp.off && e_tile + 4LL * LPT <= seg_end;
-    if (interior) {
-      if constexpr (M > 0) {
-        Lane<M, MODE, SAME> L[U];
-#pragma unroll
-        for (int j = 0; j < U; ++j) {
-          const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
-          L[j].load(A, e, e + snap_shift);
-        }
-#pragma unroll
-        for (int j = 0; j < U; ++j) {
-          const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
-          L[j].compute_store(A, e, sa.acc);
-        }
-      }
-    } else {
-      for (int j = 0; j < U; ++j) {
-        const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
-        if (e >= seg_end) break;
-        bool done = false;
-        if constexpr (M > 0) {
-          if (sp.vec_ok && e >= sp.off && e + 4 <= seg_end) {
-            Lane<M, MODE, SAME> L1;
-            L1.load(A, e, e + snap_shift);
-            L1.compute_store(A, e, sa.acc);
-            done = true;
-          }
-        }
-        if (!done) {
-          for (int k = 0; k < 4; ++k) {
-            const long long ee = e + k;
-            if (ee >= sp.off && ee < seg_end) scalar_element<MODE, SAME>(A, ee, ee + snap_shift, sa.acc);
-          }
-        }
-      }
-    }
+    if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
+    ragged_lane<0, MODE, SAME>(A, tw.sp, tw.tile_start(tile) + 4LL * threadIdx.x, sa.acc);
   }
   if (A.partial) sa.finish(h.n_ids, A.partial);
 }
@@ -228,7 +242,7 @@ k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ plan,
         const PlanHeader* __restrict__ hdr, double* __restrict__ partial) {
   const PlanHeader h = *hdr;
   constexpr int LPT = kThreads * U;
-  SlotAccumulator sa;
+  SlotAccumulator sa(kThreads / 32);
   int seg = 0, seg_loaded = -1;
   SegPlan sp;
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {

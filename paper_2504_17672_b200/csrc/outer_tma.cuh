@@ -1,0 +1,232 @@
+// The fused outer-step kernel for the instantiated worker counts: worker tiles are staged through
+// shared memory by the TMA unit (1-D bulk asynchronous copies), in both directions.
+//
+// One CTA per SM: warps 0-7 compute, warp 8 holds the producer thread.  A stage is one tile
+// (1024 elements = 4 KB) of every stream the mode reads; S stages keep about 160 KB of loads in
+// flight per SM, which plain register loads cannot hold.  Per tile:
+//   producer : waits until the stage is free, arms the stage's "full" barrier with the byte count,
+//              issues one bulk copy global->shared per stream;
+//   consumers: wait on "full", read their 16-byte lane of every stream from shared memory, do the
+//              arithmetic of outer.cuh in registers, write the outputs IN PLACE in the stage,
+//              fence towards the async proxy, barrier;
+//   thread 0 : issues one bulk copy shared->global per output stream, commits them as a group,
+//              waits until the PREVIOUS tile's group has finished reading its stage and hands that
+//              stage back to the producer ("empty" barrier).
+// Tiles that are ragged or whose snapshot placement is not 16-byte compatible never enter the
+// pipeline: the consumers process them straight from global memory (ragged_lane); producer and
+// consumers agree on which tiles those are from the plan alone.
+//
+// Every wait is bounded.  When one runs out the kernel records COCODC_ERR_TIMEOUT, all consumers
+// leave the loop in the same iteration, thread 0 drains its own stores, and the CTA returns.
+// Only this GPU's memory is read; no cluster multicast is used.
+#pragma once
+
+#include "outer.cuh"
+
+namespace cocodc {
+
+constexpr int kProducerThreads = 32;
+constexpr int kTmaThreads = kThreads + kProducerThreads;
+constexpr unsigned kTileBytes = kTileElems * sizeof(float);   // one stream's share of a stage
+constexpr int kWaitLimit = 1 << 22;                           // polls of a barrier before giving up
+constexpr int kMaxStages = 10;
+
+// ---- PTX wrappers ------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// false if the phase did not complete within the poll limit
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity) {
+  for (int i = 0; i < kWaitLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ void bulk_load(unsigned dst_smem, const void* src, unsigned bytes, unsigned bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, unsigned src_smem, unsigned bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+
+// ---- stage layout ----------------------------------------------------------------------------
+// Slots of kTileElems floats each: [recorded x nS][current x nN][global][momentum x nU][delta x nX].
+// Outputs overwrite inputs in place; the mean pseudo-gradient, when asked for, goes to the first
+// recorded slot (its content is in registers by then), or to the extra slot when there is none.
+template <int M, int MODE, bool SAME>
+struct StageLayout {
+  static constexpr int nS = SAME ? 0 : M;
+  static constexpr int nN = (MODE == MODE_OUTER_ONLY) ? 0 : M;
+  static constexpr int nU = (MODE == MODE_MERGE_ONLY) ? 0 : 1;
+  static constexpr int nX = (SAME && MODE == MODE_FUSED) ? 1 : 0;
+  static constexpr int kSnap = 0;
+  static constexpr int kNow = nS;
+  static constexpr int kGlobal = nS + nN;
+  static constexpr int kMomentum = kGlobal + 1;
+  static constexpr int kDelta = (nX == 1) ? (kMomentum + nU) : kSnap;
+  static constexpr int kLoaded = nS + nN + 1 + nU;       // streams brought in by the producer
+  static constexpr int kSlots = kLoaded + nX;
+  static constexpr unsigned kStageBytes = kSlots * kTileBytes;
+  static constexpr int kStagesRaw = (160 * 1024) / kStageBytes;
+  static constexpr int kStages = kStagesRaw < 3 ? 3 : (kStagesRaw > kMaxStages ? kMaxStages : kStagesRaw);
+  static constexpr unsigned kSmemBytes = kStages * kStageBytes;
+  static_assert(kSmemBytes <= 227 * 1024, "stages do not fit in shared memory");
+  static_assert(SAME ? (MODE != MODE_OUTER_ONLY) : true, "zero-delay mode needs the merge");
+};
+
+template <int M, int MODE, bool SAME>
+__global__ void __launch_bounds__(kTmaThreads, 1)
+k_outer_tma(const OuterArgs A) {
+  using L = StageLayout<M, MODE, SAME>;
+  constexpr int S = L::kStages;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  float* const stages = reinterpret_cast<float*>(smem_raw);
+  __shared__ __align__(8) unsigned long long full_bar[S];
+  __shared__ __align__(8) unsigned long long empty_bar[S];
+  __shared__ volatile int s_fail;
+
+  const int tid = threadIdx.x;
+  const PlanHeader h = *A.hdr;
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // ------------------------------------------------------------------ producer
+  if (tid >= kThreads) {
+    if (tid != kThreads) return;
+    TileWalker tw(A.plan, h.n_seg);
+    int k = 0;   // staged tiles issued so far
+    for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+      tw.seek(tile);
+      const long long e0 = tw.tile_start(tile);
+      if (!tw.interior(e0)) continue;
+      const int s = k % S;
+      if (k >= S && !mbar_wait_bounded(smem_u32(&empty_bar[s]), ((k / S) - 1) & 1)) {
+        record_status(A.status, A.err_timeout);
+        s_fail = 1;
+        return;
+      }
+      if (s_fail) return;
+      const unsigned bar = smem_u32(&full_bar[s]);
+      float* st = stages + (size_t)s * L::kSlots * kTileElems;
+      const long long snap_e0 = e0 + (tw.sp.snap_off - tw.sp.off);
+      mbar_expect_tx(bar, L::kLoaded * kTileBytes);
+#pragma unroll
+      for (int m = 0; m < L::nS; ++m)
+        bulk_load(smem_u32(st + (L::kSnap + m) * kTileElems), A.w_snap + m * A.snap_stride + snap_e0, kTileBytes, bar);
+#pragma unroll
+      for (int m = 0; m < L::nN; ++m)
+        bulk_load(smem_u32(st + (L::kNow + m) * kTileElems), A.w_now + m * A.now_stride + e0, kTileBytes, bar);
+      bulk_load(smem_u32(st + L::kGlobal * kTileElems), A.theta_g + e0, kTileBytes, bar);
+      if (L::nU) bulk_load(smem_u32(st + L::kMomentum * kTileElems), A.momentum + e0, kTileBytes, bar);
+      ++k;
+    }
+    return;
+  }
+
+  // ------------------------------------------------------------------ consumers
+  SlotAccumulator sa(kThreads / 32);
+  TileWalker tw(A.plan, h.n_seg);
+  int k = 0;           // staged tiles consumed so far
+  bool failed = false;
+  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+    if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
+    const long long e0 = tw.tile_start(tile);
+    if (!tw.interior(e0)) {
+      ragged_lane<M, MODE, SAME>(A, tw.sp, e0 + 4LL * tid, sa.acc);
+      continue;
+    }
+    const int s = k % S;
+    if (!mbar_wait_bounded(smem_u32(&full_bar[s]), (k / S) & 1)) {
+      record_status(A.status, A.err_timeout);
+      s_fail = 1;
+    }
+    consumer_barrier();
+    if (s_fail) {                             // uniform: every consumer sees the flag after the barrier
+      // give the loads that were issued for this stage one more bounded chance to land before the
+      // CTA gives its shared memory back
+      if (tid == 0) mbar_wait_bounded(smem_u32(&full_bar[s]), (k / S) & 1);
+      failed = true;
+      break;
+    }
+    float* st = stages + (size_t)s * L::kSlots * kTileElems;
+    {
+      Lane<M, MODE, SAME> ln;
+      auto slot = [&](int idx) -> float4& { return reinterpret_cast<float4*>(st + idx * kTileElems)[tid]; };
+      ln.thg = slot(L::kGlobal);
+      if (L::nU) ln.u = slot(L::kMomentum);
+      if (SAME) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kNow + m);
+      } else {
+#pragma unroll
+        for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kSnap + m);
+        if (L::nN) {
+#pragma unroll
+          for (int m = 0; m < M; ++m) ln.a[m] = slot(L::kNow + m);
+        }
+      }
+      ln.compute(A, sa.acc);
+      if (MODE != MODE_MERGE_ONLY) {
+        slot(L::kGlobal) = ln.thg;
+        slot(L::kMomentum) = ln.u;
+        if (A.delta_out) slot(L::kDelta) = ln.delta;
+      }
+      if (MODE != MODE_OUTER_ONLY) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) slot(L::kNow + m) = ln.out(m);
+      }
+    }
+    fence_async_shared();     // make the generic-proxy writes visible to the bulk stores
+    consumer_barrier();
+    if (tid == 0) {
+      if (MODE != MODE_OUTER_ONLY) {
+#pragma unroll
+        for (int m = 0; m < M; ++m)
+          bulk_store(A.w_now + m * A.now_stride + e0, smem_u32(st + (L::kNow + m) * kTileElems), kTileBytes);
+      }
+      if (MODE != MODE_MERGE_ONLY) {
+        bulk_store(A.theta_g + e0, smem_u32(st + L::kGlobal * kTileElems), kTileBytes);
+        bulk_store(A.momentum + e0, smem_u32(st + L::kMomentum * kTileElems), kTileBytes);
+        if (A.delta_out) bulk_store(A.delta_out + e0, smem_u32(st + L::kDelta * kTileElems), kTileBytes);
+      }
+      bulk_commit();
+      if (k >= 1) {   // the previous staged tile's stores have read their stage: release it
+        bulk_wait_read_all_but_one();
+        mbar_arrive(smem_u32(&empty_bar[(k - 1) % S]));
+      }
+    }
+    ++k;
+  }
+  if (tid == 0) bulk_wait_all();     // this thread's stores are complete before the CTA exits
+  if (failed) return;
+  if (A.partial) sa.finish(h.n_ids, A.partial);
+}
+
+}  // namespace cocodc

@@ -98,7 +98,7 @@ k_plan(const int* __restrict__ ids, const int* __restrict__ n_ids_p, int K,
       const long long lanes = (sp.off - sp.abase + sp.len + 3) >> 2;
       tiles += (lanes + lanes_per_tile - 1) / lanes_per_tile;
       pos += sp.len;
-      if (tiles > 0x7fffffffLL) { overflow = true; break; }
+      if (tiles > 0x3fffffffLL) { overflow = true; break; }  // tile + gridDim.x must not wrap
     }
   }
   if (overflow) {
@@ -118,7 +118,7 @@ k_plan(const int* __restrict__ ids, const int* __restrict__ n_ids_p, int K,
 // A persistent CTA walks its tiles in increasing order, so the fragment slot it
 // works on never decreases.  Every thread keeps a double accumulator for the
 // current slot; when the slot changes the warp reduces it and lane 0 writes
-// partial[(slot*gridDim.x + blockIdx.x)*warps + warp].  Slots a CTA never
+// partial[(slot*gridDim.x + blockIdx.x)*warps + warp] (warps = accumulating warps per CTA).  Slots a CTA never
 // touched get an explicit zero, so the finalize kernel can sum every entry
 // without the buffer being cleared first.  The tile-to-CTA map is static,
 // hence the summation order - and the rounded result - is the same every run.
@@ -132,9 +132,11 @@ __device__ __forceinline__ double warp_sum(double v) {
 struct SlotAccumulator {
   double acc = 0.0;
   int slot = 0;
+  int warps;   // accumulating warps per CTA (warps 0 .. warps-1 must all call the methods below)
+
+  __device__ __forceinline__ explicit SlotAccumulator(int accumulating_warps) : warps(accumulating_warps) {}
 
   __device__ __forceinline__ void flush_to(int new_slot, double* __restrict__ partial) {
-    const int warps = blockDim.x >> 5;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     double v = warp_sum(acc);
     if (lane == 0) {
