@@ -185,6 +185,8 @@ void fold_coefficients(const cocodc_hyper* h, bool zero_delay, OuterArgs* A) {
   A->mu = h->momentum;
   A->M = h->M;
   A->Mf = (float)h->M;
+  A->inv_M = 1.0f / (float)h->M;
+  A->M_pow2 = ((h->M & (h->M - 1)) == 0) ? 1 : 0;
 }
 
 void set_status_sink(const cocodc_ctx* c, OuterArgs* A) {

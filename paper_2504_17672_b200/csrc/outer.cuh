@@ -38,6 +38,8 @@ struct OuterArgs {
   float c1, c2;             // target = G + c1*d + c2*d*d*D
   float alpha, one_minus_alpha;
   float Mf;                 // (float)M
+  float inv_M;              // 1/M, exact when M is a power of two
+  int M_pow2;               // 1 if M is a power of two
 };
 
 // ---- memory access helpers -------------------------------------------------
@@ -49,11 +51,20 @@ __device__ __forceinline__ float ld1(const float* p) { return __ldcs(p); }
 __device__ __forceinline__ void st1(float* p, float v) { __stcs(p, v); }
 
 // ---- the arithmetic of one element -----------------------------------------
-// S1-S3.  Differences first, summed in worker order, then divided by M (Eq. 1);
-// u' = mu*u + Delta, G = thg + eta*(Delta + mu*u') (Eq. 2, Nesterov).
-__device__ __forceinline__ void outer_update(float sum, float thg, float u, const OuterArgs& A,
-                                             float& Delta, float& u_new, float& G) {
-  Delta = __fdiv_rn(sum, A.Mf);
+// S2.  The sum of the workers' pseudo-gradients divided by M (Eq. 1).  For a power of two the
+// product with 1/M is the correctly rounded quotient, bit for bit, and it has no data-dependent
+// slow path (the IEEE division routine branches on zero or tiny numerators, which costs bandwidth
+// once many elements have converged).  Other M use the IEEE division.
+template <int M>
+__device__ __forceinline__ float mean_of_sum(float sum, const OuterArgs& A) {
+  if constexpr (M > 0 && (M & (M - 1)) == 0) return __fmul_rn(sum, 1.0f / (float)M);
+  else if constexpr (M > 0) return __fdiv_rn(sum, (float)M);
+  else return A.M_pow2 ? __fmul_rn(sum, A.inv_M) : __fdiv_rn(sum, A.Mf);
+}
+
+// S3.  u' = mu*u + Delta, G = thg + eta*(Delta + mu*u') (Eq. 2, Nesterov).
+__device__ __forceinline__ void outer_update(float Delta, float thg, float u, const OuterArgs& A,
+                                             float& u_new, float& G) {
   u_new = __fmaf_rn(A.mu, u, Delta);
   const float t = __fmaf_rn(A.mu, u_new, Delta);
   G = __fmaf_rn(A.eta, t, thg);
@@ -84,8 +95,9 @@ __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, 
   } else {
     float sum = 0.f;
     for (int m = 0; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(ld1(A.w_snap + m * A.snap_stride + snap_e), thg));
-    float Delta, u_new;
-    outer_update(sum, thg, ld1(A.momentum + e), A, Delta, u_new, G);
+    const float Delta = mean_of_sum<0>(sum, A);
+    float u_new;
+    outer_update(Delta, thg, ld1(A.momentum + e), A, u_new, G);
     acc += (double)__fmul_rn(Delta, Delta);
     st1(A.theta_g + e, G);
     st1(A.momentum + e, u_new);
@@ -137,8 +149,9 @@ struct Lane {
         float sum = __fsub_rn(comp(b[0], k), t);
 #pragma unroll
         for (int m = 1; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(comp(b[m], k), t));
-        float Delta, u_new, G;
-        outer_update(sum, t, comp(u, k), A, Delta, u_new, G);
+        const float Delta = mean_of_sum<M>(sum, A);
+        float u_new, G;
+        outer_update(Delta, t, comp(u, k), A, u_new, G);
         comp(delta, k) = Delta; comp(u, k) = u_new; comp(thg, k) = G;
         sq = __fmaf_rn(Delta, Delta, sq);
       }
