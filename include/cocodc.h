@@ -263,6 +263,38 @@ cocodc_status cocodc_snapshot_host(cocodc_ctx* ctx, const float* w_now, float* w
                                    int32_t M, const int32_t* ids, int32_t n_ids, void* stream);
 
 /*
+ * (No counterpart in the paper: this is an interface variant, not a step of the method.)
+ * cocodc_fragment_scores for callers that cannot allocate device memory - code running inside an
+ * allocator hook or a memory-pool callback, processes whose device memory is handed out up front
+ * and whose runtime heap is closed, latency-critical paths that must not hit an allocation's
+ * implicit synchronisation.  Such callers cannot use cocodc_create either, so the fragment table
+ * is passed directly (host arrays, validated on every call) and no context is involved.
+ *
+ * Same result as cocodc_fragment_scores: norms[p] = ||delta_g restricted to fragment p||_2,
+ * scores[p] = norms[p] / max(1, interval[p]) (interval NULL means 1).  A non-finite norm is
+ * written as it is; there is no status word.
+ *
+ * The scratch (per-CTA partial sums, about 1.2 MB) is a fixed __device__ array inside the library
+ * image: every GPU that loads the library holds it until the process exits.  Its size bounds the
+ * problem: K <= COCODC_NOALLOC_MAX_K fragments and n_segments <= COCODC_NOALLOC_MAX_SEGMENTS;
+ * anything larger returns COCODC_ERR_INVALID_ARG.  The call itself makes no cudaMalloc/cudaFree
+ * and calls no allocating library routine; it launches two kernels on `stream`.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current) and caches it; make that first call outside any stream capture.
+ * All calls on a device share the one array: each call rewrites every entry it later reads, so the
+ * previous call's contents never matter, but two calls that overlap on the GPU (different streams,
+ * different threads) race on it - serialise them.
+ *   partition  host; delta_g dev fp32[N], 16-byte aligned; interval dev int64[K] or NULL;
+ *   norms, scores dev fp32[K]; device = the CUDA device the pointers belong to
+ */
+#define COCODC_NOALLOC_MAX_K 64
+#define COCODC_NOALLOC_MAX_SEGMENTS 64
+cocodc_status cocodc_fragment_scores_noalloc(const cocodc_partition* partition, const float* delta_g,
+                                             const int64_t* interval, float* norms, float* scores,
+                                             int32_t device, void* stream);
+
+/*
  * Waits for the stream, then returns and clears the device status word
  * (COCODC_OK if nothing was recorded since the last poll).
  */

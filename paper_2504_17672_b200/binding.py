@@ -26,7 +26,9 @@ EXPORTS = (
     "cocodc_create", "cocodc_destroy", "cocodc_sync_budget", "cocodc_fragment_scores",
     "cocodc_select_fragments", "cocodc_outer_step", "cocodc_outer_step_host", "cocodc_merge", "cocodc_snapshot", "cocodc_snapshot_host",
     "cocodc_poll_status", "cocodc_launch_count", "cocodc_status_string",
+    "cocodc_fragment_scores_noalloc",
 )
+NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
 
 class CocodcError(RuntimeError):
@@ -87,6 +89,7 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_snapshot_host.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, i32, vp]
     lib.cocodc_merge.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp]
     lib.cocodc_snapshot.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp]
+    lib.cocodc_fragment_scores_noalloc.argtypes = [ctypes.POINTER(_Partition), vp, vp, vp, vp, i32, vp]
     lib.cocodc_poll_status.argtypes = [vp, vp]
     lib.cocodc_launch_count.argtypes = [vp]
     lib.cocodc_launch_count.restype = i64
@@ -129,6 +132,25 @@ def cocodc_sync_budget(K: int, H: int, gamma: float, Tc: float, Ts: float):
     N, h = ctypes.c_int64(), ctypes.c_int64()
     _check(_lib.cocodc_sync_budget(K, H, gamma, Tc, Ts, ctypes.byref(N), ctypes.byref(h)), "cocodc_sync_budget")
     return N.value, h.value
+
+
+def cocodc_fragment_scores_noalloc(N: int, frag_seg_ptr, seg_offset, seg_len, delta_g, interval, norms, scores,
+                                   device: int = 0, stream=None) -> None:
+    """Fragment norms and scores without a context and without any device allocation.
+
+    For callers that may not allocate on the device (allocator hooks, pre-partitioned memory,
+    allocation-free hot paths): the library's own fixed scratch array is used instead of context
+    memory.  At most NOALLOC_MAX_K fragments / NOALLOC_MAX_SEGMENTS segments; calls that overlap on
+    the GPU race on that array, so keep them on one stream.  The fragment table is host data."""
+    ptr = np.ascontiguousarray(frag_seg_ptr, dtype=np.int32)
+    off = np.ascontiguousarray(seg_offset, dtype=np.int64)
+    ln = np.ascontiguousarray(seg_len, dtype=np.int64)
+    part = _Partition(int(N), len(ptr) - 1, len(off),
+                      ptr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                      off.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)),
+                      ln.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)))
+    _check(_lib.cocodc_fragment_scores_noalloc(ctypes.byref(part), _p(delta_g), _p(interval), _p(norms), _p(scores),
+                                               int(device), _stream(stream)), "cocodc_fragment_scores_noalloc")
 
 
 class Context:

@@ -45,7 +45,7 @@ constexpr int kPlanThreads = 256;
 constexpr int kMaxK = 1024;
 
 // ids == nullptr means "all K fragments in index order" (stand-alone scoring).
-__global__ void __launch_bounds__(kPlanThreads)
+static __global__ void __launch_bounds__(kPlanThreads)
 k_plan(const int* __restrict__ ids, const int* __restrict__ n_ids_p, int K,
        const int* __restrict__ frag_seg_ptr, const long long* __restrict__ seg_off,
        const long long* __restrict__ seg_len, const long long* __restrict__ snap_offset,
@@ -162,7 +162,7 @@ constexpr int kFinalizeThreads = 256;
 // square root, form the score of Eq. 10 and (for a completion) stamp last_sync.
 //   mode 0: completion - I_p = max(1, t_p - last_sync[p]); last_sync[p] = t_l
 //   mode 1: stand-alone scoring - I_p = max(1, interval[p]) or 1; last_sync untouched
-__global__ void __launch_bounds__(kFinalizeThreads)
+static __global__ void __launch_bounds__(kFinalizeThreads)
 k_finalize_scores(const PlanHeader* __restrict__ hdr, const int* __restrict__ ids,
                   const double* __restrict__ partial, int entries_per_slot,
                   int mode, long long t_p, long long t_l, const long long* __restrict__ interval,
@@ -202,7 +202,7 @@ k_finalize_scores(const PlanHeader* __restrict__ hdr, const int* __restrict__ id
 // device staging in chunks: each chunk is a one-segment plan, and the chunk's
 // sum of squares is added to its fragment's running total in chunk order.
 // ---------------------------------------------------------------------------
-__global__ void k_plan_chunk(long long len, long long snap_off, int lanes_per_tile,
+static __global__ void k_plan_chunk(long long len, long long snap_off, int lanes_per_tile,
                              SegPlan* __restrict__ plan, PlanHeader* __restrict__ hdr) {
   SegPlan sp;
   sp.off = 0; sp.len = len; sp.snap_off = snap_off; sp.abase = 0;
@@ -213,7 +213,7 @@ __global__ void k_plan_chunk(long long len, long long snap_off, int lanes_per_ti
   hdr->n_seg = 1; hdr->n_ids = 1; hdr->pad = 0;
 }
 
-__global__ void __launch_bounds__(kFinalizeThreads)
+static __global__ void __launch_bounds__(kFinalizeThreads)
 k_accumulate_chunk(const double* __restrict__ partial, int entries, double* __restrict__ total) {
   __shared__ double red[kFinalizeThreads];
   double s = 0.0;
@@ -228,7 +228,7 @@ k_accumulate_chunk(const double* __restrict__ partial, int entries, double* __re
   if (threadIdx.x == 0) *total += red[0];
 }
 
-__global__ void k_finalize_from_sums(const double* __restrict__ sums, const int* __restrict__ ids, int n,
+static __global__ void k_finalize_from_sums(const double* __restrict__ sums, const int* __restrict__ ids, int n,
                                      long long t_p, long long t_l, long long* __restrict__ last_sync,
                                      float* __restrict__ norms, float* __restrict__ scores,
                                      int* __restrict__ status, int err_nonfinite) {
