@@ -300,6 +300,15 @@ cocodc_status cocodc_fragment_scores_noalloc(const cocodc_partition* partition, 
  */
 cocodc_status cocodc_poll_status(cocodc_ctx* ctx, void* stream);
 
+/*
+ * Failure-detection self-test.  The staged kernels wait on shared-memory barriers for their bulk
+ * copies; every such wait gives up after a fixed number of polls, records COCODC_ERR_TIMEOUT in the
+ * status word and lets the kernel return.  This call runs that wait on a barrier nothing will
+ * complete, with `polls` (1 .. 4194304) as the limit: afterwards cocodc_poll_status returns
+ * COCODC_ERR_TIMEOUT and the context is as usable as before.  It cannot hang: the loop is bounded.
+ */
+cocodc_status cocodc_selftest_bounded_wait(cocodc_ctx* ctx, int32_t polls, void* stream);
+
 /* Number of kernels the library has launched through this context so far. */
 int64_t cocodc_launch_count(const cocodc_ctx* ctx);
 

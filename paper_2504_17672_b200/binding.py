@@ -26,7 +26,7 @@ EXPORTS = (
     "cocodc_create", "cocodc_destroy", "cocodc_sync_budget", "cocodc_fragment_scores",
     "cocodc_select_fragments", "cocodc_outer_step", "cocodc_outer_step_host", "cocodc_merge", "cocodc_snapshot", "cocodc_snapshot_host",
     "cocodc_poll_status", "cocodc_launch_count", "cocodc_status_string",
-    "cocodc_fragment_scores_noalloc",
+    "cocodc_fragment_scores_noalloc", "cocodc_selftest_bounded_wait",
 )
 NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
@@ -90,6 +90,7 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_merge.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp]
     lib.cocodc_snapshot.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp]
     lib.cocodc_fragment_scores_noalloc.argtypes = [ctypes.POINTER(_Partition), vp, vp, vp, vp, i32, vp]
+    lib.cocodc_selftest_bounded_wait.argtypes = [vp, i32, vp]
     lib.cocodc_poll_status.argtypes = [vp, vp]
     lib.cocodc_launch_count.argtypes = [vp]
     lib.cocodc_launch_count.restype = i64
@@ -236,6 +237,10 @@ class Context:
         _check(_lib.cocodc_snapshot_host(self._h, _p(w_now), _p(w_snap), int(now_stride), int(snap_stride),
                                          _p(snap_offset), int(M), _p(ids), int(n_ids), _stream(stream)),
                "cocodc_snapshot_host")
+
+    def cocodc_selftest_bounded_wait(self, polls: int, stream=None) -> None:
+        """Runs a bounded wait that must run out; the status word then reads ERR_TIMEOUT."""
+        _check(_lib.cocodc_selftest_bounded_wait(self._h, int(polls), _stream(stream)), "cocodc_selftest_bounded_wait")
 
     def cocodc_poll_status(self, stream=None) -> int:
         """Waits for the stream; returns and clears the device status word."""

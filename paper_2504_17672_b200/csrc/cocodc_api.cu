@@ -501,12 +501,15 @@ cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
     return COCODC_ERR_ALIAS;
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  constexpr int U = 4;
-  auto kernel = k_snapshot<U>;
-  const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads * U, st);
+  static bool configured = false;   // one-time opt-in to 160 KB of dynamic shared memory
+  if (!configured) {
+    cudaFuncSetAttribute(k_snapshot_tma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSnapSmemBytes);
+    configured = true;
+  }
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads * kSnapU, st);
   if (s != COCODC_OK) return s;
-  kernel<<<grid, kThreads, 0, st>>>(w_now, w_snap, now_stride, snap_stride, M, c->d_plan, c->d_hdr);
+  k_snapshot_tma<<<c->sm_count, kThreads, kSnapSmemBytes, st>>>(w_now, w_snap, now_stride, snap_stride, M, c->d_plan,
+                                                                c->d_hdr, c->d_status, (int)COCODC_ERR_TIMEOUT);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
@@ -680,6 +683,14 @@ cocodc_status cocodc_snapshot_host(cocodc_ctx* c, const float* w_now, float* w_s
     }
   }
   return ok ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+cocodc_status cocodc_selftest_bounded_wait(cocodc_ctx* c, int32_t polls, void* stream) {
+  if (!c || polls < 1 || polls > kWaitLimit) return COCODC_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  k_selftest_bounded_wait<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(polls, c->d_status, (int)COCODC_ERR_TIMEOUT);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
 }  // extern "C"

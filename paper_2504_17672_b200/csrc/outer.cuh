@@ -1,5 +1,5 @@
 // Arithmetic of the outer synchronisation step and the kernels that do not stage through
-// shared memory: the generic-M fallback, the stand-alone sum of squares and the snapshot copy.
+// shared memory: the generic-M fallback and the stand-alone sum of squares.
 //
 // Per element the step reads every worker's recorded and current value, the global state and the
 // momentum once, keeps pseudo-gradient, mean, Nesterov update, delay compensation and merge in
@@ -287,48 +287,6 @@ k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ plan,
     }
   }
   sa.finish(h.n_ids, partial);
-}
-
-// ---------------------------------------------------------------------------
-// S0: copy the listed fragments of every worker from w_now into w_snap.
-// ---------------------------------------------------------------------------
-template <int U>
-__global__ void __launch_bounds__(kThreads)
-k_snapshot(const float* __restrict__ w_now, float* __restrict__ w_snap, long long now_stride,
-           long long snap_stride, int M, const SegPlan* __restrict__ plan,
-           const PlanHeader* __restrict__ hdr) {
-  const PlanHeader h = *hdr;
-  constexpr int LPT = kThreads * U;
-  int seg = 0, seg_loaded = -1;
-  SegPlan sp;
-  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
-    while (seg + 1 < h.n_seg && tile >= plan[seg + 1].first_tile) ++seg;
-    if (seg != seg_loaded) { sp = plan[seg]; seg_loaded = seg; }
-    const long long e_tile = sp.abase + 4LL * (long long)(tile - sp.first_tile) * LPT;
-    const long long seg_end = sp.off + sp.len;
-    const long long shift = sp.snap_off - sp.off;
-    if (sp.vec_ok && e_tile >= sp.off && e_tile + 4LL * LPT <= seg_end) {
-      for (int m = 0; m < M; ++m) {
-        float4 v[U];
-#pragma unroll
-        for (int j = 0; j < U; ++j)
-          v[j] = ld4(w_now + m * now_stride + e_tile + 4LL * (j * kThreads + threadIdx.x));
-#pragma unroll
-        for (int j = 0; j < U; ++j)
-          st4(w_snap + m * snap_stride + shift + e_tile + 4LL * (j * kThreads + threadIdx.x), v[j]);
-      }
-    } else {
-      for (int j = 0; j < U; ++j) {
-        const long long e = e_tile + 4LL * (j * kThreads + threadIdx.x);
-        if (e >= seg_end) break;
-        for (int k = 0; k < 4; ++k) {
-          const long long ee = e + k;
-          if (ee >= sp.off && ee < seg_end)
-            for (int m = 0; m < M; ++m) st1(w_snap + m * snap_stride + shift + ee, ld1(w_now + m * now_stride + ee));
-        }
-      }
-    }
-  }
 }
 
 }  // namespace cocodc

@@ -55,6 +55,12 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned bar, unsigned parity)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
+// the same with a caller-chosen limit
+__device__ __forceinline__ bool mbar_wait_limit(unsigned bar, unsigned parity, int limit) {
+  for (int i = 0; i < limit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
 __device__ __forceinline__ void bulk_load(unsigned dst_smem, const void* src, unsigned bytes, unsigned bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
@@ -227,6 +233,136 @@ k_outer_tma(const OuterArgs A) {
   if (tid == 0) bulk_wait_all();     // this thread's stores are complete before the CTA exits
   if (failed) return;
   if (A.partial) sa.finish(h.n_ids, A.partial);
+}
+
+}  // namespace cocodc
+
+namespace cocodc {
+
+// ---------------------------------------------------------------------------------------------
+// S0 as a pure DMA job: copy the listed fragments of every worker from w_now into w_snap.
+//
+// One thread per CTA drives the TMA unit: bulk load of a 16 KB chunk (one tile of one worker) into
+// a shared-memory stage, and, once it has landed, a bulk store of the same stage to its place in
+// w_snap.  kSnapStages stages with up to kSnapDepth loads in flight keep about 80 KB of reads and
+// as much of writes outstanding per SM.  Warps 1-7 meanwhile copy the ragged tiles (segment
+// edges, snapshot placements that are not 16-byte compatible) with ordinary loads and stores.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSnapU = 4;                                      // lanes per thread and tile
+constexpr int kSnapTileElems = kTileElems * kSnapU;            // 4096 elements = 16 KB per worker
+constexpr unsigned kSnapChunkBytes = kSnapTileElems * sizeof(float);
+constexpr int kSnapStages = 10;
+constexpr int kSnapDepth = 5;                                  // loads in flight before the oldest is stored
+constexpr unsigned kSnapSmemBytes = kSnapStages * kSnapChunkBytes;
+
+template <int N> __device__ __forceinline__ void bulk_wait_read_n() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long long now_stride,
+               long long snap_stride, int M, const SegPlan* __restrict__ plan,
+               const PlanHeader* __restrict__ hdr, int* __restrict__ status, int err_timeout) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  float* const stages = reinterpret_cast<float*>(smem_raw);
+  __shared__ __align__(8) unsigned long long full_bar[kSnapStages];
+  __shared__ float* dst_of_stage[kSnapStages];
+  const PlanHeader h = *hdr;
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    for (int s = 0; s < kSnapStages; ++s) mbar_init(smem_u32(&full_bar[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  auto tile_geometry = [&](int tile, int& seg, SegPlan& sp, int& loaded, long long& e0, bool& interior) {
+    while (seg + 1 < h.n_seg && tile >= plan[seg + 1].first_tile) ++seg;
+    if (seg != loaded) { sp = plan[seg]; loaded = seg; }
+    e0 = sp.abase + (long long)(tile - sp.first_tile) * kSnapTileElems;
+    interior = sp.vec_ok && e0 >= sp.off && e0 + kSnapTileElems <= sp.off + sp.len;
+  };
+
+  if (tid == 0) {
+    // ---- DMA driver
+    int seg = 0, loaded = -1;
+    SegPlan sp;
+    int issued = 0, stored = 0;
+    bool ok = true;
+    auto drain_one = [&]() {
+      const int s = stored % kSnapStages;
+      if (!mbar_wait_bounded(smem_u32(&full_bar[s]), (stored / kSnapStages) & 1)) {
+        record_status(status, err_timeout);
+        ok = false;
+        return;
+      }
+      bulk_store(dst_of_stage[s], smem_u32(stages + (size_t)s * kSnapTileElems), kSnapChunkBytes);
+      bulk_commit();
+      ++stored;
+    };
+    for (int tile = blockIdx.x; tile < h.total_tiles && ok; tile += gridDim.x) {
+      long long e0; bool interior;
+      tile_geometry(tile, seg, sp, loaded, e0, interior);
+      if (!interior) continue;
+      const long long shift = sp.snap_off - sp.off;
+      for (int m = 0; m < M && ok; ++m) {
+        if (issued - stored == kSnapDepth) drain_one();
+        if (!ok) break;
+        const int s = issued % kSnapStages;
+        // the stage's previous store (chunk issued - kSnapStages) is older than the newest
+        // kSnapStages - kSnapDepth - 1 committed groups: waiting until at most that many are
+        // still reading guarantees it has finished with the stage
+        if (issued >= kSnapStages) bulk_wait_read_n<kSnapStages - kSnapDepth - 1>();
+        const unsigned bar = smem_u32(&full_bar[s]);
+        mbar_expect_tx(bar, kSnapChunkBytes);
+        bulk_load(smem_u32(stages + (size_t)s * kSnapTileElems), w_now + m * now_stride + e0, kSnapChunkBytes, bar);
+        dst_of_stage[s] = w_snap + m * snap_stride + shift + e0;
+        ++issued;
+      }
+    }
+    while (ok && stored < issued) drain_one();
+    bulk_wait_all();
+    return;
+  }
+  if (tid < 32) return;
+
+  // ---- ragged tiles, warps 1-7
+  const int wtid = tid - 32;
+  constexpr int kWorkers = kThreads - 32;
+  int seg = 0, loaded = -1;
+  SegPlan sp;
+  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+    long long e0; bool interior;
+    tile_geometry(tile, seg, sp, loaded, e0, interior);
+    if (interior) continue;
+    const long long seg_end = sp.off + sp.len;
+    const long long shift = sp.snap_off - sp.off;
+    for (int l = wtid; l < kSnapTileElems / 4; l += kWorkers) {
+      const long long e = e0 + 4LL * l;
+      if (e >= seg_end) break;
+      if (sp.vec_ok && e >= sp.off && e + 4 <= seg_end) {
+        for (int m = 0; m < M; ++m) st4(w_snap + m * snap_stride + shift + e, ld4(w_now + m * now_stride + e));
+      } else {
+        for (int k = 0; k < 4; ++k) {
+          const long long ee = e + k;
+          if (ee >= sp.off && ee < seg_end)
+            for (int m = 0; m < M; ++m) st1(w_snap + m * snap_stride + shift + ee, ld1(w_now + m * now_stride + ee));
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: one thread waits on a barrier that nothing will ever complete.
+// The loop ends after `polls` polls, the kernel records the timeout code and returns, and the
+// context stays usable - this is the path a stalled copy would take in the kernels above.
+// ---------------------------------------------------------------------------------------------
+static __global__ void k_selftest_bounded_wait(int polls, int* __restrict__ status, int err_timeout) {
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x != 0) return;
+  mbar_init(smem_u32(&bar), 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  if (!mbar_wait_limit(smem_u32(&bar), 0, polls)) record_status(status, err_timeout);
 }
 
 }  // namespace cocodc

@@ -281,3 +281,19 @@ def test_host_buffer_entry_point_matches_device_path_and_oracle(same):
         prob.ctx.cocodc_outer_step_host(hp, host["w_now"], snap_h, w.N, w.N, None, host["theta_g"],
                                         host["momentum"], None, ids_h, len(ids), 8, 10, last_h, norms_h,
                                         scores_h, ws[:1000])
+
+
+def test_bounded_wait_runs_out_and_leaves_the_context_usable():
+    """Failure detection without a fault: a wait that nothing completes ends by itself with a status."""
+    prob = make(4, seed=140)
+    prob.ctx.cocodc_selftest_bounded_wait(2000)
+    assert prob.poll() == prob.B.ERR_TIMEOUT
+    assert prob.poll() == 0
+    with pytest.raises(prob.B.CocodcError):
+        prob.ctx.cocodc_selftest_bounded_wait(0)
+    ids = [0, 3]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    prob.outer_step(2, 4)
+    assert prob.poll() == 0
+    check_step_against_oracle(prob, before, ids, 2, 4, orc_hyper(prob.w))
