@@ -65,9 +65,16 @@ __device__ __forceinline__ void bulk_load(unsigned dst_smem, const void* src, un
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void bulk_store(void* dst, unsigned src_smem, unsigned bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes)
-               : "memory");
+// Outputs are not read again by this kernel: their lines are marked evict-first in L2 so that they
+// drain to DRAM early instead of displacing the loads that follow (measured: +1% bandwidth).
+__device__ __forceinline__ unsigned long long l2_evict_first_policy() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_store(void* dst, unsigned src_smem, unsigned bytes, unsigned long long policy) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;"
+               ::"l"(dst), "r"(src_smem), "r"(bytes), "l"(policy) : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_read_all_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
@@ -159,6 +166,7 @@ k_outer_tma(const OuterArgs A) {
   // ------------------------------------------------------------------ consumers
   SlotAccumulator sa(kThreads / 32);
   TileWalker tw(A.plan, h.n_seg);
+  const unsigned long long store_policy = l2_evict_first_policy();
   int k = 0;           // staged tiles consumed so far
   bool failed = false;
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
@@ -215,12 +223,12 @@ k_outer_tma(const OuterArgs A) {
       if (MODE != MODE_OUTER_ONLY) {
 #pragma unroll
         for (int m = 0; m < M; ++m)
-          bulk_store(A.w_now + m * A.now_stride + e0, smem_u32(st + (L::kNow + m) * kTileElems), kTileBytes);
+          bulk_store(A.w_now + m * A.now_stride + e0, smem_u32(st + (L::kNow + m) * kTileElems), kTileBytes, store_policy);
       }
       if (MODE != MODE_MERGE_ONLY) {
-        bulk_store(A.theta_g + e0, smem_u32(st + L::kGlobal * kTileElems), kTileBytes);
-        bulk_store(A.momentum + e0, smem_u32(st + L::kMomentum * kTileElems), kTileBytes);
-        if (A.delta_out) bulk_store(A.delta_out + e0, smem_u32(st + L::kDelta * kTileElems), kTileBytes);
+        bulk_store(A.theta_g + e0, smem_u32(st + L::kGlobal * kTileElems), kTileBytes, store_policy);
+        bulk_store(A.momentum + e0, smem_u32(st + L::kMomentum * kTileElems), kTileBytes, store_policy);
+        if (A.delta_out) bulk_store(A.delta_out + e0, smem_u32(st + L::kDelta * kTileElems), kTileBytes, store_policy);
       }
       bulk_commit();
       if (k >= 1) {   // the previous staged tile's stores have read their stage: release it
@@ -288,6 +296,7 @@ k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long
     SegPlan sp;
     int issued = 0, stored = 0;
     bool ok = true;
+    const unsigned long long store_policy = l2_evict_first_policy();
     auto drain_one = [&]() {
       const int s = stored % kSnapStages;
       if (!mbar_wait_bounded(smem_u32(&full_bar[s]), (stored / kSnapStages) & 1)) {
@@ -295,7 +304,7 @@ k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long
         ok = false;
         return;
       }
-      bulk_store(dst_of_stage[s], smem_u32(stages + (size_t)s * kSnapTileElems), kSnapChunkBytes);
+      bulk_store(dst_of_stage[s], smem_u32(stages + (size_t)s * kSnapTileElems), kSnapChunkBytes, store_policy);
       bulk_commit();
       ++stored;
     };
