@@ -69,7 +69,7 @@ class ClockSampler:
     def __enter__(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -266,7 +266,7 @@ def run_ours(args):
     peak, peak_kind = read_peaks()
     bpp = bytes_per_param(w.M)
     achieved = params_local * bpp / outer_seconds / 1e9
-    traffic = read_traffic_note(w)
+    traffic = read_traffic_note(w, params_local / K)
     out = {
         "metric": METRIC, "value": total_params / max_seconds, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": max_seconds / K * 1e3, "higher_is_better": True, "scaling": "weak",
@@ -297,17 +297,89 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def read_traffic_note(w):
-    """DRAM bytes per launch from the committed ncu summary, if it covers the current kernel."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    if not os.path.exists(path):
-        return None
+def run_sweep(args):
+    """Compensation sweep at the 1B shape: tau x lambda x fraction of the 32 fragments completing per call.
+
+    Timing only (parity of the same variants is a test): per variant a few launches of cocodc_outer_step over
+    the first n fragments, fused-kernel GB/s from CUDA events.  Prints one JSON line with all variants."""
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
+    from paper_2504_17672_b200 import binding as B
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    w = synth.get_workload("sweep_1b")
+    bufs = synth.generate(w, device)
+    ptr, off, ln = w.partition.csr()
+    ctx = B.Context(w.N, ptr, off, ln, w.M, device=0)
+    K = w.K
+    scores = torch.full((K,), float("inf"), dtype=torch.float32, device=device)
+    norms = torch.zeros(K, dtype=torch.float32, device=device)
+    last_sync = torch.zeros(K, dtype=torch.int64, device=device)
+    ids = torch.arange(K, dtype=torch.int32, device=device)
+    n_ids = torch.zeros(1, dtype=torch.int32, device=device)
+    frag = int(w.partition.frag_sizes[0])
+    peak, peak_kind = read_peaks()
+    bpp = bytes_per_param(w.M)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    variants = []
+    reps = max(3, args.steps // 4)
+    t = 0
+    for frac in (0.25, 0.5, 1.0):
+        n = int(round(frac * K))
+        n_ids.fill_(n)
+        for tau in (1, 2, 4, 8):
+            for lam in (0.0, 0.25, 0.5, 1.0):
+                hp = B.Hyper(M=w.M, H=w.H, tau=tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=lam, alpha=w.alpha)
+
+                def launch():
+                    nonlocal t
+                    t += tau
+                    ctx.cocodc_outer_step(hp, bufs.w_now, bufs.w_snap, bufs.now_stride, bufs.snap_stride, None,
+                                          bufs.theta_g, bufs.momentum, None, ids, n_ids, t, t + tau, last_sync,
+                                          norms, scores)
+                launch()
+                torch.cuda.synchronize(device)
+                a.record()
+                for _ in range(reps):
+                    launch()
+                b.record()
+                torch.cuda.synchronize(device)
+                ms = a.elapsed_time(b) / reps
+                gbs = n * frag * bpp / ms / 1e6
+                variants.append({"tau": tau, "lambda": lam, "fraction": frac, "fragments": n, "ms": ms,
+                                 "gbs": gbs, "frac_of_peak": gbs / peak})
+    status = ctx.cocodc_poll_status()
+    g = [v["gbs"] for v in variants]
+    print(json.dumps({"metric": "outer_step_gbs_per_variant", "workload": w.name, "unit": "GB/s", "peak": peak,
+                      "peak_kind": f"of {peak_kind}", "launches_per_variant": reps, "status": int(status),
+                      "min": min(g), "median": statistics.median(g), "max": max(g), "variants": variants}))
+
+
+def kernel_source_sha() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("outer.cuh", "outer_tma.cuh", "plan.cuh"):
+        with open(os.path.join(ROOT, "paper_2504_17672_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def read_traffic_note(w, params_per_launch: float):
+    """DRAM bytes per launch of the fused kernel: bytes per parameter measured by ncu on the small case
+    (profiles/dram_traffic.txt) scaled by the parameters of one launch; None if the kernel sources changed
+    since the capture or no capture covers this worker count."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
     try:
         with open(path) as f:
-            d = json.load(f)
-        return d.get(w.name)
-    except (OSError, ValueError):
+            lines = [l.split() for l in f if l.startswith("kernel=")]
+    except OSError:
         return None
+    sha = kernel_source_sha()
+    for fields in lines:
+        d = dict(x.split("=", 1) for x in fields)
+        if d.get("kernel") == "k_outer_tma" and int(d.get("M", -1)) == w.M and d.get("source_sha") == sha:
+            return float(d["bytes_per_param"]) * params_per_launch
+    return None
 
 
 # --------------------------------------------------------------------------------------------
@@ -459,7 +531,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=list(synth.WORKLOAD_NAMES), default=DEFAULT_WORKLOAD)
@@ -469,11 +541,14 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="wall time spent timing the oracle")
     ap.add_argument("--cpu-sample", type=int, default=16_000_000, help="parameters in the oracle's sample")
     ap.add_argument("--reference-sample", type=int, default=8_000_000)
+    ap.add_argument("--sweep", action="store_true", help="time the 48 variants of the 1B compensation sweep")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args)
 

@@ -1,0 +1,110 @@
+"""The schedule driver around the path (Section 2.1 time line, Section 3.2) in the paper's own setting:
+M = 4 workers, H = 100, tau = 5, K = 4 strided shards of three layers, lambda = 0.5, gamma = 0.4, which gives
+8 synchronisations per H steps (Section 4.1), one fragment per decision (Algorithm 2).
+
+Every event is checked against the oracle from the GPU's own state just before it (selection bit-exact,
+completion within the parity tolerance), and the schedule's guarantees are checked at the end."""
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import reference as orc
+from helpers import TOL_NORM, TOL_PARAM, assert_close, fragments_of, np_
+
+pytestmark = pytest.mark.gpu
+
+
+def strided_workload(layer=3001, layers=12, shards=4, M=4):
+    frs = [[(l * layer, layer) for l in range(k, layers, shards)] for k in range(shards)]
+    total = layer * layers
+    return synth.small_workload((total + 4 - total % 4, frs), M=M, seed=31, tau=5, H=100,
+                                lam=0.5, budget_kind="count", budget=1)
+
+
+def test_round_driver_in_the_papers_setting():
+    from paper_2504_17672_b200 import binding as B
+    from paper_2504_17672_b200.schedule import RoundDriver
+    w = strided_workload()
+    frs = fragments_of(w)
+    bufs = synth.generate(w, "cuda")
+    ptr, off, ln = w.partition.csr()
+    ctx = B.Context(w.N, ptr, off, ln, w.M)
+    hyper = B.Hyper(M=w.M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam, alpha=1.0)
+    drv = RoundDriver(ctx, hyper, bufs.w_now, bufs.theta_g, bufs.momentum, w.partition.frag_sizes,
+                      gamma=0.4, Tc=0.2, Ts=1.0, budget_kind=B.BUDGET_COUNT, budget=1)
+    assert (drv.N_sync, drv.h) == (8, 12)                       # "8 synchronizations per H steps"
+    ohp = orc.Hyper(M=w.M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam, alpha=1.0)
+    log = {"initiated": [], "completed": [], "pre": None, "worst": 0.0}
+
+    def state():
+        return dict(w_now=np_(bufs.w_now).copy(), theta_g=np_(bufs.theta_g).copy(), momentum=np_(bufs.momentum).copy(),
+                    scores=np_(drv.scores).copy(), last_sync=np_(drv.last_sync).copy(),
+                    ineligible=np_(drv.ineligible).copy(), norms=np_(drv.norms).copy())
+
+    def observer(kind, phase, slot, t):
+        if phase == "before":
+            log["pre"] = state()
+            if kind == "complete":
+                log["pre"]["pool"] = np_(slot.pool).copy()
+                log["pre"]["pool_off"] = np_(slot.pool_off).copy()
+                log["pre"]["ids"] = np_(slot.ids)[:int(slot.n_ids.item())].tolist()
+                log["pre"]["t_p"] = slot.t_p
+            return
+        pre, post = log["pre"], state()
+        assert ctx.cocodc_poll_status() == 0
+        if kind == "initiate":
+            mask, ids, n = orc.select_fragments(pre["scores"], pre["last_sync"], w.partition.frag_sizes, t, w.H,
+                                                orc.BUDGET_COUNT, 1, pre["ineligible"])
+            got = np_(slot.ids)[:int(slot.n_ids.item())].tolist()
+            assert got == ids.tolist() and np.array_equal(np_(slot.mask), mask)
+            assert not any(pre["ineligible"][p] for p in got)          # never a fragment that is in flight
+            assert np.array_equal(post["ineligible"], pre["ineligible"] + mask)
+            po = np_(slot.pool_off)
+            exp_pool = orc.snapshot(frs, pre["w_now"], got, w.M, po, np_(slot.pool))
+            assert np.array_equal(np_(slot.pool), exp_pool)             # S0 recorded exactly the chosen fragments
+            log["initiated"].append((t, got))
+        else:
+            ids = pre["ids"]
+            res, new_last = orc.outer_step(frs, ohp, pre["w_now"], pre["pool"], pre["theta_g"], pre["momentum"], ids,
+                                           pre["t_p"], t, pre["last_sync"], snap_offset=pre["pool_off"])
+            assert t - pre["t_p"] == w.tau
+            for p in ids:
+                r = res[p]
+                log["worst"] = max(log["worst"], *assert_close(orc.gather_fragment(frs, post["theta_g"], p), r.theta_g,
+                                                               TOL_PARAM, "theta_g"))
+                assert_close(orc.gather_fragment(frs, post["momentum"], p), r.momentum, TOL_PARAM, "momentum")
+                wn = orc.gather_fragment(frs, post["w_now"], p)
+                for m in range(w.M):
+                    assert_close(wn[m], r.w_now[m], TOL_PARAM, f"w_now[{m}]")
+                assert abs(post["scores"][p] - r.score) <= TOL_NORM * r.score
+            assert np.array_equal(post["last_sync"], new_last)
+            log["completed"].append((t, ids))
+
+    drv.observer = observer
+    gen = torch.Generator(device="cuda").manual_seed(77)
+    T = 230
+    for t in range(1, T + 1):
+        # local training: every worker moves a little
+        bufs.w_now.add_(torch.randn(bufs.w_now.shape, generator=gen, device="cuda") * 2e-4)
+        drv.after_local_step(t)
+
+    starts = [t for t, _ in log["initiated"]]
+    assert starts == list(range(12, T + 1, 12))                                   # every h = 12 steps
+    assert [ids for _, ids in log["initiated"][:4]] == [[0], [1], [2], [3]]        # never-synced first, in order
+    assert [t for t, _ in log["completed"]] == [s + w.tau for s in starts if s + w.tau <= T]
+    # at least K synchronisations per H steps, 8 with this gamma
+    for lo in range(12, T - w.H, 12):
+        in_window = [ids[0] for t, ids in log["initiated"] if lo <= t < lo + w.H]
+        assert len(in_window) >= 8
+        # the staleness rule of Algorithm 2 brings every fragment back within H steps of its last
+        # completion, up to the delay and the wait for the next initiation slot(s)
+        wide = [ids[0] for t, ids in log["initiated"] if lo <= t < lo + w.H + 2 * drv.h]
+        assert set(wide) == {0, 1, 2, 3}
+    # no fragment goes stale: time since its last completed sync stays below H plus one interval and the delay
+    last = np_(drv.last_sync)
+    assert np.all(T - last < w.H + 2 * drv.h + w.tau)
+    counts = np.bincount([ids[0] for _, ids in log["initiated"]], minlength=4)
+    assert counts.min() >= 2 and counts.sum() == len(starts)
+    assert log["worst"] <= TOL_PARAM
