@@ -149,9 +149,9 @@ def pool_capacity(w: synth.Workload) -> int:
 class DeviceJob:
     """Workload resident in HBM plus its schedule state, stepped through the C-ABI binding."""
 
-    def __init__(self, w: synth.Workload, device: torch.device):
+    def __init__(self, w: synth.Workload, device: torch.device, variant: str = "cocodc"):
         from paper_2504_17672_b200 import binding as B
-        self.B, self.w, self.dev = B, w, device
+        self.B, self.w, self.dev, self.variant = B, w, device, variant
         ptr, off, ln = w.partition.csr()
         self.ctx = B.Context(w.N, ptr, off, ln, w.M, device=device.index or 0)
         K = w.K
@@ -169,6 +169,10 @@ class DeviceJob:
         self.t = w.tau
         self.hyper = B.Hyper(M=w.M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam,
                              alpha=w.alpha)
+        if variant == "streaming_diloco":      # Eq. 1-3 only: no compensation, blend with alpha = 0.5
+            self.hyper.comp_mode, self.hyper.alpha = B.COMP_NONE, 0.5
+        elif variant == "diloco":              # blocking sync of the whole model: snapshot = current, no delay
+            self.hyper.comp_mode, self.hyper.tau = B.COMP_NONE, 0
         # first selection, then generate the buffers with the selected fragments' snapshots in the pool
         self.select()
         torch.cuda.synchronize(device)
@@ -177,6 +181,9 @@ class DeviceJob:
         offs = {p: int(self.pool_off[p].item()) for p in ids0}
         self.bufs = synth.generate(w, device, snap_layout="pool", pool_ids=ids0, pool_offsets=offs,
                                    pool_len=pool_capacity(w))
+        if variant == "diloco":
+            self.ids.copy_(torch.arange(K, dtype=torch.int32, device=device))
+            self.n_ids.fill_(K)
 
     def select(self):
         w = self.w
@@ -185,6 +192,11 @@ class DeviceJob:
 
     def outer(self):
         b, w = self.bufs, self.w
+        if self.variant == "diloco":
+            self.ctx.cocodc_outer_step(self.hyper, b.w_now, b.w_now, b.now_stride, b.now_stride, None,
+                                       b.theta_g, b.momentum, None, self.ids, self.n_ids, self.t, self.t,
+                                       self.last_sync, self.norms, self.scores)
+            return
         self.ctx.cocodc_outer_step(self.hyper, b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off,
                                    b.theta_g, b.momentum, None, self.ids, self.n_ids, self.t, self.t + w.tau,
                                    self.last_sync, self.norms, self.scores)
@@ -204,6 +216,9 @@ class DeviceJob:
         if log_ids is not None:
             log_ids.copy_(self.ids)
             log_n.copy_(self.n_ids)
+        if self.variant == "diloco":
+            self.t += self.w.H
+            return
         self.t += self.w.tau
         self.select()
         self.snapshot()
@@ -223,7 +238,7 @@ def run_ours(args):
     w = synth.get_workload(args.workload)
     if world > 1:
         w = w.with_(seed=w.seed + 1000 * rank)   # every rank owns a different shard of the same shape
-    job = DeviceJob(w, device)
+    job = DeviceJob(w, device, args.variant)
     K, W = args.steps, args.warmup
     log_ids = torch.full((K, w.K), -1, dtype=torch.int32, device=device)
     log_n = torch.zeros((K, 1), dtype=torch.int32, device=device)
@@ -264,16 +279,19 @@ def run_ours(args):
     total_params, max_seconds = aggregate(params_local, seconds, world, backend_ready)
 
     peak, peak_kind = read_peaks()
-    bpp = bytes_per_param(w.M)
+    bpp = bytes_per_param(w.M) if args.variant != "diloco" else 8 * w.M + 16   # zero delay: one read of w_now
+    snap_bpp = 8 * w.M if args.variant != "diloco" else 0
     achieved = params_local * bpp / outer_seconds / 1e9
-    traffic = read_traffic_note(w, params_local / K)
+    traffic = read_traffic_note(w, params_local / K) if args.variant != "diloco" else None
     out = {
         "metric": METRIC, "value": total_params / max_seconds, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": max_seconds / K * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "N": w.N, "K": w.K, "M": w.M, "tau": w.tau, "H": w.H,
                    "budget": f"{w.budget} {w.budget_kind}", "params_per_step": params_local / K,
-                   "step": "outer_step(S1-S6) + select(S7) + snapshot(S0)", "snapshot_layout": "pool",
+                   "variant": args.variant,
+                   "step": ("outer_step(S1-S6) + select(S7) + snapshot(S0)" if args.variant != "diloco"
+                            else "outer_step(S1-S6) over all fragments, blocking"), "snapshot_layout": "pool",
                    "l2": "inputs larger than L2 (every step streams GBs)", "parallelism": f"replicas x{world}"},
         "gpu_launches": int(launches),
         "clocks": clocks.result,
@@ -281,9 +299,9 @@ def run_ours(args):
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": achieved / 8000.0, "bytes_per_param": bpp,
                      "ms_per_launch": outer_seconds / K * 1e3, "traffic": traffic},
-        "step_gbs": (params_local * (bpp + 8 * w.M)) / seconds / 1e9,
+        "step_gbs": (params_local * (bpp + snap_bpp)) / seconds / 1e9,
     }
-    if rank == 0 and not args.no_e2e:
+    if rank == 0 and not args.no_e2e and args.variant == "cocodc":
         out["e2e"] = run_e2e(job, args)
     elif rank == 0:
         out["e2e"] = None
@@ -541,6 +559,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="wall time spent timing the oracle")
     ap.add_argument("--cpu-sample", type=int, default=16_000_000, help="parameters in the oracle's sample")
     ap.add_argument("--reference-sample", type=int, default=8_000_000)
+    ap.add_argument("--variant", choices=["cocodc", "streaming_diloco", "diloco"], default="cocodc",
+                    help="which method's arithmetic the step runs (the baselines are modes of the same kernels)")
     ap.add_argument("--sweep", action="store_true", help="time the 48 variants of the 1B compensation sweep")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
