@@ -197,7 +197,9 @@ cocodc_status cocodc_select_fragments(cocodc_ctx* ctx, const float* scores, cons
  *   ids dev int32[<=K] distinct fragment ids; n_ids dev int32[1]
  *   last_sync dev int64[K]; norms, scores dev fp32[K] (needed with STAGE_SCORE)
  * Errors: INVALID_ARG, ALIGNMENT, ALIAS (buffers overlapping other than w_snap == w_now), CUDA.
- * Device-side: an id outside [0,K) or listed twice processes nothing and sets INVALID_ARG.
+ * Device-side: an id outside [0,K) or listed twice, a listed fragment without a place in the pool
+ * (snap_offset[p] < 0) or whose packed snapshot would not fit inside one row (snap_offset[p] + n_p >
+ * snap_stride) processes nothing and sets INVALID_ARG.
  */
 cocodc_status cocodc_outer_step(cocodc_ctx* ctx, const cocodc_hyper* hyper,
                                 float* w_now, const float* w_snap,

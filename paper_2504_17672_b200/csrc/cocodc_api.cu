@@ -85,9 +85,9 @@ int grid_for(cocodc_ctx* c, const void* kernel) {
 }
 
 cocodc_status launch_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_ids,
-                          const int64_t* snap_offset, int lanes_per_tile, cudaStream_t st) {
+                          const int64_t* snap_offset, long long snap_row_len, int lanes_per_tile, cudaStream_t st) {
   k_plan<<<1, kPlanThreads, 0, st>>>(ids, n_ids, c->K, c->d_frag_seg_ptr, c->d_seg_off, c->d_seg_len,
-                                     reinterpret_cast<const long long*>(snap_offset), lanes_per_tile,
+                                     reinterpret_cast<const long long*>(snap_offset), snap_row_len, lanes_per_tile,
                                      c->n_segments, c->d_plan, c->d_hdr, c->d_status,
                                      (int)COCODC_ERR_INVALID_ARG);
   c->launches++;
@@ -145,7 +145,7 @@ cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool sam
                            const int32_t* n_ids, const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
   const Variant v = pick_variant(A.M, mode, same);
   const int grid = variant_grid(c, v);
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads, st);
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, A.snap_stride, kThreads, st);
   if (s != COCODC_OK) return s;
   v.kernel<<<grid, v.threads, v.smem, st>>>(A);
   c->launches++;
@@ -187,6 +187,13 @@ void fold_coefficients(const cocodc_hyper* h, bool zero_delay, OuterArgs* A) {
   A->Mf = (float)h->M;
   A->inv_M = 1.0f / (float)h->M;
   A->M_pow2 = ((h->M & (h->M - 1)) == 0) ? 1 : 0;
+}
+
+// elements of fragment p (host copy of the table)
+long long fragment_elems(const cocodc_ctx* c, int p) {
+  long long n = 0;
+  for (int s = c->h_frag_seg_ptr[p]; s < c->h_frag_seg_ptr[p + 1]; ++s) n += c->h_seg_len[s];
+  return n;
 }
 
 void set_status_sink(const cocodc_ctx* c, OuterArgs* A) {
@@ -356,7 +363,7 @@ cocodc_status cocodc_fragment_scores(cocodc_ctx* c, const float* delta_g, const 
   constexpr int U = 4;
   auto kernel = k_sumsq<U>;
   const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
-  cocodc_status s = launch_plan(c, nullptr, nullptr, nullptr, kThreads * U, st);
+  cocodc_status s = launch_plan(c, nullptr, nullptr, nullptr, 0, kThreads * U, st);
   if (s != COCODC_OK) return s;
   kernel<<<grid, kThreads, 0, st>>>(delta_g, c->d_plan, c->d_hdr, c->d_partial);
   c->launches++;
@@ -506,7 +513,7 @@ cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
     cudaFuncSetAttribute(k_snapshot_tma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSnapSmemBytes);
     configured = true;
   }
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, kThreads * kSnapU, st);
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, snap_stride, kThreads * kSnapU, st);
   if (s != COCODC_OK) return s;
   k_snapshot_tma<<<c->sm_count, kThreads, kSnapSmemBytes, st>>>(w_now, w_snap, now_stride, snap_stride, M, c->d_plan,
                                                                 c->d_hdr, c->d_status, (int)COCODC_ERR_TIMEOUT);
@@ -539,7 +546,8 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
     for (int j = 0; j < n_ids; ++j) {
       const int p = ids[j];
       if (p < 0 || p >= K || seen[p]) return COCODC_ERR_INVALID_ARG;
-      if (snap_offset && snap_offset[p] < 0) return COCODC_ERR_INVALID_ARG;
+      if (snap_offset && (snap_offset[p] < 0 || snap_offset[p] + fragment_elems(c, p) > snap_stride))
+        return COCODC_ERR_INVALID_ARG;   // no place, or not inside one row of the pool
       seen[p] = 1;
     }
     std::vector<Range> r;
@@ -665,7 +673,8 @@ cocodc_status cocodc_snapshot_host(cocodc_ctx* c, const float* w_now, float* w_s
   if (now_stride < c->N || snap_stride < (snap_offset ? 1 : c->N)) return COCODC_ERR_INVALID_ARG;
   for (int j = 0; j < n_ids; ++j) {
     if (ids[j] < 0 || ids[j] >= c->K) return COCODC_ERR_INVALID_ARG;
-    if (snap_offset && snap_offset[ids[j]] < 0) return COCODC_ERR_INVALID_ARG;
+    if (snap_offset && (snap_offset[ids[j]] < 0 || snap_offset[ids[j]] + fragment_elems(c, ids[j]) > snap_stride))
+      return COCODC_ERR_INVALID_ARG;
   }
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);

@@ -49,7 +49,7 @@ static __global__ void __launch_bounds__(kPlanThreads)
 k_plan(const int* __restrict__ ids, const int* __restrict__ n_ids_p, int K,
        const int* __restrict__ frag_seg_ptr, const long long* __restrict__ seg_off,
        const long long* __restrict__ seg_len, const long long* __restrict__ snap_offset,
-       int lanes_per_tile, int plan_capacity, SegPlan* __restrict__ plan,
+       long long snap_row_len, int lanes_per_tile, int plan_capacity, SegPlan* __restrict__ plan,
        PlanHeader* __restrict__ hdr, int* __restrict__ status, int err_invalid) {
   __shared__ int seen[kMaxK];
   __shared__ int bad;
@@ -94,6 +94,8 @@ k_plan(const int* __restrict__ ids, const int* __restrict__ n_ids_p, int K,
       sp.slot = j;
       sp.frag = p;
       sp.vec_ok = (((sp.snap_off - sp.off) & 3LL) == 0) ? 1 : 0;
+      // a packed snapshot must lie inside one row of the pool the caller described
+      if (snap_offset != nullptr && sp.snap_off + sp.len > snap_row_len) { overflow = true; break; }
       plan[ns++] = sp;
       const long long lanes = (sp.off - sp.abase + sp.len + 3) >> 2;
       tiles += (lanes + lanes_per_tile - 1) / lanes_per_tile;

@@ -161,6 +161,12 @@ def test_sweep_1b_variants():
             if prob is None:
                 prob = GpuProblem(w, bufs)
             prob.w = w
+            if i > 1:
+                # fresh outer state for every variant: repeated completions from the same snapshots would drive
+                # the mean pseudo-gradient to the cancellation limit of fp32 (|Delta| << |delta_m|), where an
+                # error bound relative to the output no longer applies
+                bufs.momentum.normal_(0.0, 1e-3)
+                bufs.theta_g.add_(bufs.momentum)
             n = int(round(frac * w.K))
             ids = list(range(n))
             _sampled_round(prob, ids, t, t + tau, orc_hyper(w), full_norm=1)

@@ -129,6 +129,16 @@ def test_snapshot_pool_layouts(aligned):
     after = prob.host_state()
     for k in ("w_now", "theta_g", "momentum", "last_sync"):
         assert np.array_equal(before[k], after[k])
+    # a placement that would run past the end of a pool row is refused too (no out-of-bounds read or write)
+    prob.set_ids([1])
+    prob.bufs.snap_offset[1] = prob.bufs.w_snap.shape[1] - 100
+    prob.outer_step(12, 13)
+    assert prob.poll() == prob.B.ERR_INVALID_ARG
+    prob.snapshot()
+    assert prob.poll() == prob.B.ERR_INVALID_ARG
+    after = prob.host_state()
+    for k in ("w_now", "w_snap", "theta_g", "momentum", "last_sync"):
+        assert np.array_equal(before[k], after[k])
 
 
 def test_snapshot_kernel_copies_exactly_the_listed_fragments():
