@@ -63,6 +63,12 @@ static double merged_value(double a, double b, double G, double lambda, double a
  * Outputs (double): theta_g_out[i] = G, u_out[i] = u', delta_out[i] = Delta,
  * now_out[m*n + i] = merged local value.  do_merge = 0 leaves now_out alone.
  * Returns sum_i Delta_i^2 accumulated in element order (for Eq. 10's norm).
+ *
+ * Worker-per-device deployment (Section 2.1: each worker all-reduces its pseudo-gradient): if
+ * recv_sum is not NULL it holds, per element, the sum over ALL M_total workers of their
+ * pseudo-gradients as delivered by the all-reduce (fp32), and Eq. 1's mean is recv_sum[i] / M_total;
+ * the M local workers in snap/now are then only merged.  recv_sum == NULL: the mean is formed from
+ * the M stacked workers as above.
  */
 double cocodc_oracle_outer_elements(
     long n, int M,
@@ -71,19 +77,25 @@ double cocodc_oracle_outer_elements(
     const float *theta_g, const float *u,
     double eta, double mu, double lambda, double alpha, long tau, long H,
     int comp_mode, int sign_mode, int do_merge,
+    const float *recv_sum, int M_total,
     double *now_out, double *theta_g_out, double *u_out, double *delta_out)
 {
     long double sumsq = 0.0L;
     for (long i = 0; i < n; ++i) {
         double thg = (double)theta_g[i];
-        /* pseudo-gradient of every worker (Section 2.1) and their mean, Eq. 1:
-         * differences first, summed in worker order, then divided by M */
-        double sum = 0.0;
-        for (int m = 0; m < M; ++m) {
-            double delta_m = (double)snap[(size_t)m * snap_stride + i] - thg;
-            sum += delta_m;
+        double Delta;
+        if (recv_sum) {
+            Delta = (double)recv_sum[i] / (double)M_total;       /* Eq. 1 from the all-reduced sum */
+        } else {
+            /* pseudo-gradient of every worker (Section 2.1) and their mean, Eq. 1:
+             * differences first, summed in worker order, then divided by M */
+            double sum = 0.0;
+            for (int m = 0; m < M; ++m) {
+                double delta_m = (double)snap[(size_t)m * snap_stride + i] - thg;
+                sum += delta_m;
+            }
+            Delta = sum / (double)M;
         }
-        double Delta = sum / (double)M;
         /* outer optimizer, Eq. 2 */
         double u_new = mu * (double)u[i] + Delta;
         double G = thg + eta * (Delta + mu * u_new);
@@ -121,6 +133,20 @@ void cocodc_oracle_merge_elements(
             now_out[(size_t)m * n + i] =
                 merged_value(a, b, G, lambda, alpha, tau, H, comp_mode, sign_mode);
         }
+    }
+}
+
+/* What one device contributes to the all-reduce of Section 2.1: the sum over its M local workers
+ * of the pseudo-gradients theta^m_{p,t_p} - theta^g_{p,t_p-H}, per element. */
+void cocodc_oracle_pseudo_gradient_sum(long n, int M, const float *snap, long snap_stride,
+                                       const float *theta_g, double *sum_out)
+{
+    for (long i = 0; i < n; ++i) {
+        double thg = (double)theta_g[i];
+        double sum = 0.0;
+        for (int m = 0; m < M; ++m)
+            sum += (double)snap[(size_t)m * snap_stride + i] - thg;
+        sum_out[i] = sum;
     }
 }
 

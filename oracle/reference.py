@@ -42,7 +42,9 @@ def _clib():
         d, l, i, p = ctypes.c_double, ctypes.c_long, ctypes.c_int, ctypes.c_void_p
         lib.cocodc_oracle_outer_elements.restype = d
         lib.cocodc_oracle_outer_elements.argtypes = [
-            l, i, p, l, p, l, p, p, d, d, d, d, l, l, i, i, i, p, p, p, p]
+            l, i, p, l, p, l, p, p, d, d, d, d, l, l, i, i, i, p, i, p, p, p, p]
+        lib.cocodc_oracle_pseudo_gradient_sum.restype = None
+        lib.cocodc_oracle_pseudo_gradient_sum.argtypes = [l, i, p, l, p, p]
         lib.cocodc_oracle_merge_elements.restype = None
         lib.cocodc_oracle_merge_elements.argtypes = [l, i, p, l, p, l, p, d, d, l, l, i, i, p]
         lib.cocodc_oracle_sumsq.restype = d
@@ -183,14 +185,20 @@ def outer_step(fragments: Fragments, hp: Hyper, w_now: np.ndarray, w_snap: np.nd
                theta_g: np.ndarray, momentum: np.ndarray, ids: Sequence[int],
                t_p: int, t_l: int, last_sync: Sequence[int],
                snap_offset: Optional[Sequence[int]] = None, do_merge: bool = True,
-               threads: int = 1):
+               threads: int = 1, recv_sum: Optional[np.ndarray] = None, M_total: Optional[int] = None):
     """Run Eq. 1-2, Algorithm 1 / Eq. 3 and Eq. 10 on the fragments in `ids`.
 
     w_now, w_snap: float32 [M, .]; theta_g, momentum: float32 [N].  w_snap is
     laid out like w_now unless snap_offset[p] gives fragment p's start inside a
     packed row.  Inputs are not modified.
+    recv_sum (float32 [N]) and M_total: the worker-per-device deployment of Section 2.1 - the all-reduced
+    sum of all M_total workers' pseudo-gradients is given, and the M local workers are only merged.
     Returns (results {p: FragmentResult}, new last_sync int64[K]).
     """
+    if recv_sum is not None:
+        recv_sum = _f32(recv_sum)
+        if not M_total or M_total < 1:
+            raise ValueError("M_total must accompany recv_sum")
     lib = _clib()
     w_now, w_snap, theta_g, momentum = _f32(w_now), _f32(w_snap), _f32(theta_g), _f32(momentum)
     M = hp.M
@@ -227,6 +235,7 @@ def outer_step(fragments: Fragments, hp: Hyper, w_now: np.ndarray, w_snap: np.nd
                     _ptr(theta_g, off + lo), _ptr(momentum, off + lo),
                     hp.outer_lr, hp.momentum, hp.lam, hp.alpha, hp.tau, hp.H,
                     hp.comp_mode, hp.sign_mode, 1 if do_merge else 0,
+                    None if recv_sum is None else _ptr(recv_sum, off + lo), int(M_total or 0),
                     blk.ctypes.data if do_merge else None,
                     _ptr(out_g, pos + lo), _ptr(out_u, pos + lo), _ptr(out_d, pos + lo))
                 if do_merge:
@@ -246,6 +255,27 @@ def outer_step(fragments: Fragments, hp: Hyper, w_now: np.ndarray, w_snap: np.nd
         results[p] = FragmentResult(out_now, out_g, out_u, out_d, sumsq, norm, norm / interval)
         new_last[p] = int(t_l)
     return results, new_last
+
+
+def pseudo_gradient_sum(fragments: Fragments, M: int, w_snap: np.ndarray, theta_g: np.ndarray, ids: Sequence[int],
+                        snap_offset: Optional[Sequence[int]] = None) -> Dict[int, np.ndarray]:
+    """Per listed fragment, the sum over the M local workers of theta^m_{p,t_p} - theta^g (what one device
+    hands to the all-reduce of Section 2.1), float64 [n_p], segments concatenated."""
+    lib = _clib()
+    w_snap, theta_g = _f32(w_snap), _f32(theta_g)
+    snap_stride = w_snap.strides[0] // 4
+    out: Dict[int, np.ndarray] = {}
+    for p in [int(q) for q in ids]:
+        n_p = sum(l for _, l in fragments[p])
+        res = np.empty(n_p, dtype=np.float64)
+        pos = 0
+        for off, ln in fragments[p]:
+            sb = _snap_base(snap_offset, p, off, pos)
+            lib.cocodc_oracle_pseudo_gradient_sum(ln, M, _ptr(w_snap, sb), snap_stride, _ptr(theta_g, off),
+                                                  _ptr(res, pos))
+            pos += ln
+        out[p] = res
+    return out
 
 
 def _split(n: int, parts: int):

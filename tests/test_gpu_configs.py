@@ -167,6 +167,7 @@ def test_sweep_1b_variants():
                 # error bound relative to the output no longer applies
                 bufs.momentum.normal_(0.0, 1e-3)
                 bufs.theta_g.add_(bufs.momentum)
+                bufs.momentum.normal_(0.0, 1e-3)      # independent of the shift just applied to theta_g
             n = int(round(frac * w.K))
             ids = list(range(n))
             _sampled_round(prob, ids, t, t + tau, orc_hyper(w), full_norm=1)

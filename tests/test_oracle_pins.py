@@ -411,3 +411,33 @@ def test_selection_is_deterministic_and_rejects_nan():
         orc.select_fragments([1.0, float("nan")], [0, 0], [1, 1], 1, 100, orc.BUDGET_COUNT, 1)
     mask, ids, n = orc.select_fragments([1.0, 2.0], [0, 0], [1, 1], 1, 100, orc.BUDGET_COUNT, 1, [1, 1])
     assert n == 0 and mask.sum() == 0
+
+
+# ------------------------------------------------------------------ worker-per-device deployment (Section 2.1)
+
+def test_received_sum_mode_equals_stacked_workers():
+    """Two devices with two workers each, their pseudo-gradient sums all-reduced, reproduce the four stacked workers."""
+    M, n = 4, 500
+    now, snap, thg, mom = rand_inputs(M, n, seed=21)
+    # quantise so that every partial sum is exact in fp32 and the comparison can be bit for bit
+    q = lambda x: (np.round(x * 2.0 ** 16) / 2.0 ** 16).astype(np.float32)
+    snap, thg = q(snap), q(thg)
+    frs = one_fragment(n)
+    parts = [orc.pseudo_gradient_sum(frs, 2, np.ascontiguousarray(snap[d * 2:d * 2 + 2]), thg, [0])[0] for d in range(2)]
+    np.testing.assert_array_equal(parts[0], (snap[0].astype(np.float64) - thg) + (snap[1].astype(np.float64) - thg))
+    total = (parts[0] + parts[1]).astype(np.float32)
+    assert np.array_equal(total.astype(np.float64), parts[0] + parts[1])
+    hp4 = orc.Hyper(M=4, tau=3)
+    full = run_single(hp4, now, snap, thg, mom)
+    for d in range(2):
+        hp2 = orc.Hyper(M=2, tau=3)
+        res, last = orc.outer_step(frs, hp2, np.ascontiguousarray(now[d * 2:d * 2 + 2]),
+                                   np.ascontiguousarray(snap[d * 2:d * 2 + 2]), thg, mom, [0], 10, 12, [0],
+                                   recv_sum=total, M_total=4)
+        r = res[0]
+        np.testing.assert_array_equal(r.theta_g, full.theta_g)
+        np.testing.assert_array_equal(r.momentum, full.momentum)
+        np.testing.assert_array_equal(r.w_now, full.w_now[d * 2:d * 2 + 2])
+        assert r.norm == full.norm and list(last) == [12]
+    with pytest.raises(ValueError):
+        orc.outer_step(frs, orc.Hyper(M=2), now[:2], snap[:2], thg, mom, [0], 10, 12, [0], recv_sum=total)
