@@ -210,6 +210,34 @@ cocodc_status cocodc_outer_step(cocodc_ctx* ctx, const cocodc_hyper* hyper,
                                 float* norms, float* scores, uint32_t stages, void* stream);
 
 /*
+ * Worker-per-device deployment (Section 2.1: every worker all-reduces its pseudo-gradient).  When a
+ * device holds only M of the M_total workers, Eq. 1's sum spans devices:
+ *
+ *   cocodc_pseudo_gradient_sum   S1 + the local part of S2: sum_out[i] = sum over this device's M
+ *                                workers of (w_snap[m][i] - theta_g[i]) for the listed fragments, at their
+ *                                native offsets in sum_out (dev fp32[N]); other elements are not touched.
+ *   (the caller all-reduces sum_out over the devices, e.g. with NCCL)
+ *   cocodc_outer_step_received   S2-S6 as cocodc_outer_step (all stages), except that
+ *                                Delta = delta_sum[i] / M_total; hyper->M is the local worker count, whose
+ *                                w_now rows are merged.  delta_g_out may be NULL, or delta_sum itself
+ *                                (replaced by Delta in place).
+ *
+ * With M_total == hyper->M and delta_sum produced by cocodc_pseudo_gradient_sum on the same buffers the
+ * result is bit-identical to cocodc_outer_step.  Layout, alignment and device-side error rules as there;
+ * w_snap == w_now (zero delay) is not accepted here.
+ */
+cocodc_status cocodc_pseudo_gradient_sum(cocodc_ctx* ctx, const float* w_snap, int64_t snap_stride,
+                                         const int64_t* snap_offset, const float* theta_g, int32_t M,
+                                         float* sum_out, const int32_t* ids, const int32_t* n_ids, void* stream);
+cocodc_status cocodc_outer_step_received(cocodc_ctx* ctx, const cocodc_hyper* hyper, int32_t M_total,
+                                         float* w_now, const float* w_snap,
+                                         int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                         float* theta_g, float* momentum, const float* delta_sum,
+                                         float* delta_g_out, const int32_t* ids, const int32_t* n_ids,
+                                         int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                         float* norms, float* scores, void* stream);
+
+/*
  * S4-S5 alone (Algorithm 1, or Eq. 3 for COMP_NONE), given the new global state:
  * w_now[m][i] = (1-alpha)*w_now[m][i] + alpha*target_m with G = theta_g_new[i].
  * Together with cocodc_outer_step(stages without MERGE) this is the unfused path.

@@ -27,6 +27,7 @@ EXPORTS = (
     "cocodc_select_fragments", "cocodc_outer_step", "cocodc_outer_step_host", "cocodc_merge", "cocodc_snapshot", "cocodc_snapshot_host",
     "cocodc_poll_status", "cocodc_launch_count", "cocodc_status_string",
     "cocodc_fragment_scores_noalloc", "cocodc_selftest_bounded_wait",
+    "cocodc_pseudo_gradient_sum", "cocodc_outer_step_received",
 )
 NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
@@ -91,6 +92,9 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_snapshot.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp]
     lib.cocodc_fragment_scores_noalloc.argtypes = [ctypes.POINTER(_Partition), vp, vp, vp, vp, i32, vp]
     lib.cocodc_selftest_bounded_wait.argtypes = [vp, i32, vp]
+    lib.cocodc_pseudo_gradient_sum.argtypes = [vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
+    lib.cocodc_outer_step_received.argtypes = [vp, ctypes.POINTER(_Hyper), i32, vp, vp, i64, i64, vp, vp, vp, vp,
+                                               vp, vp, vp, i64, i64, vp, vp, vp, vp]
     lib.cocodc_poll_status.argtypes = [vp, vp]
     lib.cocodc_launch_count.argtypes = [vp]
     lib.cocodc_launch_count.restype = i64
@@ -217,6 +221,22 @@ class Context:
                                            _p(last_sync), _p(norms), _p(scores), 1 if snap_on_device else 0, _p(workspace),
                                            workspace.numel() * workspace.element_size(), _stream(stream)),
                "cocodc_outer_step_host")
+
+    def cocodc_pseudo_gradient_sum(self, w_snap, snap_stride: int, snap_offset, theta_g, M: int, sum_out,
+                                   ids, n_ids, stream=None) -> None:
+        _check(_lib.cocodc_pseudo_gradient_sum(self._h, _p(w_snap), int(snap_stride), _p(snap_offset), _p(theta_g),
+                                               int(M), _p(sum_out), _p(ids), _p(n_ids), _stream(stream)),
+               "cocodc_pseudo_gradient_sum")
+
+    def cocodc_outer_step_received(self, hyper: Hyper, M_total: int, w_now, w_snap, now_stride: int,
+                                   snap_stride: int, snap_offset, theta_g, momentum, delta_sum, delta_g_out,
+                                   ids, n_ids, t_p: int, t_l: int, last_sync, norms, scores, stream=None) -> None:
+        h = hyper._c()
+        _check(_lib.cocodc_outer_step_received(self._h, ctypes.byref(h), int(M_total), _p(w_now), _p(w_snap),
+                                               int(now_stride), int(snap_stride), _p(snap_offset), _p(theta_g),
+                                               _p(momentum), _p(delta_sum), _p(delta_g_out), _p(ids), _p(n_ids),
+                                               int(t_p), int(t_l), _p(last_sync), _p(norms), _p(scores),
+                                               _stream(stream)), "cocodc_outer_step_received")
 
     def cocodc_merge(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                      theta_g_new, ids, n_ids, stream=None) -> None:

@@ -131,6 +131,15 @@ Variant pick_variant(int M) {
 }
 
 Variant pick_variant(int M, int mode, bool same) {
+  if (mode == MODE_FUSED_RECV) {   // one more stream per stage: staged up to four local workers
+    switch (M) {
+      case 1: return staged_variant<1, MODE_FUSED_RECV, false>();
+      case 2: return staged_variant<2, MODE_FUSED_RECV, false>();
+      case 3: return staged_variant<3, MODE_FUSED_RECV, false>();
+      case 4: return staged_variant<4, MODE_FUSED_RECV, false>();
+      default: return Variant{k_outer_generic<MODE_FUSED_RECV, false>, kThreads, 0u, false};
+    }
+  }
   if (mode == MODE_OUTER_ONLY) return pick_variant<MODE_OUTER_ONLY, false>(M);
   if (mode == MODE_MERGE_ONLY) return same ? pick_variant<MODE_MERGE_ONLY, true>(M) : pick_variant<MODE_MERGE_ONLY, false>(M);
   return same ? pick_variant<MODE_FUSED, true>(M) : pick_variant<MODE_FUSED, false>(M);
@@ -392,15 +401,25 @@ cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const 
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
-cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
-                                float* w_now, const float* w_snap,
-                                int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
-                                float* theta_g, float* momentum, float* delta_g_out,
-                                const int32_t* ids, const int32_t* n_ids,
-                                int64_t t_p, int64_t t_l, int64_t* last_sync,
-                                float* norms, float* scores, uint32_t stages, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// cocodc_outer_step and cocodc_outer_step_received: the latter passes the all-reduced sum of every
+// worker's pseudo-gradients (delta_sum) and the total worker count it is to be divided by.
+cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
+                              float* w_now, const float* w_snap,
+                              int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                              float* theta_g, float* momentum, float* delta_g_out,
+                              const int32_t* ids, const int32_t* n_ids,
+                              int64_t t_p, int64_t t_l, int64_t* last_sync,
+                              float* norms, float* scores, uint32_t stages, void* stream,
+                              const float* delta_sum, int32_t M_total) {
   cocodc_status s = check_hyper(c, h);
   if (s != COCODC_OK) return s;
+  const bool received = delta_sum != nullptr;
+  if (received && (M_total < h->M || stages != COCODC_STAGE_ALL)) return COCODC_ERR_INVALID_ARG;
+  if (received && !aligned16(delta_sum)) return COCODC_ERR_ALIGNMENT;
   if (!(stages & COCODC_STAGE_OUTER) || (stages & ~COCODC_STAGE_ALL)) return COCODC_ERR_INVALID_ARG;
   const bool do_merge = (stages & COCODC_STAGE_MERGE) != 0;
   const bool do_score = (stages & COCODC_STAGE_SCORE) != 0;
@@ -411,6 +430,7 @@ cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
   const long long N = c->N;
   if (snap_stride < (snap_offset ? 1 : N) || (do_merge && now_stride < N)) return COCODC_ERR_INVALID_ARG;
   const bool same = do_merge && (w_snap == w_now) && (snap_stride == now_stride) && (snap_offset == nullptr);
+  if (received && same) return COCODC_ERR_INVALID_ARG;   // the received sum belongs to recorded snapshots
   if (h->tau == 0 && h->comp_mode == COCODC_COMP_TAYLOR && do_merge && !same) return COCODC_ERR_INVALID_ARG;
   if (!aligned16(w_snap) || !aligned16(theta_g) || !aligned16(momentum) || (snap_stride & 3)) return COCODC_ERR_ALIGNMENT;
   if (do_merge && (!aligned16(w_now) || (now_stride & 3))) return COCODC_ERR_ALIGNMENT;
@@ -430,6 +450,11 @@ cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
       const Range rs = range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N));
       for (const Range& x : r) if (overlap(rs, x)) return COCODC_ERR_ALIAS;
     }
+    if (received) {   // delta_g_out may be the same buffer as delta_sum (updated in place), nothing else may
+      const Range rd = range_of(delta_sum, N);
+      for (const Range& x : r)
+        if (overlap(rd, x) && !(delta_g_out == delta_sum && x.lo == rd.lo)) return COCODC_ERR_ALIAS;
+    }
   }
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -441,13 +466,20 @@ cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
   A.theta_g = theta_g;
   A.momentum = momentum;
   A.delta_out = delta_g_out;
+  A.delta_in = delta_sum;
   A.plan = c->d_plan;
   A.hdr = c->d_hdr;
   A.partial = do_score ? c->d_partial : nullptr;
   fold_coefficients(h, same, &A);
+  if (received) {   // Eq. 1 divides the received sum by the number of workers that contributed to it
+    A.Mf = (float)M_total;
+    A.inv_M = 1.0f / (float)M_total;
+    A.M_pow2 = ((M_total & (M_total - 1)) == 0) ? 1 : 0;
+  }
   set_status_sink(c, &A);
   int grid = 0;
-  s = launch_outer(c, A, do_merge ? MODE_FUSED : MODE_OUTER_ONLY, same, ids, n_ids, snap_offset, st, &grid);
+  const int mode = received ? MODE_FUSED_RECV : (do_merge ? MODE_FUSED : MODE_OUTER_ONLY);
+  s = launch_outer(c, A, mode, same, ids, n_ids, snap_offset, st, &grid);
   if (s != COCODC_OK) return s;
   if (do_score) {
     k_finalize_scores<<<c->K, kFinalizeThreads, 0, st>>>(
@@ -457,6 +489,64 @@ cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
     if (cudaGetLastError() != cudaSuccess) return COCODC_ERR_CUDA;
   }
   return COCODC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
+                                float* w_now, const float* w_snap,
+                                int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                float* theta_g, float* momentum, float* delta_g_out,
+                                const int32_t* ids, const int32_t* n_ids,
+                                int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                float* norms, float* scores, uint32_t stages, void* stream) {
+  return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
+                         ids, n_ids, t_p, t_l, last_sync, norms, scores, stages, stream, nullptr, 0);
+}
+
+cocodc_status cocodc_outer_step_received(cocodc_ctx* c, const cocodc_hyper* h, int32_t M_total,
+                                         float* w_now, const float* w_snap,
+                                         int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                         float* theta_g, float* momentum, const float* delta_sum,
+                                         float* delta_g_out, const int32_t* ids, const int32_t* n_ids,
+                                         int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                         float* norms, float* scores, void* stream) {
+  if (!delta_sum) return COCODC_ERR_INVALID_ARG;
+  return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
+                         ids, n_ids, t_p, t_l, last_sync, norms, scores, COCODC_STAGE_ALL, stream, delta_sum, M_total);
+}
+
+cocodc_status cocodc_pseudo_gradient_sum(cocodc_ctx* c, const float* w_snap, int64_t snap_stride,
+                                         const int64_t* snap_offset, const float* theta_g, int32_t M,
+                                         float* sum_out, const int32_t* ids, const int32_t* n_ids, void* stream) {
+  if (!c || !w_snap || !theta_g || !sum_out || !ids || !n_ids) return COCODC_ERR_INVALID_ARG;
+  if (M < 1 || M > c->max_M) return COCODC_ERR_INVALID_ARG;
+  const long long N = c->N;
+  if (snap_stride < (snap_offset ? 1 : N)) return COCODC_ERR_INVALID_ARG;
+  if (!aligned16(w_snap) || !aligned16(theta_g) || !aligned16(sum_out) || (snap_stride & 3)) return COCODC_ERR_ALIGNMENT;
+  const Range ro = range_of(sum_out, N);
+  if (overlap(ro, range_of(theta_g, N)) ||
+      overlap(ro, range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N))))
+    return COCODC_ERR_ALIAS;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  void (*kernel)(const float*, long long, const float*, float*, int, const SegPlan*, const PlanHeader*);
+  switch (M) {
+    case 1: kernel = k_pseudo_sum<1>; break;
+    case 2: kernel = k_pseudo_sum<2>; break;
+    case 3: kernel = k_pseudo_sum<3>; break;
+    case 4: kernel = k_pseudo_sum<4>; break;
+    case 8: kernel = k_pseudo_sum<8>; break;
+    default: kernel = k_pseudo_sum<0>; break;
+  }
+  const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, snap_stride, kThreads, st);
+  if (s != COCODC_OK) return s;
+  kernel<<<grid, kThreads, 0, st>>>(w_snap, snap_stride, theta_g, sum_out, M, c->d_plan, c->d_hdr);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
 cocodc_status cocodc_merge(cocodc_ctx* c, const cocodc_hyper* h,

@@ -18,7 +18,9 @@ namespace cocodc {
 constexpr int kThreads = 256;        // consumer threads per CTA; a tile is kThreads lanes of 16 bytes
 constexpr int kTileElems = 4 * kThreads;
 
-enum : int { MODE_FUSED = 0, MODE_OUTER_ONLY = 1, MODE_MERGE_ONLY = 2 };
+// MODE_FUSED_RECV: as MODE_FUSED, but Eq. 1's sum over ALL workers arrives ready-made (delta_in, the result
+// of the all-reduce when every device holds only some of the workers) and is divided by the total count.
+enum : int { MODE_FUSED = 0, MODE_OUTER_ONLY = 1, MODE_MERGE_ONLY = 2, MODE_FUSED_RECV = 3 };
 
 struct OuterArgs {
   float* w_now;             // [M][now_stride]
@@ -28,6 +30,7 @@ struct OuterArgs {
   float* theta_g;           // in/out (MODE_MERGE_ONLY: read only, the new global state)
   float* momentum;          // in/out
   float* delta_out;         // optional
+  const float* delta_in;    // MODE_FUSED_RECV: received sum of all workers' pseudo-gradients
   const SegPlan* plan;
   const PlanHeader* hdr;
   double* partial;          // nullptr: no score accumulation
@@ -37,9 +40,9 @@ struct OuterArgs {
   float eta, mu;            // outer learning rate, Nesterov momentum
   float c1, c2;             // target = G + c1*d + c2*d*d*D
   float alpha, one_minus_alpha;
-  float Mf;                 // (float)M
-  float inv_M;              // 1/M, exact when M is a power of two
-  int M_pow2;               // 1 if M is a power of two
+  float Mf;                 // divisor of Eq. 1 as float: M, or the total worker count in MODE_FUSED_RECV
+  float inv_M;              // its reciprocal, exact when it is a power of two
+  int M_pow2;               // 1 if the divisor is a power of two
 };
 
 // ---- memory access helpers -------------------------------------------------
@@ -94,7 +97,11 @@ __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, 
     G = thg;
   } else {
     float sum = 0.f;
-    for (int m = 0; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(ld1(A.w_snap + m * A.snap_stride + snap_e), thg));
+    if (MODE == MODE_FUSED_RECV) {
+      sum = ld1(A.delta_in + e);
+    } else {
+      for (int m = 0; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(ld1(A.w_snap + m * A.snap_stride + snap_e), thg));
+    }
     const float Delta = mean_of_sum<0>(sum, A);
     float u_new;
     outer_update(Delta, thg, ld1(A.momentum + e), A, u_new, G);
@@ -113,7 +120,8 @@ __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, 
 }
 
 // Registers of one 16-byte lane (four consecutive elements) of every stream.
-// compute() works in place: afterwards thg holds G, u holds u', delta holds Delta and the merged
+// compute() works in place: afterwards thg holds G, u holds u', delta holds Delta (on entry, in
+// MODE_FUSED_RECV, the received sum) and the merged
 // local parameters sit in out(m) (= a[m], or b[m] when the snapshot is the current state).
 template <int M, int MODE, bool SAME>
 struct Lane {
@@ -132,6 +140,7 @@ struct Lane {
   __device__ __forceinline__ void load(const OuterArgs& A, long long e, long long snap_e) {
     thg = ld4(A.theta_g + e);
     if (MODE != MODE_MERGE_ONLY) u = ld4(A.momentum + e);
+    if (MODE == MODE_FUSED_RECV) delta = ld4(A.delta_in + e);
 #pragma unroll
     for (int m = 0; m < M; ++m) b[m] = ld4(A.w_snap + m * A.snap_stride + snap_e);
     if (kHasNow) {
@@ -146,10 +155,15 @@ struct Lane {
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         const float t = comp(thg, k);
-        float sum = __fsub_rn(comp(b[0], k), t);
+        float Delta;
+        if (MODE == MODE_FUSED_RECV) {
+          Delta = mean_of_sum<0>(comp(delta, k), A);      // delta holds the received sum on entry
+        } else {
+          float sum = __fsub_rn(comp(b[0], k), t);
 #pragma unroll
-        for (int m = 1; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(comp(b[m], k), t));
-        const float Delta = mean_of_sum<M>(sum, A);
+          for (int m = 1; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(comp(b[m], k), t));
+          Delta = mean_of_sum<M>(sum, A);
+        }
         float u_new, G;
         outer_update(Delta, t, comp(u, k), A, u_new, G);
         comp(delta, k) = Delta; comp(u, k) = u_new; comp(thg, k) = G;
@@ -244,6 +258,62 @@ k_outer_generic(const OuterArgs A) {
     ragged_lane<0, MODE, SAME>(A, tw.sp, tw.tile_start(tile) + 4LL * threadIdx.x, sa.acc);
   }
   if (A.partial) sa.finish(h.n_ids, A.partial);
+}
+
+// ---------------------------------------------------------------------------
+// S1 and the local part of S2 for the worker-per-device deployment (Section 2.1): the sum over this
+// device's M workers of theta^m_{p,t_p} - theta^g, written at the fragments' native offsets of
+// sum_out.  That buffer is what the all-reduce across devices then sums.
+// ---------------------------------------------------------------------------
+template <int M>   // 0: runtime worker count
+__global__ void __launch_bounds__(kThreads)
+k_pseudo_sum(const float* __restrict__ w_snap, long long snap_stride, const float* __restrict__ theta_g,
+             float* __restrict__ sum_out, int M_runtime, const SegPlan* __restrict__ plan,
+             const PlanHeader* __restrict__ hdr) {
+  const PlanHeader h = *hdr;
+  const int Mw = (M > 0) ? M : M_runtime;
+  TileWalker tw(plan, h.n_seg);
+  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+    tw.seek(tile);
+    const SegPlan& sp = tw.sp;
+    const long long e = tw.tile_start(tile) + 4LL * threadIdx.x;
+    const long long seg_end = sp.off + sp.len;
+    const long long shift = sp.snap_off - sp.off;
+    if (e >= seg_end) continue;
+    if (sp.vec_ok && e >= sp.off && e + 4 <= seg_end) {
+      const float4 t = ld4(theta_g + e);
+      float4 acc;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) comp(acc, k) = 0.f;
+#pragma unroll
+      for (int m = 0; m < (M > 0 ? M : 1); ++m) {
+        if (M > 0) {
+          const float4 b = ld4(w_snap + m * snap_stride + shift + e);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            comp(acc, k) = (m == 0) ? __fsub_rn(comp(b, k), comp(t, k))
+                                    : __fadd_rn(comp(acc, k), __fsub_rn(comp(b, k), comp(t, k)));
+        }
+      }
+      if (M == 0) {
+        for (int m = 0; m < Mw; ++m) {
+          const float4 b = ld4(w_snap + m * snap_stride + shift + e);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) comp(acc, k) = __fadd_rn(comp(acc, k), __fsub_rn(comp(b, k), comp(t, k)));
+        }
+      }
+      st4(sum_out + e, acc);
+    } else {
+      for (int k = 0; k < 4; ++k) {
+        const long long ee = e + k;
+        if (ee < sp.off || ee >= seg_end) continue;
+        const float t = ld1(theta_g + ee);
+        float acc = 0.f;
+        for (int m = 0; m < Mw; ++m) acc = __fadd_rn(acc, __fsub_rn(ld1(w_snap + m * snap_stride + shift + ee), t));
+        st1(sum_out + ee, acc);
+      }
+    }
+  }
 }
 
 // ---------------------------------------------------------------------------

@@ -83,7 +83,8 @@ __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 
 // ---- stage layout ----------------------------------------------------------------------------
-// Slots of kTileElems floats each: [recorded x nS][current x nN][global][momentum x nU][delta x nX].
+// Slots of kTileElems floats each: [recorded x nS][current x nN][global][momentum x nU][received sum x nR]
+// [delta x nX].
 // Outputs overwrite inputs in place; the mean pseudo-gradient, when asked for, goes to the first
 // recorded slot (its content is in registers by then), or to the extra slot when there is none.
 template <int M, int MODE, bool SAME>
@@ -91,20 +92,23 @@ struct StageLayout {
   static constexpr int nS = SAME ? 0 : M;
   static constexpr int nN = (MODE == MODE_OUTER_ONLY) ? 0 : M;
   static constexpr int nU = (MODE == MODE_MERGE_ONLY) ? 0 : 1;
+  static constexpr int nR = (MODE == MODE_FUSED_RECV) ? 1 : 0;     // received sum of pseudo-gradients
   static constexpr int nX = (SAME && MODE == MODE_FUSED) ? 1 : 0;
   static constexpr int kSnap = 0;
   static constexpr int kNow = nS;
   static constexpr int kGlobal = nS + nN;
   static constexpr int kMomentum = kGlobal + 1;
-  static constexpr int kDelta = (nX == 1) ? (kMomentum + nU) : kSnap;
-  static constexpr int kLoaded = nS + nN + 1 + nU;       // streams brought in by the producer
+  static constexpr int kDeltaIn = kMomentum + nU;
+  static constexpr int kDelta = (nR == 1 || nX == 1) ? (kMomentum + nU) : kSnap;
+  static constexpr int kLoaded = nS + nN + 1 + nU + nR;  // streams brought in by the producer
   static constexpr int kSlots = kLoaded + nX;
   static constexpr unsigned kStageBytes = kSlots * kTileBytes;
   static constexpr int kStagesRaw = (160 * 1024) / kStageBytes;
   static constexpr int kStages = kStagesRaw < 3 ? 3 : (kStagesRaw > kMaxStages ? kMaxStages : kStagesRaw);
   static constexpr unsigned kSmemBytes = kStages * kStageBytes;
   static_assert(kSmemBytes <= 227 * 1024, "stages do not fit in shared memory");
-  static_assert(SAME ? (MODE != MODE_OUTER_ONLY) : true, "zero-delay mode needs the merge");
+  static_assert(SAME ? (MODE != MODE_OUTER_ONLY && MODE != MODE_FUSED_RECV) : true,
+                "zero-delay mode needs the merge and local pseudo-gradients");
 };
 
 template <int M, int MODE, bool SAME>
@@ -158,6 +162,7 @@ k_outer_tma(const OuterArgs A) {
         bulk_load(smem_u32(st + (L::kNow + m) * kTileElems), A.w_now + m * A.now_stride + e0, kTileBytes, bar);
       bulk_load(smem_u32(st + L::kGlobal * kTileElems), A.theta_g + e0, kTileBytes, bar);
       if (L::nU) bulk_load(smem_u32(st + L::kMomentum * kTileElems), A.momentum + e0, kTileBytes, bar);
+      if (L::nR) bulk_load(smem_u32(st + L::kDeltaIn * kTileElems), A.delta_in + e0, kTileBytes, bar);
       ++k;
     }
     return;
@@ -195,6 +200,7 @@ k_outer_tma(const OuterArgs A) {
       auto slot = [&](int idx) -> float4& { return reinterpret_cast<float4*>(st + idx * kTileElems)[tid]; };
       ln.thg = slot(L::kGlobal);
       if (L::nU) ln.u = slot(L::kMomentum);
+      if (L::nR) ln.delta = slot(L::kDeltaIn);
       if (SAME) {
 #pragma unroll
         for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kNow + m);

@@ -1,0 +1,161 @@
+"""Worker-per-device deployment (Section 2.1): pseudo-gradient sums per device, all-reduced, then the
+completion from the received sum.  One GPU stands in for the devices one after the other (no kernel waits
+on another); the cross-rank part is torch.distributed's all-reduce."""
+
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import reference as orc
+from helpers import (GpuProblem, TOL_NORM, TOL_PARAM, assert_close, fragments_of, np_, orc_hyper)
+from test_gpu_parity_small import RAGGED
+
+pytestmark = pytest.mark.gpu
+
+
+def make(M, seed, **kw):
+    w = synth.small_workload(RAGGED, M=M, seed=seed, scale_kind="loguniform")
+    return GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3, **kw))
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 8])
+def test_two_phase_on_one_device_is_bit_identical_to_the_fused_step(M):
+    a = make(M, seed=200 + M)
+    b = make(M, seed=200 + M)
+    ids = [4, 0, 2, 1]
+    for prob in (a, b):
+        prob.set_ids(ids)
+    da = torch.zeros(a.w.N, device="cuda")
+    a.outer_step(6, 9, delta_out=da)
+    before = b.host_state()
+    sum_buf = torch.full((b.w.N,), 7.0, device="cuda")
+    bb = b.bufs
+    b.ctx.cocodc_pseudo_gradient_sum(bb.w_snap, bb.snap_stride, None, bb.theta_g, M, sum_buf, b.ids, b.n_ids)
+    # phase one against the oracle, and nothing outside the listed fragments written
+    exp = orc.pseudo_gradient_sum(fragments_of(b.w), M, before["w_snap"], before["theta_g"], ids)
+    got = np_(sum_buf)
+    touched = np.zeros(b.w.N, dtype=bool)
+    for p in ids:
+        assert_close(orc.gather_fragment(fragments_of(b.w), got, p), exp[p], TOL_PARAM, f"sum[{p}]")
+        for o, l in b.w.partition.fragments[p]:
+            touched[o:o + l] = True
+    assert np.all(got[~touched] == 7.0)
+    b.ctx.cocodc_outer_step_received(b.hyper(), M, bb.w_now, bb.w_snap, bb.now_stride, bb.snap_stride, None,
+                                     bb.theta_g, bb.momentum, sum_buf, sum_buf, b.ids, b.n_ids, 6, 9,
+                                     b.last_sync, b.norms, b.scores)
+    assert b.poll() == 0
+    for x, y in ((a.bufs.w_now, bb.w_now), (a.bufs.theta_g, bb.theta_g), (a.bufs.momentum, bb.momentum),
+                 (a.scores, b.scores), (a.norms, b.norms), (a.last_sync, b.last_sync)):
+        assert torch.equal(x, y)
+    t = torch.from_numpy(touched).cuda()
+    assert torch.equal(da[t], sum_buf[t])                      # delta written in place of the received sum
+
+
+def test_two_devices_with_two_workers_each():
+    """Workers 0-1 on one device, 2-3 on another, replicated outer state; the sums are added as an all-reduce would."""
+    full = make(4, seed=210, snap_layout="pool", pool_ids=[3, 1, 0])
+    w = full.w
+    frs = fragments_of(w)
+    ids = [1, 3, 0]
+    before = full.host_state()
+    devs = []
+    for d in range(2):
+        w2 = w.with_(M=2)
+        bufs = synth.DeviceBuffers(theta_g=full.bufs.theta_g.clone(), momentum=full.bufs.momentum.clone(),
+                                   w_now=full.bufs.w_now[2 * d:2 * d + 2].clone(),
+                                   w_snap=full.bufs.w_snap[2 * d:2 * d + 2].clone(),
+                                   snap_offset=full.bufs.snap_offset.clone(), scales=full.bufs.scales)
+        prob = GpuProblem(w2, bufs)
+        prob.set_ids(ids)
+        prob.sum = torch.zeros(w.N, device="cuda")
+        b = prob.bufs
+        prob.ctx.cocodc_pseudo_gradient_sum(b.w_snap, b.snap_stride, b.snap_offset, b.theta_g, 2, prob.sum,
+                                            prob.ids, prob.n_ids)
+        devs.append(prob)
+    total = devs[0].sum + devs[1].sum                         # what the all-reduce delivers to both
+    ohp = orc_hyper(w)
+    for d, prob in enumerate(devs):
+        b = prob.bufs
+        prob.ctx.cocodc_outer_step_received(prob.hyper(), 4, b.w_now, b.w_snap, b.now_stride, b.snap_stride,
+                                            b.snap_offset, b.theta_g, b.momentum, total, None, prob.ids, prob.n_ids,
+                                            8, 10, prob.last_sync, prob.norms, prob.scores)
+        assert prob.poll() == 0
+        res, new_last = orc.outer_step(frs, orc_hyper(w, M=2), before["w_now"][2 * d:2 * d + 2],
+                                       before["w_snap"][2 * d:2 * d + 2], before["theta_g"], before["momentum"], ids,
+                                       8, 10, before["last_sync"], snap_offset=before["snap_offset"],
+                                       recv_sum=np_(total), M_total=4)
+        after = prob.host_state()
+        for p in ids:
+            r = res[p]
+            assert_close(orc.gather_fragment(frs, after["theta_g"], p), r.theta_g, TOL_PARAM, "theta_g")
+            assert_close(orc.gather_fragment(frs, after["momentum"], p), r.momentum, TOL_PARAM, "momentum")
+            wn = orc.gather_fragment(frs, after["w_now"], p)
+            for m in range(2):
+                assert_close(wn[m], r.w_now[m], TOL_PARAM, f"w_now[{m}]")
+            assert abs(after["norms"][p] - r.norm) <= TOL_NORM * r.norm
+        assert np.array_equal(after["last_sync"], new_last)
+    # the replicated state stays identical on both devices, bit for bit
+    for k in ("theta_g", "momentum"):
+        assert torch.equal(getattr(devs[0].bufs, k), getattr(devs[1].bufs, k))
+    assert torch.equal(devs[0].scores, devs[1].scores)
+    # and agrees with all four workers stacked on one device
+    full.set_ids(ids)
+    full.outer_step(8, 10)
+    assert_close(np_(devs[0].bufs.theta_g), np_(full.bufs.theta_g).astype(np.float64), TOL_PARAM, "vs stacked")
+
+
+def test_received_mode_validation():
+    prob = make(2, seed=220)
+    b, B = prob.bufs, prob.B
+    prob.set_ids([0])
+    s = torch.zeros(prob.w.N, device="cuda")
+
+    def code(**kw):
+        a = dict(hyper=prob.hyper(), M_total=2, w_now=b.w_now, w_snap=b.w_snap, now_stride=b.now_stride,
+                 snap_stride=b.snap_stride, snap_offset=None, theta_g=b.theta_g, momentum=b.momentum, delta_sum=s,
+                 delta_g_out=None, ids=prob.ids, n_ids=prob.n_ids, t_p=1, t_l=2, last_sync=prob.last_sync,
+                 norms=prob.norms, scores=prob.scores)
+        a.update(kw)
+        with pytest.raises(B.CocodcError) as e:
+            prob.ctx.cocodc_outer_step_received(**a)
+        return e.value.code
+
+    assert code(M_total=1) == B.ERR_INVALID_ARG                 # fewer workers in total than held locally
+    assert code(delta_sum=None) == B.ERR_INVALID_ARG
+    assert code(delta_sum=b.theta_g) == B.ERR_ALIAS
+    assert code(w_snap=b.w_now, snap_stride=b.now_stride) == B.ERR_INVALID_ARG   # zero delay is not a two-phase case
+    assert code(delta_sum=s[1:]) == B.ERR_ALIGNMENT
+    with pytest.raises(B.CocodcError) as e:
+        prob.ctx.cocodc_pseudo_gradient_sum(b.w_snap, b.snap_stride, None, b.theta_g, 2, b.theta_g, prob.ids, prob.n_ids)
+    assert e.value.code == B.ERR_ALIAS
+
+
+def test_complete_fragments_through_nccl_world_of_one():
+    """The glue (kernel, all-reduce, kernel) on a one-rank NCCL group equals the fused step."""
+    import torch.distributed as dist
+    from paper_2504_17672_b200 import distributed as D
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        a, b = make(4, seed=230), make(4, seed=230)
+        ids = [2, 4, 0]
+        for prob in (a, b):
+            prob.set_ids(ids)
+        a.outer_step(3, 7)
+        bb = b.bufs
+        sum_buf = torch.zeros(b.w.N, device="cuda")
+        D.complete_fragments(b.ctx, b.hyper(), 4, fragments_of(b.w), ids, b.ids, b.n_ids, bb.w_now, bb.w_snap, None,
+                             bb.theta_g, bb.momentum, sum_buf, 3, 7, b.last_sync, b.norms, b.scores)
+        assert b.poll() == 0
+        for x, y in ((a.bufs.w_now, bb.w_now), (a.bufs.theta_g, bb.theta_g), (a.bufs.momentum, bb.momentum),
+                     (a.scores, b.scores)):
+            assert torch.equal(x, y)
+    finally:
+        dist.destroy_process_group()

@@ -50,6 +50,18 @@ def _worker(rank, world, port, out):
         allsel = [None] * world
         dist.all_gather_object(allsel, sel)
         assert allsel[0] == allsel[1] == [1]
+        # worker-per-device deployment: the listed fragments' ranges of the per-rank sums are all-reduced in place
+        from paper_2504_17672_b200 import distributed as D
+        frs = [[(3, 100), (700, 57)], [(103, 250)], [(400, 299)]]
+        ranges = D.fragment_ranges(frs, [2, 0])
+        assert ranges == [(400, 299), (3, 100), (700, 57)]
+        buf = torch.full((1000,), float(rank + 1))
+        calls = D.allreduce_ranges(buf, ranges, bucket_elems=128)
+        assert calls == 3 + 1 + 1
+        exp = torch.full((1000,), float(rank + 1))
+        for o, l in ranges:
+            exp[o:o + l] = 3.0                                    # 1 + 2 summed over the two ranks
+        assert torch.equal(buf, exp)
         out.put((rank, "ok"))
     except Exception as e:  # pragma: no cover
         out.put((rank, repr(e)))
