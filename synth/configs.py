@@ -174,12 +174,26 @@ def _llama_3b() -> Workload:
         notes="Llama-3B-shaped: 26 layer fragments + one embeddings fragment")
 
 
+def _paper_150m() -> Workload:
+    """The shape of the paper's own experiment (Section 4.1): a LLaMA-style decoder of 12 layers and about
+    150 M parameters cut into 4 shards of 3 layers in a strided pattern, M = 4, H = 100, tau = 5, lambda = 0.5,
+    one fragment per decision (Algorithm 2).  Width 1024 / FFN 2816 give 12.85 M parameters per layer."""
+    layers, shards = 12, 4
+    layer, _, _ = _llama_shape(layers, 1024, 2816, 32000)
+    frags = [tuple((l * layer, layer) for l in range(k, layers, shards)) for k in range(shards)]
+    part = Partition(N=layers * layer, fragments=tuple(frags))
+    return Workload(
+        name="paper_150m", partition=part, M=4, tau=5, H=100, lam=0.5, budget_kind="count", budget=1, seed=5,
+        scale_kind="loguniform", notes="12 layers in 4 strided shards of 3 layers (Section 4.1)")
+
+
 _BUILDERS = {
     "tiny": _tiny,
     "gpt2_small": _gpt2_small,
     "llama_1b": _llama_1b,
     "sweep_1b": _sweep_1b,
     "llama_3b": _llama_3b,
+    "paper_150m": _paper_150m,
 }
 WORKLOAD_NAMES = tuple(_BUILDERS)
 

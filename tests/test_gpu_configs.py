@@ -71,6 +71,24 @@ def test_gpt2_small_full_parity():
     check_step_against_oracle(prob, before, ids, 20, 20 + w.tau, orc_hyper(w))
 
 
+def test_paper_150m_strided_shards_full_parity():
+    """The paper's own setting (Section 4.1): 4 strided shards of 3 layers, one shard per completion."""
+    w = synth.get_workload("paper_150m")
+    prob = GpuProblem(w, synth.generate(w, "cuda"))
+    t = 0
+    seen = []
+    for rnd in range(2):
+        t += 12
+        before = prob.host_state()
+        prob.select(t)
+        ids = np_(prob.ids)[:int(prob.n_ids.item())].tolist()
+        prob.outer_step(t, t + w.tau)
+        assert prob.poll() == 0
+        check_step_against_oracle(prob, before, ids, t, t + w.tau, orc_hyper(w))
+        seen += ids
+    assert seen == [0, 1]                     # never-synced shards first, in index order
+
+
 def _sampled_round(prob, ids, t_p, t_l, ohp, full_norm=2, same=False):
     w = prob.w
     ids = [int(p) for p in ids]

@@ -13,6 +13,7 @@ def test_workload_shapes():
         "llama_1b": (953_223_168, 16, 4),
         "sweep_1b": (953_223_168, 32, 4),
         "llama_3b": (3_426_473_600, 27, 4),
+        "paper_150m": (154_165_248, 4, 4),
     }
     for name, (N, K, M) in expect.items():
         w = synth.get_workload(name)
