@@ -1,23 +1,22 @@
-// The fused outer-step kernel for the instantiated worker counts: worker tiles are staged through
-// shared memory by the TMA unit (1-D bulk asynchronous copies), in both directions.
+// The fused outer-step kernel for the instantiated worker counts: the inputs of every tile are brought
+// into shared memory by the TMA unit (1-D bulk asynchronous copies); the outputs leave from registers.
 //
 // One CTA per SM: warps 0-7 compute, warp 8 holds the producer thread.  A stage is one tile
-// (1024 elements = 4 KB) of every stream the mode reads; S stages keep about 160 KB of loads in
-// flight per SM, which plain register loads cannot hold.  Per tile:
-//   producer : waits until the stage is free, arms the stage's "full" barrier with the byte count,
-//              issues one bulk copy global->shared per stream;
-//   consumers: wait on "full", read their 16-byte lane of every stream from shared memory, do the
-//              arithmetic of outer.cuh in registers, write the outputs IN PLACE in the stage,
-//              fence towards the async proxy, barrier;
-//   thread 0 : issues one bulk copy shared->global per output stream, commits them as a group,
-//              waits until the PREVIOUS tile's group has finished reading its stage and hands that
-//              stage back to the producer ("empty" barrier).
+// (1024 elements = 4 KB) of every stream the mode reads.  Per tile:
+//   producer : waits until the stage is free ("empty" barrier, one arrival per consumer thread), arms the
+//              stage's "full" barrier with the byte count, issues one bulk copy global->shared per stream;
+//   consumers: wait on "full", read their 16-byte lane of every stream from shared memory into registers,
+//              arrive on "empty" at once (the stage can be refilled while they compute), do the arithmetic
+//              of outer.cuh, and write their outputs with streaming 16-byte stores.
+// How far the producer runs ahead is the tuning knob: measured on B200, bandwidth peaks at 16-20
+// outstanding 4 KB copies per SM (64-80 KB in flight) and falls by 5-8 % at twice that, so the ring has
+// only as many stages as that takes (2 at M = 4), not as many as shared memory would hold.
 // Tiles that are ragged or whose snapshot placement is not 16-byte compatible never enter the
 // pipeline: the consumers process them straight from global memory (ragged_lane); producer and
 // consumers agree on which tiles those are from the plan alone.
 //
-// Every wait is bounded.  When one runs out the kernel records COCODC_ERR_TIMEOUT, all consumers
-// leave the loop in the same iteration, thread 0 drains its own stores, and the CTA returns.
+// Every wait is bounded.  When one runs out the thread records COCODC_ERR_TIMEOUT, raises a flag the
+// others poll, and leaves; no thread waits on a barrier another thread could have abandoned.
 // Only this GPU's memory is read; no cluster multicast is used.
 #pragma once
 
@@ -83,28 +82,23 @@ __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy
 __device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 
 // ---- stage layout ----------------------------------------------------------------------------
-// Slots of kTileElems floats each: [recorded x nS][current x nN][global][momentum x nU][received sum x nR]
-// [delta x nX].
-// Outputs overwrite inputs in place; the mean pseudo-gradient, when asked for, goes to the first
-// recorded slot (its content is in registers by then), or to the extra slot when there is none.
+// Slots of kTileElems floats each: [recorded x nS][current x nN][global][momentum x nU][received sum x nR].
 template <int M, int MODE, bool SAME>
 struct StageLayout {
   static constexpr int nS = SAME ? 0 : M;
   static constexpr int nN = (MODE == MODE_OUTER_ONLY) ? 0 : M;
   static constexpr int nU = (MODE == MODE_MERGE_ONLY) ? 0 : 1;
   static constexpr int nR = (MODE == MODE_FUSED_RECV) ? 1 : 0;     // received sum of pseudo-gradients
-  static constexpr int nX = (SAME && MODE == MODE_FUSED) ? 1 : 0;
   static constexpr int kSnap = 0;
   static constexpr int kNow = nS;
   static constexpr int kGlobal = nS + nN;
   static constexpr int kMomentum = kGlobal + 1;
   static constexpr int kDeltaIn = kMomentum + nU;
-  static constexpr int kDelta = (nR == 1 || nX == 1) ? (kMomentum + nU) : kSnap;
   static constexpr int kLoaded = nS + nN + 1 + nU + nR;  // streams brought in by the producer
-  static constexpr int kSlots = kLoaded + nX;
-  static constexpr unsigned kStageBytes = kSlots * kTileBytes;
-  static constexpr int kStagesRaw = (160 * 1024) / kStageBytes;
-  static constexpr int kStages = kStagesRaw < 3 ? 3 : (kStagesRaw > kMaxStages ? kMaxStages : kStagesRaw);
+  static constexpr unsigned kStageBytes = kLoaded * kTileBytes;
+  // about 72 KB of copies in flight (see the note at the top), never fewer than two stages
+  static constexpr int kStagesRaw = (72 * 1024) / kStageBytes;
+  static constexpr int kStages = kStagesRaw < 2 ? 2 : (kStagesRaw > kMaxStages ? kMaxStages : kStagesRaw);
   static constexpr unsigned kSmemBytes = kStages * kStageBytes;
   static_assert(kSmemBytes <= 227 * 1024, "stages do not fit in shared memory");
   static_assert(SAME ? (MODE != MODE_OUTER_ONLY && MODE != MODE_FUSED_RECV) : true,
@@ -127,7 +121,7 @@ k_outer_tma(const OuterArgs A) {
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
-      mbar_init(smem_u32(&empty_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), kThreads);   // every consumer thread releases its own lane
     }
     s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -151,7 +145,7 @@ k_outer_tma(const OuterArgs A) {
       }
       if (s_fail) return;
       const unsigned bar = smem_u32(&full_bar[s]);
-      float* st = stages + (size_t)s * L::kSlots * kTileElems;
+      float* st = stages + (size_t)s * L::kLoaded * kTileElems;
       const long long snap_e0 = e0 + (tw.sp.snap_off - tw.sp.off);
       mbar_expect_tx(bar, L::kLoaded * kTileBytes);
 #pragma unroll
@@ -171,7 +165,6 @@ k_outer_tma(const OuterArgs A) {
   // ------------------------------------------------------------------ consumers
   SlotAccumulator sa(kThreads / 32);
   TileWalker tw(A.plan, h.n_seg);
-  const unsigned long long store_policy = l2_evict_first_policy();
   int k = 0;           // staged tiles consumed so far
   bool failed = false;
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
@@ -182,70 +175,38 @@ k_outer_tma(const OuterArgs A) {
       continue;
     }
     const int s = k % S;
-    if (!mbar_wait_bounded(smem_u32(&full_bar[s]), (k / S) & 1)) {
+    // the verdict is taken per warp, so that a warp never splits around the full-warp shuffles of the
+    // score accumulation
+    const bool landed = !s_fail && mbar_wait_bounded(smem_u32(&full_bar[s]), (k / S) & 1);
+    if (!__all_sync(0xffffffffu, landed)) {
       record_status(A.status, A.err_timeout);
       s_fail = 1;
-    }
-    consumer_barrier();
-    if (s_fail) {                             // uniform: every consumer sees the flag after the barrier
-      // give the loads that were issued for this stage one more bounded chance to land before the
-      // CTA gives its shared memory back
-      if (tid == 0) mbar_wait_bounded(smem_u32(&full_bar[s]), (k / S) & 1);
       failed = true;
       break;
     }
-    float* st = stages + (size_t)s * L::kSlots * kTileElems;
-    {
-      Lane<M, MODE, SAME> ln;
-      auto slot = [&](int idx) -> float4& { return reinterpret_cast<float4*>(st + idx * kTileElems)[tid]; };
-      ln.thg = slot(L::kGlobal);
-      if (L::nU) ln.u = slot(L::kMomentum);
-      if (L::nR) ln.delta = slot(L::kDeltaIn);
-      if (SAME) {
+    const float* st = stages + (size_t)s * L::kLoaded * kTileElems;
+    Lane<M, MODE, SAME> ln;
+    auto slot = [&](int idx) -> const float4& { return reinterpret_cast<const float4*>(st + idx * kTileElems)[tid]; };
+    ln.thg = slot(L::kGlobal);
+    if (L::nU) ln.u = slot(L::kMomentum);
+    if (L::nR) ln.delta = slot(L::kDeltaIn);
+    if (SAME) {
 #pragma unroll
-        for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kNow + m);
-      } else {
+      for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kNow + m);
+    } else {
 #pragma unroll
-        for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kSnap + m);
-        if (L::nN) {
+      for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kSnap + m);
+      if (L::nN) {
 #pragma unroll
-          for (int m = 0; m < M; ++m) ln.a[m] = slot(L::kNow + m);
-        }
-      }
-      ln.compute(A, sa.acc);
-      if (MODE != MODE_MERGE_ONLY) {
-        slot(L::kGlobal) = ln.thg;
-        slot(L::kMomentum) = ln.u;
-        if (A.delta_out) slot(L::kDelta) = ln.delta;
-      }
-      if (MODE != MODE_OUTER_ONLY) {
-#pragma unroll
-        for (int m = 0; m < M; ++m) slot(L::kNow + m) = ln.out(m);
+        for (int m = 0; m < M; ++m) ln.a[m] = slot(L::kNow + m);
       }
     }
-    fence_async_shared();     // make the generic-proxy writes visible to the bulk stores
-    consumer_barrier();
-    if (tid == 0) {
-      if (MODE != MODE_OUTER_ONLY) {
-#pragma unroll
-        for (int m = 0; m < M; ++m)
-          bulk_store(A.w_now + m * A.now_stride + e0, smem_u32(st + (L::kNow + m) * kTileElems), kTileBytes, store_policy);
-      }
-      if (MODE != MODE_MERGE_ONLY) {
-        bulk_store(A.theta_g + e0, smem_u32(st + L::kGlobal * kTileElems), kTileBytes, store_policy);
-        bulk_store(A.momentum + e0, smem_u32(st + L::kMomentum * kTileElems), kTileBytes, store_policy);
-        if (A.delta_out) bulk_store(A.delta_out + e0, smem_u32(st + L::kDelta * kTileElems), kTileBytes, store_policy);
-      }
-      bulk_commit();
-      if (k >= 1) {   // the previous staged tile's stores have read their stage: release it
-        bulk_wait_read_all_but_one();
-        mbar_arrive(smem_u32(&empty_bar[(k - 1) % S]));
-      }
-    }
+    mbar_arrive(smem_u32(&empty_bar[s]));   // this thread's lane is in registers: its share of the stage is free
+    ln.compute(A, sa.acc);
+    ln.store(A, e0 + 4LL * tid);
     ++k;
   }
-  if (tid == 0) bulk_wait_all();     // this thread's stores are complete before the CTA exits
-  if (failed) return;
+  if (failed) return;     // warp-uniform by construction
   if (A.partial) sa.finish(h.n_ids, A.partial);
 }
 
@@ -258,15 +219,15 @@ namespace cocodc {
 //
 // One thread per CTA drives the TMA unit: bulk load of a 16 KB chunk (one tile of one worker) into
 // a shared-memory stage, and, once it has landed, a bulk store of the same stage to its place in
-// w_snap.  kSnapStages stages with up to kSnapDepth loads in flight keep about 80 KB of reads and
-// as much of writes outstanding per SM.  Warps 1-7 meanwhile copy the ragged tiles (segment
+// w_snap.  kSnapStages stages with up to kSnapDepth loads in flight keep 48 KB of reads and as much of
+// writes outstanding per SM (measured optimum: 48-64 KB; 80 KB and more lose 5 %).  Warps 1-7 meanwhile copy the ragged tiles (segment
 // edges, snapshot placements that are not 16-byte compatible) with ordinary loads and stores.
 // ---------------------------------------------------------------------------------------------
 constexpr int kSnapU = 4;                                      // lanes per thread and tile
 constexpr int kSnapTileElems = kTileElems * kSnapU;            // 4096 elements = 16 KB per worker
 constexpr unsigned kSnapChunkBytes = kSnapTileElems * sizeof(float);
-constexpr int kSnapStages = 10;
-constexpr int kSnapDepth = 5;                                  // loads in flight before the oldest is stored
+constexpr int kSnapStages = 6;
+constexpr int kSnapDepth = 3;                                  // loads in flight before the oldest is stored
 constexpr unsigned kSnapSmemBytes = kSnapStages * kSnapChunkBytes;
 
 template <int N> __device__ __forceinline__ void bulk_wait_read_n() {
