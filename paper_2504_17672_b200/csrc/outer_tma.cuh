@@ -217,17 +217,17 @@ namespace cocodc {
 // ---------------------------------------------------------------------------------------------
 // S0 as a pure DMA job: copy the listed fragments of every worker from w_now into w_snap.
 //
-// One thread per CTA drives the TMA unit: bulk load of a 16 KB chunk (one tile of one worker) into
+// One thread per CTA drives the TMA unit: bulk load of a 32 KB chunk (one tile of one worker) into
 // a shared-memory stage, and, once it has landed, a bulk store of the same stage to its place in
-// w_snap.  kSnapStages stages with up to kSnapDepth loads in flight keep 48 KB of reads and as much of
+// w_snap.  kSnapStages stages with up to kSnapDepth loads in flight keep 64 KB of reads and as much of
 // writes outstanding per SM (measured optimum: 48-64 KB; 80 KB and more lose 5 %).  Warps 1-7 meanwhile copy the ragged tiles (segment
 // edges, snapshot placements that are not 16-byte compatible) with ordinary loads and stores.
 // ---------------------------------------------------------------------------------------------
-constexpr int kSnapU = 4;                                      // lanes per thread and tile
-constexpr int kSnapTileElems = kTileElems * kSnapU;            // 4096 elements = 16 KB per worker
+constexpr int kSnapU = 8;                                      // lanes per thread and tile
+constexpr int kSnapTileElems = kTileElems * kSnapU;            // 8192 elements = 32 KB per worker
 constexpr unsigned kSnapChunkBytes = kSnapTileElems * sizeof(float);
-constexpr int kSnapStages = 6;
-constexpr int kSnapDepth = 3;                                  // loads in flight before the oldest is stored
+constexpr int kSnapStages = 4;
+constexpr int kSnapDepth = 2;                                  // loads in flight before the oldest is stored
 constexpr unsigned kSnapSmemBytes = kSnapStages * kSnapChunkBytes;
 
 template <int N> __device__ __forceinline__ void bulk_wait_read_n() {
