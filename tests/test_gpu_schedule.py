@@ -108,3 +108,17 @@ def test_round_driver_in_the_papers_setting():
     counts = np.bincount([ids[0] for _, ids in log["initiated"]], minlength=4)
     assert counts.min() >= 2 and counts.sum() == len(starts)
     assert log["worst"] <= TOL_PARAM
+
+
+@pytest.mark.parametrize("variant,lam,tau", [("diloco", 0.0, 0), ("streaming_diloco", 0.0, 4), ("cocodc", 0.0, 4),
+                                             ("cocodc", 0.5, 4), ("cocodc", 0.5, 8)])
+def test_toy_training_converges_under_every_variant(variant, lam, tau):
+    """Workers with different quadratic objectives, synchronised through the library under a delay, reach the
+    optimum of the mean objective; the run is reproducible from its seed."""
+    from paper_2504_17672_b200.toy import run_toy
+    r = run_toy(variant, lam=lam, tau=tau if variant != "diloco" else 4, steps=300, seed=3)
+    again = run_toy(variant, lam=lam, tau=tau if variant != "diloco" else 4, steps=300, seed=3)
+    assert r.losses == again.losses
+    assert r.syncs >= 300 // 20
+    start, final = r.losses[0][1], r.final
+    assert np.isfinite(final) and final < 0.02 * start, (start, final)
