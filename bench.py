@@ -373,6 +373,95 @@ def run_sweep(args):
                       "min": min(g), "median": statistics.median(g), "max": max(g), "variants": variants}))
 
 
+def run_micro(args):
+    """Every streaming entry point on its own, on the llama_1b buffers: algorithmic GB/s from CUDA events.
+
+    Rows: the fused step and its modes, the unfused halves, snapshot, stand-alone scores (with and without a
+    context), and the two calls of the worker-per-device deployment."""
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
+    from paper_2504_17672_b200 import binding as B
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    w = synth.get_workload(args.workload)
+    bufs = synth.generate(w, device)                 # full-size snapshot buffer: every fragment has a snapshot
+    ptr, off, ln = w.partition.csr()
+    ctx = B.Context(w.N, ptr, off, ln, w.M, device=0)
+    K, M = w.K, w.M
+    sizes = w.partition.frag_sizes
+    chosen = [int(p) for p in np.argsort(-sizes, kind="stable")[:max(1, min(4, K))]]
+    n = int(sizes[chosen].sum())
+    ids = torch.tensor(chosen + [-1] * (K - len(chosen)), dtype=torch.int32, device=device)
+    n_ids = torch.tensor([len(chosen)], dtype=torch.int32, device=device)
+    scores = torch.zeros(K, device=device)
+    norms = torch.zeros(K, device=device)
+    last_sync = torch.zeros(K, dtype=torch.int64, device=device)
+    scratch = torch.zeros(w.N, device=device)
+    hp = B.Hyper(M=M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam, alpha=w.alpha)
+    b = bufs
+    peak, peak_kind = read_peaks()
+    t = [0]
+
+    def outer(stages=7, delta=None, snap=None):
+        t[0] += w.tau
+        s = b.w_snap if snap is None else snap
+        ctx.cocodc_outer_step(hp, b.w_now, s, b.now_stride, s.stride(0), None, b.theta_g, b.momentum, delta,
+                              ids, n_ids, t[0], t[0] + w.tau, last_sync, norms, scores, stages)
+
+    hp0 = B.Hyper(M=M, H=w.H, tau=0, outer_lr=w.outer_lr, momentum=w.momentum, lam=0.0, alpha=1.0,
+                  comp_mode=B.COMP_NONE)
+
+    def zero_delay():
+        t[0] += w.tau
+        ctx.cocodc_outer_step(hp0, b.w_now, b.w_now, b.now_stride, b.now_stride, None, b.theta_g, b.momentum, None,
+                              ids, n_ids, t[0], t[0], last_sync, norms, scores, 7)
+
+    def received():
+        t[0] += w.tau
+        ctx.cocodc_outer_step_received(hp, M, b.w_now, b.w_snap, b.now_stride, b.snap_stride, None, b.theta_g,
+                                       b.momentum, scratch, None, ids, n_ids, t[0], t[0] + w.tau, last_sync,
+                                       norms, scores)
+
+    rows = [
+        ("cocodc_outer_step, all stages (S1-S6)", 12 * M + 16, n, lambda: outer()),
+        ("cocodc_outer_step + delta_g_out", 12 * M + 20, n, lambda: outer(delta=scratch)),
+        ("cocodc_outer_step, zero delay (w_snap == w_now)", 8 * M + 16, n, zero_delay),
+        ("cocodc_outer_step, OUTER|SCORE only (S1-S3, S6)", 4 * M + 16, n, lambda: outer(stages=5)),
+        ("cocodc_merge (S4-S5)", 12 * M + 4, n,
+         lambda: ctx.cocodc_merge(hp, b.w_now, b.w_snap, b.now_stride, b.snap_stride, None, b.theta_g, ids, n_ids)),
+        ("cocodc_snapshot (S0)", 8 * M, n,
+         lambda: ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, None, M, ids, n_ids)),
+        ("cocodc_pseudo_gradient_sum", 4 * M + 8, n,
+         lambda: ctx.cocodc_pseudo_gradient_sum(b.w_snap, b.snap_stride, None, b.theta_g, M, scratch, ids, n_ids)),
+        ("cocodc_outer_step_received", 12 * M + 20, n, received),
+        ("cocodc_fragment_scores (all fragments)", 4, w.N,
+         lambda: ctx.cocodc_fragment_scores(b.theta_g, None, norms, scores)),
+    ]
+    if K <= B.NOALLOC_MAX_K and len(off) <= B.NOALLOC_MAX_SEGMENTS:
+        rows.append(("cocodc_fragment_scores_noalloc (all fragments)", 4, w.N,
+                     lambda: B.cocodc_fragment_scores_noalloc(w.N, ptr, off, ln, b.theta_g, None, norms, scores)))
+    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = max(5, args.steps // 5)
+    out = []
+    for name, bpp, params, fn in rows:
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize(device)
+        ev_a.record()
+        for _ in range(reps):
+            fn()
+        ev_b.record()
+        torch.cuda.synchronize(device)
+        ms = ev_a.elapsed_time(ev_b) / reps
+        gbs = params * bpp / ms / 1e6
+        out.append({"entry": name, "bytes_per_param": bpp, "params": params, "ms": ms, "gbs": gbs,
+                    "frac_of_peak": gbs / peak})
+    status = ctx.cocodc_poll_status()
+    print(json.dumps({"metric": "entry_point_gbs", "workload": w.name, "unit": "GB/s", "peak": peak,
+                      "peak_kind": f"of {peak_kind}", "launches_per_entry": reps, "fragments": chosen,
+                      "status": int(status), "entries": out}))
+
+
 def kernel_source_sha() -> str:
     import hashlib
     h = hashlib.sha256()
@@ -561,6 +650,7 @@ def main():
     ap.add_argument("--reference-sample", type=int, default=8_000_000)
     ap.add_argument("--variant", choices=["cocodc", "streaming_diloco", "diloco"], default="cocodc",
                     help="which method's arithmetic the step runs (the baselines are modes of the same kernels)")
+    ap.add_argument("--micro", action="store_true", help="time every streaming entry point on its own")
     ap.add_argument("--sweep", action="store_true", help="time the 48 variants of the 1B compensation sweep")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
@@ -569,6 +659,8 @@ def main():
         run_reference(args)
     elif args.sweep:
         run_sweep(args)
+    elif args.micro:
+        run_micro(args)
     else:
         run_ours(args)
 
