@@ -307,3 +307,52 @@ def test_bounded_wait_runs_out_and_leaves_the_context_usable():
     prob.outer_step(2, 4)
     assert prob.poll() == 0
     check_step_against_oracle(prob, before, ids, 2, 4, orc_hyper(prob.w))
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_partitions_layouts_and_modes(seed):
+    """Randomised sweep: fragment tables with gaps, odd offsets and several segments, random worker counts,
+    id lists, snapshot layouts (plain / packed pool with arbitrary offsets), sign modes, mixing factors."""
+    rng = np.random.default_rng(1000 + seed)
+    M = int(rng.choice([1, 2, 3, 4, 4, 4, 6, 8]))
+    K = int(rng.integers(1, 7))
+    pos, frs = int(rng.integers(0, 9)), []
+    for p in range(K):
+        segs = []
+        for _ in range(int(rng.integers(1, 4))):
+            ln = int(rng.choice([1, 3, 4, 5, 1023, 1024, 1025, 2048, 4099, 9000, 20_000]))
+            segs.append((pos, ln))
+            pos += ln + int(rng.choice([0, 0, 1, 3, 4, 17]))
+        frs.append(segs)
+    N = pos + (-pos) % 4 + 4
+    w = synth.small_workload((N, frs), M=M, seed=seed, scale_kind="loguniform", tau=int(rng.integers(1, 9)),
+                             lam=float(rng.choice([0.0, 0.5, 1.0])))
+    ids = [int(p) for p in rng.permutation(K)[:int(rng.integers(1, K + 1))]]
+    layout = rng.choice(["full", "pool", "pool_odd"])
+    kw = {}
+    if layout != "full":
+        kw = dict(snap_layout="pool", pool_ids=ids)
+        if layout == "pool_odd":
+            offs, cur = {}, int(rng.integers(0, 4))
+            for p in ids:
+                offs[p] = cur
+                cur += w.partition.frag_size(p) + int(rng.integers(0, 6))
+            kw.update(pool_offsets=offs, pool_len=cur + 8 - cur % 4)
+    prob = GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3, **kw))
+    prob.set_ids(ids)
+    sign = int(rng.integers(0, 3))
+    alpha = float(rng.choice([1.0, 1.0, 0.5]))
+    comp = int(rng.choice([1, 1, 0]))
+    delta = torch.full((w.N,), 3.0, device="cuda") if rng.random() < 0.5 else None
+    before = prob.host_state()
+    t_p = int(rng.integers(1, 50))
+    prob.outer_step(t_p, t_p + w.tau, hyper=prob.hyper(sign_mode=sign, alpha=alpha, comp_mode=comp), delta_out=delta)
+    assert prob.poll() == 0
+    check_step_against_oracle(prob, before, ids, t_p, t_p + w.tau,
+                              orc_hyper(w, sign_mode=sign, alpha=alpha, comp_mode=comp), delta_out=delta)
+    # S0 on the same table and layout
+    snap_before = prob.host_state()
+    prob.snapshot()
+    assert prob.poll() == 0
+    exp = orc.snapshot(fragments_of(w), snap_before["w_now"], ids, M, snap_before["snap_offset"], snap_before["w_snap"])
+    assert np.array_equal(np_(prob.bufs.w_snap), exp)
