@@ -12,7 +12,7 @@ and integer-valued: walking a fragment's segments, Eq. 10's score, Algorithm
 Parity pins (tests/test_oracle_pins.py): closed forms and worked values for
 every function here.  Unpinned by the paper itself: which of the three sign
 readings of Eq. 4/Eq. 7 the authors ran, and the outer optimizer's exact
-formula and settings (the paper only says "e.g. SGD with Nesterov momentum");
+formula and settings (the paper names SGD with Nesterov momentum only as an example of OuterOptim);
 the Nesterov reading is pinned to the torch CPU optimizer of that name.
 """
 

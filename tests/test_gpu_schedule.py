@@ -34,7 +34,7 @@ def test_round_driver_in_the_papers_setting():
     hyper = B.Hyper(M=w.M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam, alpha=1.0)
     drv = RoundDriver(ctx, hyper, bufs.w_now, bufs.theta_g, bufs.momentum, w.partition.frag_sizes,
                       gamma=0.4, Tc=0.2, Ts=1.0, budget_kind=B.BUDGET_COUNT, budget=1)
-    assert (drv.N_sync, drv.h) == (8, 12)                       # "8 synchronizations per H steps"
+    assert (drv.N_sync, drv.h) == (8, 12)                       # Section 4.1: eight synchronisations per H steps with these settings
     ohp = orc.Hyper(M=w.M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam, alpha=1.0)
     log = {"initiated": [], "completed": [], "pre": None, "worst": 0.0}
 
