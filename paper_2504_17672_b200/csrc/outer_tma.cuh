@@ -93,8 +93,10 @@ struct StageLayout {
   static constexpr int kDeltaIn = kMomentum + nU;
   static constexpr int kLoaded = nS + nN + 1 + nU + nR;  // streams brought in by the producer
   static constexpr unsigned kStageBytes = kLoaded * kTileBytes;
-  // about 72 KB of copies in flight (see the note at the top), never fewer than two stages
-  static constexpr int kStagesRaw = (72 * 1024) / kStageBytes;
+  // about 72 KB of copies in flight (see the note at the top), never fewer than two stages; the
+  // read-heavy OUTER_ONLY mode (3 reads per write) measures best one stage deeper
+  static constexpr int kInFlightBytes = (MODE == MODE_OUTER_ONLY ? 96 : 72) * 1024;
+  static constexpr int kStagesRaw = kInFlightBytes / kStageBytes;
   static constexpr int kStages = kStagesRaw < 2 ? 2 : (kStagesRaw > kMaxStages ? kMaxStages : kStagesRaw);
   static constexpr unsigned kSmemBytes = kStages * kStageBytes;
   static_assert(kSmemBytes <= 227 * 1024, "stages do not fit in shared memory");
