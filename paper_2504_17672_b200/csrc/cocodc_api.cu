@@ -40,6 +40,7 @@ struct cocodc_ctx {
   int* d_status = nullptr;
   long long launches = 0;
   std::vector<std::pair<const void*, int>> occupancy;  // kernel -> resident CTAs per SM
+  std::vector<const void*> smem_opted_in;              // kernels whose dynamic shared memory limit was raised on this device
   // host copy of the fragment table (host-buffer entry point walks it on the host)
   std::vector<int> h_frag_seg_ptr;
   std::vector<long long> h_seg_off, h_seg_len;
@@ -107,13 +108,16 @@ struct Variant {
 template <int M, int MODE, bool SAME>
 Variant staged_variant() {
   using L = StageLayout<M, MODE, SAME>;
-  auto kernel = k_outer_tma<M, MODE, SAME>;
-  static bool configured = false;   // one-time opt-in to more than 48 KB of dynamic shared memory
-  if (!configured) {
-    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L::kSmemBytes);
-    configured = true;
-  }
-  return Variant{kernel, kTmaThreads, L::kSmemBytes, true};
+  return Variant{k_outer_tma<M, MODE, SAME>, kTmaThreads, L::kSmemBytes, true};
+}
+
+// More than 48 KB of dynamic shared memory needs a one-time opt-in per kernel and device (the
+// caller has made the context's device current).
+void opt_in_shared_memory(cocodc_ctx* c, const void* kernel, unsigned bytes) {
+  if (bytes <= 48u * 1024u) return;
+  for (const void* k : c->smem_opted_in) if (k == kernel) return;
+  cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  c->smem_opted_in.push_back(kernel);
 }
 
 // Instantiated worker counts are staged through shared memory by TMA; any other M takes the
@@ -154,6 +158,7 @@ cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool sam
                            const int32_t* n_ids, const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
   const Variant v = pick_variant(A.M, mode, same);
   const int grid = variant_grid(c, v);
+  opt_in_shared_memory(c, reinterpret_cast<const void*>(v.kernel), v.smem);
   cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, A.snap_stride, kThreads, st);
   if (s != COCODC_OK) return s;
   v.kernel<<<grid, v.threads, v.smem, st>>>(A);
@@ -598,11 +603,7 @@ cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
     return COCODC_ERR_ALIAS;
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  static bool configured = false;   // one-time opt-in to 160 KB of dynamic shared memory
-  if (!configured) {
-    cudaFuncSetAttribute(k_snapshot_tma, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSnapSmemBytes);
-    configured = true;
-  }
+  opt_in_shared_memory(c, reinterpret_cast<const void*>(k_snapshot_tma), kSnapSmemBytes);
   cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, snap_stride, kThreads * kSnapU, st);
   if (s != COCODC_OK) return s;
   k_snapshot_tma<<<c->sm_count, kThreads, kSnapSmemBytes, st>>>(w_now, w_snap, now_stride, snap_stride, M, c->d_plan,
@@ -664,6 +665,7 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Variant v = pick_variant(M, MODE_FUSED, same);
   const int grid = variant_grid(c, v);
+  opt_in_shared_memory(c, reinterpret_cast<const void*>(v.kernel), v.smem);
   const int entries = grid * (kThreads / 32);
   bool ok = true;
   auto CK = [&](cudaError_t e) { ok = ok && (e == cudaSuccess); };
