@@ -120,8 +120,7 @@ void opt_in_shared_memory(cocodc_ctx* c, const void* kernel, unsigned bytes) {
   c->smem_opted_in.push_back(kernel);
 }
 
-// Instantiated worker counts are staged through shared memory by TMA; any other M takes the
-// generic element loop.
+// Worker counts 1..8 are staged through shared memory by TMA; larger M take the generic element loop.
 template <int MODE, bool SAME>
 Variant pick_variant(int M) {
   switch (M) {
@@ -129,6 +128,9 @@ Variant pick_variant(int M) {
     case 2: return staged_variant<2, MODE, SAME>();
     case 3: return staged_variant<3, MODE, SAME>();
     case 4: return staged_variant<4, MODE, SAME>();
+    case 5: return staged_variant<5, MODE, SAME>();
+    case 6: return staged_variant<6, MODE, SAME>();
+    case 7: return staged_variant<7, MODE, SAME>();
     case 8: return staged_variant<8, MODE, SAME>();
     default: return Variant{k_outer_generic<MODE, SAME>, kThreads, 0u, false};
   }
