@@ -35,21 +35,30 @@ BUDGET_COUNT, BUDGET_PARAMS = 0, 1
 _lib = None
 
 
+def load_library(path: str):
+    """Load a build of cocodc_oracle.c and declare its signatures (tests also load deliberately broken builds)."""
+    lib = ctypes.CDLL(path)
+    _declare(lib)
+    return lib
+
+
+def _declare(lib):
+    d, l, i, p = ctypes.c_double, ctypes.c_long, ctypes.c_int, ctypes.c_void_p
+    lib.cocodc_oracle_outer_elements.restype = d
+    lib.cocodc_oracle_outer_elements.argtypes = [
+        l, i, p, l, p, l, p, p, d, d, d, d, l, l, i, i, i, p, i, p, p, p, p]
+    lib.cocodc_oracle_pseudo_gradient_sum.restype = None
+    lib.cocodc_oracle_pseudo_gradient_sum.argtypes = [l, i, p, l, p, p]
+    lib.cocodc_oracle_merge_elements.restype = None
+    lib.cocodc_oracle_merge_elements.argtypes = [l, i, p, l, p, l, p, d, d, l, l, i, i, p]
+    lib.cocodc_oracle_sumsq.restype = d
+    lib.cocodc_oracle_sumsq.argtypes = [l, p]
+
+
 def _clib():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(_build.build())
-        d, l, i, p = ctypes.c_double, ctypes.c_long, ctypes.c_int, ctypes.c_void_p
-        lib.cocodc_oracle_outer_elements.restype = d
-        lib.cocodc_oracle_outer_elements.argtypes = [
-            l, i, p, l, p, l, p, p, d, d, d, d, l, l, i, i, i, p, i, p, p, p, p]
-        lib.cocodc_oracle_pseudo_gradient_sum.restype = None
-        lib.cocodc_oracle_pseudo_gradient_sum.argtypes = [l, i, p, l, p, p]
-        lib.cocodc_oracle_merge_elements.restype = None
-        lib.cocodc_oracle_merge_elements.argtypes = [l, i, p, l, p, l, p, d, d, l, l, i, i, p]
-        lib.cocodc_oracle_sumsq.restype = d
-        lib.cocodc_oracle_sumsq.argtypes = [l, p]
-        _lib = lib
+        _lib = load_library(_build.build())
     return _lib
 
 
