@@ -356,3 +356,59 @@ def test_random_partitions_layouts_and_modes(seed):
     assert prob.poll() == 0
     exp = orc.snapshot(fragments_of(w), snap_before["w_now"], ids, M, snap_before["snap_offset"], snap_before["w_snap"])
     assert np.array_equal(np_(prob.bufs.w_snap), exp)
+
+
+def _check_pooled(prob, before, ids, t_p, t_l):
+    """Parity over all listed fragments taken together (fragments of one or a few elements leave the
+    per-fragment measure nothing to normalise by when an output is small against its operands)."""
+    w = prob.w
+    frs = fragments_of(w)
+    res, new_last = orc.outer_step(frs, orc_hyper(w), before["w_now"], before["w_snap"], before["theta_g"],
+                                   before["momentum"], ids, t_p, t_l, before["last_sync"])
+    after = prob.host_state()
+    cat = lambda f: np.concatenate([f(p) for p in ids], axis=-1)
+    assert_close(cat(lambda p: orc.gather_fragment(frs, after["theta_g"], p)), cat(lambda p: res[p].theta_g), TOL_PARAM, "theta_g")
+    assert_close(cat(lambda p: orc.gather_fragment(frs, after["momentum"], p)), cat(lambda p: res[p].momentum), TOL_PARAM, "momentum")
+    for m in range(w.M):
+        assert_close(cat(lambda p: orc.gather_fragment(frs, after["w_now"], p)[m]), cat(lambda p: res[p].w_now[m]), TOL_PARAM, f"w_now[{m}]")
+    norms = np.array([res[p].norm for p in ids])
+    got = after["norms"][ids]
+    big = norms > 1e-3 * norms.max()
+    assert np.all(np.abs(got[big] - norms[big]) <= 1e-5 * norms[big])
+    assert np.all(np.abs(got[~big] - norms[~big]) <= 1e-5 * norms.max())
+    assert np.array_equal(after["last_sync"], new_last)
+    untouched = ~touched_mask(w, ids)
+    for k in ("theta_g", "momentum"):
+        assert np.array_equal(after[k][untouched], before[k][untouched])
+    assert np.array_equal(after["w_now"][:, untouched], before["w_now"][:, untouched])
+
+
+def test_maximum_fragment_count():
+    """K = 1024 fragments (the limit of a context), many of them shorter than a tile, all completed in one call."""
+    rng = np.random.default_rng(5)
+    sizes = rng.choice([1, 7, 255, 257, 1023, 1024, 1500], size=1024).tolist()
+    offs = np.concatenate([[0], np.cumsum(sizes)])
+    total = int(offs[-1])
+    w = synth.small_workload((total + 8 - total % 4, [[(int(o), int(l))] for o, l in zip(offs[:-1], sizes)]),
+                             M=2, seed=150)
+    prob = GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3))
+    ids = rng.permutation(1024).tolist()
+    prob.set_ids(ids)
+    before = prob.host_state()
+    prob.outer_step(3, 4)
+    assert prob.poll() == 0
+    _check_pooled(prob, before, ids, 3, 4)
+    # selection over all 1024 under a parameter budget, feeding the next completion
+    prob.select(t_now=50, budget_kind=1, budget=int(sum(sizes) // 3))
+    n = int(prob.n_ids.item())
+    got = np_(prob.ids)[:n].tolist()
+    _, eids, en = orc.select_fragments(np_(prob.scores), np_(prob.last_sync), w.partition.frag_sizes, 50, w.H,
+                                       orc.BUDGET_PARAMS, int(sum(sizes) // 3))
+    assert n == en and got == eids.tolist()
+    before = prob.host_state()
+    prob.outer_step(50, 52)
+    assert prob.poll() == 0
+    _check_pooled(prob, before, got, 50, 52)
+    with pytest.raises(prob.B.CocodcError):
+        ptr = np.arange(1026, dtype=np.int32)
+        prob.B.Context(1025, ptr, np.arange(1025), np.ones(1025, dtype=np.int64), 1)
