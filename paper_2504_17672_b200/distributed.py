@@ -46,3 +46,18 @@ def complete_fragments(ctx, hyper, M_total: int, fragments, ids_host: Sequence[i
     ctx.cocodc_outer_step_received(hyper, M_total, w_now, w_snap, w_now.stride(0), w_snap.stride(0), snap_offset,
                                    theta_g, momentum, sum_buf, None, ids_dev, n_ids_dev, t_p, t_l,
                                    last_sync, norms, scores)
+
+
+def combine_sharded_norms(norms_local: torch.Tensor, interval: torch.Tensor = None, group=None):
+    """Parameter-range sharding: every rank holds a slice of each fragment (all workers of that slice), so
+    the element-wise steps need no exchange and only Eq. 10's norm spans ranks.  Given the norms each rank
+    computed over its own slices, returns (norms, scores) of the whole fragments, identical on every rank:
+    one all-reduce of K doubles (the sums of squares), then R_p = norm_p / max(1, I_p)."""
+    sq = norms_local.double() ** 2
+    dist.all_reduce(sq, op=dist.ReduceOp.SUM, group=group)
+    norms = sq.sqrt()
+    if interval is None:
+        scores = norms.clone()
+    else:
+        scores = norms / interval.clamp(min=1).double()
+    return norms.float(), scores.float()

@@ -62,6 +62,12 @@ def _worker(rank, world, port, out):
         for o, l in ranges:
             exp[o:o + l] = 3.0                                    # 1 + 2 summed over the two ranks
         assert torch.equal(buf, exp)
+        # parameter-range sharding: fragment norms from per-rank slices, one all-reduce of K sums of squares
+        full = torch.arange(1, 13, dtype=torch.float32).reshape(3, 4)          # 3 fragments of 4 elements
+        mine = full[:, 2 * rank:2 * rank + 2]                                  # each rank owns half of every fragment
+        n, sc = D.combine_sharded_norms(mine.norm(dim=1), torch.tensor([0, 2, 5]))
+        assert torch.allclose(n, full.norm(dim=1), rtol=1e-6)
+        assert torch.allclose(sc, full.norm(dim=1) / torch.tensor([1.0, 2.0, 5.0]), rtol=1e-6)
         out.put((rank, "ok"))
     except Exception as e:  # pragma: no cover
         out.put((rank, repr(e)))
