@@ -210,6 +210,26 @@ cocodc_status cocodc_outer_step(cocodc_ctx* ctx, const cocodc_hyper* hyper,
                                 float* norms, float* scores, uint32_t stages, void* stream);
 
 /*
+ * cocodc_select_fragments and cocodc_outer_step with their step numbers read from DEVICE memory at run time
+ * (t_now, t_p, t_l: dev int64[1] each) instead of passed by value.  Everything else is identical.  A schedule
+ * step (completion, selection, snapshot) contains no host-side value that changes from step to step any more,
+ * so it can be recorded once in a CUDA graph and replayed while a device-side counter advances - which is
+ * what makes small workloads, whose step is a handful of microsecond kernels, launch-bound no longer.
+ */
+cocodc_status cocodc_select_fragments_at(cocodc_ctx* ctx, const float* scores, const int64_t* last_sync,
+                                         const uint8_t* ineligible, const int64_t* t_now, int64_t H,
+                                         int32_t budget_kind, int64_t budget,
+                                         uint8_t* mask, int32_t* ids, int32_t* n_sel,
+                                         int64_t* pool_offset, void* stream);
+cocodc_status cocodc_outer_step_at(cocodc_ctx* ctx, const cocodc_hyper* hyper,
+                                   float* w_now, const float* w_snap,
+                                   int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                   float* theta_g, float* momentum, float* delta_g_out,
+                                   const int32_t* ids, const int32_t* n_ids,
+                                   const int64_t* t_p, const int64_t* t_l, int64_t* last_sync,
+                                   float* norms, float* scores, uint32_t stages, void* stream);
+
+/*
  * Worker-per-device deployment (Section 2.1: every worker all-reduces its pseudo-gradient).  When a
  * device holds only M of the M_total workers, Eq. 1's sum spans devices:
  *

@@ -28,6 +28,7 @@ EXPORTS = (
     "cocodc_poll_status", "cocodc_launch_count", "cocodc_status_string",
     "cocodc_fragment_scores_noalloc", "cocodc_selftest_bounded_wait",
     "cocodc_pseudo_gradient_sum", "cocodc_outer_step_received",
+    "cocodc_select_fragments_at", "cocodc_outer_step_at",
 )
 NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
@@ -92,6 +93,9 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_snapshot.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, vp, vp]
     lib.cocodc_fragment_scores_noalloc.argtypes = [ctypes.POINTER(_Partition), vp, vp, vp, vp, i32, vp]
     lib.cocodc_selftest_bounded_wait.argtypes = [vp, i32, vp]
+    lib.cocodc_select_fragments_at.argtypes = [vp, vp, vp, vp, vp, i64, i32, i64, vp, vp, vp, vp, vp]
+    lib.cocodc_outer_step_at.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, vp,
+                                         vp, vp, vp, vp, vp, u32, vp]
     lib.cocodc_pseudo_gradient_sum.argtypes = [vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
     lib.cocodc_outer_step_received.argtypes = [vp, ctypes.POINTER(_Hyper), i32, vp, vp, i64, i64, vp, vp, vp, vp,
                                                vp, vp, vp, i64, i64, vp, vp, vp, vp]
@@ -221,6 +225,23 @@ class Context:
                                            _p(last_sync), _p(norms), _p(scores), 1 if snap_on_device else 0, _p(workspace),
                                            workspace.numel() * workspace.element_size(), _stream(stream)),
                "cocodc_outer_step_host")
+
+    def cocodc_select_fragments_at(self, scores, last_sync, ineligible, t_now, H: int, budget_kind: int,
+                                   budget: int, mask, ids, n_sel, pool_offset=None, stream=None) -> None:
+        """As cocodc_select_fragments with t_now a device int64[1] tensor."""
+        _check(_lib.cocodc_select_fragments_at(self._h, _p(scores), _p(last_sync), _p(ineligible), _p(t_now), int(H),
+                                               int(budget_kind), int(budget), _p(mask), _p(ids), _p(n_sel),
+                                               _p(pool_offset), _stream(stream)), "cocodc_select_fragments_at")
+
+    def cocodc_outer_step_at(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
+                             theta_g, momentum, delta_g_out, ids, n_ids, t_p, t_l, last_sync,
+                             norms, scores, stages: int = STAGE_ALL, stream=None) -> None:
+        """As cocodc_outer_step with t_p and t_l device int64[1] tensors."""
+        h = hyper._c()
+        _check(_lib.cocodc_outer_step_at(self._h, ctypes.byref(h), _p(w_now), _p(w_snap), int(now_stride),
+                                         int(snap_stride), _p(snap_offset), _p(theta_g), _p(momentum),
+                                         _p(delta_g_out), _p(ids), _p(n_ids), _p(t_p), _p(t_l), _p(last_sync),
+                                         _p(norms), _p(scores), int(stages), _stream(stream)), "cocodc_outer_step_at")
 
     def cocodc_pseudo_gradient_sum(self, w_snap, snap_stride: int, snap_offset, theta_g, M: int, sum_out,
                                    ids, n_ids, stream=None) -> None:

@@ -384,26 +384,9 @@ cocodc_status cocodc_fragment_scores(cocodc_ctx* c, const float* delta_g, const 
   kernel<<<grid, kThreads, 0, st>>>(delta_g, c->d_plan, c->d_hdr, c->d_partial);
   c->launches++;
   k_finalize_scores<<<c->K, kFinalizeThreads, 0, st>>>(
-      c->d_hdr, nullptr, c->d_partial, grid * (kThreads / 32), 1, 0, 0,
+      c->d_hdr, nullptr, c->d_partial, grid * (kThreads / 32), 1, 0, 0, nullptr, nullptr,
       reinterpret_cast<const long long*>(interval), nullptr, norms, scores, c->d_status,
       (int)COCODC_ERR_NONFINITE);
-  c->launches++;
-  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
-}
-
-cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
-                                      const uint8_t* ineligible, int64_t t_now, int64_t H,
-                                      int32_t budget_kind, int64_t budget,
-                                      uint8_t* mask, int32_t* ids, int32_t* n_sel,
-                                      int64_t* pool_offset, void* stream) {
-  if (!c || !scores || !last_sync || !mask || !ids || !n_sel) return COCODC_ERR_INVALID_ARG;
-  if (H < 1 || budget < 0) return COCODC_ERR_INVALID_ARG;
-  if (budget_kind != COCODC_BUDGET_COUNT && budget_kind != COCODC_BUDGET_PARAMS) return COCODC_ERR_INVALID_ARG;
-  DeviceGuard guard(c->device);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  k_select<<<1, kSelectThreads, 0, st>>>(c->K, scores, reinterpret_cast<const long long*>(last_sync), ineligible,
-                                         c->d_frag_size, t_now, H, budget_kind, budget, mask, ids, n_sel,
-                                         reinterpret_cast<long long*>(pool_offset), c->d_status, (int)COCODC_ERR_NONFINITE);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
@@ -411,6 +394,22 @@ cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const 
 }  // extern "C"
 
 namespace {
+cocodc_status select_impl(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
+                          const uint8_t* ineligible, int64_t t_now, const int64_t* t_now_dev, int64_t H,
+                          int32_t budget_kind, int64_t budget,
+                          uint8_t* mask, int32_t* ids, int32_t* n_sel,
+                          int64_t* pool_offset, void* stream) {
+  if (!c || !scores || !last_sync || !mask || !ids || !n_sel) return COCODC_ERR_INVALID_ARG;
+  if (H < 1 || budget < 0) return COCODC_ERR_INVALID_ARG;
+  if (budget_kind != COCODC_BUDGET_COUNT && budget_kind != COCODC_BUDGET_PARAMS) return COCODC_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  k_select<<<1, kSelectThreads, 0, st>>>(c->K, scores, reinterpret_cast<const long long*>(last_sync), ineligible,
+                                         c->d_frag_size, t_now, reinterpret_cast<const long long*>(t_now_dev), H, budget_kind, budget, mask, ids, n_sel,
+                                         reinterpret_cast<long long*>(pool_offset), c->d_status, (int)COCODC_ERR_NONFINITE);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
 
 // cocodc_outer_step and cocodc_outer_step_received: the latter passes the all-reduced sum of every
 // worker's pseudo-gradients (delta_sum) and the total worker count it is to be divided by.
@@ -421,7 +420,8 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
                               const int32_t* ids, const int32_t* n_ids,
                               int64_t t_p, int64_t t_l, int64_t* last_sync,
                               float* norms, float* scores, uint32_t stages, void* stream,
-                              const float* delta_sum, int32_t M_total) {
+                              const float* delta_sum, int32_t M_total,
+                              const int64_t* t_p_dev = nullptr, const int64_t* t_l_dev = nullptr) {
   cocodc_status s = check_hyper(c, h);
   if (s != COCODC_OK) return s;
   const bool received = delta_sum != nullptr;
@@ -434,6 +434,7 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
   if (do_merge && !w_now) return COCODC_ERR_INVALID_ARG;
   if (do_score && (!last_sync || !norms || !scores)) return COCODC_ERR_INVALID_ARG;
   if (t_l < t_p) return COCODC_ERR_INVALID_ARG;
+  if ((t_p_dev == nullptr) != (t_l_dev == nullptr)) return COCODC_ERR_INVALID_ARG;
   const long long N = c->N;
   if (snap_stride < (snap_offset ? 1 : N) || (do_merge && now_stride < N)) return COCODC_ERR_INVALID_ARG;
   const bool same = do_merge && (w_snap == w_now) && (snap_stride == now_stride) && (snap_offset == nullptr);
@@ -490,7 +491,8 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
   if (s != COCODC_OK) return s;
   if (do_score) {
     k_finalize_scores<<<c->K, kFinalizeThreads, 0, st>>>(
-        c->d_hdr, ids, c->d_partial, grid * (kThreads / 32), 0, t_p, t_l, nullptr,
+        c->d_hdr, ids, c->d_partial, grid * (kThreads / 32), 0, t_p, t_l,
+        reinterpret_cast<const long long*>(t_p_dev), reinterpret_cast<const long long*>(t_l_dev), nullptr,
         reinterpret_cast<long long*>(last_sync), norms, scores, c->d_status, (int)COCODC_ERR_NONFINITE);
     c->launches++;
     if (cudaGetLastError() != cudaSuccess) return COCODC_ERR_CUDA;
@@ -523,6 +525,37 @@ cocodc_status cocodc_outer_step_received(cocodc_ctx* c, const cocodc_hyper* h, i
   if (!delta_sum) return COCODC_ERR_INVALID_ARG;
   return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
                          ids, n_ids, t_p, t_l, last_sync, norms, scores, COCODC_STAGE_ALL, stream, delta_sum, M_total);
+}
+
+cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
+                                      const uint8_t* ineligible, int64_t t_now, int64_t H,
+                                      int32_t budget_kind, int64_t budget,
+                                      uint8_t* mask, int32_t* ids, int32_t* n_sel,
+                                      int64_t* pool_offset, void* stream) {
+  return select_impl(c, scores, last_sync, ineligible, t_now, nullptr, H, budget_kind, budget, mask, ids, n_sel,
+                     pool_offset, stream);
+}
+
+cocodc_status cocodc_select_fragments_at(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
+                                         const uint8_t* ineligible, const int64_t* t_now, int64_t H,
+                                         int32_t budget_kind, int64_t budget,
+                                         uint8_t* mask, int32_t* ids, int32_t* n_sel,
+                                         int64_t* pool_offset, void* stream) {
+  if (!t_now) return COCODC_ERR_INVALID_ARG;
+  return select_impl(c, scores, last_sync, ineligible, 0, t_now, H, budget_kind, budget, mask, ids, n_sel,
+                     pool_offset, stream);
+}
+
+cocodc_status cocodc_outer_step_at(cocodc_ctx* c, const cocodc_hyper* h,
+                                   float* w_now, const float* w_snap,
+                                   int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                   float* theta_g, float* momentum, float* delta_g_out,
+                                   const int32_t* ids, const int32_t* n_ids,
+                                   const int64_t* t_p, const int64_t* t_l, int64_t* last_sync,
+                                   float* norms, float* scores, uint32_t stages, void* stream) {
+  if (!t_p || !t_l) return COCODC_ERR_INVALID_ARG;
+  return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
+                         ids, n_ids, 0, 0, last_sync, norms, scores, stages, stream, nullptr, 0, t_p, t_l);
 }
 
 cocodc_status cocodc_pseudo_gradient_sum(cocodc_ctx* c, const float* w_snap, int64_t snap_stride,

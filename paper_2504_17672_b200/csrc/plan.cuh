@@ -167,7 +167,8 @@ constexpr int kFinalizeThreads = 256;
 static __global__ void __launch_bounds__(kFinalizeThreads)
 k_finalize_scores(const PlanHeader* __restrict__ hdr, const int* __restrict__ ids,
                   const double* __restrict__ partial, int entries_per_slot,
-                  int mode, long long t_p, long long t_l, const long long* __restrict__ interval,
+                  int mode, long long t_p, long long t_l, const long long* __restrict__ t_p_dev,
+                  const long long* __restrict__ t_l_dev, const long long* __restrict__ interval,
                   long long* __restrict__ last_sync, float* __restrict__ norms,
                   float* __restrict__ scores, int* __restrict__ status, int err_nonfinite) {
   __shared__ double red[kFinalizeThreads];
@@ -188,6 +189,9 @@ k_finalize_scores(const PlanHeader* __restrict__ hdr, const int* __restrict__ id
   const double norm = sqrt(red[0]);
   long long I = 1;
   if (mode == 0) {
+    // step numbers kept in device memory (graph replay) take precedence over the launch arguments
+    if (t_p_dev) t_p = *t_p_dev;
+    if (t_l_dev) t_l = *t_l_dev;
     I = t_p - last_sync[p];
     last_sync[p] = t_l;
   } else if (interval != nullptr) {

@@ -15,7 +15,7 @@ constexpr int kSelectThreads = 1024;
 __global__ void __launch_bounds__(kSelectThreads)
 k_select(int K, const float* __restrict__ scores, const long long* __restrict__ last_sync,
          const unsigned char* __restrict__ ineligible, const long long* __restrict__ frag_size,
-         long long t_now, long long H, int budget_kind, long long budget,
+         long long t_now, const long long* __restrict__ t_now_dev, long long H, int budget_kind, long long budget,
          unsigned char* __restrict__ mask, int* __restrict__ ids, int* __restrict__ n_sel,
          long long* __restrict__ pool_offset, int* __restrict__ status, int err_nonfinite) {
   __shared__ float s_score[kMaxK];
@@ -24,6 +24,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   __shared__ int s_nan;
   __shared__ int s_count;
   const int p = threadIdx.x;
+  if (t_now_dev) t_now = *t_now_dev;   // step number kept in device memory (graph replay)
   if (p == 0) { s_nan = 0; s_count = 0; }
   __syncthreads();
   if (p < K) {

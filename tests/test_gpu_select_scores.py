@@ -133,3 +133,62 @@ def test_standalone_scores(frs):
     x[7] = float("nan")
     ctx.cocodc_fragment_scores(x, None, norms, scores)
     assert ctx.cocodc_poll_status() == B.ERR_NONFINITE
+
+
+def test_schedule_step_replayed_from_a_cuda_graph_equals_eager_steps():
+    """Completion + selection + snapshot with device-resident step numbers, recorded once and replayed: bit-identical
+    to the same steps issued call by call."""
+    w = synth.get_workload("tiny")
+    from paper_2504_17672_b200 import binding as B
+
+    def fresh():
+        prob = GpuProblem(w, synth.generate(w, "cuda", snap_layout="pool", pool_ids=[0, 1], momentum_sigma=1e-3))
+        prob.pool_off = prob.bufs.snap_offset
+        prob.scores.copy_(torch.arange(w.K, 0, -1, dtype=torch.float32, device="cuda"))
+        prob.set_ids([0, 1])
+        return prob
+
+    tau = w.tau
+    # eager reference: five steps with host-side step numbers
+    a = fresh()
+    t = 10
+    for _ in range(5):
+        b = a.bufs
+        a.ctx.cocodc_outer_step(a.hyper(), b.w_now, b.w_snap, b.now_stride, b.snap_stride, a.pool_off, b.theta_g,
+                                b.momentum, None, a.ids, a.n_ids, t, t + tau, a.last_sync, a.norms, a.scores)
+        t += tau
+        a.ctx.cocodc_select_fragments(a.scores, a.last_sync, None, t, w.H, B.BUDGET_COUNT, w.budget, a.mask, a.ids,
+                                      a.n_ids, a.pool_off)
+        a.ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, a.pool_off, w.M, a.ids, a.n_ids)
+    assert a.poll() == 0
+
+    # the same through a graph: clock[0] = t_p, clock[1] = t_l = the next selection's t_now
+    g = fresh()
+    clock = torch.tensor([10, 10 + tau], dtype=torch.int64, device="cuda")
+
+    def step():
+        b = g.bufs
+        g.ctx.cocodc_outer_step_at(g.hyper(), b.w_now, b.w_snap, b.now_stride, b.snap_stride, g.pool_off, b.theta_g,
+                                   b.momentum, None, g.ids, g.n_ids, clock[0:1], clock[1:2], g.last_sync, g.norms,
+                                   g.scores)
+        g.ctx.cocodc_select_fragments_at(g.scores, g.last_sync, None, clock[1:2], w.H, B.BUDGET_COUNT, w.budget,
+                                         g.mask, g.ids, g.n_ids, g.pool_off)
+        g.ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, g.pool_off, w.M, g.ids, g.n_ids)
+        clock.add_(tau)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                                   # warm-up outside the capture (first-use set-up of the kernels)
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for _ in range(4):                           # one eager warm-up step + four replays (recording runs nothing)
+        graph.replay()
+    torch.cuda.synchronize()
+    assert g.poll() == 0
+    assert int(clock[0].item()) == 10 + 5 * tau
+    for x, y in ((a.bufs.w_now, g.bufs.w_now), (a.bufs.theta_g, g.bufs.theta_g), (a.bufs.momentum, g.bufs.momentum),
+                 (a.bufs.w_snap, g.bufs.w_snap), (a.scores, g.scores), (a.last_sync, g.last_sync), (a.ids, g.ids)):
+        assert torch.equal(x, y)
