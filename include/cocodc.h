@@ -324,7 +324,7 @@ cocodc_status cocodc_snapshot_host(cocodc_ctx* ctx, const float* w_now, float* w
  * scores[p] = norms[p] / max(1, interval[p]) (interval NULL means 1).  A non-finite norm is
  * written as it is; there is no status word.
  *
- * The scratch (per-CTA partial sums, about 1.2 MB) is a fixed __device__ array inside the library
+ * The scratch (per-CTA partial sums, about 0.6 MB) is a fixed __device__ array inside the library
  * image: every GPU that loads the library holds it until the process exits.  Its size bounds the
  * problem: K <= COCODC_NOALLOC_MAX_K fragments and n_segments <= COCODC_NOALLOC_MAX_SEGMENTS;
  * anything larger returns COCODC_ERR_INVALID_ARG.  The call itself makes no cudaMalloc/cudaFree

@@ -31,10 +31,10 @@ namespace {
 
 constexpr int kNoallocMaxK = COCODC_NOALLOC_MAX_K;
 constexpr int kNoallocMaxSeg = COCODC_NOALLOC_MAX_SEGMENTS;
-constexpr int kGrid = 296;                 // fixed launch width: the scratch is sized for it
+constexpr int kGrid = 1184;                // fixed launch width (8 CTAs on each of 148 SMs): the scratch is sized for it
 constexpr int kWarps = kThreads / 32;
 constexpr int kU = 4;                      // 16-byte lanes per thread and tile
-constexpr size_t kScratchDoubles = (size_t)kNoallocMaxK * kGrid * kWarps;
+constexpr size_t kScratchDoubles = (size_t)kNoallocMaxK * kGrid;   // one double per (fragment, CTA)
 constexpr size_t kNoallocScratchBytes = kScratchDoubles * sizeof(double);
 static_assert(kNoallocScratchBytes <= (2u << 20), "the fixed scratch is meant to stay modest");
 
@@ -48,14 +48,46 @@ struct PlanTable {
   SegPlan seg[kNoallocMaxSeg];
 };
 
+// Per-CTA running sum of squares of the current fragment.  When the fragment changes (the same tile, hence
+// the same moment, for every thread of the CTA) the warps reduce, thread 0 adds the warp sums in warp order
+// and writes partial[fragment * gridDim.x + CTA]; fragments the CTA never touched get an explicit zero.
+struct CtaAccumulator {
+  double acc = 0.0;
+  int slot = 0;
+  double* warp_sums;   // shared, one per warp
+
+  __device__ __forceinline__ explicit CtaAccumulator(double* shared_warp_sums) : warp_sums(shared_warp_sums) {}
+  __device__ __forceinline__ void flush_to(int new_slot, double* __restrict__ partial) {
+    const double v = warp_sum(acc);
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      double s = 0.0;
+      for (int w = 0; w < kWarps; ++w) s += warp_sums[w];
+      partial[(size_t)slot * gridDim.x + blockIdx.x] = s;
+      for (int z = slot + 1; z < new_slot; ++z) partial[(size_t)z * gridDim.x + blockIdx.x] = 0.0;
+    }
+    __syncthreads();
+    acc = 0.0;
+    slot = new_slot;
+  }
+  __device__ __forceinline__ void advance(int new_slot, double* __restrict__ partial) {
+    if (new_slot != slot) flush_to(new_slot, partial);
+  }
+  __device__ __forceinline__ void finish(int n_ids, double* __restrict__ partial) {
+    if (slot < n_ids) flush_to(n_ids, partial);
+  }
+};
+
 // Variant of k_sumsq that reads its plan from the argument block and writes its partial sums to
-// the scratch array.  Every (fragment, CTA, warp) entry that the finalize kernel reads is written
+// the scratch array.  Every (fragment, CTA) entry that the finalize kernel reads is written
 // by this kernel in the same call (untouched ones with an explicit zero), so what an earlier call
 // left in the array is never read and nothing has to be cleared.
 __global__ void __launch_bounds__(kThreads)
 k_sumsq_table(const float* __restrict__ x, const __grid_constant__ PlanTable plan, double* __restrict__ partial) {
   constexpr int LPT = kThreads * kU;
-  SlotAccumulator sa(kWarps);
+  __shared__ double warp_sums[kWarps];
+  CtaAccumulator sa(warp_sums);
   int seg = 0;
   for (int tile = blockIdx.x; tile < plan.hdr.total_tiles; tile += gridDim.x) {
     while (seg + 1 < plan.hdr.n_seg && tile >= plan.seg[seg + 1].first_tile) ++seg;
@@ -184,7 +216,7 @@ extern "C" cocodc_status cocodc_fragment_scores_noalloc(const cocodc_partition* 
   if (prev != device && cudaSetDevice(device) != cudaSuccess) return COCODC_ERR_CUDA;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
   k_sumsq_table<<<kGrid, kThreads, 0, cs>>>(delta_g, table, scratch);
-  k_finalize_table<<<K, kFinalizeThreads, 0, cs>>>(scratch, kGrid * kWarps,
+  k_finalize_table<<<K, kFinalizeThreads, 0, cs>>>(scratch, kGrid,
                                                    reinterpret_cast<const long long*>(interval), norms, scores);
   const cudaError_t e = cudaGetLastError();
   if (prev != device) cudaSetDevice(prev);
