@@ -147,6 +147,7 @@ Variant pick_variant(int M, int mode, bool same) {
     }
   }
   if (mode == MODE_OUTER_ONLY) return pick_variant<MODE_OUTER_ONLY, false>(M);
+  if (mode == MODE_PSEUDO_SUM) return pick_variant<MODE_PSEUDO_SUM, false>(M);
   if (mode == MODE_MERGE_ONLY) return same ? pick_variant<MODE_MERGE_ONLY, true>(M) : pick_variant<MODE_MERGE_ONLY, false>(M);
   return same ? pick_variant<MODE_FUSED, true>(M) : pick_variant<MODE_FUSED, false>(M);
 }
@@ -572,21 +573,15 @@ cocodc_status cocodc_pseudo_gradient_sum(cocodc_ctx* c, const float* w_snap, int
     return COCODC_ERR_ALIAS;
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  void (*kernel)(const float*, long long, const float*, float*, int, const SegPlan*, const PlanHeader*);
-  switch (M) {
-    case 1: kernel = k_pseudo_sum<1>; break;
-    case 2: kernel = k_pseudo_sum<2>; break;
-    case 3: kernel = k_pseudo_sum<3>; break;
-    case 4: kernel = k_pseudo_sum<4>; break;
-    case 8: kernel = k_pseudo_sum<8>; break;
-    default: kernel = k_pseudo_sum<0>; break;
-  }
-  const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, snap_stride, kThreads, st);
-  if (s != COCODC_OK) return s;
-  kernel<<<grid, kThreads, 0, st>>>(w_snap, snap_stride, theta_g, sum_out, M, c->d_plan, c->d_hdr);
-  c->launches++;
-  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+  OuterArgs A{};
+  A.w_snap = w_snap; A.snap_stride = snap_stride; A.now_stride = N;
+  A.theta_g = const_cast<float*>(theta_g);   // read only in this mode
+  A.delta_out = sum_out;
+  A.plan = c->d_plan; A.hdr = c->d_hdr; A.partial = nullptr;
+  A.status = c->d_status; A.err_timeout = COCODC_ERR_TIMEOUT;
+  A.M = M;
+  int grid = 0;
+  return launch_outer(c, A, MODE_PSEUDO_SUM, false, ids, n_ids, snap_offset, st, &grid);
 }
 
 cocodc_status cocodc_merge(cocodc_ctx* c, const cocodc_hyper* h,

@@ -20,7 +20,11 @@ constexpr int kTileElems = 4 * kThreads;
 
 // MODE_FUSED_RECV: as MODE_FUSED, but Eq. 1's sum over ALL workers arrives ready-made (delta_in, the result
 // of the all-reduce when every device holds only some of the workers) and is divided by the total count.
-enum : int { MODE_FUSED = 0, MODE_OUTER_ONLY = 1, MODE_MERGE_ONLY = 2, MODE_FUSED_RECV = 3 };
+// MODE_PSEUDO_SUM: only S1 and the local part of S2 -- the sum over this device's workers of
+// theta^m_{p,t_p} - theta^g goes to delta_out (what the all-reduce of Section 2.1 then sums); nothing else is touched.
+enum : int { MODE_FUSED = 0, MODE_OUTER_ONLY = 1, MODE_MERGE_ONLY = 2, MODE_FUSED_RECV = 3, MODE_PSEUDO_SUM = 4 };
+__host__ __device__ constexpr bool mode_updates_global(int mode) { return mode == MODE_FUSED || mode == MODE_OUTER_ONLY || mode == MODE_FUSED_RECV; }
+__host__ __device__ constexpr bool mode_merges(int mode) { return mode == MODE_FUSED || mode == MODE_MERGE_ONLY || mode == MODE_FUSED_RECV; }
 
 struct OuterArgs {
   float* w_now;             // [M][now_stride]
@@ -92,6 +96,12 @@ template <int MODE, bool SAME>
 __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, long long snap_e, double& acc) {
   const int M = A.M;
   const float thg = ld1(A.theta_g + e);
+  if (MODE == MODE_PSEUDO_SUM) {
+    float sum = 0.f;
+    for (int m = 0; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(ld1(A.w_snap + m * A.snap_stride + snap_e), thg));
+    st1(A.delta_out + e, sum);
+    return;
+  }
   float G;
   if (MODE == MODE_MERGE_ONLY) {
     G = thg;
@@ -110,7 +120,7 @@ __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, 
     st1(A.momentum + e, u_new);
     if (A.delta_out) st1(A.delta_out + e, Delta);
   }
-  if (MODE != MODE_OUTER_ONLY) {
+  if (mode_merges(MODE)) {
     for (int m = 0; m < M; ++m) {
       const float b = ld1(A.w_snap + m * A.snap_stride + snap_e);
       const float a = SAME ? b : ld1(A.w_now + m * A.now_stride + e);
@@ -125,7 +135,7 @@ __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, 
 // local parameters sit in out(m) (= a[m], or b[m] when the snapshot is the current state).
 template <int M, int MODE, bool SAME>
 struct Lane {
-  static constexpr bool kHasNow = (MODE != MODE_OUTER_ONLY) && !SAME;
+  static constexpr bool kHasNow = mode_merges(MODE) && !SAME;
   float4 b[M];
   float4 a[kHasNow ? M : 1];
   float4 thg;
@@ -139,7 +149,7 @@ struct Lane {
 
   __device__ __forceinline__ void load(const OuterArgs& A, long long e, long long snap_e) {
     thg = ld4(A.theta_g + e);
-    if (MODE != MODE_MERGE_ONLY) u = ld4(A.momentum + e);
+    if (mode_updates_global(MODE)) u = ld4(A.momentum + e);
     if (MODE == MODE_FUSED_RECV) delta = ld4(A.delta_in + e);
 #pragma unroll
     for (int m = 0; m < M; ++m) b[m] = ld4(A.w_snap + m * A.snap_stride + snap_e);
@@ -150,7 +160,17 @@ struct Lane {
   }
 
   __device__ __forceinline__ void compute(const OuterArgs& A, double& acc) {
-    if (MODE != MODE_MERGE_ONLY) {
+    if (MODE == MODE_PSEUDO_SUM) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float t = comp(thg, k);
+        float sum = __fsub_rn(comp(b[0], k), t);
+#pragma unroll
+        for (int m = 1; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(comp(b[m], k), t));
+        comp(delta, k) = sum;
+      }
+    }
+    if (mode_updates_global(MODE)) {
       float sq = 0.f;
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
@@ -171,7 +191,7 @@ struct Lane {
       }
       acc += (double)sq;
     }
-    if (MODE != MODE_OUTER_ONLY) {
+    if (mode_merges(MODE)) {
 #pragma unroll
       for (int m = 0; m < M; ++m) {
 #pragma unroll
@@ -185,12 +205,13 @@ struct Lane {
   }
 
   __device__ __forceinline__ void store(const OuterArgs& A, long long e) {
-    if (MODE != MODE_MERGE_ONLY) {
+    if (MODE == MODE_PSEUDO_SUM) st4(A.delta_out + e, delta);
+    if (mode_updates_global(MODE)) {
       st4(A.theta_g + e, thg);
       st4(A.momentum + e, u);
       if (A.delta_out) st4(A.delta_out + e, delta);
     }
-    if (MODE != MODE_OUTER_ONLY) {
+    if (mode_merges(MODE)) {
 #pragma unroll
       for (int m = 0; m < M; ++m) st4(A.w_now + m * A.now_stride + e, out(m));
     }
@@ -258,62 +279,6 @@ k_outer_generic(const OuterArgs A) {
     ragged_lane<0, MODE, SAME>(A, tw.sp, tw.tile_start(tile) + 4LL * threadIdx.x, sa.acc);
   }
   if (A.partial) sa.finish(h.n_ids, A.partial);
-}
-
-// ---------------------------------------------------------------------------
-// S1 and the local part of S2 for the worker-per-device deployment (Section 2.1): the sum over this
-// device's M workers of theta^m_{p,t_p} - theta^g, written at the fragments' native offsets of
-// sum_out.  That buffer is what the all-reduce across devices then sums.
-// ---------------------------------------------------------------------------
-template <int M>   // 0: runtime worker count
-__global__ void __launch_bounds__(kThreads)
-k_pseudo_sum(const float* __restrict__ w_snap, long long snap_stride, const float* __restrict__ theta_g,
-             float* __restrict__ sum_out, int M_runtime, const SegPlan* __restrict__ plan,
-             const PlanHeader* __restrict__ hdr) {
-  const PlanHeader h = *hdr;
-  const int Mw = (M > 0) ? M : M_runtime;
-  TileWalker tw(plan, h.n_seg);
-  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
-    tw.seek(tile);
-    const SegPlan& sp = tw.sp;
-    const long long e = tw.tile_start(tile) + 4LL * threadIdx.x;
-    const long long seg_end = sp.off + sp.len;
-    const long long shift = sp.snap_off - sp.off;
-    if (e >= seg_end) continue;
-    if (sp.vec_ok && e >= sp.off && e + 4 <= seg_end) {
-      const float4 t = ld4(theta_g + e);
-      float4 acc;
-#pragma unroll
-      for (int k = 0; k < 4; ++k) comp(acc, k) = 0.f;
-#pragma unroll
-      for (int m = 0; m < (M > 0 ? M : 1); ++m) {
-        if (M > 0) {
-          const float4 b = ld4(w_snap + m * snap_stride + shift + e);
-#pragma unroll
-          for (int k = 0; k < 4; ++k)
-            comp(acc, k) = (m == 0) ? __fsub_rn(comp(b, k), comp(t, k))
-                                    : __fadd_rn(comp(acc, k), __fsub_rn(comp(b, k), comp(t, k)));
-        }
-      }
-      if (M == 0) {
-        for (int m = 0; m < Mw; ++m) {
-          const float4 b = ld4(w_snap + m * snap_stride + shift + e);
-#pragma unroll
-          for (int k = 0; k < 4; ++k) comp(acc, k) = __fadd_rn(comp(acc, k), __fsub_rn(comp(b, k), comp(t, k)));
-        }
-      }
-      st4(sum_out + e, acc);
-    } else {
-      for (int k = 0; k < 4; ++k) {
-        const long long ee = e + k;
-        if (ee < sp.off || ee >= seg_end) continue;
-        const float t = ld1(theta_g + ee);
-        float acc = 0.f;
-        for (int m = 0; m < Mw; ++m) acc = __fadd_rn(acc, __fsub_rn(ld1(w_snap + m * snap_stride + shift + ee), t));
-        st1(sum_out + ee, acc);
-      }
-    }
-  }
 }
 
 // ---------------------------------------------------------------------------

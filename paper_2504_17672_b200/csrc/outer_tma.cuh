@@ -83,8 +83,8 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 template <int M, int MODE, bool SAME>
 struct StageLayout {
   static constexpr int nS = SAME ? 0 : M;
-  static constexpr int nN = (MODE == MODE_OUTER_ONLY) ? 0 : M;
-  static constexpr int nU = (MODE == MODE_MERGE_ONLY) ? 0 : 1;
+  static constexpr int nN = mode_merges(MODE) ? M : 0;
+  static constexpr int nU = mode_updates_global(MODE) ? 1 : 0;
   static constexpr int nR = (MODE == MODE_FUSED_RECV) ? 1 : 0;     // received sum of pseudo-gradients
   static constexpr int kSnap = 0;
   static constexpr int kNow = nS;
@@ -94,13 +94,15 @@ struct StageLayout {
   static constexpr int kLoaded = nS + nN + 1 + nU + nR;  // streams brought in by the producer
   static constexpr unsigned kStageBytes = kLoaded * kTileBytes;
   // about 72 KB of copies in flight (see the note at the top), never fewer than two stages; the
-  // read-heavy OUTER_ONLY mode (3 reads per write) measures best one stage deeper
-  static constexpr int kInFlightBytes = (MODE == MODE_OUTER_ONLY ? 96 : 72) * 1024;
+  // read-heavy modes measure best with more: OUTER_ONLY (3 reads per write) one stage deeper,
+  // PSEUDO_SUM (M + 1 reads per write) at 100 KB
+  static constexpr int kInFlightBytes =
+      (MODE == MODE_PSEUDO_SUM ? 100 : MODE == MODE_OUTER_ONLY ? 96 : 72) * 1024;
   static constexpr int kStagesRaw = kInFlightBytes / kStageBytes;
   static constexpr int kStages = kStagesRaw < 2 ? 2 : (kStagesRaw > kMaxStages ? kMaxStages : kStagesRaw);
   static constexpr unsigned kSmemBytes = kStages * kStageBytes;
   static_assert(kSmemBytes <= 227 * 1024, "stages do not fit in shared memory");
-  static_assert(SAME ? (MODE != MODE_OUTER_ONLY && MODE != MODE_FUSED_RECV) : true,
+  static_assert(SAME ? (MODE == MODE_FUSED || MODE == MODE_MERGE_ONLY) : true,
                 "zero-delay mode needs the merge and local pseudo-gradients");
 };
 
