@@ -80,7 +80,10 @@ typedef enum {
   COCODC_SIGN_DESCENT = 2
 } cocodc_sign_mode;
 
-typedef enum { COCODC_BUDGET_COUNT = 0, COCODC_BUDGET_PARAMS = 1 } cocodc_budget_kind;
+/* COUNT and PARAMS walk the priority order greedily; PARAMS_EXACT (an option the paper does not have)
+ * solves the parameter budget as a knapsack, see cocodc_select_fragments. */
+typedef enum { COCODC_BUDGET_COUNT = 0, COCODC_BUDGET_PARAMS = 1, COCODC_BUDGET_PARAMS_EXACT = 2 } cocodc_budget_kind;
+#define COCODC_EXACT_MAX_CANDIDATES 24
 
 /* Stages of cocodc_outer_step. */
 #define COCODC_STAGE_OUTER 1u   /* S1-S3: update theta_g and momentum (required) */
@@ -168,6 +171,16 @@ cocodc_status cocodc_fragment_scores(cocodc_ctx* ctx, const float* delta_g, cons
  *   budget + (largest fragment) elements (PARAMS), or the `budget` largest fragments (COUNT),
  *   plus 4 per fragment for rounding, always suffices.
  * A NaN score selects nothing and sets COCODC_ERR_NONFINITE.
+ *
+ * PARAMS_EXACT (no counterpart in the paper, whose Algorithm 2 picks one fragment per decision): the
+ * fragments that must go first -- the overdue ones and those with score +Inf -- are walked as for PARAMS;
+ * among the remaining eligible fragments the subset with the largest sum of scores whose sizes fit what is
+ * left of the budget is taken (sum formed in double in priority order; equal sums go to the subset that,
+ * written as a bit string over the priority order with the first fragment as lowest bit, is the smaller
+ * number).  If nothing was taken at all, the first fragment of the order is (a decision always returns one).
+ * ids lists the forced fragments first, then the subset in priority order.  At most
+ * COCODC_EXACT_MAX_CANDIDATES fragments may remain for the subset search (it enumerates all subsets); more
+ * selects nothing and sets COCODC_ERR_INVALID_ARG in the status word.
  */
 cocodc_status cocodc_select_fragments(cocodc_ctx* ctx, const float* scores, const int64_t* last_sync,
                                       const uint8_t* ineligible, int64_t t_now, int64_t H,

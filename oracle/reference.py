@@ -30,7 +30,7 @@ from . import build as _build
 
 COMP_NONE, COMP_TAYLOR = 0, 1
 SIGN_FORWARD, SIGN_PRINTED, SIGN_DESCENT = 0, 1, 2
-BUDGET_COUNT, BUDGET_PARAMS = 0, 1
+BUDGET_COUNT, BUDGET_PARAMS, BUDGET_PARAMS_EXACT = 0, 1, 2
 
 _lib = None
 
@@ -142,13 +142,20 @@ def select_fragments(scores: Sequence[float], last_sync: Sequence[int], sizes: S
     to the lower index (Eq. 11; +inf marks never-synced fragments).  The head
     of the order is always taken (Algorithm 2 always returns a fragment); each
     later fragment is taken iff its cost (1, or its size) still fits.
+
+    BUDGET_PARAMS_EXACT is an option outside the paper (its Algorithm 2 returns one fragment per decision):
+    the walk stops at the first fragment that is neither overdue nor never-synced (score +inf); the fragments
+    from there on are a knapsack, solved by trying every subset -- largest sum of scores (added in priority
+    order) among those whose sizes fit the rest of the budget, equal sums to the subset tried first when
+    subsets are numbered with the first fragment of the order as the lowest bit.  If nothing at all was taken,
+    the first fragment of the order is.
     Returns (mask uint8[K], ids int32[n_sel] in admission order, n_sel).
     """
     K = len(scores)
     R = [float(s) for s in scores]
     if any(math.isnan(r) for r in R):
         raise ValueError("NaN score")
-    if budget < 0 or budget_kind not in (BUDGET_COUNT, BUDGET_PARAMS):
+    if budget < 0 or budget_kind not in (BUDGET_COUNT, BUDGET_PARAMS, BUDGET_PARAMS_EXACT):
         raise ValueError("bad budget")
     elig = [p for p in range(K) if ineligible is None or not ineligible[p]]
     overdue = [p for p in elig if int(t_now) - int(last_sync[p]) >= H]
@@ -158,12 +165,33 @@ def select_fragments(scores: Sequence[float], last_sync: Sequence[int], sizes: S
     mask = np.zeros(K, dtype=np.uint8)
     ids: List[int] = []
     remaining = int(budget)
+    free: List[int] = []
     for j, p in enumerate(order):
+        if budget_kind == BUDGET_PARAMS_EXACT and p not in overdue and R[p] != math.inf:
+            free = order[j:]
+            break
         cost = 1 if budget_kind == BUDGET_COUNT else int(sizes[p])
         if j == 0 or cost <= remaining:
             mask[p] = 1
             ids.append(p)
             remaining -= cost
+    if free:
+        best_value, best_subset = None, 0
+        for subset in range(1 << len(free)):
+            members = [p for j, p in enumerate(free) if (subset >> j) & 1]
+            if sum(int(sizes[p]) for p in members) > remaining:
+                continue
+            value = 0.0
+            for p in members:
+                value += R[p]
+            if best_value is None or value > best_value:
+                best_value, best_subset = value, subset
+        if best_subset == 0 and not ids:
+            best_subset = 1
+        for j, p in enumerate(free):
+            if (best_subset >> j) & 1:
+                mask[p] = 1
+                ids.append(p)
     return mask, np.asarray(ids, dtype=np.int32), len(ids)
 
 

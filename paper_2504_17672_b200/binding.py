@@ -19,7 +19,7 @@ from . import build as _build
 OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_NONFINITE, ERR_TIMEOUT, ERR_CUDA, ERR_NOMEM = range(8)
 COMP_NONE, COMP_TAYLOR = 0, 1
 SIGN_FORWARD, SIGN_PRINTED, SIGN_DESCENT = 0, 1, 2
-BUDGET_COUNT, BUDGET_PARAMS = 0, 1
+BUDGET_COUNT, BUDGET_PARAMS, BUDGET_PARAMS_EXACT = 0, 1, 2
 STAGE_OUTER, STAGE_MERGE, STAGE_SCORE, STAGE_ALL = 1, 2, 4, 7
 
 EXPORTS = (

@@ -402,12 +402,15 @@ cocodc_status select_impl(cocodc_ctx* c, const float* scores, const int64_t* las
                           int64_t* pool_offset, void* stream) {
   if (!c || !scores || !last_sync || !mask || !ids || !n_sel) return COCODC_ERR_INVALID_ARG;
   if (H < 1 || budget < 0) return COCODC_ERR_INVALID_ARG;
-  if (budget_kind != COCODC_BUDGET_COUNT && budget_kind != COCODC_BUDGET_PARAMS) return COCODC_ERR_INVALID_ARG;
+  if (budget_kind != COCODC_BUDGET_COUNT && budget_kind != COCODC_BUDGET_PARAMS &&
+      budget_kind != COCODC_BUDGET_PARAMS_EXACT)
+    return COCODC_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   k_select<<<1, kSelectThreads, 0, st>>>(c->K, scores, reinterpret_cast<const long long*>(last_sync), ineligible,
                                          c->d_frag_size, t_now, reinterpret_cast<const long long*>(t_now_dev), H, budget_kind, budget, mask, ids, n_sel,
-                                         reinterpret_cast<long long*>(pool_offset), c->d_status, (int)COCODC_ERR_NONFINITE);
+                                         reinterpret_cast<long long*>(pool_offset), c->d_status, (int)COCODC_ERR_NONFINITE,
+                                         (int)COCODC_ERR_INVALID_ARG);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }

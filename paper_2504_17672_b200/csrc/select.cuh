@@ -11,13 +11,14 @@
 namespace cocodc {
 
 constexpr int kSelectThreads = 1024;
+constexpr int kExactMaxFree = 24;    // knapsack candidates enumerated at most (2^24 subsets)
 
 __global__ void __launch_bounds__(kSelectThreads)
 k_select(int K, const float* __restrict__ scores, const long long* __restrict__ last_sync,
          const unsigned char* __restrict__ ineligible, const long long* __restrict__ frag_size,
          long long t_now, const long long* __restrict__ t_now_dev, long long H, int budget_kind, long long budget,
          unsigned char* __restrict__ mask, int* __restrict__ ids, int* __restrict__ n_sel,
-         long long* __restrict__ pool_offset, int* __restrict__ status, int err_nonfinite) {
+         long long* __restrict__ pool_offset, int* __restrict__ status, int err_nonfinite, int err_too_many) {
   __shared__ float s_score[kMaxK];
   __shared__ unsigned char s_class[kMaxK];  // 0 = ineligible, 1 = ordinary, 2 = overdue
   __shared__ int s_order[kMaxK];
@@ -63,22 +64,100 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     atomicAdd(&s_count, 1);
   }
   __syncthreads();
-  if (p != 0) return;
-  long long remaining = budget;
-  long long pool_pos = 0;   // next free element of the snapshot pool (kept a multiple of 4)
-  int n = 0;
+  // ---- the walk under the budget ---------------------------------------------------------------
+  // COUNT and PARAMS budgets: thread 0 walks the whole order.  EXACT (not in the paper): it walks only the
+  // fragments that must go first -- the overdue ones and those never synchronised (score +inf) -- and the
+  // rest of the order becomes a knapsack that all threads solve by enumeration below.
+  __shared__ long long s_remaining;
+  __shared__ long long s_pool_pos;   // next free element of the snapshot pool (kept a multiple of 4)
+  __shared__ int s_n;                // fragments admitted so far
+  __shared__ int s_free_begin;       // first position of the order that belongs to the knapsack
   const int n_elig = s_count;
-  for (int j = 0; j < n_elig; ++j) {
-    const int f = s_order[j];
-    const long long cost = (budget_kind == 0) ? 1 : frag_size[f];
-    if (j == 0 || cost <= remaining) {   // the head of the order is always taken
-      mask[f] = 1;
-      ids[n++] = f;
-      remaining -= cost;
-      if (pool_offset) {
-        pool_offset[f] = pool_pos;
-        pool_pos = (pool_pos + frag_size[f] + 3) & ~3LL;
+  const bool exact = (budget_kind == 2);
+  if (p == 0) {
+    long long remaining = budget, pool_pos = 0;
+    int n = 0, j = 0;
+    for (; j < n_elig; ++j) {
+      const int f = s_order[j];
+      if (exact && s_class[f] != 2 && s_score[f] != INFINITY) break;
+      const long long cost = (budget_kind == 0) ? 1 : frag_size[f];
+      if (j == 0 || cost <= remaining) {   // the head of the order is always taken
+        mask[f] = 1;
+        ids[n++] = f;
+        remaining -= cost;
+        if (pool_offset) {
+          pool_offset[f] = pool_pos;
+          pool_pos = (pool_pos + frag_size[f] + 3) & ~3LL;
+        }
       }
+    }
+    s_remaining = remaining; s_pool_pos = pool_pos; s_n = n; s_free_begin = j;
+  }
+  __syncthreads();
+  const int n_free = n_elig - s_free_begin;
+  if (!exact || n_free == 0) {
+    if (p == 0) *n_sel = s_n;
+    return;
+  }
+  if (n_free > kExactMaxFree) {      // too many candidates to enumerate: report it, select nothing
+    if (p < K) { mask[p] = 0; ids[p] = -1; if (pool_offset) pool_offset[p] = -1; }
+    if (p == 0) { *n_sel = 0; record_status(status, err_too_many); }
+    return;
+  }
+  // ---- knapsack over the remaining order by enumeration ------------------------------------------
+  // Subset m has bit j set when the j-th remaining fragment (in priority order) is in it.  Its value is the
+  // sum of the scores, added in double in that order; the best feasible subset wins, equal values go to
+  // the smaller m (which prefers fragments earlier in the order).
+  __shared__ double s_val[kExactMaxFree];
+  __shared__ long long s_size[kExactMaxFree];
+  __shared__ double s_best_val[kSelectThreads];
+  __shared__ unsigned s_best_mask[kSelectThreads];
+  if (p < n_free) {
+    const int f = s_order[s_free_begin + p];
+    s_val[p] = (double)s_score[f];
+    s_size[p] = frag_size[f];
+  }
+  __syncthreads();
+  const long long room = s_remaining;
+  double best_val = -1.0;            // below every feasible value only when scores are non-negative ...
+  unsigned best_mask = 0xffffffffu;  // ... so feasibility is tracked by the mask: all ones = none found
+  const unsigned total = 1u << n_free;
+  for (unsigned m = p; m < total; m += kSelectThreads) {
+    long long size = 0;
+    double val = 0.0;
+    for (int j = 0; j < n_free; ++j)
+      if ((m >> j) & 1u) { size += s_size[j]; val += s_val[j]; }
+    if (size <= room && (best_mask == 0xffffffffu || val > best_val)) { best_val = val; best_mask = m; }
+  }
+  s_best_val[p] = best_val;
+  s_best_mask[p] = best_mask;
+  __syncthreads();
+  for (int w = kSelectThreads / 2; w > 0; w >>= 1) {
+    if (p < w) {
+      const double v = s_best_val[p + w];
+      const unsigned m = s_best_mask[p + w];
+      const unsigned mine = s_best_mask[p];
+      if (m != 0xffffffffu && (mine == 0xffffffffu || v > s_best_val[p] || (v == s_best_val[p] && m < mine))) {
+        s_best_val[p] = v;
+        s_best_mask[p] = m;
+      }
+    }
+    __syncthreads();
+  }
+  if (p != 0) return;
+  unsigned chosen = s_best_mask[0];
+  if (chosen == 0xffffffffu) chosen = 0;             // nothing fits (the budget is already overdrawn)
+  if (chosen == 0 && s_n == 0) chosen = 1;           // a decision always returns a fragment (Algorithm 2)
+  int n = s_n;
+  long long pool_pos = s_pool_pos;
+  for (int j = 0; j < n_free; ++j) {
+    if (!((chosen >> j) & 1u)) continue;
+    const int f = s_order[s_free_begin + j];
+    mask[f] = 1;
+    ids[n++] = f;
+    if (pool_offset) {
+      pool_offset[f] = pool_pos;
+      pool_pos = (pool_pos + frag_size[f] + 3) & ~3LL;
     }
   }
   *n_sel = n;

@@ -55,6 +55,73 @@ def test_selection_matches_oracle_bit_for_bit(K):
             assert np.array_equal(got[:en], eids) and (got[en:] == -1).all()
 
 
+@pytest.mark.parametrize("K", [1, 3, 8, 12, 15])
+def test_exact_budget_selection_matches_oracle_bit_for_bit(K):
+    """The knapsack option (outside the paper): same subsets, same order, same pool places as the oracle's
+    search over all subsets, with forced (overdue / never-synced) and ineligible fragments mixed in."""
+    rng = np.random.default_rng(100 + K)
+    w, ctx, B = selection_problem(K, rng)
+    sizes = w.partition.frag_sizes
+    dev = "cuda"
+    mask = torch.zeros(K, dtype=torch.uint8, device=dev)
+    ids = torch.zeros(K, dtype=torch.int32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    pool_off = torch.zeros(K, dtype=torch.int64, device=dev)
+    for trial in range(10):
+        if trial % 2:
+            scores = rng.choice(np.array([0.0, 0.5, 1.0, 1.0, 2.5, 3.0, np.inf], dtype=np.float32), size=K)
+        else:
+            scores = rng.random(K).astype(np.float32)
+        last = np.where(rng.random(K) < 0.15, 0, 150).astype(np.int64)
+        inel = (rng.random(K) < 0.25).astype(np.uint8) if trial % 3 else None
+        budget = int(rng.integers(0, sizes.sum() + 1))
+        ctx.cocodc_select_fragments(torch.from_numpy(scores).to(dev), torch.from_numpy(last).to(dev),
+                                    None if inel is None else torch.from_numpy(inel).to(dev),
+                                    200, 100, B.BUDGET_PARAMS_EXACT, budget, mask, ids, n_sel, pool_off)
+        assert ctx.cocodc_poll_status() == 0
+        emask, eids, en = orc.select_fragments(scores, last, sizes, 200, 100, orc.BUDGET_PARAMS_EXACT, budget, inel)
+        assert int(n_sel.item()) == en
+        assert np.array_equal(np_(mask), emask)
+        got = np_(ids)
+        assert np.array_equal(got[:en], eids) and (got[en:] == -1).all()
+        po, pos = np_(pool_off), 0
+        for p in eids:
+            assert po[p] == pos
+            pos = (pos + int(sizes[p]) + 3) // 4 * 4
+        assert all(po[p] == -1 for p in range(K) if not emask[p])
+
+
+def test_exact_budget_at_the_candidate_limit():
+    """24 candidates (2^24 subsets): integer scores and sizes, so the optimum value is the textbook table's; one more
+    candidate is reported through the status word and selects nothing."""
+    from paper_2504_17672_b200 import binding as B
+    rng = np.random.default_rng(77)
+    for K, expect_error in ((24, False), (25, True)):
+        sizes = rng.integers(4, 60, size=K)
+        w, ctx, _ = selection_problem(K, rng, sizes=sizes)
+        R = rng.integers(1, 100, size=K).astype(np.float32)
+        budget = int(sizes.sum() // 3)
+        mask = torch.zeros(K, dtype=torch.uint8, device="cuda")
+        ids = torch.zeros(K, dtype=torch.int32, device="cuda")
+        n_sel = torch.full((1,), -5, dtype=torch.int32, device="cuda")
+        ctx.cocodc_select_fragments(torch.from_numpy(R).cuda(), torch.full((K,), 150, dtype=torch.int64, device="cuda"),
+                                    None, 200, 100, B.BUDGET_PARAMS_EXACT, budget, mask, ids, n_sel)
+        status = ctx.cocodc_poll_status()
+        if expect_error:
+            assert status == B.ERR_INVALID_ARG and int(n_sel.item()) == 0 and int(mask.sum().item()) == 0
+            continue
+        assert status == 0
+        n = int(n_sel.item())
+        chosen = np_(ids)[:n]
+        assert len(set(chosen.tolist())) == n and np_(mask).sum() == n
+        assert sizes[chosen].sum() <= budget
+        table = np.zeros(budget + 1)
+        for p in range(K):
+            for c in range(budget, int(sizes[p]) - 1, -1):
+                table[c] = max(table[c], table[c - int(sizes[p])] + float(R[p]))
+        assert float(R[chosen].sum()) == table[budget]
+
+
 def test_selection_rejects_nan_scores():
     rng = np.random.default_rng(1)
     w, ctx, B = selection_problem(6, rng)

@@ -119,7 +119,9 @@ def _py_pins():
     out = [pins.test_sync_budget_never_below_K, pins.test_budget_one_is_algorithm_2,
            pins.test_never_synced_fragments_go_first_in_index_order, pins.test_count_budget_brute_force,
            pins.test_params_budget_brute_force, pins.test_selection_is_deterministic_and_rejects_nan,
-           pins.test_norm_closed_forms, pins.test_unprocessed_fragments_are_not_reported_and_layouts_agree]
+           pins.test_norm_closed_forms, pins.test_unprocessed_fragments_are_not_reported_and_layouts_agree,
+           pins.test_exact_budget_matches_the_textbook_knapsack_table,
+           pins.test_exact_budget_forced_fragments_ties_and_head]
     for row in pins.rows("schedule_sizing.txt"):
         out.append(lambda row=row: pins.test_sync_budget_golden(row))
     return out
@@ -142,6 +144,9 @@ PY_MUTATIONS = [
     ("parameter budget counted in fragments", "select_fragments",
      lambda f: (lambda scores, last_sync, sizes, t_now, H, kind, budget, ineligible=None:
                 f(scores, last_sync, [1] * len(sizes), t_now, H, kind, budget, ineligible))),
+    ("exact budget falls back to the greedy walk", "select_fragments",
+     lambda f: (lambda scores, last_sync, sizes, t_now, H, kind, budget, ineligible=None:
+                f(scores, last_sync, sizes, t_now, H, min(kind, 1), budget, ineligible))),
     ("score not divided by the interval", "fragment_scores",
      lambda f: (lambda fragments, delta_g, interval=None: f(fragments, delta_g, None))),
 ]

@@ -402,6 +402,57 @@ def test_params_budget_brute_force():
         assert all(sizes[p] > left for p in elig if not mask[p])         # nothing skipped still fits
 
 
+def test_exact_budget_matches_the_textbook_knapsack_table():
+    """The subset search (an option outside the paper) against the 0/1-knapsack dynamic programme over
+    capacities: integer scores, so every sum is exact and the optimum value is unique."""
+    rng = np.random.default_rng(23)
+    for trial in range(40):
+        K = int(rng.integers(1, 11))
+        sizes = rng.integers(1, 30, size=K)
+        R = rng.integers(0, 50, size=K).astype(np.float32)
+        budget = int(rng.integers(0, sizes.sum() + 1))
+        last = np.full(K, 95)
+        mask, ids, n = orc.select_fragments(R, last, sizes, 100, 100, orc.BUDGET_PARAMS_EXACT, budget)
+        table = np.zeros(budget + 1)                                   # best value within capacity c
+        for p in range(K):
+            for c in range(budget, int(sizes[p]) - 1, -1):
+                table[c] = max(table[c], table[c - int(sizes[p])] + float(R[p]))
+        chosen = list(ids)
+        assert mask.sum() == n == len(set(chosen)) and all(mask[p] for p in chosen)
+        if sizes[chosen].sum() > budget:                                # only the always-admitted head may overdraw
+            assert n == 1 and table[budget] == 0.0 and chosen[0] == int(np.lexsort((np.arange(K), -R))[0])
+        else:
+            assert R[chosen].sum() == table[budget] or (table[budget] == 0.0 and n == 1)
+        g_mask, g_ids, _ = orc.select_fragments(R, last, sizes, 100, 100, orc.BUDGET_PARAMS, budget)
+        if sizes[list(g_ids)].sum() <= budget and sizes[chosen].sum() <= budget:
+            assert R[chosen].sum() >= R[list(g_ids)].sum()              # never worse than the greedy walk
+
+
+def test_exact_budget_forced_fragments_ties_and_head():
+    sizes = [10, 10, 10, 10, 10]
+    # fragment 3 overdue, fragment 1 never synced: both forced first (overdue before +inf), as in the greedy walk
+    R = np.array([5.0, np.inf, 7.0, 1.0, 6.0], dtype=np.float32)
+    last = [95, 95, 95, 0, 95]
+    mask, ids, n = orc.select_fragments(R, last, sizes, 100, 100, orc.BUDGET_PARAMS_EXACT, 40)
+    assert list(ids) == [3, 1, 2, 4]                                   # forced, then the best pair by score order
+    # equal scores and sizes, room for one: the fragment earlier in the order (lower index) wins
+    mask, ids, n = orc.select_fragments([2.0, 2.0, 2.0], [95] * 3, [10, 10, 10], 100, 100, orc.BUDGET_PARAMS_EXACT, 15)
+    assert list(ids) == [0]
+    # one big fragment beats two small ones where the greedy walk (score order) would take the small ones
+    R = [4.0, 3.0, 6.5]
+    mask, ids, n = orc.select_fragments(R, [95] * 3, [5, 5, 10], 100, 100, orc.BUDGET_PARAMS_EXACT, 10)
+    assert list(ids) == [0, 1]                                          # 7.0 > 6.5
+    mask, ids, n = orc.select_fragments([4.0, 2.0, 6.5], [95] * 3, [5, 5, 10], 100, 100, orc.BUDGET_PARAMS_EXACT, 10)
+    assert list(ids) == [2]                                             # 6.5 > 6.0
+    # nothing fits: a decision still returns the head of the order
+    mask, ids, n = orc.select_fragments([1.0, 9.0], [95] * 2, [50, 60], 100, 100, orc.BUDGET_PARAMS_EXACT, 10)
+    assert list(ids) == [1]
+    # ineligible fragments never enter
+    mask, ids, n = orc.select_fragments([1.0, 9.0, 3.0], [95] * 3, [5, 5, 5], 100, 100, orc.BUDGET_PARAMS_EXACT, 10,
+                                        [0, 1, 0])
+    assert list(ids) == [2, 0]
+
+
 def test_selection_is_deterministic_and_rejects_nan():
     R = np.array([1.0, 3.0, 3.0, np.inf], dtype=np.float32)
     a = orc.select_fragments(R, [0] * 4, [1] * 4, 10, 100, orc.BUDGET_COUNT, 3)
