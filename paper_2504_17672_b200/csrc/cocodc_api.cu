@@ -136,6 +136,26 @@ Variant pick_variant(int M) {
   }
 }
 
+template <int M>
+Variant inplace_variant() {
+  return Variant{k_outer_inplace<M>, kInplaceThreads, InplaceLayout<M>::kSmemBytes, true};
+}
+
+// the fused step with zero delay: the in-place pipeline for the staged worker counts
+Variant pick_zero_delay_variant(int M) {
+  switch (M) {
+    case 1: return inplace_variant<1>();
+    case 2: return inplace_variant<2>();
+    case 3: return inplace_variant<3>();
+    case 4: return inplace_variant<4>();
+    case 5: return inplace_variant<5>();
+    case 6: return inplace_variant<6>();
+    case 7: return inplace_variant<7>();
+    case 8: return inplace_variant<8>();
+    default: return Variant{k_outer_generic<MODE_FUSED, true>, kThreads, 0u, false};
+  }
+}
+
 Variant pick_variant(int M, int mode, bool same) {
   if (mode == MODE_FUSED_RECV) {   // one more stream per stage: staged up to four local workers
     switch (M) {
@@ -149,7 +169,7 @@ Variant pick_variant(int M, int mode, bool same) {
   if (mode == MODE_OUTER_ONLY) return pick_variant<MODE_OUTER_ONLY, false>(M);
   if (mode == MODE_PSEUDO_SUM) return pick_variant<MODE_PSEUDO_SUM, false>(M);
   if (mode == MODE_MERGE_ONLY) return same ? pick_variant<MODE_MERGE_ONLY, true>(M) : pick_variant<MODE_MERGE_ONLY, false>(M);
-  return same ? pick_variant<MODE_FUSED, true>(M) : pick_variant<MODE_FUSED, false>(M);
+  return same ? pick_zero_delay_variant(M) : pick_variant<MODE_FUSED, false>(M);
 }
 
 int variant_grid(cocodc_ctx* c, const Variant& v) {

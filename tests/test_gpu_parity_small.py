@@ -57,7 +57,7 @@ def test_no_compensation_is_streaming_diloco():
     check_step_against_oracle(prob, before, ids, 5, 7, orc_hyper(prob.w, comp_mode=orc.COMP_NONE, alpha=0.25))
 
 
-@pytest.mark.parametrize("M", [2, 4, 6])
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 6, 7, 8, 9])
 def test_zero_delay_blocking_sync(M):
     """w_snap == w_now: the DiLoCo case; every worker leaves with the new global state."""
     prob = make(M, seed=40)
