@@ -435,9 +435,21 @@ def run_micro(args):
         ("cocodc_pseudo_gradient_sum", 4 * M + 8, n,
          lambda: ctx.cocodc_pseudo_gradient_sum(b.w_snap, b.snap_stride, None, b.theta_g, M, scratch, ids, n_ids)),
         ("cocodc_outer_step_received", 12 * M + 20, n, received),
+        ("cocodc_outer_step_received_peers, 2 buffers of partial sums (all on this GPU)", 12 * M + 16 + 8, n,
+         lambda: received_peers(2)),
+        ("cocodc_outer_step_received_peers, 4 buffers of partial sums (all on this GPU)", 12 * M + 16 + 16, n,
+         lambda: received_peers(4)),
         ("cocodc_fragment_scores (all fragments)", 4, w.N,
          lambda: ctx.cocodc_fragment_scores(b.theta_g, None, norms, scores)),
     ]
+    more = [torch.zeros(w.N, device=device) for _ in range(3)]
+
+    def received_peers(R):
+        t[0] += w.tau
+        ctx.cocodc_outer_step_received_peers(hp, M * R, b.w_now, b.w_snap, b.now_stride, b.snap_stride, None,
+                                             b.theta_g, b.momentum, ([scratch] + more)[:R], None, ids, n_ids, t[0],
+                                             t[0] + w.tau, last_sync, norms, scores)
+
     if K <= B.NOALLOC_MAX_K and len(off) <= B.NOALLOC_MAX_SEGMENTS:
         rows.append(("cocodc_fragment_scores_noalloc (all fragments)", 4, w.N,
                      lambda: B.cocodc_fragment_scores_noalloc(w.N, ptr, off, ln, b.theta_g, None, norms, scores)))

@@ -271,6 +271,31 @@ cocodc_status cocodc_outer_step_received(cocodc_ctx* ctx, const cocodc_hyper* hy
                                          float* norms, float* scores, void* stream);
 
 /*
+ * The same step with the exchange of Section 2.1 folded in: instead of one all-reduced buffer the call takes
+ * the n_sums (1..COCODC_MAX_SUMS) buffers that cocodc_pseudo_gradient_sum wrote on the contributing devices
+ * and adds them itself, in the listed order, while it streams the fragment:
+ *   Delta = (delta_sums[0][i] + delta_sums[1][i] + ... ) / M_total      (fp32, left to right)
+ * so the summed pseudo-gradient is never written to or re-read from memory.  delta_sums is a HOST array of
+ * device pointers (dev fp32[N] each, 16-byte aligned); entries may point into other devices' memory that is
+ * mapped into this process (peer access, CUDA IPC or a symmetric-memory allocation): the kernel reads them
+ * with ordinary, non-multicast bulk loads, each element once.  Every device that lists the buffers in the same
+ * order computes bit-identical Delta, theta_g and momentum.  The caller orders the calls across devices: all
+ * cocodc_pseudo_gradient_sum calls must have completed before any device starts this call, and no buffer may
+ * be overwritten until every device has finished it (a barrier on the host, or stream events, before and
+ * after).  delta_g_out may be NULL or one of the listed buffers of THIS device (replaced by Delta in place).
+ * With n_sums == 1 this is cocodc_outer_step_received.
+ */
+#define COCODC_MAX_SUMS 8
+cocodc_status cocodc_outer_step_received_peers(cocodc_ctx* ctx, const cocodc_hyper* hyper, int32_t M_total,
+                                               float* w_now, const float* w_snap,
+                                               int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                               float* theta_g, float* momentum,
+                                               const float* const* delta_sums, int32_t n_sums,
+                                               float* delta_g_out, const int32_t* ids, const int32_t* n_ids,
+                                               int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                               float* norms, float* scores, void* stream);
+
+/*
  * S4-S5 alone (Algorithm 1, or Eq. 3 for COMP_NONE), given the new global state:
  * w_now[m][i] = (1-alpha)*w_now[m][i] + alpha*target_m with G = theta_g_new[i].
  * Together with cocodc_outer_step(stages without MERGE) this is the unfused path.

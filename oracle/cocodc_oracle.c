@@ -65,10 +65,10 @@ static double merged_value(double a, double b, double G, double lambda, double a
  * Returns sum_i Delta_i^2 accumulated in element order (for Eq. 10's norm).
  *
  * Worker-per-device deployment (Section 2.1: each worker all-reduces its pseudo-gradient): if
- * recv_sum is not NULL it holds, per element, the sum over ALL M_total workers of their
- * pseudo-gradients as delivered by the all-reduce (fp32), and Eq. 1's mean is recv_sum[i] / M_total;
- * the M local workers in snap/now are then only merged.  recv_sum == NULL: the mean is formed from
- * the M stacked workers as above.
+ * n_recv > 0, recv_sums[0..n_recv-1] hold, per element, sums of pseudo-gradients (fp32) that together
+ * cover ALL M_total workers - one buffer if the exchange has already added them up, one per contributing
+ * device otherwise - and Eq. 1's mean is their total / M_total; the M local workers in snap/now are then
+ * only merged.  n_recv == 0: the mean is formed from the M stacked workers as above.
  */
 double cocodc_oracle_outer_elements(
     long n, int M,
@@ -77,15 +77,18 @@ double cocodc_oracle_outer_elements(
     const float *theta_g, const float *u,
     double eta, double mu, double lambda, double alpha, long tau, long H,
     int comp_mode, int sign_mode, int do_merge,
-    const float *recv_sum, int M_total,
+    const float *const *recv_sums, int n_recv, int M_total,
     double *now_out, double *theta_g_out, double *u_out, double *delta_out)
 {
     long double sumsq = 0.0L;
     for (long i = 0; i < n; ++i) {
         double thg = (double)theta_g[i];
         double Delta;
-        if (recv_sum) {
-            Delta = (double)recv_sum[i] / (double)M_total;       /* Eq. 1 from the all-reduced sum */
+        if (n_recv > 0) {
+            double total = 0.0;                                  /* Eq. 1 from the exchanged sums */
+            for (int r = 0; r < n_recv; ++r)
+                total += (double)recv_sums[r][i];
+            Delta = total / (double)M_total;
         } else {
             /* pseudo-gradient of every worker (Section 2.1) and their mean, Eq. 1:
              * differences first, summed in worker order, then divided by M */

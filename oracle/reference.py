@@ -46,7 +46,7 @@ def _declare(lib):
     d, l, i, p = ctypes.c_double, ctypes.c_long, ctypes.c_int, ctypes.c_void_p
     lib.cocodc_oracle_outer_elements.restype = d
     lib.cocodc_oracle_outer_elements.argtypes = [
-        l, i, p, l, p, l, p, p, d, d, d, d, l, l, i, i, i, p, i, p, p, p, p]
+        l, i, p, l, p, l, p, p, d, d, d, d, l, l, i, i, i, p, i, i, p, p, p, p]
     lib.cocodc_oracle_pseudo_gradient_sum.restype = None
     lib.cocodc_oracle_pseudo_gradient_sum.argtypes = [l, i, p, l, p, p]
     lib.cocodc_oracle_merge_elements.restype = None
@@ -228,12 +228,15 @@ def outer_step(fragments: Fragments, hp: Hyper, w_now: np.ndarray, w_snap: np.nd
     w_now, w_snap: float32 [M, .]; theta_g, momentum: float32 [N].  w_snap is
     laid out like w_now unless snap_offset[p] gives fragment p's start inside a
     packed row.  Inputs are not modified.
-    recv_sum (float32 [N]) and M_total: the worker-per-device deployment of Section 2.1 - the all-reduced
-    sum of all M_total workers' pseudo-gradients is given, and the M local workers are only merged.
+    recv_sum and M_total: the worker-per-device deployment of Section 2.1 - the sum of all M_total workers'
+    pseudo-gradients is given, either all-reduced already (float32 [N]) or as the contributing devices' partial
+    sums (a sequence of float32 [N] arrays, added up here), and the M local workers are only merged.
     Returns (results {p: FragmentResult}, new last_sync int64[K]).
     """
+    recv_list = []
     if recv_sum is not None:
-        recv_sum = _f32(recv_sum)
+        recv_list = [_f32(recv_sum)] if isinstance(recv_sum, np.ndarray) and recv_sum.ndim == 1 \
+            else [_f32(x) for x in recv_sum]
         if not M_total or M_total < 1:
             raise ValueError("M_total must accompany recv_sum")
     lib = _clib()
@@ -272,7 +275,8 @@ def outer_step(fragments: Fragments, hp: Hyper, w_now: np.ndarray, w_snap: np.nd
                     _ptr(theta_g, off + lo), _ptr(momentum, off + lo),
                     hp.outer_lr, hp.momentum, hp.lam, hp.alpha, hp.tau, hp.H,
                     hp.comp_mode, hp.sign_mode, 1 if do_merge else 0,
-                    None if recv_sum is None else _ptr(recv_sum, off + lo), int(M_total or 0),
+                    (ctypes.c_void_p * max(1, len(recv_list)))(*[_ptr(x, off + lo) for x in recv_list]),
+                    len(recv_list), int(M_total or 0),
                     blk.ctypes.data if do_merge else None,
                     _ptr(out_g, pos + lo), _ptr(out_u, pos + lo), _ptr(out_d, pos + lo))
                 if do_merge:

@@ -28,7 +28,7 @@ EXPORTS = (
     "cocodc_poll_status", "cocodc_launch_count", "cocodc_status_string",
     "cocodc_fragment_scores_noalloc", "cocodc_selftest_bounded_wait",
     "cocodc_pseudo_gradient_sum", "cocodc_outer_step_received",
-    "cocodc_select_fragments_at", "cocodc_outer_step_at",
+    "cocodc_select_fragments_at", "cocodc_outer_step_at", "cocodc_outer_step_received_peers",
 )
 NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
@@ -99,6 +99,8 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_pseudo_gradient_sum.argtypes = [vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
     lib.cocodc_outer_step_received.argtypes = [vp, ctypes.POINTER(_Hyper), i32, vp, vp, i64, i64, vp, vp, vp, vp,
                                                vp, vp, vp, i64, i64, vp, vp, vp, vp]
+    lib.cocodc_outer_step_received_peers.argtypes = [vp, ctypes.POINTER(_Hyper), i32, vp, vp, i64, i64, vp, vp, vp,
+                                                     ctypes.POINTER(vp), i32, vp, vp, vp, i64, i64, vp, vp, vp, vp]
     lib.cocodc_poll_status.argtypes = [vp, vp]
     lib.cocodc_launch_count.argtypes = [vp]
     lib.cocodc_launch_count.restype = i64
@@ -258,6 +260,20 @@ class Context:
                                                _p(momentum), _p(delta_sum), _p(delta_g_out), _p(ids), _p(n_ids),
                                                int(t_p), int(t_l), _p(last_sync), _p(norms), _p(scores),
                                                _stream(stream)), "cocodc_outer_step_received")
+
+    def cocodc_outer_step_received_peers(self, hyper: Hyper, M_total: int, w_now, w_snap, now_stride: int,
+                                         snap_stride: int, snap_offset, theta_g, momentum, delta_sums, delta_g_out,
+                                         ids, n_ids, t_p: int, t_l: int, last_sync, norms, scores,
+                                         stream=None) -> None:
+        """delta_sums: sequence of device tensors (or integer device addresses, e.g. of peer-mapped buffers)."""
+        h = hyper._c()
+        addrs = [int(x) if isinstance(x, int) else x.data_ptr() for x in delta_sums]
+        arr = (ctypes.c_void_p * len(addrs))(*addrs)
+        _check(_lib.cocodc_outer_step_received_peers(self._h, ctypes.byref(h), int(M_total), _p(w_now), _p(w_snap),
+                                                     int(now_stride), int(snap_stride), _p(snap_offset), _p(theta_g),
+                                                     _p(momentum), arr, len(addrs), _p(delta_g_out), _p(ids),
+                                                     _p(n_ids), int(t_p), int(t_l), _p(last_sync), _p(norms),
+                                                     _p(scores), _stream(stream)), "cocodc_outer_step_received_peers")
 
     def cocodc_merge(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                      theta_g_new, ids, n_ids, stream=None) -> None:

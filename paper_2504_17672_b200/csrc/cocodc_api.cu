@@ -40,7 +40,7 @@ struct cocodc_ctx {
   int* d_status = nullptr;
   long long launches = 0;
   std::vector<std::pair<const void*, int>> occupancy;  // kernel -> resident CTAs per SM
-  std::vector<const void*> smem_opted_in;              // kernels whose dynamic shared memory limit was raised on this device
+  std::vector<std::pair<const void*, unsigned>> smem_opted_in;   // kernels opted in to large shared memory, with the size
   // host copy of the fragment table (host-buffer entry point walks it on the host)
   std::vector<int> h_frag_seg_ptr;
   std::vector<long long> h_seg_off, h_seg_len;
@@ -115,9 +115,15 @@ Variant staged_variant() {
 // caller has made the context's device current).
 void opt_in_shared_memory(cocodc_ctx* c, const void* kernel, unsigned bytes) {
   if (bytes <= 48u * 1024u) return;
-  for (const void* k : c->smem_opted_in) if (k == kernel) return;
+  for (auto& k : c->smem_opted_in) {
+    if (k.first != kernel) continue;
+    if (k.second >= bytes) return;
+    cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    k.second = bytes;
+    return;
+  }
   cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  c->smem_opted_in.push_back(kernel);
+  c->smem_opted_in.emplace_back(kernel, bytes);
 }
 
 // Worker counts 1..8 are staged through shared memory by TMA; larger M take the generic element loop.
@@ -156,13 +162,21 @@ Variant pick_zero_delay_variant(int M) {
   }
 }
 
-Variant pick_variant(int M, int mode, bool same) {
-  if (mode == MODE_FUSED_RECV) {   // one more stream per stage: staged up to four local workers
+// received-sum mode: n_recv more streams per stage, ring sized at run time; staged up to four local workers
+template <int M>
+Variant received_variant(int n_recv) {
+  const int loaded = StageLayout<M, MODE_FUSED_RECV, false>::kLoaded + n_recv;
+  return Variant{k_outer_tma<M, MODE_FUSED_RECV, false>, kTmaThreads,
+                 (unsigned)(stages_for(loaded) * loaded) * kTileBytes, true};
+}
+
+Variant pick_variant(int M, int mode, bool same, int n_recv = 0) {
+  if (mode == MODE_FUSED_RECV) {
     switch (M) {
-      case 1: return staged_variant<1, MODE_FUSED_RECV, false>();
-      case 2: return staged_variant<2, MODE_FUSED_RECV, false>();
-      case 3: return staged_variant<3, MODE_FUSED_RECV, false>();
-      case 4: return staged_variant<4, MODE_FUSED_RECV, false>();
+      case 1: return received_variant<1>(n_recv);
+      case 2: return received_variant<2>(n_recv);
+      case 3: return received_variant<3>(n_recv);
+      case 4: return received_variant<4>(n_recv);
       default: return Variant{k_outer_generic<MODE_FUSED_RECV, false>, kThreads, 0u, false};
     }
   }
@@ -179,7 +193,7 @@ int variant_grid(cocodc_ctx* c, const Variant& v) {
 // plan + streaming kernel for a device-resident id list
 cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool same, const int32_t* ids,
                            const int32_t* n_ids, const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
-  const Variant v = pick_variant(A.M, mode, same);
+  const Variant v = pick_variant(A.M, mode, same, A.n_recv);
   const int grid = variant_grid(c, v);
   opt_in_shared_memory(c, reinterpret_cast<const void*>(v.kernel), v.smem);
   cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, A.snap_stride, kThreads, st);
@@ -444,13 +458,16 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
                               const int32_t* ids, const int32_t* n_ids,
                               int64_t t_p, int64_t t_l, int64_t* last_sync,
                               float* norms, float* scores, uint32_t stages, void* stream,
-                              const float* delta_sum, int32_t M_total,
+                              const float* const* delta_sums, int32_t n_sums, int32_t M_total,
                               const int64_t* t_p_dev = nullptr, const int64_t* t_l_dev = nullptr) {
   cocodc_status s = check_hyper(c, h);
   if (s != COCODC_OK) return s;
-  const bool received = delta_sum != nullptr;
-  if (received && (M_total < h->M || stages != COCODC_STAGE_ALL)) return COCODC_ERR_INVALID_ARG;
-  if (received && !aligned16(delta_sum)) return COCODC_ERR_ALIGNMENT;
+  const bool received = n_sums > 0;
+  if (received && (M_total < h->M || stages != COCODC_STAGE_ALL || n_sums > kMaxRecv)) return COCODC_ERR_INVALID_ARG;
+  for (int r = 0; r < n_sums; ++r) {
+    if (!delta_sums[r]) return COCODC_ERR_INVALID_ARG;
+    if (!aligned16(delta_sums[r])) return COCODC_ERR_ALIGNMENT;
+  }
   if (!(stages & COCODC_STAGE_OUTER) || (stages & ~COCODC_STAGE_ALL)) return COCODC_ERR_INVALID_ARG;
   const bool do_merge = (stages & COCODC_STAGE_MERGE) != 0;
   const bool do_score = (stages & COCODC_STAGE_SCORE) != 0;
@@ -482,10 +499,11 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
       const Range rs = range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N));
       for (const Range& x : r) if (overlap(rs, x)) return COCODC_ERR_ALIAS;
     }
-    if (received) {   // delta_g_out may be the same buffer as delta_sum (updated in place), nothing else may
-      const Range rd = range_of(delta_sum, N);
+    // delta_g_out may be the same buffer as one of the sums (updated in place), nothing else may
+    for (int q = 0; q < n_sums; ++q) {
+      const Range rd = range_of(delta_sums[q], N);
       for (const Range& x : r)
-        if (overlap(rd, x) && !(delta_g_out == delta_sum && x.lo == rd.lo)) return COCODC_ERR_ALIAS;
+        if (overlap(rd, x) && !(delta_g_out == delta_sums[q] && x.lo == rd.lo)) return COCODC_ERR_ALIAS;
     }
   }
   DeviceGuard guard(c->device);
@@ -498,7 +516,8 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
   A.theta_g = theta_g;
   A.momentum = momentum;
   A.delta_out = delta_g_out;
-  A.delta_in = delta_sum;
+  for (int r = 0; r < n_sums; ++r) A.delta_in[r] = delta_sums[r];
+  A.n_recv = n_sums;
   A.plan = c->d_plan;
   A.hdr = c->d_hdr;
   A.partial = do_score ? c->d_partial : nullptr;
@@ -536,7 +555,7 @@ cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
                                 int64_t t_p, int64_t t_l, int64_t* last_sync,
                                 float* norms, float* scores, uint32_t stages, void* stream) {
   return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
-                         ids, n_ids, t_p, t_l, last_sync, norms, scores, stages, stream, nullptr, 0);
+                         ids, n_ids, t_p, t_l, last_sync, norms, scores, stages, stream, nullptr, 0, 0);
 }
 
 cocodc_status cocodc_outer_step_received(cocodc_ctx* c, const cocodc_hyper* h, int32_t M_total,
@@ -548,7 +567,21 @@ cocodc_status cocodc_outer_step_received(cocodc_ctx* c, const cocodc_hyper* h, i
                                          float* norms, float* scores, void* stream) {
   if (!delta_sum) return COCODC_ERR_INVALID_ARG;
   return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
-                         ids, n_ids, t_p, t_l, last_sync, norms, scores, COCODC_STAGE_ALL, stream, delta_sum, M_total);
+                         ids, n_ids, t_p, t_l, last_sync, norms, scores, COCODC_STAGE_ALL, stream, &delta_sum, 1, M_total);
+}
+
+cocodc_status cocodc_outer_step_received_peers(cocodc_ctx* c, const cocodc_hyper* h, int32_t M_total,
+                                               float* w_now, const float* w_snap,
+                                               int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
+                                               float* theta_g, float* momentum,
+                                               const float* const* delta_sums, int32_t n_sums,
+                                               float* delta_g_out, const int32_t* ids, const int32_t* n_ids,
+                                               int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                               float* norms, float* scores, void* stream) {
+  if (!delta_sums || n_sums < 1) return COCODC_ERR_INVALID_ARG;
+  return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
+                         ids, n_ids, t_p, t_l, last_sync, norms, scores, COCODC_STAGE_ALL, stream, delta_sums, n_sums,
+                         M_total);
 }
 
 cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
@@ -579,7 +612,7 @@ cocodc_status cocodc_outer_step_at(cocodc_ctx* c, const cocodc_hyper* h,
                                    float* norms, float* scores, uint32_t stages, void* stream) {
   if (!t_p || !t_l) return COCODC_ERR_INVALID_ARG;
   return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
-                         ids, n_ids, 0, 0, last_sync, norms, scores, stages, stream, nullptr, 0, t_p, t_l);
+                         ids, n_ids, 0, 0, last_sync, norms, scores, stages, stream, nullptr, 0, 0, t_p, t_l);
 }
 
 cocodc_status cocodc_pseudo_gradient_sum(cocodc_ctx* c, const float* w_snap, int64_t snap_stride,

@@ -26,6 +26,8 @@ enum : int { MODE_FUSED = 0, MODE_OUTER_ONLY = 1, MODE_MERGE_ONLY = 2, MODE_FUSE
 __host__ __device__ constexpr bool mode_updates_global(int mode) { return mode == MODE_FUSED || mode == MODE_OUTER_ONLY || mode == MODE_FUSED_RECV; }
 __host__ __device__ constexpr bool mode_merges(int mode) { return mode == MODE_FUSED || mode == MODE_MERGE_ONLY || mode == MODE_FUSED_RECV; }
 
+constexpr int kMaxRecv = 8;          // buffers of partial sums a received-sum step can add up
+
 struct OuterArgs {
   float* w_now;             // [M][now_stride]
   const float* w_snap;      // [M][snap_stride]
@@ -34,7 +36,8 @@ struct OuterArgs {
   float* theta_g;           // in/out (MODE_MERGE_ONLY: read only, the new global state)
   float* momentum;          // in/out
   float* delta_out;         // optional
-  const float* delta_in;    // MODE_FUSED_RECV: received sum of all workers' pseudo-gradients
+  const float* delta_in[kMaxRecv];   // MODE_FUSED_RECV: sums of pseudo-gradients, one buffer per contributing device
+  int n_recv;               // how many of them (added in this order, so every device that lists them alike gets the same bits)
   const SegPlan* plan;
   const PlanHeader* hdr;
   double* partial;          // nullptr: no score accumulation
@@ -56,6 +59,23 @@ __device__ __forceinline__ float4 ld4(const float* p) { return __ldcs(reinterpre
 __device__ __forceinline__ void st4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
 __device__ __forceinline__ float ld1(const float* p) { return __ldcs(p); }
 __device__ __forceinline__ void st1(float* p, float v) { __stcs(p, v); }
+
+// The received sum of Eq. 1: the listed buffers added in order (a single buffer when a collective has already
+// summed them; one buffer per device when they are read straight from the peers' memory).
+__device__ __forceinline__ float received_sum1(const OuterArgs& A, long long e) {
+  float s = ld1(A.delta_in[0] + e);
+  for (int r = 1; r < A.n_recv; ++r) s = __fadd_rn(s, ld1(A.delta_in[r] + e));
+  return s;
+}
+__device__ __forceinline__ float4 add4(float4 a, const float4& b) {
+  a.x = __fadd_rn(a.x, b.x); a.y = __fadd_rn(a.y, b.y); a.z = __fadd_rn(a.z, b.z); a.w = __fadd_rn(a.w, b.w);
+  return a;
+}
+__device__ __forceinline__ float4 received_sum4(const OuterArgs& A, long long e) {
+  float4 s = ld4(A.delta_in[0] + e);
+  for (int r = 1; r < A.n_recv; ++r) s = add4(s, ld4(A.delta_in[r] + e));
+  return s;
+}
 
 // ---- the arithmetic of one element -----------------------------------------
 // S2.  The sum of the workers' pseudo-gradients divided by M (Eq. 1).  For a power of two the
@@ -108,7 +128,7 @@ __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, 
   } else {
     float sum = 0.f;
     if (MODE == MODE_FUSED_RECV) {
-      sum = ld1(A.delta_in + e);
+      sum = received_sum1(A, e);
     } else {
       for (int m = 0; m < M; ++m) sum = __fadd_rn(sum, __fsub_rn(ld1(A.w_snap + m * A.snap_stride + snap_e), thg));
     }
@@ -150,7 +170,7 @@ struct Lane {
   __device__ __forceinline__ void load(const OuterArgs& A, long long e, long long snap_e) {
     thg = ld4(A.theta_g + e);
     if (mode_updates_global(MODE)) u = ld4(A.momentum + e);
-    if (MODE == MODE_FUSED_RECV) delta = ld4(A.delta_in + e);
+    if (MODE == MODE_FUSED_RECV) delta = received_sum4(A, e);
 #pragma unroll
     for (int m = 0; m < M; ++m) b[m] = ld4(A.w_snap + m * A.snap_stride + snap_e);
     if (kHasNow) {

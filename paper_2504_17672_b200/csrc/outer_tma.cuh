@@ -78,20 +78,28 @@ __device__ __forceinline__ void bulk_store(void* dst, unsigned src_smem, unsigne
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
+// Ring depth of the received-sum mode, whose stage size is known only at run time: about 72 KB of
+// copies in flight, at least two stages (host and device use the same function).
+__host__ __device__ constexpr int stages_for(int loaded_streams) {
+  const int raw = (72 * 1024) / (loaded_streams * (int)kTileBytes);
+  return raw < 2 ? 2 : (raw > kMaxStages ? kMaxStages : raw);
+}
+
 // ---- stage layout ----------------------------------------------------------------------------
-// Slots of kTileElems floats each: [recorded x nS][current x nN][global][momentum x nU][received sum x nR].
+// Slots of kTileElems floats each: [recorded x nS][current x nN][global][momentum x nU], then, in
+// MODE_FUSED_RECV, one slot per buffer of received sums (a run-time count, so that mode sizes its ring at
+// run time: stages_for()).
 template <int M, int MODE, bool SAME>
 struct StageLayout {
   static constexpr int nS = SAME ? 0 : M;
   static constexpr int nN = mode_merges(MODE) ? M : 0;
   static constexpr int nU = mode_updates_global(MODE) ? 1 : 0;
-  static constexpr int nR = (MODE == MODE_FUSED_RECV) ? 1 : 0;     // received sum of pseudo-gradients
   static constexpr int kSnap = 0;
   static constexpr int kNow = nS;
   static constexpr int kGlobal = nS + nN;
   static constexpr int kMomentum = kGlobal + 1;
   static constexpr int kDeltaIn = kMomentum + nU;
-  static constexpr int kLoaded = nS + nN + 1 + nU + nR;  // streams brought in by the producer
+  static constexpr int kLoaded = nS + nN + 1 + nU;       // streams brought in by the producer (plus the received sums)
   static constexpr unsigned kStageBytes = kLoaded * kTileBytes;
   // about 72 KB of copies in flight (see the note at the top), never fewer than two stages; the
   // read-heavy modes measure best with more: OUTER_ONLY (3 reads per write) one stage deeper,
@@ -110,11 +118,14 @@ template <int M, int MODE, bool SAME>
 __global__ void __launch_bounds__(kTmaThreads, 1)
 k_outer_tma(const OuterArgs A) {
   using L = StageLayout<M, MODE, SAME>;
-  constexpr int S = L::kStages;
+  constexpr bool kRecv = (MODE == MODE_FUSED_RECV);
+  const int n_recv = kRecv ? A.n_recv : 0;
+  const int loaded = L::kLoaded + n_recv;                       // streams per stage
+  const int S = kRecv ? stages_for(loaded) : L::kStages;        // a compile-time constant unless kRecv
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* const stages = reinterpret_cast<float*>(smem_raw);
-  __shared__ __align__(8) unsigned long long full_bar[S];
-  __shared__ __align__(8) unsigned long long empty_bar[S];
+  __shared__ __align__(8) unsigned long long full_bar[kMaxStages];
+  __shared__ __align__(8) unsigned long long empty_bar[kMaxStages];
   __shared__ volatile int s_fail;
 
   const int tid = threadIdx.x;
@@ -146,9 +157,9 @@ k_outer_tma(const OuterArgs A) {
       }
       if (s_fail) return;
       const unsigned bar = smem_u32(&full_bar[s]);
-      float* st = stages + (size_t)s * L::kLoaded * kTileElems;
+      float* st = stages + (size_t)s * loaded * kTileElems;
       const long long snap_e0 = e0 + (tw.sp.snap_off - tw.sp.off);
-      mbar_expect_tx(bar, L::kLoaded * kTileBytes);
+      mbar_expect_tx(bar, loaded * kTileBytes);
 #pragma unroll
       for (int m = 0; m < L::nS; ++m)
         bulk_load(smem_u32(st + (L::kSnap + m) * kTileElems), A.w_snap + m * A.snap_stride + snap_e0, kTileBytes, bar);
@@ -157,7 +168,8 @@ k_outer_tma(const OuterArgs A) {
         bulk_load(smem_u32(st + (L::kNow + m) * kTileElems), A.w_now + m * A.now_stride + e0, kTileBytes, bar);
       bulk_load(smem_u32(st + L::kGlobal * kTileElems), A.theta_g + e0, kTileBytes, bar);
       if (L::nU) bulk_load(smem_u32(st + L::kMomentum * kTileElems), A.momentum + e0, kTileBytes, bar);
-      if (L::nR) bulk_load(smem_u32(st + L::kDeltaIn * kTileElems), A.delta_in + e0, kTileBytes, bar);
+      for (int r = 0; r < n_recv; ++r)
+        bulk_load(smem_u32(st + (L::kDeltaIn + r) * kTileElems), A.delta_in[r] + e0, kTileBytes, bar);
       ++k;
     }
     return;
@@ -185,12 +197,15 @@ k_outer_tma(const OuterArgs A) {
       failed = true;
       break;
     }
-    const float* st = stages + (size_t)s * L::kLoaded * kTileElems;
+    const float* st = stages + (size_t)s * loaded * kTileElems;
     Lane<M, MODE, SAME> ln;
     auto slot = [&](int idx) -> const float4& { return reinterpret_cast<const float4*>(st + idx * kTileElems)[tid]; };
     ln.thg = slot(L::kGlobal);
     if (L::nU) ln.u = slot(L::kMomentum);
-    if (L::nR) ln.delta = slot(L::kDeltaIn);
+    if (kRecv) {
+      ln.delta = slot(L::kDeltaIn);
+      for (int r = 1; r < n_recv; ++r) ln.delta = add4(ln.delta, slot(L::kDeltaIn + r));
+    }
     if (SAME) {
 #pragma unroll
       for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kNow + m);

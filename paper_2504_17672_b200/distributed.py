@@ -4,14 +4,15 @@ M_total workers, and Eq. 1's sum over all workers is an all-reduce of the per-ra
     cocodc_pseudo_gradient_sum  ->  all-reduce of the listed fragments' ranges  ->  cocodc_outer_step_received
 
 The all-reduce is torch.distributed's (NCCL over NVLink on GPUs, gloo in CPU tests); received data lands
-in this rank's own memory before any kernel reads it.  The global state, the momentum and the schedule
+in this rank's own memory before any kernel reads it.  complete_fragments_peers is the variant without a
+collective: the step itself adds the ranks' sums, read from the peers' mapped memory.  The global state, the momentum and the schedule
 arrays are replicated: every rank computes the same outer update from the same reduced sum, which keeps
 them identical without further exchange (the determinism argument of Section 3.2).
 """
 
 from __future__ import annotations
 
-from typing import Iterable, Sequence, Tuple
+from typing import Callable, Iterable, Sequence, Tuple
 
 import torch
 import torch.distributed as dist
@@ -46,6 +47,28 @@ def complete_fragments(ctx, hyper, M_total: int, fragments, ids_host: Sequence[i
     ctx.cocodc_outer_step_received(hyper, M_total, w_now, w_snap, w_now.stride(0), w_snap.stride(0), snap_offset,
                                    theta_g, momentum, sum_buf, None, ids_dev, n_ids_dev, t_p, t_l,
                                    last_sync, norms, scores)
+
+
+def complete_fragments_peers(ctx, hyper, M_total: int, rank: int, sum_bufs: Sequence, ids_dev, n_ids_dev,
+                             w_now, w_snap, snap_offset, theta_g, momentum, t_p: int, t_l: int,
+                             last_sync, norms, scores, barrier: Callable[[], None]) -> None:
+    """The same completion with the exchange folded into the step: no all-reduce, every rank reads the other
+    ranks' pseudo-gradient sums straight from their memory while it streams the fragment.
+
+    sum_buf[r] is rank r's fp32 [N] buffer as seen from THIS process, for every rank in the same order:
+    sum_bufs[rank] a tensor of this device, the others tensors or integer device addresses of peer memory mapped
+    into this process (peer access between devices of one process, CUDA IPC handles, or a symmetric-memory
+    allocation).  `barrier()` must return only when the work every rank has issued so far has finished on its
+    device (for instance stream synchronisation followed by a process-group barrier): it separates the ranks'
+    writes of their sums from the reads by the others, and those reads from the next overwrite.  The sums are
+    added left to right in fp32 by every rank alike, so the replicated state stays bit-identical."""
+    own = sum_bufs[rank]
+    ctx.cocodc_pseudo_gradient_sum(w_snap, w_snap.stride(0), snap_offset, theta_g, hyper.M, own, ids_dev, n_ids_dev)
+    barrier()
+    ctx.cocodc_outer_step_received_peers(hyper, M_total, w_now, w_snap, w_now.stride(0), w_snap.stride(0),
+                                         snap_offset, theta_g, momentum, list(sum_bufs), None, ids_dev, n_ids_dev,
+                                         t_p, t_l, last_sync, norms, scores)
+    barrier()
 
 
 def combine_sharded_norms(norms_local: torch.Tensor, interval: torch.Tensor = None, group=None):

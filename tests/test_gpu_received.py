@@ -108,6 +108,138 @@ def test_two_devices_with_two_workers_each():
     assert_close(np_(devs[0].bufs.theta_g), np_(full.bufs.theta_g).astype(np.float64), TOL_PARAM, "vs stacked")
 
 
+@pytest.mark.parametrize("R,M_local", [(1, 2), (2, 1), (2, 2), (3, 1), (4, 1), (4, 4), (8, 1), (8, 3), (2, 5)])
+def test_partial_sums_added_inside_the_step(R, M_local):
+    """R devices' partial sums handed to the step as R buffers (on a deployment: the peers' mapped memory; here R
+    buffers of one GPU).  Against the oracle's total of the partial sums, and bit for bit against the single-buffer
+    entry point fed the same left-to-right fp32 sum."""
+    M_total = R * M_local
+    full = make(M_total, seed=300 + 10 * R + M_local, snap_layout="pool", pool_ids=[2, 4, 0])
+    w, frs, ids = full.w, fragments_of(full.w), [4, 0, 2]
+    before = full.host_state()
+    w_loc = w.with_(M=M_local)
+    sums = []
+    for d in range(R):                      # phase one on every "device": its local workers' pseudo-gradient sum
+        rows = slice(d * M_local, (d + 1) * M_local)
+        prob = GpuProblem(w_loc, synth.DeviceBuffers(theta_g=full.bufs.theta_g, momentum=full.bufs.momentum,
+                                                     w_now=full.bufs.w_now[rows], w_snap=full.bufs.w_snap[rows],
+                                                     snap_offset=full.bufs.snap_offset, scales=full.bufs.scales))
+        prob.set_ids(ids)
+        buf = torch.zeros(w.N, device="cuda")
+        b = prob.bufs
+        prob.ctx.cocodc_pseudo_gradient_sum(b.w_snap, full.bufs.snap_stride, b.snap_offset, b.theta_g, M_local, buf,
+                                            prob.ids, prob.n_ids)
+        sums.append(buf)
+    total = sums[0].clone()
+    for x in sums[1:]:
+        total += x                           # fp32, left to right: what the kernel does
+    out = {}
+    for which in ("peers", "single"):        # device 0 completes, once per entry point, from identical state
+        rows = slice(0, M_local)
+        bufs = synth.DeviceBuffers(theta_g=full.bufs.theta_g.clone(), momentum=full.bufs.momentum.clone(),
+                                   w_now=full.bufs.w_now[rows].clone(), w_snap=full.bufs.w_snap[rows].clone(),
+                                   snap_offset=full.bufs.snap_offset.clone(), scales=full.bufs.scales)
+        prob = GpuProblem(w_loc, bufs)
+        prob.set_ids(ids)
+        b = prob.bufs
+        delta = torch.zeros(w.N, device="cuda")
+        args = (b.w_now, b.w_snap, b.now_stride, b.snap_stride, b.snap_offset, b.theta_g, b.momentum)
+        tail = (delta, prob.ids, prob.n_ids, 8, 10, prob.last_sync, prob.norms, prob.scores)
+        if which == "peers":
+            prob.ctx.cocodc_outer_step_received_peers(prob.hyper(), M_total, *args, sums, *tail)
+        else:
+            prob.ctx.cocodc_outer_step_received(prob.hyper(), M_total, *args, total, *tail)
+        assert prob.poll() == 0
+        out[which] = (prob, delta)
+    pp, dp = out["peers"]
+    ps, ds = out["single"]
+    for x, y in ((pp.bufs.w_now, ps.bufs.w_now), (pp.bufs.theta_g, ps.bufs.theta_g), (pp.bufs.momentum, ps.bufs.momentum),
+                 (pp.scores, ps.scores), (pp.norms, ps.norms), (pp.last_sync, ps.last_sync), (dp, ds)):
+        assert torch.equal(x, y)
+    res, new_last = orc.outer_step(frs, orc_hyper(w, M=M_local), before["w_now"][:M_local], before["w_snap"][:M_local],
+                                   before["theta_g"], before["momentum"], ids, 8, 10, before["last_sync"],
+                                   snap_offset=before["snap_offset"], recv_sum=[np_(x) for x in sums], M_total=M_total)
+    after = pp.host_state()
+    for p in ids:
+        r = res[p]
+        assert_close(orc.gather_fragment(frs, after["theta_g"], p), r.theta_g, TOL_PARAM, "theta_g")
+        assert_close(orc.gather_fragment(frs, after["momentum"], p), r.momentum, TOL_PARAM, "momentum")
+        assert_close(orc.gather_fragment(frs, np_(dp), p), r.delta_g, TOL_PARAM, "delta_g")
+        wn = orc.gather_fragment(frs, after["w_now"], p)
+        for m in range(M_local):
+            assert_close(wn[m], r.w_now[m], TOL_PARAM, f"w_now[{m}]")
+        assert abs(after["norms"][p] - r.norm) <= TOL_NORM * r.norm
+    assert np.array_equal(after["last_sync"], new_last)
+
+
+def test_peer_glue_two_ranks_taken_in_turn():
+    """distributed.complete_fragments_peers for two ranks of two workers, run one after the other on one GPU: the
+    barrier of the rank that goes first stands in for the other rank's arrival (it runs that rank's phase one)."""
+    from paper_2504_17672_b200 import distributed as D
+    full = make(4, seed=240)
+    w, ids = full.w, [0, 3, 1]
+    ranks = []
+    for d in range(2):
+        bufs = synth.DeviceBuffers(theta_g=full.bufs.theta_g.clone(), momentum=full.bufs.momentum.clone(),
+                                   w_now=full.bufs.w_now[2 * d:2 * d + 2].clone(),
+                                   w_snap=full.bufs.w_snap[2 * d:2 * d + 2].clone(), snap_offset=None,
+                                   scales=full.bufs.scales)
+        prob = GpuProblem(w.with_(M=2), bufs)
+        prob.set_ids(ids)
+        ranks.append(prob)
+    sums = [torch.zeros(w.N, device="cuda") for _ in range(2)]
+    calls = []
+
+    def barrier_of_rank0():
+        calls.append("barrier")
+        if len(calls) == 1:                    # the other rank reaches the barrier: its sum is in place
+            p1 = ranks[1]
+            p1.ctx.cocodc_pseudo_gradient_sum(p1.bufs.w_snap, p1.bufs.snap_stride, None, p1.bufs.theta_g, 2, sums[1],
+                                              p1.ids, p1.n_ids)
+
+    for r, prob in enumerate(ranks):
+        b = prob.bufs
+        D.complete_fragments_peers(prob.ctx, prob.hyper(), 4, r, sums, prob.ids, prob.n_ids, b.w_now, b.w_snap, None,
+                                   b.theta_g, b.momentum, 5, 9, prob.last_sync, prob.norms, prob.scores,
+                                   barrier_of_rank0 if r == 0 else (lambda: None))
+        assert prob.poll() == 0
+    assert calls == ["barrier", "barrier"]
+    for k in ("theta_g", "momentum"):
+        assert torch.equal(getattr(ranks[0].bufs, k), getattr(ranks[1].bufs, k))     # replicated state: same bits
+    assert torch.equal(ranks[0].scores, ranks[1].scores)
+    full.set_ids(ids)
+    full.outer_step(5, 9)
+    assert_close(np_(ranks[0].bufs.theta_g), np_(full.bufs.theta_g).astype(np.float64), TOL_PARAM, "vs stacked")
+    for d in range(2):
+        assert_close(np_(ranks[d].bufs.w_now), np_(full.bufs.w_now[2 * d:2 * d + 2]).astype(np.float64), TOL_PARAM,
+                     "w_now vs stacked")
+
+
+def test_partial_sums_validation():
+    prob = make(2, seed=221)
+    b, B = prob.bufs, prob.B
+    prob.set_ids([0])
+    bufs = [torch.zeros(prob.w.N, device="cuda") for _ in range(9)]
+
+    def code(sums, out=None):
+        with pytest.raises(B.CocodcError) as e:
+            prob.ctx.cocodc_outer_step_received_peers(prob.hyper(), 4, b.w_now, b.w_snap, b.now_stride, b.snap_stride,
+                                                      None, b.theta_g, b.momentum, sums, out, prob.ids, prob.n_ids,
+                                                      1, 2, prob.last_sync, prob.norms, prob.scores)
+        return e.value.code
+
+    assert code([]) == B.ERR_INVALID_ARG
+    assert code(bufs) == B.ERR_INVALID_ARG                      # more than the eight buffers a step adds up
+    assert code([bufs[0], b.momentum]) == B.ERR_ALIAS
+    assert code([bufs[0], bufs[1][1:]]) == B.ERR_ALIGNMENT
+    assert code([bufs[0], 0]) == B.ERR_INVALID_ARG              # a null entry
+    # in place on one of the listed buffers is allowed
+    prob.ctx.cocodc_outer_step_received_peers(prob.hyper(), 4, b.w_now, b.w_snap, b.now_stride, b.snap_stride, None,
+                                              b.theta_g, b.momentum, bufs[:2], bufs[1], prob.ids, prob.n_ids, 1, 2,
+                                              prob.last_sync, prob.norms, prob.scores)
+    assert prob.poll() == 0
+
+
 def test_received_mode_validation():
     prob = make(2, seed=220)
     b, B = prob.bufs, prob.B

@@ -103,3 +103,29 @@ def test_reference_arm_runs_only_on_rank_zero(monkeypatch, capsys):
     import json
     line = json.loads(capsys.readouterr().out)
     assert line["impl"] == "reference" and line["value"] > 0 and line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_peer_glue_orders_sum_barrier_step_barrier():
+    """complete_fragments_peers (host logic only, a recording stand-in for the context): this rank's sum goes to its
+    own buffer, a barrier separates it from the step that reads every rank's buffer in rank order, and a second
+    barrier keeps the buffers alive until every rank has read them."""
+    from types import SimpleNamespace
+    import torch
+    from paper_2504_17672_b200 import distributed as D
+    log = []
+
+    class Recorder:
+        def cocodc_pseudo_gradient_sum(self, w_snap, stride, snap_offset, theta_g, M, out, ids, n_ids):
+            log.append(("sum", out, M))
+
+        def cocodc_outer_step_received_peers(self, hyper, M_total, w_now, w_snap, ns, ss, so, thg, mom, sums, dout,
+                                             ids, n_ids, t_p, t_l, last, norms, scores):
+            log.append(("step", list(sums), M_total, t_p, t_l))
+
+    bufs = ["rank0-buffer", "rank1-buffer", "rank2-buffer"]
+    t = torch.zeros(2, 8)
+    D.complete_fragments_peers(Recorder(), SimpleNamespace(M=2), 6, 1, bufs, None, None, t, t, None, None, None, 4, 7,
+                               None, None, None, lambda: log.append(("barrier",)))
+    assert [x[0] for x in log] == ["sum", "barrier", "step", "barrier"]
+    assert log[0][1] == "rank1-buffer" and log[0][2] == 2
+    assert log[2][1] == bufs and log[2][2:] == (6, 4, 7)

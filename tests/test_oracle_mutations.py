@@ -52,8 +52,9 @@ C_MUTATIONS = [
     ("sum of squares sums plain values", "s += (long double)x[i] * (long double)x[i];", "s += (long double)x[i];"),
     ("worker rows transposed in the merge", "double a = (double)now[(size_t)m * now_stride + i];\n                double b = (double)snap[(size_t)m * snap_stride + i];\n                now_out[(size_t)m * n + i] =",
      "double a = (double)now[(size_t)(M - 1 - m) * now_stride + i];\n                double b = (double)snap[(size_t)m * snap_stride + i];\n                now_out[(size_t)m * n + i] ="),
-    ("received sum divided by the local worker count", "Delta = (double)recv_sum[i] / (double)M_total;",
-     "Delta = (double)recv_sum[i] / (double)M;"),
+    ("received sum divided by the local worker count", "Delta = total / (double)M_total;",
+     "Delta = total / (double)M;"),
+    ("only the first device's partial sum is used", "for (int r = 0; r < n_recv; ++r)", "for (int r = 0; r < 1; ++r)"),
     ("per-device sum skips the last worker", "for (int m = 0; m < M; ++m)\n            sum += (double)snap[(size_t)m * snap_stride + i] - thg;",
      "for (int m = 0; m + 1 < M || m == 0; ++m)\n            sum += (double)snap[(size_t)m * snap_stride + i] - thg;"),
 ]

@@ -490,5 +490,11 @@ def test_received_sum_mode_equals_stacked_workers():
         np.testing.assert_array_equal(r.momentum, full.momentum)
         np.testing.assert_array_equal(r.w_now, full.w_now[d * 2:d * 2 + 2])
         assert r.norm == full.norm and list(last) == [12]
+        # the same from the two devices' partial sums, left for the step to add up
+        res2, _ = orc.outer_step(frs, hp2, np.ascontiguousarray(now[d * 2:d * 2 + 2]),
+                                 np.ascontiguousarray(snap[d * 2:d * 2 + 2]), thg, mom, [0], 10, 12, [0],
+                                 recv_sum=[parts[0].astype(np.float32), parts[1].astype(np.float32)], M_total=4)
+        np.testing.assert_array_equal(res2[0].theta_g, full.theta_g)
+        np.testing.assert_array_equal(res2[0].w_now, full.w_now[d * 2:d * 2 + 2])
     with pytest.raises(ValueError):
         orc.outer_step(frs, orc.Hyper(M=2), now[:2], snap[:2], thg, mom, [0], 10, 12, [0], recv_sum=total)
