@@ -14,7 +14,7 @@
 #include <vector>
 
 #include "outer.cuh"
-#include "outer_tma.cuh"
+#include "outer_ring.cuh"
 #include "plan.cuh"
 #include "select.cuh"
 
@@ -103,7 +103,17 @@ struct Variant {
   int threads;
   unsigned smem;
   bool one_cta_per_sm;   // staged kernel: persistent, one CTA per SM; otherwise sized by occupancy
+  int ring_slots = 0;    // k_outer_ring only
 };
+
+// Worker counts without a compile-time instance: the slot-ring kernel, or, when even the recorded values of
+// one tile do not fit its ring, the element loop.
+template <int MODE, bool SAME>
+Variant runtime_variant(int M) {
+  const int slots = ring_slots_for(MODE, M);
+  if (slots == 0) return Variant{k_outer_generic<MODE, SAME>, kThreads, 0u, false};
+  return Variant{k_outer_ring<MODE, SAME>, kRingThreads, (unsigned)slots * kTileBytes, true, slots};
+}
 
 template <int M, int MODE, bool SAME>
 Variant staged_variant() {
@@ -138,7 +148,7 @@ Variant pick_variant(int M) {
     case 6: return staged_variant<6, MODE, SAME>();
     case 7: return staged_variant<7, MODE, SAME>();
     case 8: return staged_variant<8, MODE, SAME>();
-    default: return Variant{k_outer_generic<MODE, SAME>, kThreads, 0u, false};
+    default: return runtime_variant<MODE, SAME>(M);
   }
 }
 
@@ -158,7 +168,7 @@ Variant pick_zero_delay_variant(int M) {
     case 6: return inplace_variant<6>();
     case 7: return inplace_variant<7>();
     case 8: return inplace_variant<8>();
-    default: return Variant{k_outer_generic<MODE_FUSED, true>, kThreads, 0u, false};
+    default: return runtime_variant<MODE_FUSED, true>(M);
   }
 }
 
@@ -177,7 +187,7 @@ Variant pick_variant(int M, int mode, bool same, int n_recv = 0) {
       case 2: return received_variant<2>(n_recv);
       case 3: return received_variant<3>(n_recv);
       case 4: return received_variant<4>(n_recv);
-      default: return Variant{k_outer_generic<MODE_FUSED_RECV, false>, kThreads, 0u, false};
+      default: return runtime_variant<MODE_FUSED_RECV, false>(M);
     }
   }
   if (mode == MODE_OUTER_ONLY) return pick_variant<MODE_OUTER_ONLY, false>(M);
@@ -198,7 +208,9 @@ cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool sam
   opt_in_shared_memory(c, reinterpret_cast<const void*>(v.kernel), v.smem);
   cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, A.snap_stride, kThreads, st);
   if (s != COCODC_OK) return s;
-  v.kernel<<<grid, v.threads, v.smem, st>>>(A);
+  OuterArgs args = A;
+  args.ring_slots = v.ring_slots;
+  v.kernel<<<grid, v.threads, v.smem, st>>>(args);
   c->launches++;
   *grid_out = grid;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
@@ -806,6 +818,7 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
         A.theta_g = d_thg;
         A.momentum = d_u;
         A.delta_out = delta_g_out ? d_delta : nullptr;
+        A.ring_slots = v.ring_slots;
         k_plan_chunk<<<1, 1, 0, st>>>(cnt, snap_on_device ? sbase + lo : 0, kThreads, c->d_plan, c->d_hdr);
         v.kernel<<<grid, v.threads, v.smem, st>>>(A);
         k_accumulate_chunk<<<1, kFinalizeThreads, 0, st>>>(c->d_partial, entries, c->d_frag_sumsq + j);

@@ -309,12 +309,54 @@ def test_bounded_wait_runs_out_and_leaves_the_context_usable():
     check_step_against_oracle(prob, before, ids, 2, 4, orc_hyper(prob.w))
 
 
+# several tiles per CTA (148 CTAs x 1024-element tiles), ragged edges, an odd start
+MANY_TILES = (1_300_000, [[(4, 600_001)], [(600_008, 650_000)], [(1_250_009, 40_000)]])
+
+
+@pytest.mark.parametrize("M", [9, 13, 16, 34, 49])
+def test_worker_counts_beyond_the_instantiated_ones(M):
+    """Run-time worker counts (slot-ring kernel; 49 recorded tiles no longer fit its ring, so the fused mode takes the
+    element loop there): fused step, unfused halves bit-identical to it, zero delay, and the two-phase calls."""
+    a = make(M, seed=500 + M, frs=MANY_TILES, snap_layout="pool", pool_ids=[1, 0, 2])
+    ids = [1, 0, 2]
+    a.set_ids(ids)
+    before = a.host_state()
+    delta = torch.full((a.w.N,), 7.0, dtype=torch.float32, device="cuda")
+    a.outer_step(t_p=10, t_l=12, delta_out=delta)
+    assert a.poll() == 0
+    check_step_against_oracle(a, before, ids, 10, 12, orc_hyper(a.w), delta_out=delta)
+    # S1-S3 + S6, then S4-S5: same bits as the fused step
+    b = make(M, seed=500 + M, frs=MANY_TILES, snap_layout="pool", pool_ids=[1, 0, 2])
+    b.set_ids(ids)
+    b.outer_step(10, 12, stages=1 | 4)
+    b.merge(b.bufs.theta_g)
+    # pseudo-gradient sum + received sum: same bits again
+    c = make(M, seed=500 + M, frs=MANY_TILES, snap_layout="pool", pool_ids=[1, 0, 2])
+    c.set_ids(ids)
+    cb = c.bufs
+    s = torch.zeros(c.w.N, device="cuda")
+    c.ctx.cocodc_pseudo_gradient_sum(cb.w_snap, cb.snap_stride, cb.snap_offset, cb.theta_g, M, s, c.ids, c.n_ids)
+    c.ctx.cocodc_outer_step_received(c.hyper(), M, cb.w_now, cb.w_snap, cb.now_stride, cb.snap_stride, cb.snap_offset,
+                                     cb.theta_g, cb.momentum, s, None, c.ids, c.n_ids, 10, 12, c.last_sync, c.norms,
+                                     c.scores)
+    assert b.poll() == 0 and c.poll() == 0
+    for other in (b, c):
+        for x, y in ((a.bufs.w_now, other.bufs.w_now), (a.bufs.theta_g, other.bufs.theta_g),
+                     (a.bufs.momentum, other.bufs.momentum), (a.scores, other.scores), (a.norms, other.norms)):
+            assert torch.equal(x, y)
+    # zero delay on the state the first step left
+    before = a.host_state()
+    a.outer_step(100, 100, hyper=a.hyper(tau=0), w_snap=a.bufs.w_now)
+    assert a.poll() == 0
+    check_step_against_oracle(a, before, ids, 100, 100, orc_hyper(a.w, tau=0), same=True)
+
+
 @pytest.mark.parametrize("seed", range(12))
 def test_random_partitions_layouts_and_modes(seed):
     """Randomised sweep: fragment tables with gaps, odd offsets and several segments, random worker counts,
     id lists, snapshot layouts (plain / packed pool with arbitrary offsets), sign modes, mixing factors."""
     rng = np.random.default_rng(1000 + seed)
-    M = int(rng.choice([1, 2, 3, 4, 4, 4, 6, 8]))
+    M = int(rng.choice([1, 2, 3, 4, 4, 4, 6, 8, 11]))
     K = int(rng.integers(1, 7))
     pos, frs = int(rng.integers(0, 9)), []
     for p in range(K):
