@@ -297,7 +297,7 @@ def run_ours(args):
         "gpu_launches": int(launches),
         "clocks": clocks.result,
         "roofline": {"bound": "hbm", "kernel": (f"{'k_outer_inplace' if args.variant == 'diloco' else 'k_outer_tma'}<{w.M}> (fused S1-S6)"
-                                               if w.M <= 8 else "k_outer_generic (fused S1-S6)"), "achieved": achieved, "peak": peak,
+                                               if w.M <= 8 else "k_outer_ring (fused S1-S6)"), "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "frac_of_nominal_8TBs": achieved / 8000.0, "bytes_per_param": bpp,
                      "ms_per_launch": outer_seconds / K * 1e3,
