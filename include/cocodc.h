@@ -278,7 +278,7 @@ cocodc_status cocodc_outer_step_received(cocodc_ctx* ctx, const cocodc_hyper* hy
  * so the summed pseudo-gradient is never written to or re-read from memory.  delta_sums is a HOST array of
  * device pointers (dev fp32[N] each, 16-byte aligned); entries may point into other devices' memory that is
  * mapped into this process (peer access, CUDA IPC or a symmetric-memory allocation): the kernel reads them
- * with ordinary, non-multicast bulk loads, each element once.  Every device that lists the buffers in the same
+ * with ordinary one-CTA bulk copies (no cluster-wide form), each element once.  Every device that lists the buffers in the same
  * order computes bit-identical Delta, theta_g and momentum.  The caller orders the calls across devices: all
  * cocodc_pseudo_gradient_sum calls must have completed before any device starts this call, and no buffer may
  * be overwritten until every device has finished it (a barrier on the host, or stream events, before and

@@ -15,7 +15,7 @@
 // About 80 KB of slots beyond those held are what the producer can have in flight.
 //
 // Waits are bounded and verdicts are taken per warp, as in k_outer_tma.  Only this GPU's memory and mapped
-// peer buffers of received sums are read, with non-multicast bulk loads.
+// peer buffers of received sums are read, with plain one-CTA bulk copies.
 #pragma once
 
 #include "outer_tma.cuh"

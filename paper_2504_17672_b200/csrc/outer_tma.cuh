@@ -17,7 +17,8 @@
 //
 // Every wait is bounded.  When one runs out the thread records COCODC_ERR_TIMEOUT, raises a flag the
 // others poll, and leaves; no thread waits on a barrier another thread could have abandoned.
-// Only this GPU's memory is read; no cluster multicast is used.
+// Every copy is a plain one-CTA bulk copy (no cluster-wide form); only this GPU's memory is read, apart from
+// buffers of received sums that the caller may have mapped from a peer.
 #pragma once
 
 #include "outer.cuh"
