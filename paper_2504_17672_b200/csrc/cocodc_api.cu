@@ -118,7 +118,7 @@ Variant runtime_variant(int M) {
 template <int M, int MODE, bool SAME>
 Variant staged_variant() {
   using L = StageLayout<M, MODE, SAME>;
-  return Variant{k_outer_tma<M, MODE, SAME>, kTmaThreads, L::kSmemBytes, true};
+  return Variant{k_outer_tma<M, MODE, SAME>, tma_threads(M), L::kSmemBytes, true};
 }
 
 // More than 48 KB of dynamic shared memory needs a one-time opt-in per kernel and device (the
@@ -176,7 +176,7 @@ Variant pick_zero_delay_variant(int M) {
 template <int M>
 Variant received_variant(int n_recv) {
   const int loaded = StageLayout<M, MODE_FUSED_RECV, false>::kLoaded + n_recv;
-  return Variant{k_outer_tma<M, MODE_FUSED_RECV, false>, kTmaThreads,
+  return Variant{k_outer_tma<M, MODE_FUSED_RECV, false>, tma_threads(M),
                  (unsigned)(stages_for(loaded) * loaded) * kTileBytes, true};
 }
 

@@ -25,8 +25,12 @@
 
 namespace cocodc {
 
-constexpr int kProducerThreads = 32;
-constexpr int kTmaThreads = kThreads + kProducerThreads;
+// Producer warps of k_outer_tma (one issuing thread each).  One thread starts a 4 KB copy every few hundred
+// cycles; from seven workers on (16 and more copies per tile) a second one shares the streams (measured: +0.5 %
+// at M = 7, +1.6 % at M = 8, nothing at M = 4 and 6, -1 % at M = 5).
+__host__ __device__ constexpr int tma_producers(int M) { return M >= 7 ? 2 : 1; }
+__host__ __device__ constexpr int tma_threads(int M) { return kThreads + 32 * tma_producers(M); }
+constexpr int kTmaThreads = kThreads + 32;      // kernels with a single producer warp
 constexpr unsigned kTileBytes = kTileElems * sizeof(float);   // one stream's share of a stage
 constexpr int kWaitLimit = 1 << 22;                           // polls of a barrier before giving up
 constexpr int kMaxStages = 10;
@@ -116,7 +120,7 @@ struct StageLayout {
 };
 
 template <int M, int MODE, bool SAME>
-__global__ void __launch_bounds__(kTmaThreads, 1)
+__global__ void __launch_bounds__(tma_threads(M), 1)
 k_outer_tma(const OuterArgs A) {
   using L = StageLayout<M, MODE, SAME>;
   constexpr bool kRecv = (MODE == MODE_FUSED_RECV);
@@ -141,9 +145,21 @@ k_outer_tma(const OuterArgs A) {
   }
   __syncthreads();
 
-  // ------------------------------------------------------------------ producer
+  // ------------------------------------------------------------------ producer(s)
+  // With two producers the streams of a stage are dealt out in turn; both wait for the stage to be free,
+  // the first arms the barrier with the whole byte count (a copy of the other that completes before that only
+  // runs the count negative for a moment: the phase cannot end before the arming arrival).
   if (tid >= kThreads) {
-    if (tid != kThreads) return;
+    if ((tid & 31) != 0) return;
+    constexpr int P = tma_producers(M);
+    const int me = (tid - kThreads) >> 5;
+    int turn = 0;
+    auto mine = [&]() -> bool {
+      if (P == 1) return true;
+      const bool yes = (turn == me);
+      turn = (turn + 1 == P) ? 0 : turn + 1;
+      return yes;
+    };
     TileWalker tw(A.plan, h.n_seg);
     int k = 0;   // staged tiles issued so far
     for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
@@ -160,17 +176,17 @@ k_outer_tma(const OuterArgs A) {
       const unsigned bar = smem_u32(&full_bar[s]);
       float* st = stages + (size_t)s * loaded * kTileElems;
       const long long snap_e0 = e0 + (tw.sp.snap_off - tw.sp.off);
-      mbar_expect_tx(bar, loaded * kTileBytes);
+      if (me == 0) mbar_expect_tx(bar, loaded * kTileBytes);
 #pragma unroll
       for (int m = 0; m < L::nS; ++m)
-        bulk_load(smem_u32(st + (L::kSnap + m) * kTileElems), A.w_snap + m * A.snap_stride + snap_e0, kTileBytes, bar);
+        if (mine()) bulk_load(smem_u32(st + (L::kSnap + m) * kTileElems), A.w_snap + m * A.snap_stride + snap_e0, kTileBytes, bar);
 #pragma unroll
       for (int m = 0; m < L::nN; ++m)
-        bulk_load(smem_u32(st + (L::kNow + m) * kTileElems), A.w_now + m * A.now_stride + e0, kTileBytes, bar);
-      bulk_load(smem_u32(st + L::kGlobal * kTileElems), A.theta_g + e0, kTileBytes, bar);
-      if (L::nU) bulk_load(smem_u32(st + L::kMomentum * kTileElems), A.momentum + e0, kTileBytes, bar);
+        if (mine()) bulk_load(smem_u32(st + (L::kNow + m) * kTileElems), A.w_now + m * A.now_stride + e0, kTileBytes, bar);
+      if (mine()) bulk_load(smem_u32(st + L::kGlobal * kTileElems), A.theta_g + e0, kTileBytes, bar);
+      if (L::nU && mine()) bulk_load(smem_u32(st + L::kMomentum * kTileElems), A.momentum + e0, kTileBytes, bar);
       for (int r = 0; r < n_recv; ++r)
-        bulk_load(smem_u32(st + (L::kDeltaIn + r) * kTileElems), A.delta_in[r] + e0, kTileBytes, bar);
+        if (mine()) bulk_load(smem_u32(st + (L::kDeltaIn + r) * kTileElems), A.delta_in[r] + e0, kTileBytes, bar);
       ++k;
     }
     return;
