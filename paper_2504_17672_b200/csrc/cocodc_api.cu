@@ -110,9 +110,9 @@ struct Variant {
 // one tile do not fit its ring, the element loop.
 template <int MODE, bool SAME>
 Variant runtime_variant(int M) {
-  const int slots = ring_slots_for(MODE, M);
-  if (slots == 0) return Variant{k_outer_generic<MODE, SAME>, kThreads, 0u, false};
-  return Variant{k_outer_ring<MODE, SAME>, kRingThreads, (unsigned)slots * kTileBytes, true, slots};
+  const int chunks = ring_chunks_for(MODE, M);
+  if (chunks == 0) return Variant{k_outer_generic<MODE, SAME>, kThreads, 0u, false};
+  return Variant{k_outer_ring<MODE, SAME>, kRingThreads, (unsigned)chunks * kChunkBytes, true, chunks};
 }
 
 template <int M, int MODE, bool SAME>

@@ -50,7 +50,7 @@ struct OuterArgs {
   float Mf;                 // divisor of Eq. 1 as float: M, or the total worker count in MODE_FUSED_RECV
   float inv_M;              // its reciprocal, exact when it is a power of two
   int M_pow2;               // 1 if the divisor is a power of two
-  int ring_slots;           // k_outer_ring: 4 KB slots in its shared-memory ring
+  int ring_slots;           // k_outer_ring: chunks in its shared-memory ring
 };
 
 // ---- memory access helpers -------------------------------------------------

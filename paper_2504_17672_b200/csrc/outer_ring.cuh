@@ -2,17 +2,20 @@
 // four local workers in the received-sum mode): the same arithmetic and the same TMA staging as
 // k_outer_tma, with the worker count a run-time value.
 //
-// Shared memory is a ring of 4 KB slots, each one tile of ONE stream, each with its own "full" and "empty"
-// barrier.  The producer thread walks the tiles and, per tile, issues the streams in the order the
-// arithmetic needs them:
-//     theta_g, momentum, received sums,            (what the mode reads of them)
-//     recorded values of workers 0 .. M-1,         (modes that form the local pseudo-gradient sum)
-//     then per worker its current values           (modes that merge; preceded by the recorded values of that
-//                                                   worker when they were not loaded above)
-// The consumers take the slots in the same order.  Slots are released as soon as their lane is in a register,
-// except the recorded values in the fused mode: they are needed twice (Eq. 1's sum, then Eq. 5-7 per worker),
-// so they stay in the ring until their worker has been merged, and the ring is sized M slots larger for it.
-// About 80 KB of slots beyond those held are what the producer can have in flight.
+// Shared memory is a ring of 16 KB chunks.  A chunk holds one tile (4 KB) of up to four streams and has one
+// "full" and one "empty" barrier.  Per tile the producers fill chunks in the order the arithmetic needs them:
+//     head   : theta_g, momentum, received sums            (what the mode reads of them, four to a chunk)
+//     sum    : recorded values of workers 0 .. M-1, four workers to a chunk   (modes that form the local sum)
+//     merge  : current values, four workers to a chunk (fused mode), or recorded and current values of two
+//              workers to a chunk (modes that merge without having summed)
+// and the consumers take them in the same order, four (two) workers at a time.  Chunks are handed back as soon
+// as their lanes are in registers, except the recorded values in the fused mode: they are needed twice (Eq. 1's
+// sum, then Eq. 5-7 per worker), so those chunks stay in the ring until their workers have been merged, and the
+// ring is that much larger.
+//
+// Why chunks: with one barrier pair per 4 KB stream-tile the kernel tops out near 6 million tiles per second and
+// SM (5.4 TB/s at M = 16, and the same 20 % short at M = 4) whatever the number of producers, the ring size or
+// the polling instruction; the cost sits in the per-barrier hand-shake, so four streams share one.
 //
 // Waits are bounded and verdicts are taken per warp, as in k_outer_tma.  Only this GPU's memory and mapped
 // peer buffers of received sums are read, with plain one-CTA bulk copies.
@@ -22,26 +25,27 @@
 
 namespace cocodc {
 
-constexpr int kRingMaxSlots = 54;      // 216 KB of the 227 KB a CTA may use
-constexpr int kRingFreeSlots = 20;     // slots beyond the held ones: what may be in flight (80 KB)
+constexpr int kChunkStreams = 4;                                   // stream-tiles per chunk
+constexpr unsigned kChunkBytes = kChunkStreams * kTileBytes;       // 16 KB
+constexpr int kRingMaxChunks = 13;                                 // 208 KB of the 227 KB a CTA may use
+constexpr int kRingFreeChunks = 6;                                 // chunks beyond the held ones: 96 KB in flight at most
+constexpr int kRingProducers = 4;                                  // producer threads (one per warp), a chunk each in turn
+constexpr int kRingThreads = kThreads + 32 * kRingProducers;
 
 __host__ __device__ constexpr bool mode_sums_locally(int mode) {
   return mode == MODE_FUSED || mode == MODE_OUTER_ONLY || mode == MODE_PSEUDO_SUM;
 }
-// recorded values stay in the ring from the sum to the merge
-__host__ __device__ constexpr int ring_held_slots(int mode, int M) {
-  return (mode_sums_locally(mode) && mode_merges(mode)) ? M : 0;
+// chunks of recorded values that stay in the ring from the sum to the merge
+__host__ __device__ constexpr int ring_held_chunks(int mode, int M) {
+  return (mode_sums_locally(mode) && mode_merges(mode)) ? (M + kChunkStreams - 1) / kChunkStreams : 0;
 }
 // 0: the worker count does not fit the ring (the caller falls back to the element loop)
-__host__ __device__ constexpr int ring_slots_for(int mode, int M) {
-  const int held = ring_held_slots(mode, M);
-  const int want = held + kRingFreeSlots;
-  const int slots = want > kRingMaxSlots ? kRingMaxSlots : want;
-  return slots >= held + 6 ? slots : 0;
+__host__ __device__ constexpr int ring_chunks_for(int mode, int M) {
+  const int held = ring_held_chunks(mode, M);
+  const int want = held + kRingFreeChunks;
+  const int chunks = want > kRingMaxChunks ? kRingMaxChunks : want;
+  return chunks >= held + 3 ? chunks : 0;
 }
-
-constexpr int kRingProducers = 4;      // producer threads (one per warp), taking the slots in turn
-constexpr int kRingThreads = kThreads + 32 * kRingProducers;
 
 template <int MODE, bool SAME>
 __global__ void __launch_bounds__(kRingThreads, 1)
@@ -51,15 +55,20 @@ k_outer_ring(const OuterArgs A) {
   constexpr bool kMerges = mode_merges(MODE);
   constexpr bool kLocalSum = mode_sums_locally(MODE);
   constexpr bool kRecv = (MODE == MODE_FUSED_RECV);
+  constexpr bool kHeld = kLocalSum && kMerges;          // recorded values wait in the ring for the merge
+  // merge phase: workers per chunk and streams per worker that are loaded then
+  constexpr int kMergeStreams = !kMerges ? 0 : kHeld ? (SAME ? 0 : 1) : (SAME ? 1 : 2);
+  constexpr int kMergeWorkers = (kMergeStreams == 2) ? 2 : 4;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* const ring = reinterpret_cast<float*>(smem_raw);
-  __shared__ __align__(8) unsigned long long full_bar[kRingMaxSlots];
-  __shared__ __align__(8) unsigned long long empty_bar[kRingMaxSlots];
+  __shared__ __align__(8) unsigned long long full_bar[kRingMaxChunks];
+  __shared__ __align__(8) unsigned long long empty_bar[kRingMaxChunks];
   __shared__ volatile int s_fail;
   const int tid = threadIdx.x;
   const int M = A.M;
-  const unsigned R = (unsigned)A.ring_slots;
+  const unsigned R = (unsigned)A.ring_slots;            // chunks in the ring
   const int n_recv = kRecv ? A.n_recv : 0;
+  const int n_head = 1 + (kUpdates ? 1 : 0) + n_recv;   // streams of the head
   const PlanHeader h = *A.hdr;
   if (tid == 0) {
     for (unsigned s = 0; s < R; ++s) {
@@ -72,47 +81,75 @@ k_outer_ring(const OuterArgs A) {
   __syncthreads();
 
   // ------------------------------------------------------------------ producers
-  // One thread issues a 4 KB copy (wait for the slot, arm its barrier, start the copy) every few hundred
-  // cycles, less than a tile of many workers needs; so kRingProducers threads share the slots round robin.
-  // Every slot has its own barriers, hence the order in which the threads get to issue does not matter.
+  // All walk the same chunk sequence; a producer fills the chunks whose turn is its own.  Every chunk has its own
+  // barriers, hence the order in which the producers get to issue does not matter.
   if (tid >= kThreads) {
     if ((tid & 31) != 0) return;
     const unsigned me = (unsigned)(tid - kThreads) >> 5;
     TileWalker tw(A.plan, h.n_seg);
-    unsigned s = 0, lap = 0;   // next slot of the ring, and how often the ring has been filled
-    unsigned turn = 0;         // whose slot the next one is
+    unsigned s = 0, lap = 0;   // next chunk of the ring, and how often the ring has been filled
+    unsigned turn = 0;         // whose chunk the next one is
     bool ok = true;
-    auto issue = [&](const float* src) {
-      if (!ok) return;
-      if (turn == me) {
+    // opens the next chunk for n streams; true if it is this producer's to fill
+    auto open = [&](int n, float*& dst, unsigned& bar) -> bool {
+      const bool mine = ok && (turn == me);
+      if (mine) {
         if (lap > 0 && (s_fail || !mbar_wait_bounded(smem_u32(&empty_bar[s]), (lap - 1) & 1))) {
           record_status(A.status, A.err_timeout);
           s_fail = 1;
           ok = false;
-          return;
+        } else {
+          bar = smem_u32(&full_bar[s]);
+          dst = ring + (size_t)s * (kChunkStreams * kTileElems);
+          mbar_expect_tx(bar, (unsigned)n * kTileBytes);
         }
-        const unsigned bar = smem_u32(&full_bar[s]);
-        mbar_expect_tx(bar, kTileBytes);
-        bulk_load(smem_u32(ring + (size_t)s * kTileElems), src, kTileBytes, bar);
       }
       if (++turn == kRingProducers) turn = 0;
       if (++s == R) { s = 0; ++lap; }
+      return mine && ok;
+    };
+    auto copy = [&](float* dst, int j, const float* src, unsigned bar) {
+      bulk_load(smem_u32(dst + j * kTileElems), src, kTileBytes, bar);
     };
     for (int tile = blockIdx.x; tile < h.total_tiles && ok; tile += gridDim.x) {
       tw.seek(tile);
       const long long e0 = tw.tile_start(tile);
       if (!tw.interior(e0)) continue;
       const long long snap_e0 = e0 + (tw.sp.snap_off - tw.sp.off);
-      issue(A.theta_g + e0);
-      if (kUpdates) issue(A.momentum + e0);
-      for (int r = 0; r < n_recv; ++r) issue(A.delta_in[r] + e0);
+      float* dst = nullptr;
+      unsigned bar = 0;
+      // head: stream i of the head is theta_g, then momentum (if read), then the received sums
+      for (int i0 = 0; i0 < n_head; i0 += kChunkStreams) {
+        const int cnt = (n_head - i0 < kChunkStreams) ? n_head - i0 : kChunkStreams;
+        if (!open(cnt, dst, bar)) continue;
+        for (int j = 0; j < cnt; ++j) {
+          const int i = i0 + j;
+          const float* src = (i == 0) ? A.theta_g + e0
+                           : (kUpdates && i == 1) ? A.momentum + e0
+                           : A.delta_in[i - 1 - (kUpdates ? 1 : 0)] + e0;
+          copy(dst, j, src, bar);
+        }
+      }
       if (kLocalSum)
-        for (int m = 0; m < M; ++m)
-          issue(SAME ? A.w_now + m * A.now_stride + e0 : A.w_snap + m * A.snap_stride + snap_e0);
-      if (kMerges && !(SAME && kLocalSum))      // fused zero delay: the current values are already in the ring
-        for (int m = 0; m < M; ++m) {
-          if (!kLocalSum && !SAME) issue(A.w_snap + m * A.snap_stride + snap_e0);
-          issue(A.w_now + m * A.now_stride + e0);
+        for (int m0 = 0; m0 < M; m0 += kChunkStreams) {
+          const int cnt = (M - m0 < kChunkStreams) ? M - m0 : kChunkStreams;
+          if (!open(cnt, dst, bar)) continue;
+          for (int j = 0; j < cnt; ++j)
+            copy(dst, j, SAME ? A.w_now + (m0 + j) * A.now_stride + e0
+                              : A.w_snap + (m0 + j) * A.snap_stride + snap_e0, bar);
+        }
+      if (kMergeStreams > 0)
+        for (int m0 = 0; m0 < M; m0 += kMergeWorkers) {
+          const int cnt = (M - m0 < kMergeWorkers) ? M - m0 : kMergeWorkers;
+          if (!open(cnt * kMergeStreams, dst, bar)) continue;
+          for (int j = 0; j < cnt; ++j) {
+            if (kMergeStreams == 2) {
+              copy(dst, 2 * j, A.w_snap + (m0 + j) * A.snap_stride + snap_e0, bar);
+              copy(dst, 2 * j + 1, A.w_now + (m0 + j) * A.now_stride + e0, bar);
+            } else {
+              copy(dst, j, A.w_now + (m0 + j) * A.now_stride + e0, bar);
+            }
+          }
         }
     }
     return;
@@ -121,10 +158,9 @@ k_outer_ring(const OuterArgs A) {
   // ------------------------------------------------------------------ consumers
   SlotAccumulator sa(kThreads / 32);
   TileWalker tw(A.plan, h.n_seg);
-  unsigned cs = 0, cphase = 0;   // next slot to take and the phase of its "full" barrier (kept incrementally:
-                                 // a division per slot and thread would cost more than the arithmetic)
+  unsigned cs = 0, cphase = 0;   // next chunk to take and the phase of its "full" barrier
   bool failed = false;
-  // waits for the next slot; the verdict is the warp's
+  // waits for the next chunk; the verdict is the warp's
   auto landed = [&]() -> bool {
     const bool ok = mbar_wait_bounded(smem_u32(&full_bar[cs]), cphase);
     if (__all_sync(0xffffffffu, ok)) return true;
@@ -133,24 +169,16 @@ k_outer_ring(const OuterArgs A) {
     failed = true;
     return false;
   };
-  auto lane_of = [&](unsigned slot) -> float4 {
-    return reinterpret_cast<const float4*>(ring + (size_t)slot * kTileElems)[tid];
+  // this thread's lane of stream j of a chunk
+  auto lane_of = [&](unsigned chunk, int j) -> float4 {
+    return reinterpret_cast<const float4*>(ring + (size_t)chunk * (kChunkStreams * kTileElems) + j * kTileElems)[tid];
   };
-  // A slot is handed back once per warp, after every lane has read its part: with up to 2M + 2 slots per tile, one
-  // arrival per thread would make the barrier updates the bottleneck.
-  auto release = [&](unsigned slot) {
+  // a chunk is handed back once per warp, after every lane has read its part
+  auto release = [&](unsigned chunk) {
     __syncwarp();
-    if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty_bar[slot]));
+    if ((tid & 31) == 0) mbar_arrive(smem_u32(&empty_bar[chunk]));
   };
   auto advance = [&]() { if (++cs == R) { cs = 0; cphase ^= 1u; } };
-  // next slot: wait, read this thread's lane, release
-  auto take = [&](float4& v) -> bool {
-    if (!landed()) return false;
-    v = lane_of(cs);
-    release(cs);
-    advance();
-    return true;
-  };
 
   for (int tile = blockIdx.x; tile < h.total_tiles && !failed; tile += gridDim.x) {
     if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
@@ -160,28 +188,48 @@ k_outer_ring(const OuterArgs A) {
       continue;
     }
     const long long e = e0 + 4LL * tid;
+    // ---- head
     float4 thg, u, sum;
-    if (!take(thg)) break;
-    if (kUpdates && !take(u)) break;
-    if (kRecv) {
-      if (!take(sum)) break;
-      for (int r = 1; r < n_recv && !failed; ++r) {
-        float4 t;
-        if (take(t)) sum = add4(sum, t);
+    for (int i0 = 0; i0 < n_head && !failed; i0 += kChunkStreams) {
+      const int cnt = (n_head - i0 < kChunkStreams) ? n_head - i0 : kChunkStreams;
+      if (!landed()) break;
+      float4 v[kChunkStreams];
+#pragma unroll
+      for (int j = 0; j < kChunkStreams; ++j)
+        if (j < cnt) v[j] = lane_of(cs, j);
+      release(cs);
+      advance();
+#pragma unroll
+      for (int j = 0; j < kChunkStreams; ++j) {
+        if (j >= cnt) continue;
+        const int i = i0 + j;
+        if (i == 0) thg = v[j];
+        else if (kUpdates && i == 1) u = v[j];
+        else if (i == 1 + (kUpdates ? 1 : 0)) sum = v[j];            // first received sum
+        else sum = add4(sum, v[j]);                                  // the others, in the order listed
       }
-      if (failed) break;
     }
-    unsigned held = cs;                // slot of worker 0's recorded values (modes that sum locally)
+    if (failed) break;
+    // ---- Eq. 1's sum over the local workers
+    unsigned held = cs;                // chunk of workers 0-3's recorded values
     if (kLocalSum) {
-      for (int m = 0; m < M && !failed; ++m) {
+      for (int m0 = 0; m0 < M && !failed; m0 += kChunkStreams) {
+        const int cnt = (M - m0 < kChunkStreams) ? M - m0 : kChunkStreams;
         if (!landed()) break;
-        const float4 b = lane_of(cs);
-        if (!kMerges) release(cs);     // otherwise kept until worker m has been merged
+        float4 b[kChunkStreams];
+#pragma unroll
+        for (int j = 0; j < kChunkStreams; ++j)
+          if (j < cnt) b[j] = lane_of(cs, j);
+        if (!kHeld) release(cs);       // otherwise kept until these workers have been merged
         advance();
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float d = __fsub_rn(comp(b, k), comp(thg, k));
-          comp(sum, k) = (m == 0) ? d : __fadd_rn(comp(sum, k), d);
+        for (int j = 0; j < kChunkStreams; ++j) {
+          if (j >= cnt) continue;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float d = __fsub_rn(comp(b[j], k), comp(thg, k));
+            comp(sum, k) = (m0 + j == 0) ? d : __fadd_rn(comp(sum, k), d);
+          }
         }
       }
       if (failed) break;
@@ -190,6 +238,7 @@ k_outer_ring(const OuterArgs A) {
       st4(A.delta_out + e, sum);
       continue;
     }
+    // ---- Eq. 2
     float4 G = thg;
     if (kUpdates) {
       float4 delta;
@@ -207,30 +256,38 @@ k_outer_ring(const OuterArgs A) {
       st4(A.momentum + e, u);
       if (A.delta_out) st4(A.delta_out + e, delta);
     }
+    // ---- Eq. 3-7 per worker
     if (kMerges) {
-      for (int m = 0; m < M && !failed; ++m) {
-        float4 a, b;
-        if (kLocalSum) {
-          b = lane_of(held);                    // landed above, still held
-          if (SAME) {
-            a = b;
-          } else {
-            if (!landed()) break;
-            a = lane_of(cs);
-            release(cs);
-            advance();
-          }
-          release(held);
-          if (++held == R) held = 0;
-        } else {
-          if (!SAME && !take(b)) break;
-          if (!take(a)) break;
-          if (SAME) b = a;
-        }
-        float4 out;
+      float* wp = A.w_now + e;         // worker m's lane of this tile
+      for (int m0 = 0; m0 < M && !failed; m0 += kMergeWorkers) {
+        const int cnt = (M - m0 < kMergeWorkers) ? M - m0 : kMergeWorkers;
+        float4 a[kMergeWorkers], b[kMergeWorkers];
+        if (kMergeStreams > 0 && !landed()) break;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) comp(out, k) = merged(comp(a, k), comp(b, k), comp(G, k), A);
-        st4(A.w_now + m * A.now_stride + e, out);
+        for (int j = 0; j < kMergeWorkers; ++j) {
+          if (j >= cnt) continue;
+          if (kHeld) {
+            b[j] = lane_of(held, j);                     // landed during the sum, still in the ring
+            a[j] = SAME ? b[j] : lane_of(cs, j);
+          } else if (kMergeStreams == 2) {
+            b[j] = lane_of(cs, 2 * j);
+            a[j] = lane_of(cs, 2 * j + 1);
+          } else {                                       // merge only, zero delay
+            a[j] = lane_of(cs, j);
+            b[j] = a[j];
+          }
+        }
+        if (kMergeStreams > 0) { release(cs); advance(); }
+        if (kHeld) { release(held); if (++held == R) held = 0; }
+#pragma unroll
+        for (int j = 0; j < kMergeWorkers; ++j) {
+          if (j >= cnt) continue;
+          float4 out;
+#pragma unroll
+          for (int k = 0; k < 4; ++k) comp(out, k) = merged(comp(a[j], k), comp(b[j], k), comp(G, k), A);
+          st4(wp, out);
+          wp += A.now_stride;
+        }
       }
     }
   }
