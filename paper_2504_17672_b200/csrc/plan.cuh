@@ -51,67 +51,87 @@ k_plan(const int* __restrict__ ids, const int* __restrict__ n_ids_p, int K,
        const long long* __restrict__ seg_len, const long long* __restrict__ snap_offset,
        long long snap_row_len, int lanes_per_tile, int plan_capacity, SegPlan* __restrict__ plan,
        PlanHeader* __restrict__ hdr, int* __restrict__ status, int err_invalid) {
+  // Three steps, so that the chains of dependent global loads (id -> segment range -> segment) run side by side
+  // for all listed fragments instead of one fragment after the other: (1) every thread sizes its fragments,
+  // (2) one thread turns the sizes into running segment and tile counts, (3) every thread writes its
+  // fragments' table entries.
   __shared__ int seen[kMaxK];
+  __shared__ int s_frag[kMaxK];            // fragment id of list position j
+  __shared__ int s_seg_base[kMaxK];        // first table entry of position j (after step 2)
+  __shared__ long long s_tiles[kMaxK];     // tiles of position j, then (after step 2) its first tile
   __shared__ int bad;
   const int tid = threadIdx.x;
   int n = (ids == nullptr) ? K : *n_ids_p;
   if (tid == 0) bad = (n < 0 || n > K) ? 1 : 0;
   for (int i = tid; i < K; i += blockDim.x) seen[i] = 0;
   __syncthreads();
-  if (!bad && ids != nullptr) {
-    for (int i = tid; i < n; i += blockDim.x) {
-      int p = ids[i];
-      if (p < 0 || p >= K) {
-        bad = 1;
-      } else if (atomicAdd(&seen[p], 1) != 0) {
-        bad = 1;
-      } else if (snap_offset != nullptr && snap_offset[p] < 0) {
-        bad = 1;  // the fragment has no slot in the snapshot pool
+  auto tiles_of = [&](long long off, long long len) -> long long {
+    const long long lanes = (off - (off & ~3LL) + len + 3) >> 2;
+    return (lanes + lanes_per_tile - 1) / lanes_per_tile;
+  };
+  if (!bad) {
+    for (int j = tid; j < n; j += blockDim.x) {
+      const int p = (ids == nullptr) ? j : ids[j];
+      if (p < 0 || p >= K) { bad = 1; continue; }
+      if (ids != nullptr && atomicAdd(&seen[p], 1) != 0) { bad = 1; continue; }
+      if (snap_offset != nullptr && snap_offset[p] < 0) { bad = 1; continue; }   // no slot in the snapshot pool
+      long long t = 0;
+      for (int sg = frag_seg_ptr[p]; sg < frag_seg_ptr[p + 1]; ++sg) t += tiles_of(seg_off[sg], seg_len[sg]);
+      s_frag[j] = p;
+      s_seg_base[j] = frag_seg_ptr[p + 1] - frag_seg_ptr[p];
+      s_tiles[j] = t;
+    }
+  }
+  __syncthreads();
+  if (tid == 0 && !bad) {
+    long long tiles = 0;
+    int ns = 0;
+    for (int j = 0; j < n; ++j) {
+      const int cnt = s_seg_base[j];
+      const long long t = s_tiles[j];
+      s_seg_base[j] = ns;
+      s_tiles[j] = tiles;
+      ns += cnt;
+      tiles += t;
+      if (ns > plan_capacity || tiles > 0x3fffffffLL) { bad = 1; break; }   // tile + gridDim.x must not wrap
+    }
+    if (!bad) {
+      hdr->total_tiles = (int)tiles;
+      hdr->n_seg = ns;
+      hdr->n_ids = n;
+      hdr->pad = 0;
+    }
+  }
+  __syncthreads();
+  if (!bad) {
+    for (int j = tid; j < n; j += blockDim.x) {
+      const int p = s_frag[j];
+      int ns = s_seg_base[j];
+      long long tiles = s_tiles[j];
+      long long pos = 0;  // elements of the fragment placed so far (packed snapshot layout)
+      for (int sg = frag_seg_ptr[p]; sg < frag_seg_ptr[p + 1]; ++sg) {
+        SegPlan sp;
+        sp.off = seg_off[sg];
+        sp.len = seg_len[sg];
+        sp.snap_off = (snap_offset != nullptr) ? snap_offset[p] + pos : sp.off;
+        sp.abase = sp.off & ~3LL;
+        sp.first_tile = (int)tiles;
+        sp.slot = j;
+        sp.frag = p;
+        sp.vec_ok = (((sp.snap_off - sp.off) & 3LL) == 0) ? 1 : 0;
+        // a packed snapshot must lie inside one row of the pool the caller described
+        if (snap_offset != nullptr && sp.snap_off + sp.len > snap_row_len) bad = 1;
+        plan[ns++] = sp;
+        tiles += tiles_of(sp.off, sp.len);
+        pos += sp.len;
       }
     }
   }
   __syncthreads();
-  if (tid != 0) return;
-  if (bad) {
+  if (tid == 0 && bad) {
     hdr->total_tiles = 0; hdr->n_seg = 0; hdr->n_ids = 0; hdr->pad = 0;
     record_status(status, err_invalid);
-    return;
   }
-  long long tiles = 0;
-  int ns = 0;
-  bool overflow = false;
-  for (int j = 0; j < n && !overflow; ++j) {
-    const int p = (ids == nullptr) ? j : ids[j];
-    long long pos = 0;  // elements of the fragment placed so far (packed snapshot layout)
-    for (int s = frag_seg_ptr[p]; s < frag_seg_ptr[p + 1]; ++s) {
-      if (ns >= plan_capacity) { overflow = true; break; }
-      SegPlan sp;
-      sp.off = seg_off[s];
-      sp.len = seg_len[s];
-      sp.snap_off = (snap_offset != nullptr) ? snap_offset[p] + pos : sp.off;
-      sp.abase = sp.off & ~3LL;
-      sp.first_tile = (int)tiles;
-      sp.slot = j;
-      sp.frag = p;
-      sp.vec_ok = (((sp.snap_off - sp.off) & 3LL) == 0) ? 1 : 0;
-      // a packed snapshot must lie inside one row of the pool the caller described
-      if (snap_offset != nullptr && sp.snap_off + sp.len > snap_row_len) { overflow = true; break; }
-      plan[ns++] = sp;
-      const long long lanes = (sp.off - sp.abase + sp.len + 3) >> 2;
-      tiles += (lanes + lanes_per_tile - 1) / lanes_per_tile;
-      pos += sp.len;
-      if (tiles > 0x3fffffffLL) { overflow = true; break; }  // tile + gridDim.x must not wrap
-    }
-  }
-  if (overflow) {
-    hdr->total_tiles = 0; hdr->n_seg = 0; hdr->n_ids = 0; hdr->pad = 0;
-    record_status(status, err_invalid);
-    return;
-  }
-  hdr->total_tiles = (int)tiles;
-  hdr->n_seg = ns;
-  hdr->n_ids = n;
-  hdr->pad = 0;
 }
 
 // ---------------------------------------------------------------------------

@@ -22,6 +22,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   __shared__ float s_score[kMaxK];
   __shared__ unsigned char s_class[kMaxK];  // 0 = ineligible, 1 = ordinary, 2 = overdue
   __shared__ int s_order[kMaxK];
+  __shared__ long long s_fsize[kMaxK];      // fragment sizes, so that the walk below reads no global memory
   __shared__ int s_nan;
   __shared__ int s_count;
   const int p = threadIdx.x;
@@ -33,6 +34,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     const bool elig = (ineligible == nullptr) || (ineligible[p] == 0);
     const bool overdue = (t_now - last_sync[p]) >= H;   // Algorithm 2's staleness test
     s_score[p] = r;
+    s_fsize[p] = frag_size[p];
     s_class[p] = elig ? (overdue ? 2 : 1) : 0;
     if (r != r) s_nan = 1;
     mask[p] = 0;
@@ -80,14 +82,14 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     for (; j < n_elig; ++j) {
       const int f = s_order[j];
       if (exact && s_class[f] != 2 && s_score[f] != INFINITY) break;
-      const long long cost = (budget_kind == 0) ? 1 : frag_size[f];
+      const long long cost = (budget_kind == 0) ? 1 : s_fsize[f];
       if (j == 0 || cost <= remaining) {   // the head of the order is always taken
         mask[f] = 1;
         ids[n++] = f;
         remaining -= cost;
         if (pool_offset) {
           pool_offset[f] = pool_pos;
-          pool_pos = (pool_pos + frag_size[f] + 3) & ~3LL;
+          pool_pos = (pool_pos + s_fsize[f] + 3) & ~3LL;
         }
       }
     }
@@ -115,7 +117,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   if (p < n_free) {
     const int f = s_order[s_free_begin + p];
     s_val[p] = (double)s_score[f];
-    s_size[p] = frag_size[f];
+    s_size[p] = s_fsize[f];
   }
   __syncthreads();
   const long long room = s_remaining;
@@ -157,7 +159,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     ids[n++] = f;
     if (pool_offset) {
       pool_offset[f] = pool_pos;
-      pool_pos = (pool_pos + frag_size[f] + 3) & ~3LL;
+      pool_pos = (pool_pos + s_fsize[f] + 3) & ~3LL;
     }
   }
   *n_sel = n;
