@@ -45,7 +45,7 @@ def test_tiny_three_rounds():
 def test_gpt2_small_full_parity():
     w = synth.get_workload("gpt2_small")
     prob = GpuProblem(w, synth.generate(w, "cuda"))
-    # round 0: complete every fragment once (the start-up round of the schedule): full element-wise parity
+    # first pass: complete every fragment once (the schedule's start-up): full element-wise parity
     all_ids = list(range(w.K))
     prob.set_ids(all_ids)
     before = prob.host_state()
@@ -53,7 +53,7 @@ def test_gpt2_small_full_parity():
     assert prob.poll() == 0
     check_step_against_oracle(prob, before, all_ids, 10, 10 + w.tau, orc_hyper(w))
     del before
-    # round 1: local training moves on, then selection under the 25 % parameter budget
+    # second pass: local training moves on, then selection under the 25 % parameter budget
     prob.snapshot()
     g = torch.Generator(device="cuda").manual_seed(11)
     for m in range(w.M):
