@@ -11,7 +11,7 @@
 //
 // The scratch is the per-CTA, per-warp partial sums of squares that the regular
 // cocodc_fragment_scores keeps in context memory.  Here it is a file-scope __device__ array of
-// kNoallocScratchBytes (about 1.2 MB); every GPU that loads the library holds it until the process
+// kNoallocScratchBytes (592 KiB); every GPU that loads the library holds it until the process
 // exits.  Limits that follow from its size: at most COCODC_NOALLOC_MAX_K fragments and
 // COCODC_NOALLOC_MAX_SEGMENTS segments.
 #include "../../include/cocodc.h"
