@@ -114,3 +114,20 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
     import paper_2504_17672_b200.binding as binding
     with pytest.raises(ImportError):
         binding._load()
+
+
+def test_plain_c_client_compiles_links_and_runs(B, tmp_path):
+    """The header is C99 and the library needs nothing but itself: gcc builds tests/abi_client.c against both."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no gcc")
+    from paper_2504_17672_b200 import build
+    lib_dir = os.path.dirname(build.LIBRARY)
+    exe = str(tmp_path / "abi_client")
+    subprocess.run([gcc, "-std=c99", "-pedantic", "-Wall", "-Wextra", "-Werror", "-I", os.path.join(ROOT, "include"),
+                    os.path.join(ROOT, "tests", "abi_client.c"), "-o", exe, "-L", lib_dir, "-lcocodc",
+                    "-Wl,-rpath," + lib_dir], check=True)
+    out = subprocess.run([exe], check=True, capture_output=True, text=True).stdout
+    assert out.strip() == "abi client ok: N=8 h=12"
