@@ -479,6 +479,74 @@ def run_micro(args):
                       "status": int(status), "entries": out}))
 
 
+def run_workers(args):
+    """The fused step, the zero-delay step and the snapshot for a range of worker counts M on one fixed shape
+    (4 fragments of --workers-fragment parameters per worker): algorithmic GB/s from CUDA events.  M = 1..8 run the
+    compile-time instances of the staged kernel, larger M the chunk-ring kernel."""
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
+    from paper_2504_17672_b200 import binding as B
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    peak, peak_kind = read_peaks()
+    frag, K = int(args.workers_fragment), 4
+    n = frag * K
+    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = max(5, args.steps // 5)
+    out = []
+    status = 0
+    for M in (1, 2, 3, 4, 5, 6, 7, 8, 9, 12, 16, 24, 34):
+        w = synth.small_workload([frag] * K, M=M, seed=7, tau=4, name=f"workers_{M}")
+        b = synth.generate(w, device)
+        ptr, off, ln = w.partition.csr()
+        ctx = B.Context(w.N, ptr, off, ln, M, device=0)
+        ids = torch.arange(K, dtype=torch.int32, device=device)
+        n_ids = torch.tensor([K], dtype=torch.int32, device=device)
+        scores = torch.zeros(K, device=device)
+        norms = torch.zeros(K, device=device)
+        last_sync = torch.zeros(K, dtype=torch.int64, device=device)
+        hp = B.Hyper(M=M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam, alpha=w.alpha)
+        hp0 = B.Hyper(M=M, H=w.H, tau=0, outer_lr=w.outer_lr, momentum=w.momentum, lam=0.0, alpha=1.0,
+                      comp_mode=B.COMP_NONE)
+        t = [0]
+
+        def fused():
+            t[0] += w.tau
+            ctx.cocodc_outer_step(hp, b.w_now, b.w_snap, b.now_stride, b.snap_stride, None, b.theta_g, b.momentum,
+                                  None, ids, n_ids, t[0], t[0] + w.tau, last_sync, norms, scores, 7)
+
+        def zero_delay():
+            t[0] += w.tau
+            ctx.cocodc_outer_step(hp0, b.w_now, b.w_now, b.now_stride, b.now_stride, None, b.theta_g, b.momentum,
+                                  None, ids, n_ids, t[0], t[0], last_sync, norms, scores, 7)
+
+        def snapshot():
+            ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, None, M, ids, n_ids)
+
+        row = {"M": M, "params": n}
+        for name, bpp, fn in (("fused", 12 * M + 16, fused), ("zero_delay", 8 * M + 16, zero_delay),
+                              ("snapshot", 8 * M, snapshot)):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize(device)
+            ev_a.record()
+            for _ in range(reps):
+                fn()
+            ev_b.record()
+            torch.cuda.synchronize(device)
+            ms = ev_a.elapsed_time(ev_b) / reps
+            row[name] = {"bytes_per_param": bpp, "ms": ms, "gbs": n * bpp / ms / 1e6,
+                         "frac_of_peak": n * bpp / ms / 1e6 / peak}
+        status = status or int(ctx.cocodc_poll_status())
+        out.append(row)
+        ctx.close()
+        del b, ctx
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "fused_step_gbs_by_worker_count", "unit": "GB/s", "peak": peak,
+                      "peak_kind": f"of {peak_kind}", "launches_per_entry": reps, "params_per_launch": n,
+                      "status": status, "rows": out}))
+
+
 def kernel_source_sha() -> str:
     import hashlib
     h = hashlib.sha256()
@@ -672,6 +740,10 @@ def main():
     ap.add_argument("--variant", choices=["cocodc", "streaming_diloco", "diloco"], default="cocodc",
                     help="which method's arithmetic the step runs (the baselines are modes of the same kernels)")
     ap.add_argument("--micro", action="store_true", help="time every streaming entry point on its own")
+    ap.add_argument("--workers", action="store_true",
+                    help="time the fused step, the zero-delay step and the snapshot for M = 1..34 workers")
+    ap.add_argument("--workers-fragment", type=int, default=24 * 1024 * 1024,
+                    help="parameters per fragment (of 4) in the --workers shape")
     ap.add_argument("--sweep", action="store_true", help="time the 48 variants of the 1B compensation sweep")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
@@ -682,6 +754,8 @@ def main():
         run_sweep(args)
     elif args.micro:
         run_micro(args)
+    elif args.workers:
+        run_workers(args)
     else:
         run_ours(args)
 

@@ -124,7 +124,7 @@ Variant staged_variant() {
 // More than 48 KB of dynamic shared memory needs a one-time opt-in per kernel and device (the
 // caller has made the context's device current).
 void opt_in_shared_memory(cocodc_ctx* c, const void* kernel, unsigned bytes) {
-  if (bytes <= 48u * 1024u) return;
+  if (bytes <= 40u * 1024u) return;   // static shared memory counts towards the 48 KB a kernel gets without opting in
   for (auto& k : c->smem_opted_in) {
     if (k.first != kernel) continue;
     if (k.second >= bytes) return;

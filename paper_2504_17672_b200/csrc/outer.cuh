@@ -48,7 +48,7 @@ struct OuterArgs {
   float c1, c2;             // target = G + c1*d + c2*d*d*D
   float alpha, one_minus_alpha;
   float Mf;                 // divisor of Eq. 1 as float: M, or the total worker count in MODE_FUSED_RECV
-  float inv_M;              // its reciprocal, exact when it is a power of two
+  float inv_M;              // its reciprocal, correctly rounded (exact when the divisor is a power of two)
   int M_pow2;               // 1 if the divisor is a power of two
   int ring_slots;           // k_outer_ring: chunks in its shared-memory ring
 };
@@ -79,15 +79,26 @@ __device__ __forceinline__ float4 received_sum4(const OuterArgs& A, long long e)
 }
 
 // ---- the arithmetic of one element -----------------------------------------
-// S2.  The sum of the workers' pseudo-gradients divided by M (Eq. 1).  For a power of two the
-// product with 1/M is the correctly rounded quotient, bit for bit, and it has no data-dependent
-// slow path (the IEEE division routine branches on zero or tiny numerators, which costs bandwidth
-// once many elements have converged).  Other M use the IEEE division.
+// S2.  The sum of the workers' pseudo-gradients divided by M (Eq. 1).  The IEEE division routine branches
+// on zero or tiny numerators, and that data-dependent slow path costs bandwidth as soon as many elements
+// have converged (every pseudo-gradient is zero right after a blocking synchronisation), so no instruction
+// here divides.  For a power of two the product with 1/M is the correctly rounded quotient, bit for bit.
+// For any other M: q0 = RN(sum * RN(1/M)) is within an ulp of the quotient, the residual sum - q0*M comes
+// exactly out of one fused multiply-add, and q0 + residual * RN(1/M) rounds to the correctly rounded
+// quotient (the usual correction step of division by iteration; it holds while the residual does not
+// underflow, i.e. for |sum| above about 2^-100, below which the result may differ by one unit of its last
+// place).  Non-finite sums keep q0, which is what the division would give.
+__device__ __forceinline__ float quotient_by_count(float sum, float count, float inv_count) {
+  const float q0 = __fmul_rn(sum, inv_count);
+  const float r = __fmaf_rn(-q0, count, sum);
+  const float q = __fmaf_rn(r, inv_count, q0);
+  return (r != 0.0f && fabsf(q0) <= 3.402823466e+38f) ? q : q0;   // r == 0: q0 is exact (keeps the sign of a zero)
+}
 template <int M>
 __device__ __forceinline__ float mean_of_sum(float sum, const OuterArgs& A) {
   if constexpr (M > 0 && (M & (M - 1)) == 0) return __fmul_rn(sum, 1.0f / (float)M);
-  else if constexpr (M > 0) return __fdiv_rn(sum, (float)M);
-  else return A.M_pow2 ? __fmul_rn(sum, A.inv_M) : __fdiv_rn(sum, A.Mf);
+  else if constexpr (M > 0) return quotient_by_count(sum, (float)M, 1.0f / (float)M);
+  else return A.M_pow2 ? __fmul_rn(sum, A.inv_M) : quotient_by_count(sum, A.Mf, A.inv_M);
 }
 
 // S3.  u' = mu*u + Delta, G = thg + eta*(Delta + mu*u') (Eq. 2, Nesterov).

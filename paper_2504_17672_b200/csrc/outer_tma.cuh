@@ -371,16 +371,27 @@ k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long
 //              stage, proxy fence, arrive on "done" (one arrival per consumer thread);
 //   storer   : waits on "done", bulk stores of the stage to theta_g, momentum and w_now, waits until they
 //              have read shared memory, arrives on "empty".
-// Loader and storer are single threads of two further warps.  About 72 KB of stages in all measured best
-// (M = 4: 3 stages 6.62 TB/s, 2 stages 5.65, 4 stages 6.17; one thread doing both jobs 6.57).
+// Loader and storer are single threads of two further warps (one thread doing both jobs: 6.57 against 6.62 TB/s
+// at M = 4).  The ring depth per worker count is measured: inplace_stages().
 // ---------------------------------------------------------------------------------------------
 constexpr int kInplaceThreads = kThreads + 64;
+
+// Stages of the in-place ring per worker count (a stage is M + 2 tiles of 4 KB), measured on B200 with 2 to 6
+// stages each (GB/s of the zero-delay step, 100 M parameters per worker; the chosen depth first):
+//   M = 1: 6 stages 6453 (5: 6351, 4: 5943)      M = 5: 3 stages 6369 (4: 6011, 2: 5725)
+//   M = 2: 4 stages 6413 (5: 6168, 3: 5829)      M = 6: 3 stages 6224 (4: 5967, 2: 5915)
+//   M = 3: 4 stages 6282 (3: 6216, 5: 5962)      M = 7: 3 stages 6187 (2: 6080, 4: 5961)
+//   M = 4: 3 stages 6501 (4: 6120, 2: 5521)      M = 8: 2 stages 6292 (3: 6165, 4: 6023)
+// Loading, updating and storing each hold a stage, so fewer than three serialise the pipeline unless a stage is
+// large; beyond about 80 KB the loads in flight crowd out the stores.
+__host__ __device__ constexpr int inplace_stages(int M) {
+  return M == 1 ? 6 : M <= 3 ? 4 : M <= 7 ? 3 : 2;
+}
 
 template <int M>
 struct InplaceLayout {
   using L = StageLayout<M, MODE_FUSED, true>;
-  static constexpr int kStagesRaw = (72 * 1024 + (int)L::kStageBytes / 2) / (int)L::kStageBytes;
-  static constexpr int kStages = kStagesRaw < 2 ? 2 : kStagesRaw;
+  static constexpr int kStages = inplace_stages(M);
   static constexpr unsigned kSmemBytes = kStages * L::kStageBytes;
   static_assert(kSmemBytes <= 227 * 1024, "stages do not fit in shared memory");
 };

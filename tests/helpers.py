@@ -16,8 +16,11 @@ def np_(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().numpy()
 
 
-def rel_errors(x: np.ndarray, y: np.ndarray):
-    """(norm-wise relative error, worst element error relative to max(|y_i|, rms(y)))."""
+def rel_errors(x: np.ndarray, y: np.ndarray, floor=None):
+    """(norm-wise relative error, worst element error relative to max(|y_i|, rms(y))).
+
+    `floor` (optional, per element): magnitude of the operands the output was formed from; where it is
+    given, errors are measured against max(|y_i|, rms(y), floor_i) and max(||y||, ||floor||)."""
     x = x.astype(np.float64).ravel()
     y = y.astype(np.float64).ravel()
     if y.size == 0:
@@ -25,16 +28,44 @@ def rel_errors(x: np.ndarray, y: np.ndarray):
     diff = np.abs(x - y)
     ny = float(np.sqrt((y * y).sum()))
     rms = ny / np.sqrt(y.size)
-    normwise = float(np.sqrt((diff * diff).sum())) / ny if ny > 0 else float(diff.max())
     denom = np.maximum(np.abs(y), rms)
+    if floor is not None:
+        f = np.abs(np.asarray(floor, dtype=np.float64).ravel())
+        ny = max(ny, float(np.sqrt((f * f).sum())))
+        denom = np.maximum(denom, f)
+    normwise = float(np.sqrt((diff * diff).sum())) / ny if ny > 0 else float(diff.max())
     elem = float((diff / np.where(denom > 0, denom, 1.0)).max())
     return normwise, elem
 
 
-def assert_close(x, y, tol=TOL_PARAM, what=""):
-    nw, el = rel_errors(np.asarray(x), np.asarray(y))
+def assert_close(x, y, tol=TOL_PARAM, what="", floor=None):
+    nw, el = rel_errors(np.asarray(x), np.asarray(y), floor)
     assert nw <= tol and el <= tol, f"{what}: norm-wise {nw:.3e}, element-wise {el:.3e} > {tol:.1e}"
     return nw, el
+
+
+# A fragment of a handful of elements has no rms to speak of: when the workers' pseudo-gradients (or the
+# momentum term and their mean) cancel in its one element, the rounding error of the operands is all that is
+# left of the output and no bound relative to the output holds; the same goes for a new global or local value
+# that happens to land near zero.  Below this size the errors are therefore measured against the operands as
+# well (rel_errors' floor).
+SMALL_FRAGMENT = 64
+
+
+def operand_floors(frs, before: dict, snap: np.ndarray, snap_offset, p: int, mu: float):
+    """(mean_m |theta^m_{t_p} - theta^g|, |mu u| + that, |theta^g|, |theta^m_{t_p}| [M, n]) per element of
+    fragment p: the magnitudes of what Eq. 1 averages, of what the momentum update adds, and of the states the
+    new global and local parameters start from.  Indexing only; no step of the method."""
+    thg = orc.gather_fragment(frs, before["theta_g"], p).astype(np.float64)
+    u = orc.gather_fragment(frs, before["momentum"], p).astype(np.float64)
+    rows, pos = [], 0
+    for off, ln in frs[p]:
+        sb = off if snap_offset is None else int(snap_offset[p]) + pos
+        rows.append(snap[:, sb:sb + ln].astype(np.float64))
+        pos += ln
+    b = np.concatenate(rows, axis=1)
+    mean_abs_delta = np.abs(b - thg[None, :]).mean(axis=0)
+    return mean_abs_delta, np.abs(mu * u) + mean_abs_delta, np.abs(thg), np.abs(b)
 
 
 def fragments_of(w: synth.Workload):
@@ -149,15 +180,20 @@ def check_step_against_oracle(prob: GpuProblem, before: dict, ids, t_p, t_l, ohp
         r = res[int(p)]
         g = orc.gather_fragment(frs, after["theta_g"], p)
         u = orc.gather_fragment(frs, after["momentum"], p)
-        worst = max(worst, *assert_close(g, r.theta_g, TOL_PARAM, f"theta_g[{p}]"))
-        worst = max(worst, *assert_close(u, r.momentum, TOL_PARAM, f"momentum[{p}]"))
+        fl_d = fl_u = fl_g = fl_b = None
+        if g.size < SMALL_FRAGMENT:
+            fl_d, fl_u, fl_g, fl_b = operand_floors(frs, before, snap, None if same else before["snap_offset"],
+                                                    int(p), ohp.momentum)
+        worst = max(worst, *assert_close(g, r.theta_g, TOL_PARAM, f"theta_g[{p}]", floor=fl_g))
+        worst = max(worst, *assert_close(u, r.momentum, TOL_PARAM, f"momentum[{p}]", floor=fl_u))
         if do_merge:
             wn = orc.gather_fragment(frs, after["w_now"], p)
             for m in range(w.M):
-                worst = max(worst, *assert_close(wn[m], r.w_now[m], TOL_PARAM, f"w_now[{m}][{p}]"))
+                worst = max(worst, *assert_close(wn[m], r.w_now[m], TOL_PARAM, f"w_now[{m}][{p}]",
+                                                 floor=None if fl_b is None else fl_b[m]))
         if delta_out is not None:
             d = orc.gather_fragment(frs, np_(delta_out), p)
-            assert_close(d, r.delta_g, TOL_PARAM, f"delta_g[{p}]")
+            assert_close(d, r.delta_g, TOL_PARAM, f"delta_g[{p}]", floor=fl_d)
         if check_scores:
             assert abs(after["norms"][p] - r.norm) <= TOL_NORM * r.norm, (p, after["norms"][p], r.norm)
             assert abs(after["scores"][p] - r.score) <= TOL_NORM * r.score, (p, after["scores"][p], r.score)

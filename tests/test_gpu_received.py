@@ -291,3 +291,33 @@ def test_complete_fragments_through_nccl_world_of_one():
             assert torch.equal(x, y)
     finally:
         dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("M_total", [3, 5, 6, 7, 9, 11, 12, 24, 49, 64])
+def test_mean_over_workers_is_the_correctly_rounded_quotient(M_total):
+    """Eq. 1's division by the worker count never runs a division instruction (its slow path on zero
+    numerators costs bandwidth); what it computes must still be the IEEE quotient.  The received-sum step
+    exposes the operation directly: Delta = delta_sum / M_total, read back through delta_g_out and compared
+    bit for bit with numpy's float32 division on zeros of both signs, huge, tiny and ordinary sums."""
+    n = 1 << 16
+    w = synth.small_workload([n], M=1, seed=300)
+    prob = GpuProblem(w, synth.generate(w, "cuda"))
+    prob.set_ids([0])
+    rng = np.random.default_rng(M_total)
+    s = (rng.standard_normal(n) * np.exp(rng.uniform(-60.0, 60.0, n))).astype(np.float32)
+    s[:64] = 0.0
+    s[64:128] = -0.0
+    s[128:192] = np.float32(M_total) * rng.integers(-1000, 1000, 64).astype(np.float32)   # exact quotients
+    s[192:200] = np.float32(3.0e38)
+    sums = torch.from_numpy(s).cuda()
+    delta = torch.full((n,), 5.0, device="cuda")
+    b = prob.bufs
+    prob.ctx.cocodc_outer_step_received(prob.hyper(), M_total, b.w_now, b.w_snap, b.now_stride, b.snap_stride, None,
+                                        b.theta_g, b.momentum, sums, delta, prob.ids, prob.n_ids, 3, 5,
+                                        prob.last_sync, prob.norms, prob.scores)
+    prob.poll()                              # sums of 1e38 make the fragment norm overflow: not what is tested here
+    want = s / np.float32(M_total)
+    got = np_(delta)
+    assert got.dtype == np.float32 and want.dtype == np.float32
+    bad = np.flatnonzero(got.view(np.uint32) != want.view(np.uint32))
+    assert bad.size == 0, (bad[:8], s[bad[:8]], got[bad[:8]], want[bad[:8]])
