@@ -480,7 +480,8 @@ def run_micro(args):
 
 
 def run_workers(args):
-    """The fused step, the zero-delay step and the snapshot for a range of worker counts M on one fixed shape
+    """The fused step, the zero-delay step, the snapshot and the two calls of the worker-per-device deployment
+    (pseudo-gradient sum, completion from a received sum) for a range of worker counts M on one fixed shape
     (4 fragments of --workers-fragment parameters per worker): algorithmic GB/s from CUDA events.  M = 1..8 run the
     compile-time instances of the staged kernel, larger M the chunk-ring kernel."""
     if not torch.cuda.is_available():
@@ -523,9 +524,21 @@ def run_workers(args):
         def snapshot():
             ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, None, M, ids, n_ids)
 
+        sums = torch.zeros(w.N, device=device)
+
+        def pseudo_sum():
+            ctx.cocodc_pseudo_gradient_sum(b.w_snap, b.snap_stride, None, b.theta_g, M, sums, ids, n_ids)
+
+        def received():      # the M workers of this device among 2M in all
+            t[0] += w.tau
+            ctx.cocodc_outer_step_received(hp, 2 * M, b.w_now, b.w_snap, b.now_stride, b.snap_stride, None,
+                                           b.theta_g, b.momentum, sums, None, ids, n_ids, t[0], t[0] + w.tau,
+                                           last_sync, norms, scores)
+
         row = {"M": M, "params": n}
         for name, bpp, fn in (("fused", 12 * M + 16, fused), ("zero_delay", 8 * M + 16, zero_delay),
-                              ("snapshot", 8 * M, snapshot)):
+                              ("snapshot", 8 * M, snapshot), ("pseudo_gradient_sum", 4 * M + 8, pseudo_sum),
+                              ("received", 12 * M + 20, received)):
             for _ in range(3):
                 fn()
             torch.cuda.synchronize(device)
@@ -741,7 +754,8 @@ def main():
                     help="which method's arithmetic the step runs (the baselines are modes of the same kernels)")
     ap.add_argument("--micro", action="store_true", help="time every streaming entry point on its own")
     ap.add_argument("--workers", action="store_true",
-                    help="time the fused step, the zero-delay step and the snapshot for M = 1..34 workers")
+                    help="time the fused step, its zero-delay and received-sum forms, the snapshot and the pseudo-gradient "
+                         "sum for M = 1..34 workers")
     ap.add_argument("--workers-fragment", type=int, default=24 * 1024 * 1024,
                     help="parameters per fragment (of 4) in the --workers shape")
     ap.add_argument("--sweep", action="store_true", help="time the 48 variants of the 1B compensation sweep")

@@ -96,14 +96,15 @@ cocodc_status launch_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_id
 }
 
 // One way to run the streaming step: which kernel, with how many threads and how much dynamic
-// shared memory, on how many CTAs.  Every variant uses tiles of kTileElems elements and eight
-// accumulating warps, so the plan and the finalize kernel do not depend on the choice.
+// shared memory, on how many CTAs, over tiles of how many lanes.  Every variant has eight accumulating
+// warps, so the finalize kernel does not depend on the choice; the plan is built for the variant's tile.
 struct Variant {
   void (*kernel)(const OuterArgs);
   int threads;
   unsigned smem;
   bool one_cta_per_sm;   // staged kernel: persistent, one CTA per SM; otherwise sized by occupancy
   int ring_slots = 0;    // k_outer_ring only
+  int lanes_per_tile = kThreads;   // 16-byte lanes of one tile: what the plan of this launch is built with
 };
 
 // Worker counts without a compile-time instance: the slot-ring kernel, or, when even the recorded values of
@@ -115,10 +116,12 @@ Variant runtime_variant(int M) {
   return Variant{k_outer_ring<MODE, SAME>, kRingThreads, (unsigned)chunks * kChunkBytes, true, chunks};
 }
 
+// The staged kernel with the tile width its number of streams calls for (tile_width()).
 template <int M, int MODE, bool SAME>
 Variant staged_variant() {
-  using L = StageLayout<M, MODE, SAME>;
-  return Variant{k_outer_tma<M, MODE, SAME>, tma_threads(M), L::kSmemBytes, true};
+  constexpr int U = tile_width(StageLayout<M, MODE, SAME, 1>::kLoaded);
+  using L = StageLayout<M, MODE, SAME, U>;
+  return Variant{k_outer_tma<M, MODE, SAME, U>, tma_threads(M), L::kSmemBytes, true, 0, kThreads * U};
 }
 
 // More than 48 KB of dynamic shared memory needs a one-time opt-in per kernel and device (the
@@ -206,7 +209,7 @@ cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool sam
   const Variant v = pick_variant(A.M, mode, same, A.n_recv);
   const int grid = variant_grid(c, v);
   opt_in_shared_memory(c, reinterpret_cast<const void*>(v.kernel), v.smem);
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, A.snap_stride, kThreads, st);
+  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, A.snap_stride, v.lanes_per_tile, st);
   if (s != COCODC_OK) return s;
   OuterArgs args = A;
   args.ring_slots = v.ring_slots;
@@ -819,7 +822,7 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
         A.momentum = d_u;
         A.delta_out = delta_g_out ? d_delta : nullptr;
         A.ring_slots = v.ring_slots;
-        k_plan_chunk<<<1, 1, 0, st>>>(cnt, snap_on_device ? sbase + lo : 0, kThreads, c->d_plan, c->d_hdr);
+        k_plan_chunk<<<1, 1, 0, st>>>(cnt, snap_on_device ? sbase + lo : 0, v.lanes_per_tile, c->d_plan, c->d_hdr);
         v.kernel<<<grid, v.threads, v.smem, st>>>(A);
         k_accumulate_chunk<<<1, kFinalizeThreads, 0, st>>>(c->d_partial, entries, c->d_frag_sumsq + j);
         c->launches += 3;

@@ -278,9 +278,11 @@ struct TileWalker {
   int n_seg;
   int seg = 0;
   int loaded = -1;
+  int tile_elems;      // elements per tile of this launch (the plan was built with tile_elems / 4 lanes per tile)
   SegPlan sp;
 
-  __device__ __forceinline__ TileWalker(const SegPlan* p, int n) : plan(p), n_seg(n) {}
+  __device__ __forceinline__ TileWalker(const SegPlan* p, int n, int tile_elems_ = kTileElems)
+      : plan(p), n_seg(n), tile_elems(tile_elems_) {}
   // returns true if the segment changed
   __device__ __forceinline__ bool seek(int tile) {
     while (seg + 1 < n_seg && tile >= plan[seg + 1].first_tile) ++seg;
@@ -290,11 +292,11 @@ struct TileWalker {
     return true;
   }
   __device__ __forceinline__ long long tile_start(int tile) const {   // first element (16-byte aligned)
-    return sp.abase + (long long)(tile - sp.first_tile) * kTileElems;
+    return sp.abase + (long long)(tile - sp.first_tile) * tile_elems;
   }
   // the whole tile lies inside the segment and every stream is 16-byte aligned there
   __device__ __forceinline__ bool interior(long long e_tile) const {
-    return sp.vec_ok && e_tile >= sp.off && e_tile + kTileElems <= sp.off + sp.len;
+    return sp.vec_ok && e_tile >= sp.off && e_tile + tile_elems <= sp.off + sp.len;
   }
 };
 

@@ -86,7 +86,8 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 // Ring depth of the received-sum mode, whose stage size is known only at run time: about 72 KB of
 // copies in flight, at least two stages (host and device use the same function).
 __host__ __device__ constexpr int stages_for(int loaded_streams) {
-  const int raw = (72 * 1024) / (loaded_streams * (int)kTileBytes);
+  const int stage = loaded_streams * (int)kTileBytes;
+  const int raw = (72 * 1024 + stage / 2) / stage;
   return raw < 2 ? 2 : (raw > kMaxStages ? kMaxStages : raw);
 }
 
@@ -94,7 +95,21 @@ __host__ __device__ constexpr int stages_for(int loaded_streams) {
 // Slots of kTileElems floats each: [recorded x nS][current x nN][global][momentum x nU], then, in
 // MODE_FUSED_RECV, one slot per buffer of received sums (a run-time count, so that mode sizes its ring at
 // run time: stages_for()).
-template <int M, int MODE, bool SAME>
+// U: tiles of kTileElems elements that one stage holds per stream (one bulk copy of U * 4 KB per stream; every
+// consumer thread then owns U lanes).  One producer thread starts a copy every few hundred cycles whatever its
+// size, so a mode that reads only two or three streams cannot be fed 4 KB at a time (the pseudo-gradient sum of
+// a single worker ran at 4.9 TB/s that way); such modes take wider tiles.  Measured on B200 (GB/s through the C
+// ABI, 100 M parameters per worker, tile widths 1 / 2 / 4 / 8 where tried):
+//   pseudo-gradient sum  M = 1 (2 streams): 4941 / - / 6190 / 6038     M = 2 (3): 5977 / 6740 / 6759 / -
+//                        M = 3 (4 streams): 6696 / 6832 / 6869 / -     M = 4 (5): 6736 / 6682 / - / -
+//   merge only           M = 1 (3 streams): 5760 / 6600 / 6766 / -     M = 2 (5): 6498 / 6792 / - / -
+//   outer update only    M = 1 (3 streams): 6237 / 6161 / 6304 / -     M = 2 (4): 6194 / 6373 / 6195 / -
+//   fused                M = 1 (4 streams): 6392 / 6404 / 6154 / -     M = 2 (6): 6495 / 6433 / - / -
+__host__ __device__ constexpr int tile_width(int loaded_streams) {
+  return loaded_streams <= 3 ? 4 : loaded_streams <= 5 ? 2 : 1;
+}
+
+template <int M, int MODE, bool SAME, int U = 1>
 struct StageLayout {
   static constexpr int nS = SAME ? 0 : M;
   static constexpr int nN = mode_merges(MODE) ? M : 0;
@@ -105,24 +120,28 @@ struct StageLayout {
   static constexpr int kMomentum = kGlobal + 1;
   static constexpr int kDeltaIn = kMomentum + nU;
   static constexpr int kLoaded = nS + nN + 1 + nU;       // streams brought in by the producer (plus the received sums)
-  static constexpr unsigned kStageBytes = kLoaded * kTileBytes;
+  static constexpr unsigned kSlotElems = U * kTileElems;  // one stream's share of a stage
+  static constexpr unsigned kStageBytes = kLoaded * U * kTileBytes;
   // about 72 KB of copies in flight (see the note at the top), never fewer than two stages; the
   // read-heavy modes measure best with more: OUTER_ONLY (3 reads per write) one stage deeper,
-  // PSEUDO_SUM (M + 1 reads per write) at 100 KB
+  // PSEUDO_SUM (M + 1 reads per write) at 100-110 KB
   static constexpr int kInFlightBytes =
-      (MODE == MODE_PSEUDO_SUM ? 100 : MODE == MODE_OUTER_ONLY ? 96 : 72) * 1024;
-  static constexpr int kStagesRaw = kInFlightBytes / kStageBytes;
+      (MODE == MODE_PSEUDO_SUM ? 110 : MODE == MODE_OUTER_ONLY ? 96 : 72) * 1024;
+  static constexpr int kStagesRaw = (kInFlightBytes + (int)kStageBytes / 2) / (int)kStageBytes;   // nearest
   static constexpr int kStages = kStagesRaw < 2 ? 2 : (kStagesRaw > kMaxStages ? kMaxStages : kStagesRaw);
   static constexpr unsigned kSmemBytes = kStages * kStageBytes;
   static_assert(kSmemBytes <= 227 * 1024, "stages do not fit in shared memory");
   static_assert(SAME ? (MODE == MODE_FUSED || MODE == MODE_MERGE_ONLY) : true,
                 "zero-delay mode needs the merge and local pseudo-gradients");
+  static_assert(U == 1 || MODE != MODE_FUSED_RECV, "the received-sum mode sizes its stages at run time for U = 1");
 };
 
-template <int M, int MODE, bool SAME>
+template <int M, int MODE, bool SAME, int U = 1>
 __global__ void __launch_bounds__(tma_threads(M), 1)
 k_outer_tma(const OuterArgs A) {
-  using L = StageLayout<M, MODE, SAME>;
+  using L = StageLayout<M, MODE, SAME, U>;
+  constexpr int kSlot = U * kTileElems;                         // elements of one stream in a stage
+  constexpr unsigned kSlotBytes = U * kTileBytes;
   constexpr bool kRecv = (MODE == MODE_FUSED_RECV);
   const int n_recv = kRecv ? A.n_recv : 0;
   const int loaded = L::kLoaded + n_recv;                       // streams per stage
@@ -160,7 +179,7 @@ k_outer_tma(const OuterArgs A) {
       turn = (turn + 1 == P) ? 0 : turn + 1;
       return yes;
     };
-    TileWalker tw(A.plan, h.n_seg);
+    TileWalker tw(A.plan, h.n_seg, kSlot);
     int k = 0;   // staged tiles issued so far
     for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
       tw.seek(tile);
@@ -174,19 +193,19 @@ k_outer_tma(const OuterArgs A) {
       }
       if (s_fail) return;
       const unsigned bar = smem_u32(&full_bar[s]);
-      float* st = stages + (size_t)s * loaded * kTileElems;
+      float* st = stages + (size_t)s * loaded * kSlot;
       const long long snap_e0 = e0 + (tw.sp.snap_off - tw.sp.off);
-      if (me == 0) mbar_expect_tx(bar, loaded * kTileBytes);
+      if (me == 0) mbar_expect_tx(bar, loaded * kSlotBytes);
 #pragma unroll
       for (int m = 0; m < L::nS; ++m)
-        if (mine()) bulk_load(smem_u32(st + (L::kSnap + m) * kTileElems), A.w_snap + m * A.snap_stride + snap_e0, kTileBytes, bar);
+        if (mine()) bulk_load(smem_u32(st + (L::kSnap + m) * kSlot), A.w_snap + m * A.snap_stride + snap_e0, kSlotBytes, bar);
 #pragma unroll
       for (int m = 0; m < L::nN; ++m)
-        if (mine()) bulk_load(smem_u32(st + (L::kNow + m) * kTileElems), A.w_now + m * A.now_stride + e0, kTileBytes, bar);
-      if (mine()) bulk_load(smem_u32(st + L::kGlobal * kTileElems), A.theta_g + e0, kTileBytes, bar);
-      if (L::nU && mine()) bulk_load(smem_u32(st + L::kMomentum * kTileElems), A.momentum + e0, kTileBytes, bar);
+        if (mine()) bulk_load(smem_u32(st + (L::kNow + m) * kSlot), A.w_now + m * A.now_stride + e0, kSlotBytes, bar);
+      if (mine()) bulk_load(smem_u32(st + L::kGlobal * kSlot), A.theta_g + e0, kSlotBytes, bar);
+      if (L::nU && mine()) bulk_load(smem_u32(st + L::kMomentum * kSlot), A.momentum + e0, kSlotBytes, bar);
       for (int r = 0; r < n_recv; ++r)
-        if (mine()) bulk_load(smem_u32(st + (L::kDeltaIn + r) * kTileElems), A.delta_in[r] + e0, kTileBytes, bar);
+        if (mine()) bulk_load(smem_u32(st + (L::kDeltaIn + r) * kSlot), A.delta_in[r] + e0, kSlotBytes, bar);
       ++k;
     }
     return;
@@ -194,14 +213,15 @@ k_outer_tma(const OuterArgs A) {
 
   // ------------------------------------------------------------------ consumers
   SlotAccumulator sa(kThreads / 32);
-  TileWalker tw(A.plan, h.n_seg);
+  TileWalker tw(A.plan, h.n_seg, kSlot);
   int k = 0;           // staged tiles consumed so far
   bool failed = false;
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
     if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
     const long long e0 = tw.tile_start(tile);
     if (!tw.interior(e0)) {
-      ragged_lane<M, MODE, SAME>(A, tw.sp, e0 + 4LL * tid, sa.acc);
+#pragma unroll
+      for (int v = 0; v < U; ++v) ragged_lane<M, MODE, SAME>(A, tw.sp, e0 + 4LL * (v * kThreads + tid), sa.acc);
       continue;
     }
     const int s = k % S;
@@ -214,29 +234,37 @@ k_outer_tma(const OuterArgs A) {
       failed = true;
       break;
     }
-    const float* st = stages + (size_t)s * loaded * kTileElems;
-    Lane<M, MODE, SAME> ln;
-    auto slot = [&](int idx) -> const float4& { return reinterpret_cast<const float4*>(st + idx * kTileElems)[tid]; };
-    ln.thg = slot(L::kGlobal);
-    if (L::nU) ln.u = slot(L::kMomentum);
-    if (kRecv) {
-      ln.delta = slot(L::kDeltaIn);
-      for (int r = 1; r < n_recv; ++r) ln.delta = add4(ln.delta, slot(L::kDeltaIn + r));
-    }
-    if (SAME) {
+    const float* st = stages + (size_t)s * loaded * kSlot;
+    Lane<M, MODE, SAME> ln[U];
 #pragma unroll
-      for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kNow + m);
-    } else {
+    for (int v = 0; v < U; ++v) {
+      auto slot = [&](int idx) -> const float4& {
+        return reinterpret_cast<const float4*>(st + idx * kSlot)[v * kThreads + tid];
+      };
+      ln[v].thg = slot(L::kGlobal);
+      if (L::nU) ln[v].u = slot(L::kMomentum);
+      if (kRecv) {
+        ln[v].delta = slot(L::kDeltaIn);
+        for (int r = 1; r < n_recv; ++r) ln[v].delta = add4(ln[v].delta, slot(L::kDeltaIn + r));
+      }
+      if (SAME) {
 #pragma unroll
-      for (int m = 0; m < M; ++m) ln.b[m] = slot(L::kSnap + m);
-      if (L::nN) {
+        for (int m = 0; m < M; ++m) ln[v].b[m] = slot(L::kNow + m);
+      } else {
 #pragma unroll
-        for (int m = 0; m < M; ++m) ln.a[m] = slot(L::kNow + m);
+        for (int m = 0; m < M; ++m) ln[v].b[m] = slot(L::kSnap + m);
+        if (L::nN) {
+#pragma unroll
+          for (int m = 0; m < M; ++m) ln[v].a[m] = slot(L::kNow + m);
+        }
       }
     }
-    mbar_arrive(smem_u32(&empty_bar[s]));   // this thread's lane is in registers: its share of the stage is free
-    ln.compute(A, sa.acc);
-    ln.store(A, e0 + 4LL * tid);
+    mbar_arrive(smem_u32(&empty_bar[s]));   // this thread's lanes are in registers: its share of the stage is free
+#pragma unroll
+    for (int v = 0; v < U; ++v) {
+      ln[v].compute(A, sa.acc);
+      ln[v].store(A, e0 + 4LL * (v * kThreads + tid));
+    }
     ++k;
   }
   if (failed) return;     // warp-uniform by construction

@@ -88,9 +88,12 @@ def test_three_consecutive_steps_carry_momentum():
     assert prob.poll() == 0
 
 
-def test_unfused_path_equals_fused_bit_for_bit():
-    a = make(4, seed=60)
-    b = make(4, seed=60)
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 6])
+def test_unfused_path_equals_fused_bit_for_bit(M):
+    """S1-S3 + S6 and S4-S5 as two calls.  The halves read few streams at small M and then run with wider
+    tiles than the fused step (4 or 2 tiles per stage), so this also covers those instances."""
+    a = make(M, seed=60)
+    b = make(M, seed=60)
     ids = [2, 1, 4]
     for prob in (a, b):
         prob.set_ids(ids)
@@ -108,6 +111,19 @@ def test_unfused_path_equals_fused_bit_for_bit():
     for p in ids:
         got = orc.gather_fragment(fragments_of(b.w), np_(b.bufs.w_now), p)
         assert_close(got, res[p], TOL_PARAM, f"merge[{p}]")
+    # the merge with zero delay (the recorded values are the current ones): Eq. 3 towards the new global state
+    before = b.host_state()
+    hp = b.hyper(alpha=0.5, comp_mode=0, tau=0)
+    bb = b.bufs
+    b.ctx.cocodc_merge(hp, bb.w_now, bb.w_now, bb.now_stride, bb.now_stride, None, bb.theta_g, b.ids, b.n_ids)
+    assert b.poll() == 0
+    res = orc.merge(fragments_of(b.w), orc_hyper(b.w, alpha=0.5, comp_mode=0, tau=0), before["w_now"],
+                    before["w_now"], before["theta_g"], ids)
+    after = np_(bb.w_now)
+    for p in ids:
+        assert_close(orc.gather_fragment(fragments_of(b.w), after, p), res[p], TOL_PARAM, f"zero-delay merge[{p}]")
+    untouched = ~touched_mask(b.w, ids)
+    assert np.array_equal(after[:, untouched], before["w_now"][:, untouched])
 
 
 @pytest.mark.parametrize("aligned", [True, False])
