@@ -139,7 +139,7 @@ def pool_capacity(w: synth.Workload) -> int:
         cap = int(w.budget + sizes[0])
     else:
         cap = int(sizes[:max(1, w.budget)].sum())
-    return (cap + 4 * w.K + 1023) // 1024 * 1024
+    return (cap + 8 * w.K + 1023) // 1024 * 1024
 
 
 # --------------------------------------------------------------------------------------------

@@ -167,9 +167,13 @@ cocodc_status cocodc_fragment_scores(cocodc_ctx* ctx, const float* delta_g, cons
  *   order; the rest set to -1); n_sel dev int32[1]
  *   pool_offset dev int64[K] or NULL: if given, the selected fragments are assigned places in a
  *   packed snapshot pool (the snap_offset argument of the calls below): admission order, back to
- *   back, each start a multiple of 4 elements; -1 for fragments not selected.  A pool row of
- *   budget + (largest fragment) elements (PARAMS), or the `budget` largest fragments (COUNT),
- *   plus 4 per fragment for rounding, always suffices.
+ *   back, each start at the next multiple of 4 elements plus (native offset of the fragment's
+ *   first segment) mod 4, so that recorded and native values share their 16-byte alignment and
+ *   the streaming calls move the fragment as vectors; -1 for fragments not selected.  A pool row
+ *   of budget + (largest fragment) elements (PARAMS), or the `budget` largest fragments (COUNT),
+ *   plus 8 per fragment for alignment, always suffices.  (Callers that place fragments themselves
+ *   should keep the same congruence: a segment whose pool position differs from its native offset
+ *   by a non-multiple of 4 is processed element by element, at a fraction of the bandwidth.)
  * A NaN score selects nothing and sets COCODC_ERR_NONFINITE.
  *
  * PARAMS_EXACT (no counterpart in the paper, whose Algorithm 2 picks one fragment per decision): the

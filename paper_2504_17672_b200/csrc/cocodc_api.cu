@@ -33,6 +33,7 @@ struct cocodc_ctx {
   long long* d_seg_off = nullptr;
   long long* d_seg_len = nullptr;
   long long* d_frag_size = nullptr;
+  long long* d_frag_first_off = nullptr;   // native offset of every fragment's first segment
   // launch scratch
   SegPlan* d_plan = nullptr;
   PlanHeader* d_hdr = nullptr;
@@ -348,6 +349,7 @@ cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, 
   ok = ok && cudaMalloc(&c->d_seg_off, sizeof(long long) * S) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_seg_len, sizeof(long long) * S) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_frag_size, sizeof(long long) * K) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_frag_first_off, sizeof(long long) * K) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_plan, sizeof(SegPlan) * S) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_hdr, sizeof(PlanHeader)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_partial, sizeof(double) * partial_elems) == cudaSuccess;
@@ -373,6 +375,11 @@ cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, 
   ok = ok && cudaMemcpy(c->d_seg_off, off.data(), sizeof(long long) * S, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->d_seg_len, len.data(), sizeof(long long) * S, cudaMemcpyHostToDevice) == cudaSuccess;
   ok = ok && cudaMemcpy(c->d_frag_size, frag_size.data(), sizeof(long long) * K, cudaMemcpyHostToDevice) == cudaSuccess;
+  {
+    std::vector<long long> first_off(K);
+    for (int p = 0; p < K; ++p) first_off[p] = part->seg_offset[part->frag_seg_ptr[p]];
+    ok = ok && cudaMemcpy(c->d_frag_first_off, first_off.data(), sizeof(long long) * K, cudaMemcpyHostToDevice) == cudaSuccess;
+  }
   ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMemset(c->d_hdr, 0, sizeof(PlanHeader)) == cudaSuccess;
   if (!ok) { cudaGetLastError(); cocodc_destroy(c); return COCODC_ERR_CUDA; }
@@ -387,6 +394,7 @@ cocodc_status cocodc_destroy(cocodc_ctx* c) {
   cudaFree(c->d_seg_off);
   cudaFree(c->d_seg_len);
   cudaFree(c->d_frag_size);
+  cudaFree(c->d_frag_first_off);
   cudaFree(c->d_plan);
   cudaFree(c->d_hdr);
   cudaFree(c->d_partial);
@@ -457,7 +465,7 @@ cocodc_status select_impl(cocodc_ctx* c, const float* scores, const int64_t* las
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   k_select<<<1, kSelectThreads, 0, st>>>(c->K, scores, reinterpret_cast<const long long*>(last_sync), ineligible,
-                                         c->d_frag_size, t_now, reinterpret_cast<const long long*>(t_now_dev), H, budget_kind, budget, mask, ids, n_sel,
+                                         c->d_frag_size, c->d_frag_first_off, t_now, reinterpret_cast<const long long*>(t_now_dev), H, budget_kind, budget, mask, ids, n_sel,
                                          reinterpret_cast<long long*>(pool_offset), c->d_status, (int)COCODC_ERR_NONFINITE,
                                          (int)COCODC_ERR_INVALID_ARG);
   c->launches++;

@@ -16,6 +16,7 @@ constexpr int kExactMaxFree = 24;    // knapsack candidates enumerated at most (
 __global__ void __launch_bounds__(kSelectThreads)
 k_select(int K, const float* __restrict__ scores, const long long* __restrict__ last_sync,
          const unsigned char* __restrict__ ineligible, const long long* __restrict__ frag_size,
+         const long long* __restrict__ frag_first_off,
          long long t_now, const long long* __restrict__ t_now_dev, long long H, int budget_kind, long long budget,
          unsigned char* __restrict__ mask, int* __restrict__ ids, int* __restrict__ n_sel,
          long long* __restrict__ pool_offset, int* __restrict__ status, int err_nonfinite, int err_too_many) {
@@ -23,6 +24,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   __shared__ unsigned char s_class[kMaxK];  // 0 = ineligible, 1 = ordinary, 2 = overdue
   __shared__ int s_order[kMaxK];
   __shared__ long long s_fsize[kMaxK];      // fragment sizes, so that the walk below reads no global memory
+  __shared__ unsigned char s_falign[kMaxK]; // native offset of the fragment's first segment, mod 4 (see place())
   __shared__ int s_nan;
   __shared__ int s_count;
   const int p = threadIdx.x;
@@ -35,6 +37,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     const bool overdue = (t_now - last_sync[p]) >= H;   // Algorithm 2's staleness test
     s_score[p] = r;
     s_fsize[p] = frag_size[p];
+    s_falign[p] = (unsigned char)(frag_first_off[p] & 3);
     s_class[p] = elig ? (overdue ? 2 : 1) : 0;
     if (r != r) s_nan = 1;
     mask[p] = 0;
@@ -72,6 +75,15 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   // rest of the order becomes a knapsack that all threads solve by enumeration below.
   __shared__ long long s_remaining;
   __shared__ long long s_pool_pos;   // next free element of the snapshot pool (kept a multiple of 4)
+  // A fragment's place in the pool starts at the next multiple of 4 plus its native offset mod 4: recorded and
+  // native values then share their 16-byte alignment, and the streaming kernels can move the fragment as
+  // vectors (a place that breaks the congruence sends the whole segment down the element-wise path, at a
+  // sixth of the bandwidth).
+  auto place = [&](int f, long long& pool_pos) {
+    const long long start = pool_pos + s_falign[f];
+    pool_offset[f] = start;
+    pool_pos = (start + s_fsize[f] + 3) & ~3LL;
+  };
   __shared__ int s_n;                // fragments admitted so far
   __shared__ int s_free_begin;       // first position of the order that belongs to the knapsack
   const int n_elig = s_count;
@@ -87,10 +99,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
         mask[f] = 1;
         ids[n++] = f;
         remaining -= cost;
-        if (pool_offset) {
-          pool_offset[f] = pool_pos;
-          pool_pos = (pool_pos + s_fsize[f] + 3) & ~3LL;
-        }
+        if (pool_offset) place(f, pool_pos);
       }
     }
     s_remaining = remaining; s_pool_pos = pool_pos; s_n = n; s_free_begin = j;
@@ -157,10 +166,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     const int f = s_order[s_free_begin + j];
     mask[f] = 1;
     ids[n++] = f;
-    if (pool_offset) {
-      pool_offset[f] = pool_pos;
-      pool_pos = (pool_pos + s_fsize[f] + 3) & ~3LL;
-    }
+    if (pool_offset) place(f, pool_pos);
   }
   *n_sel = n;
 }

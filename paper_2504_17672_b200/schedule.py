@@ -47,7 +47,7 @@ class RoundDriver:
         sizes = sorted((int(s) for s in frag_sizes), reverse=True)
         if pool_len is None:
             cap = (budget + sizes[0]) if budget_kind == B.BUDGET_PARAMS else sum(sizes[:max(1, budget)])
-            pool_len = (cap + 4 * K + 1023) // 1024 * 1024
+            pool_len = (cap + 8 * K + 1023) // 1024 * 1024
         n_slots = max(1, -(-hyper.tau // self.h)) + 1
         self.slots: List[_Slot] = [
             _Slot(ids=torch.full((K,), -1, dtype=torch.int32, device=dev),

@@ -85,9 +85,10 @@ def test_exact_budget_selection_matches_oracle_bit_for_bit(K):
         got = np_(ids)
         assert np.array_equal(got[:en], eids) and (got[en:] == -1).all()
         po, pos = np_(pool_off), 0
-        for p in eids:
-            assert po[p] == pos
-            pos = (pos + int(sizes[p]) + 3) // 4 * 4
+        for p in eids:          # next multiple of 4, plus the fragment's native offset mod 4
+            start = pos + w.partition.fragments[p][0][0] % 4
+            assert po[p] == start
+            pos = (start + int(sizes[p]) + 3) // 4 * 4
         assert all(po[p] == -1 for p in range(K) if not emask[p])
 
 
@@ -259,3 +260,45 @@ def test_schedule_step_replayed_from_a_cuda_graph_equals_eager_steps():
     for x, y in ((a.bufs.w_now, g.bufs.w_now), (a.bufs.theta_g, g.bufs.theta_g), (a.bufs.momentum, g.bufs.momentum),
                  (a.bufs.w_snap, g.bufs.w_snap), (a.scores, g.scores), (a.last_sync, g.last_sync), (a.ids, g.ids)):
         assert torch.equal(x, y)
+
+
+def test_selected_pool_places_keep_the_native_alignment():
+    """Fragments whose native offsets are not multiples of 4: the places cocodc_select_fragments hands out in
+    the snapshot pool are congruent to them mod 4 (so snapshot and completion run as vectors), do not overlap,
+    fit the documented pool size, and the chain select -> snapshot -> step matches the oracle."""
+    from helpers import check_step_against_oracle, orc_hyper
+    frs = [[(1, 9_001)], [(9_003, 12_346)], [(21_350, 4_100), (40_003, 777)], [(25_451, 5)], [(25_457, 14_001)]]
+    w = synth.small_workload((41_000, frs), M=3, seed=17, scale_kind="loguniform", tau=3)
+    K = w.K
+    sizes = w.partition.frag_sizes
+    budget = 3
+    pool_len = int(np.sort(sizes)[::-1][:budget].sum()) + 8 * K
+    pool_len += (-pool_len) % 4
+    prob = GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3, snap_layout="pool", pool_ids=[],
+                                        pool_len=pool_len))
+    dev = "cuda"
+    pool_off = prob.bufs.snap_offset
+    rng = np.random.default_rng(3)
+    for trial in range(4):
+        scores = rng.random(K).astype(np.float32)
+        prob.scores.copy_(torch.from_numpy(scores))
+        prob.ctx.cocodc_select_fragments(prob.scores, prob.last_sync, None, 10, w.H, prob.B.BUDGET_COUNT, budget,
+                                         prob.mask, prob.ids, prob.n_ids, pool_off)
+        n = int(prob.n_ids.item())
+        ids = np_(prob.ids)[:n].tolist()
+        _, eids, en = orc.select_fragments(scores, np_(prob.last_sync), sizes, 10, w.H, orc.BUDGET_COUNT, budget)
+        assert ids == eids.tolist()
+        po = np_(pool_off)
+        end = 0
+        for p in ids:
+            native = w.partition.fragments[p][0][0]
+            assert (po[p] - native) % 4 == 0 and po[p] >= end and po[p] - end < 8
+            end = po[p] + int(sizes[p])
+        assert end <= pool_len
+        prob.snapshot()
+        prob.bufs.w_now.add_(torch.randn_like(prob.bufs.w_now) * 1e-3)
+        before = prob.host_state()
+        prob.outer_step(t_p=10, t_l=13)
+        assert prob.poll() == 0
+        check_step_against_oracle(prob, before, ids, 10, 13, orc_hyper(w))
+        prob.last_sync.zero_()
