@@ -253,11 +253,13 @@ def test_nonfinite_norm_is_reported():
     assert prob.poll() == 0
 
 
+@pytest.mark.parametrize("M", [4, 1])
 @pytest.mark.parametrize("same", [False, True])
-def test_host_buffer_entry_point_matches_device_path_and_oracle(same):
-    """Parameters in host memory, streamed through a small workspace (several chunks per fragment)."""
+def test_host_buffer_entry_point_matches_device_path_and_oracle(same, M):
+    """Parameters in host memory, streamed through a small workspace (several chunks per fragment).  M = 1 runs
+    the staged kernel with two tiles per stage, so the chunk plans are built for that tile as well."""
     frs = (300_000, [[(3, 90_001), (200_010, 40_097)], [(90_004, 100_000)], [(250_000, 50_000)]])
-    w = synth.small_workload(frs, M=4, seed=130, scale_kind="loguniform")
+    w = synth.small_workload(frs, M=M, seed=130, scale_kind="loguniform")
     bufs = synth.generate(w, "cuda", momentum_sigma=1e-3)
     prob = GpuProblem(w, bufs)
     ids = [2, 0]
