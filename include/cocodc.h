@@ -173,7 +173,7 @@ cocodc_status cocodc_fragment_scores(cocodc_ctx* ctx, const float* delta_g, cons
  *   of budget + (largest fragment) elements (PARAMS), or the `budget` largest fragments (COUNT),
  *   plus 8 per fragment for alignment, always suffices.  (Callers that place fragments themselves
  *   should keep the same congruence: a segment whose pool position differs from its native offset
- *   by a non-multiple of 4 is processed element by element, at a fraction of the bandwidth.)
+ *   by a non-multiple of 4 cannot be staged by bulk copies and runs at half to two thirds of the bandwidth.)
  * A NaN score selects nothing and sets COCODC_ERR_NONFINITE.
  *
  * PARAMS_EXACT (no counterpart in the paper, whose Algorithm 2 picks one fragment per decision): the

@@ -191,6 +191,23 @@ struct Lane {
     }
   }
 
+  // The same lane when the recorded values sit at a place that is not 16-byte compatible with the native one
+  // (snap_e is any element index): they come in as four 4-byte loads per worker, everything else as vectors.
+  __device__ __forceinline__ void load_shifted(const OuterArgs& A, long long e, long long snap_e) {
+    thg = ld4(A.theta_g + e);
+    if (mode_updates_global(MODE)) u = ld4(A.momentum + e);
+    if (MODE == MODE_FUSED_RECV) delta = received_sum4(A, e);
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+      const float* p = A.w_snap + m * A.snap_stride + snap_e;
+      b[m] = make_float4(ld1(p), ld1(p + 1), ld1(p + 2), ld1(p + 3));
+    }
+    if (kHasNow) {
+#pragma unroll
+      for (int m = 0; m < M; ++m) a[m] = ld4(A.w_now + m * A.now_stride + e);
+    }
+  }
+
   __device__ __forceinline__ void compute(const OuterArgs& A, double& acc) {
     if (MODE == MODE_PSEUDO_SUM) {
 #pragma unroll
@@ -250,17 +267,19 @@ struct Lane {
   }
 };
 
-// One lane at element e of a segment, straight from global memory: a full, 16-byte-compatible lane
-// goes through registers as a vector, anything else element by element.  M = 0: always by element.
+// One lane at element e of a segment, straight from global memory: a full lane goes through registers as a
+// vector (its recorded values by element when their place is not 16-byte compatible), a partial lane element
+// by element.  M = 0: always by element.
 template <int M, int MODE, bool SAME>
 __device__ __forceinline__ void ragged_lane(const OuterArgs& A, const SegPlan& sp, long long e, double& acc) {
   const long long seg_end = sp.off + sp.len;
   const long long snap_shift = sp.snap_off - sp.off;   // snapshot index = native index + shift
   if (e >= seg_end) return;
   if constexpr (M > 0) {
-    if (sp.vec_ok && e >= sp.off && e + 4 <= seg_end) {
+    if (e >= sp.off && e + 4 <= seg_end) {
       Lane<M, MODE, SAME> L;
-      L.load(A, e, e + snap_shift);
+      if (sp.vec_ok) L.load(A, e, e + snap_shift);
+      else L.load_shifted(A, e, e + snap_shift);
       L.compute(A, acc);
       L.store(A, e);
       return;

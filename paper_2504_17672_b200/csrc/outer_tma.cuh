@@ -373,16 +373,49 @@ k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long
     if (interior) continue;
     const long long seg_end = sp.off + sp.len;
     const long long shift = sp.snap_off - sp.off;
-    for (int l = wtid; l < kSnapTileElems / 4; l += kWorkers) {
+    // one lane: false once the tile has run past the end of the segment
+    auto copy_lane = [&](int l) -> bool {
       const long long e = e0 + 4LL * l;
-      if (e >= seg_end) break;
+      if (e >= seg_end) return false;
       if (sp.vec_ok && e >= sp.off && e + 4 <= seg_end) {
         for (int m = 0; m < M; ++m) st4(w_snap + m * snap_stride + shift + e, ld4(w_now + m * now_stride + e));
+      } else if (e >= sp.off && e + 4 <= seg_end) {   // a place that is not 16-byte compatible: vector in, elements out
+        for (int m = 0; m < M; ++m) {
+          const float4 v = ld4(w_now + m * now_stride + e);
+          float* d = w_snap + m * snap_stride + shift + e;
+          st1(d, v.x); st1(d + 1, v.y); st1(d + 2, v.z); st1(d + 3, v.w);
+        }
       } else {
         for (int k = 0; k < 4; ++k) {
           const long long ee = e + k;
           if (ee >= sp.off && ee < seg_end)
             for (int m = 0; m < M; ++m) st1(w_snap + m * snap_stride + shift + ee, ld1(w_now + m * now_stride + ee));
+        }
+      }
+      return true;
+    };
+    // A segment whose place is not 16-byte compatible has no interior tiles: all of it comes through here, so
+    // full lanes go kBatch at a time per thread, loads first (enough of them in flight to matter), stores after.
+    constexpr int kBatch = 8;
+    for (int l0 = wtid; l0 < kSnapTileElems / 4; l0 += kWorkers * kBatch) {
+      const int l_last = l0 + (kBatch - 1) * kWorkers;
+      const bool batch = !sp.vec_ok && l_last < kSnapTileElems / 4 && e0 + 4LL * l0 >= sp.off &&
+                         e0 + 4LL * l_last + 4 <= seg_end;
+      if (batch) {
+        for (int m = 0; m < M; ++m) {
+          float4 v[kBatch];
+#pragma unroll
+          for (int j = 0; j < kBatch; ++j) v[j] = ld4(w_now + m * now_stride + e0 + 4LL * (l0 + j * kWorkers));
+#pragma unroll
+          for (int j = 0; j < kBatch; ++j) {
+            float* d = w_snap + m * snap_stride + shift + e0 + 4LL * (l0 + j * kWorkers);
+            st1(d, v[j].x); st1(d + 1, v[j].y); st1(d + 2, v[j].z); st1(d + 3, v[j].w);
+          }
+        }
+      } else {
+        for (int j = 0; j < kBatch; ++j) {
+          const int l = l0 + j * kWorkers;
+          if (l >= kSnapTileElems / 4 || !copy_lane(l)) break;
         }
       }
     }

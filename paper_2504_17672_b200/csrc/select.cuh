@@ -77,8 +77,8 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   __shared__ long long s_pool_pos;   // next free element of the snapshot pool (kept a multiple of 4)
   // A fragment's place in the pool starts at the next multiple of 4 plus its native offset mod 4: recorded and
   // native values then share their 16-byte alignment, and the streaming kernels can move the fragment as
-  // vectors (a place that breaks the congruence sends the whole segment down the element-wise path, at a
-  // sixth of the bandwidth).
+  // vectors staged by bulk copies (a place that breaks the congruence leaves only 4-byte accesses for the
+  // recorded values, at half to two thirds of the bandwidth).
   auto place = [&](int f, long long& pool_pos) {
     const long long start = pool_pos + s_falign[f];
     pool_offset[f] = start;
