@@ -125,7 +125,7 @@ __device__ __forceinline__ float comp(const float4& v, int k) { return reinterpr
 
 // One scalar element, any M (ragged edges, unaligned snapshot layouts, worker counts not instantiated).
 template <int MODE, bool SAME>
-__device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, long long snap_e, double& acc) {
+__device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, long long snap_e, float& sq) {
   const int M = A.M;
   const float thg = ld1(A.theta_g + e);
   if (MODE == MODE_PSEUDO_SUM) {
@@ -147,7 +147,7 @@ __device__ __forceinline__ void scalar_element(const OuterArgs& A, long long e, 
     const float Delta = mean_of_sum<0>(sum, A);
     float u_new;
     outer_update(Delta, thg, ld1(A.momentum + e), A, u_new, G);
-    acc += (double)__fmul_rn(Delta, Delta);
+    sq = __fmaf_rn(Delta, Delta, sq);   // the lane's squares add up in fp32, element order, as in Lane::compute
     st1(A.theta_g + e, G);
     st1(A.momentum + e, u_new);
     if (A.delta_out) st1(A.delta_out + e, Delta);
@@ -300,10 +300,15 @@ __device__ __forceinline__ void ragged_lane(const OuterArgs& A, const SegPlan& s
       return;
     }
   }
+  // Element by element, with the lane's sum of squares formed exactly as the vector path forms it (fp32 over
+  // the lane's elements in order, then one conversion): every kernel that walks the same tiles then arrives at
+  // the same fragment norms bit for bit, whichever path its lanes took.
+  float sq = 0.f;
   for (int k = 0; k < 4; ++k) {
     const long long ee = e + k;
-    if (ee >= sp.off && ee < seg_end) scalar_element<MODE, SAME>(A, ee, ee + snap_shift, acc);
+    if (ee >= sp.off && ee < seg_end) scalar_element<MODE, SAME>(A, ee, ee + snap_shift, sq);
   }
+  if (mode_updates_global(MODE)) acc += (double)sq;
 }
 
 // Walks the tiles of one CTA (tile = blockIdx.x + i*gridDim.x) and keeps the segment they fall in.

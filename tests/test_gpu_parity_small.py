@@ -369,10 +369,9 @@ def test_worker_counts_beyond_the_instantiated_ones(M):
     check_step_against_oracle(a, before, ids, 100, 100, orc_hyper(a.w, tau=0), same=True)
 
 
-@pytest.mark.parametrize("seed", range(12))
-def test_random_partitions_layouts_and_modes(seed):
-    """Randomised sweep: fragment tables with gaps, odd offsets and several segments, random worker counts,
-    id lists, snapshot layouts (plain / packed pool with arbitrary offsets), sign modes, mixing factors."""
+def random_problem_spec(seed):
+    """A random fragment table (gaps, odd offsets, several segments), worker count, id list and snapshot layout
+    (plain / packed pool / packed pool at arbitrary offsets); returns (rng, workload, ids, generate-kwargs)."""
     rng = np.random.default_rng(1000 + seed)
     M = int(rng.choice([1, 2, 3, 4, 4, 4, 6, 8, 11]))
     K = int(rng.integers(1, 7))
@@ -398,6 +397,15 @@ def test_random_partitions_layouts_and_modes(seed):
                 offs[p] = cur
                 cur += w.partition.frag_size(p) + int(rng.integers(0, 6))
             kw.update(pool_offsets=offs, pool_len=cur + 8 - cur % 4)
+    return rng, w, ids, kw
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_partitions_layouts_and_modes(seed):
+    """Randomised sweep: fragment tables with gaps, odd offsets and several segments, random worker counts,
+    id lists, snapshot layouts (plain / packed pool with arbitrary offsets), sign modes, mixing factors."""
+    rng, w, ids, kw = random_problem_spec(seed)
+    M = w.M
     prob = GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3, **kw))
     prob.set_ids(ids)
     sign = int(rng.integers(0, 3))
@@ -416,6 +424,41 @@ def test_random_partitions_layouts_and_modes(seed):
     assert prob.poll() == 0
     exp = orc.snapshot(fragments_of(w), snap_before["w_now"], ids, M, snap_before["snap_offset"], snap_before["w_snap"])
     assert np.array_equal(np_(prob.bufs.w_snap), exp)
+
+
+@pytest.mark.parametrize("seed", range(100, 112))
+def test_random_problems_unfused_and_two_phase_equal_the_fused_step(seed):
+    """On the same random tables and layouts: S1-S3+S6 then S4-S5 as two calls, and the worker-per-device chain
+    (pseudo-gradient sum, then the completion from that sum with every worker local), must reproduce the fused
+    step bit for bit.  The halves and the sum read few streams and run with other tile widths and ring depths
+    than the fused step, in packed and odd-offset pools too."""
+    rng, w, ids, kw = random_problem_spec(seed)
+    probs = [GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3, **kw)) for _ in range(3)]
+    for prob in probs:
+        prob.set_ids(ids)
+    a, b, c = probs
+    sign = int(rng.integers(0, 3))
+    hp = dict(sign_mode=sign, alpha=float(rng.choice([1.0, 0.5])), comp_mode=int(rng.choice([1, 1, 0])))
+    t_p = 7
+    t_l = t_p + w.tau
+    a.outer_step(t_p, t_l, hyper=a.hyper(**hp))
+    b.outer_step(t_p, t_l, hyper=b.hyper(**hp), stages=1 | 4)
+    b.merge(b.bufs.theta_g, hyper=b.hyper(**hp))
+    cb = c.bufs
+    sums = torch.full((w.N,), 3.0, device="cuda")
+    c.ctx.cocodc_pseudo_gradient_sum(cb.w_snap, cb.snap_stride, cb.snap_offset, cb.theta_g, w.M, sums, c.ids, c.n_ids)
+    c.ctx.cocodc_outer_step_received(c.hyper(**hp), w.M, cb.w_now, cb.w_snap, cb.now_stride, cb.snap_stride,
+                                     cb.snap_offset, cb.theta_g, cb.momentum, sums, None, c.ids, c.n_ids, t_p, t_l,
+                                     c.last_sync, c.norms, c.scores)
+    for other, what in ((b, "unfused"), (c, "two-phase")):
+        assert other.poll() == 0
+        for name in ("w_now", "theta_g", "momentum", "w_snap"):
+            assert torch.equal(getattr(a.bufs, name), getattr(other.bufs, name)), (what, name)
+        assert torch.equal(a.norms, other.norms) and torch.equal(a.scores, other.scores), what
+        assert torch.equal(a.last_sync, other.last_sync), what
+    assert a.poll() == 0
+    untouched = torch.from_numpy(~touched_mask(w, ids)).cuda()
+    assert bool((sums[untouched] == 3.0).all())
 
 
 def _check_pooled(prob, before, ids, t_p, t_l):
