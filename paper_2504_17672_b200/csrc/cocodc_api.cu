@@ -140,7 +140,8 @@ void opt_in_shared_memory(cocodc_ctx* c, const void* kernel, unsigned bytes) {
   c->smem_opted_in.emplace_back(kernel, bytes);
 }
 
-// Worker counts 1..8 are staged through shared memory by TMA; larger M take the generic element loop.
+// Worker counts 1..8 have compile-time instances of the staged kernel; larger M take the chunk-ring kernel
+// (or the element loop when one tile of recorded values does not fit its ring): runtime_variant().
 template <int MODE, bool SAME>
 Variant pick_variant(int M) {
   switch (M) {
@@ -314,6 +315,7 @@ cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, 
   segs.reserve(S);
   for (int p = 0; p < K; ++p) {
     if (part->frag_seg_ptr[p + 1] <= part->frag_seg_ptr[p]) return COCODC_ERR_INVALID_ARG;  // empty fragment
+    if (part->frag_seg_ptr[p + 1] > S) return COCODC_ERR_INVALID_ARG;   // would read past the segment arrays
     for (int s = part->frag_seg_ptr[p]; s < part->frag_seg_ptr[p + 1]; ++s) {
       const long long o = part->seg_offset[s], l = part->seg_len[s];
       if (o < 0 || l < 1 || o > part->N - l) return COCODC_ERR_INVALID_ARG;

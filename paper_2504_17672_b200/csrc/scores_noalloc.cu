@@ -187,6 +187,7 @@ extern "C" cocodc_status cocodc_fragment_scores_noalloc(const cocodc_partition* 
   std::pair<long long, long long> sorted[kNoallocMaxSeg];
   for (int p = 0; p < K; ++p) {
     if (part->frag_seg_ptr[p + 1] <= part->frag_seg_ptr[p]) return COCODC_ERR_INVALID_ARG;
+    if (part->frag_seg_ptr[p + 1] > S) return COCODC_ERR_INVALID_ARG;   // a pointer past the S segments the arrays hold
     for (int s = part->frag_seg_ptr[p]; s < part->frag_seg_ptr[p + 1]; ++s) {
       const long long o = part->seg_offset[s], l = part->seg_len[s];
       if (o < 0 || l < 1 || o > part->N - l) return COCODC_ERR_INVALID_ARG;

@@ -181,6 +181,8 @@ def check_step_against_oracle(prob: GpuProblem, before: dict, ids, t_p, t_l, ohp
         g = orc.gather_fragment(frs, after["theta_g"], p)
         u = orc.gather_fragment(frs, after["momentum"], p)
         fl_d = fl_u = fl_g = fl_b = None
+        # the operand floors are a contract for test partitions only: none of the named workloads may reach them
+        assert g.size >= SMALL_FRAGMENT or w.name not in synth.WORKLOAD_NAMES, (w.name, p, g.size)
         if g.size < SMALL_FRAGMENT:
             fl_d, fl_u, fl_g, fl_b = operand_floors(frs, before, snap, None if same else before["snap_offset"],
                                                     int(p), ohp.momentum)
@@ -251,7 +253,7 @@ def sample_positions(n: int, rng, n_random=100_000, edge=5000, tile=2048) -> np.
 class SampledCheck:
     """Gathers the inputs of sampled elements before a step, and checks the outputs afterwards."""
 
-    def __init__(self, prob: GpuProblem, ids, seed=0, same=False):
+    def __init__(self, prob: GpuProblem, ids, seed=0, same=False, n_random=100_000, edge=5000):
         self.prob, self.ids, self.same = prob, [int(p) for p in ids], same
         w, b = prob.w, prob.bufs
         rng = np.random.default_rng(seed)
@@ -260,7 +262,7 @@ class SampledCheck:
         self.inputs = {}
         dev = prob.dev
         for p in self.ids:
-            rel = sample_positions(w.partition.frag_size(p), rng)
+            rel = sample_positions(w.partition.frag_size(p), rng, n_random=n_random, edge=edge)
             native, snap = _fragment_index_maps(w, p, rel, so)
             ni = torch.from_numpy(native).to(dev)
             si = torch.from_numpy(snap).to(dev)
@@ -319,5 +321,71 @@ def oracle_fragment_norm(prob: GpuProblem, p: int, theta_g_before: torch.Tensor 
     snap = np.ascontiguousarray(snap)
     zeros = np.zeros(n, dtype=np.float32)
     hp = orc_hyper(w)
-    res, _ = orc.outer_step([[(0, n)]], hp, snap, snap, thg, zeros, [0], 1, 1, [0], do_merge=False)
+    res, _ = orc.outer_step([[(0, n)]], hp, snap, snap, thg, zeros, [0], 1, 1, [0], do_merge=False,
+                            threads=host_cores())
     return res[0].norm
+
+
+# --------------------------------------------------------------------------
+# full-size workloads: whole fragments, element by element, streamed through the oracle one at a time
+# --------------------------------------------------------------------------
+
+def host_cores() -> int:
+    import os
+    return len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1)
+
+
+def _gather_fragment_to_host(w: synth.Workload, t: torch.Tensor, p: int, base=None) -> np.ndarray:
+    """Fragment p of an [N] or [M, N] device tensor as one contiguous host array (segments concatenated);
+    `base`: the fragment sits packed at this element offset instead of at its native offsets."""
+    if base is not None:
+        n = w.partition.frag_size(p)
+        return np.ascontiguousarray(np_(t[..., base:base + n]))
+    return np.ascontiguousarray(np.concatenate([np_(t[..., o:o + l]) for o, l in w.partition.fragments[p]], axis=-1))
+
+
+class FullFragmentCheck:
+    """Element-by-element parity on whole fragments of a workload too large to copy to the host at once.
+
+    Before the step: the inputs of every listed fragment are copied to the host.  After it: fragment by fragment
+    the oracle runs on those inputs (element range split over the host cores) and every output element of the
+    GPU is compared with it; the oracle's norm and score of the whole fragment are compared too."""
+
+    def __init__(self, prob: GpuProblem, ids):
+        self.prob, self.ids = prob, [int(p) for p in ids]
+        w, b = prob.w, prob.bufs
+        so = None if b.snap_offset is None else np_(b.snap_offset)
+        self.inputs = {}
+        for p in self.ids:
+            self.inputs[p] = dict(
+                w_now=_gather_fragment_to_host(w, b.w_now, p),
+                w_snap=_gather_fragment_to_host(w, b.w_snap, p, None if so is None else int(so[p])),
+                theta_g=_gather_fragment_to_host(w, b.theta_g, p),
+                momentum=_gather_fragment_to_host(w, b.momentum, p))
+        self.last_sync = np_(prob.last_sync).copy()
+
+    def check(self, t_p, t_l, ohp: orc.Hyper):
+        prob = self.prob
+        w, b = prob.w, prob.bufs
+        norms, scores = np_(prob.norms), np_(prob.scores)
+        worst = 0.0
+        threads = host_cores()
+        for p in self.ids:
+            assert w.partition.frag_size(p) >= SMALL_FRAGMENT
+            x = self.inputs.pop(p)
+            n = x["theta_g"].shape[0]
+            res, _ = orc.outer_step([[(0, n)]], ohp, x["w_now"], x["w_snap"], x["theta_g"], x["momentum"], [0],
+                                    t_p, t_l, [int(self.last_sync[p])], threads=threads)
+            r = res[0]
+            del x
+            worst = max(worst, *assert_close(_gather_fragment_to_host(w, b.theta_g, p), r.theta_g, TOL_PARAM,
+                                             f"theta_g[{p}]"))
+            worst = max(worst, *assert_close(_gather_fragment_to_host(w, b.momentum, p), r.momentum, TOL_PARAM,
+                                             f"momentum[{p}]"))
+            got = _gather_fragment_to_host(w, b.w_now, p)
+            for m in range(w.M):
+                worst = max(worst, *assert_close(got[m], r.w_now[m], TOL_PARAM, f"w_now[{m}][{p}]"))
+            assert abs(norms[p] - r.norm) <= TOL_NORM * r.norm, (p, norms[p], r.norm)
+            assert abs(scores[p] - r.score) <= TOL_NORM * r.score, (p, scores[p], r.score)
+            del res, r, got
+        return worst

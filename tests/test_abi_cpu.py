@@ -87,6 +87,7 @@ def test_create_rejects_bad_partitions_before_touching_the_device(B):
         (100, [0, 1], [-4], [50]),                # negative offset
         (100, [0, 1], [0], [0]),                  # empty segment
         (100, [1, 2], [0, 50], [50, 50]),         # CSR does not start at 0
+        (100, [0, 1000, 2], [0, 50], [50, 50]),   # a pointer beyond the segment arrays, although the last one equals S
     ]
     for N, ptr, off, ln in cases:
         with pytest.raises(B.CocodcError) as e:
@@ -96,6 +97,26 @@ def test_create_rejects_bad_partitions_before_touching_the_device(B):
         with pytest.raises(B.CocodcError) as e:
             create(100, [0, 1], [0], [100], max_M=bad_M)
         assert e.value.code == B.ERR_INVALID_ARG
+
+
+def test_noalloc_entry_point_checks_its_table_before_touching_the_device(B):
+    """The table is host data validated on every call; a pointer array that is not monotone must not make the
+    host loop read past the segment arrays (the addresses below are never dereferenced: validation fails first)."""
+    fake = ctypes.c_void_p(0x10000)
+
+    def call(N, ptr, off, ln):
+        ptr = np.ascontiguousarray(ptr, dtype=np.int32)
+        off = np.ascontiguousarray(off, dtype=np.int64)
+        ln = np.ascontiguousarray(ln, dtype=np.int64)
+        part = B._Partition(N, len(ptr) - 1, len(off), ptr.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)),
+                            off.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)),
+                            ln.ctypes.data_as(ctypes.POINTER(ctypes.c_int64)))
+        return B.library().cocodc_fragment_scores_noalloc(ctypes.byref(part), fake, None, fake, fake, 0, None)
+
+    assert call(100, [0, 1000, 2], [0, 50], [50, 50]) == B.ERR_INVALID_ARG
+    assert call(100, [0, 2, 2], [0, 50], [50, 50]) == B.ERR_INVALID_ARG        # empty second fragment
+    assert call(100, [0, 1, 2], [0, 40], [50, 50]) == B.ERR_INVALID_ARG        # overlap
+    assert call(100, [0, 1, 2], [0, 60], [50, 50]) == B.ERR_INVALID_ARG        # past N
 
 
 def test_null_context_is_rejected(B):

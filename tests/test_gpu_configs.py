@@ -1,9 +1,10 @@
 """Parity on the five benchmark workloads, in the launch configuration the benchmark times.
 
-tiny and gpt2_small are compared element by element over every processed fragment.  The
-billion-parameter shapes are compared on sampled elements (edges, tile borders, random positions),
-whole-fragment norms from the oracle for two fragments, a float64 torch reduction for the rest, and
-bit-exact checksums of everything that must not change."""
+tiny, gpt2_small and paper_150m are compared element by element over every processed fragment, and so is the
+selected set of llama_1b (whole fragments streamed through the oracle one at a time).  Where a round completes
+more than the host can hold at once (llama_1b's start-up round, the 48 sweep variants, llama_3b) the comparison is
+on sampled elements (edges, tile borders, random positions), whole-fragment norms from the oracle, and bit-exact
+checksums of everything that must not change."""
 
 import numpy as np
 import pytest
@@ -11,7 +12,7 @@ import torch
 
 import synth
 from oracle import reference as orc
-from helpers import (GpuProblem, SampledCheck, check_step_against_oracle, fragment_checksums, np_,
+from helpers import (FullFragmentCheck, GpuProblem, SampledCheck, check_step_against_oracle, fragment_checksums, np_,
                      oracle_fragment_norm, orc_hyper, TOL_NORM)
 
 pytestmark = pytest.mark.gpu
@@ -89,35 +90,30 @@ def test_paper_150m_strided_shards_full_parity():
     assert seen == [0, 1]                     # never-synced shards first, in index order
 
 
-def _sampled_round(prob, ids, t_p, t_l, ohp, full_norm=2, same=False):
+def _sampled_round(prob, ids, t_p, t_l, ohp, norm_ids=None, same=False, n_random=100_000, full=False):
+    """One completion checked against the oracle.
+
+    Elements: sampled positions of every listed fragment (full=False) or every element of every listed fragment
+    (full=True).  Norms and scores: the oracle's, over whole fragments, for the fragments in norm_ids (default:
+    all listed; always all with full=True).  Everything that must not change: bit-exact checksums."""
     w = prob.w
     ids = [int(p) for p in ids]
     prob.set_ids(ids)
-    sc = SampledCheck(prob, ids, seed=t_p, same=same)
-    exp_norm = {p: oracle_fragment_norm(prob, p) for p in ids[:full_norm]} if not same else {}
-    # float64 reduction on the device for the remaining fragments (library cross-check at full size)
-    for p in ids[full_norm:]:
-        acc = 0.0
-        b = prob.bufs
-        pos = 0
-        for o, l in w.partition.fragments[p]:
-            if b.snap_offset is None or same:
-                s = (b.w_now if same else b.w_snap)[:, o:o + l]
-            else:
-                so = int(b.snap_offset[p].item()) + pos
-                s = b.w_snap[:, so:so + l]
-            d = (s.double() - b.theta_g[o:o + l].double()).mean(0)
-            acc += float((d * d).sum().item())
-            pos += l
-            del d
-        exp_norm[p] = float(np.sqrt(acc))
+    if full:
+        chk = FullFragmentCheck(prob, ids)
+        exp_norm = {}
+    else:
+        chk = SampledCheck(prob, ids, seed=t_p, same=same, n_random=n_random)
+        norm_ids = ids if norm_ids is None else [int(p) for p in norm_ids]
+        exp_norm = {p: oracle_fragment_norm(prob, p) for p in norm_ids} if not same else {}
     untouched = [p for p in range(w.K) if p not in ids]
     cs_before = {k: fragment_checksums(w, getattr(prob.bufs, k)) for k in ("theta_g", "momentum", "w_now")}
     last_before = np_(prob.last_sync).copy()
+    scores_before = np_(prob.scores).copy()
     prob.outer_step(t_p, t_l, hyper=prob.hyper(**{k: getattr(ohp, k) for k in ("tau", "lam", "alpha", "comp_mode", "sign_mode")}),
                     w_snap=prob.bufs.w_now if same else None)
     assert prob.poll() == 0
-    worst = sc.check(t_p, t_l, ohp)
+    worst = chk.check(t_p, t_l, ohp)
     cs_after = {k: fragment_checksums(w, getattr(prob.bufs, k)) for k in cs_before}
     for k in cs_before:
         assert np.array_equal(cs_before[k][untouched], cs_after[k][untouched]), f"{k} changed outside ids"
@@ -127,6 +123,7 @@ def _sampled_round(prob, ids, t_p, t_l, ohp, full_norm=2, same=False):
         assert abs(norms[p] - en) <= TOL_NORM * en, (p, norms[p], en)
         es = en / max(1, t_p - int(last_before[p]))
         assert abs(scores[p] - es) <= TOL_NORM * es
+    assert np.array_equal(scores[untouched], scores_before[untouched])
     exp_last = last_before.copy()
     exp_last[ids] = t_l
     assert np.array_equal(last, exp_last)
@@ -155,41 +152,47 @@ def test_llama_1b_selected_by_change_norm():
                                        orc.BUDGET_COUNT, w.budget)
     assert n == en == 4 and ids == eids.tolist()
     assert ids == list(np.argsort(-scores, kind="stable")[:4])
-    _sampled_round(prob, ids, 40, 40 + w.tau, ohp)
+    # the step the benchmark times (four fragments selected by change norm): every element against the oracle
+    _sampled_round(prob, ids, 40, 40 + w.tau, ohp, full=True)
 
 
 def test_sweep_1b_variants():
-    """Twelve of the 48 sweep variants, covering every tau, lambda and fraction, on one set of buffers.
+    """All 48 variants of the compensation sweep (tau x lambda x fraction of the 32 fragments) on one set of
+    buffers: sampled elements of every completed fragment, the oracle's norm of two whole fragments per variant
+    (taken in turn, so that every fragment is covered), checksums of what must not change.
 
-    tau and lambda reach the kernel only as the two scalars of the folded Eq. 6-7, the fraction only as the
-    length of the id list; the benchmark's sweep mode times all 48."""
+    tau and lambda reach the kernel as the two scalars that Eq. 6-7 fold into on the host, the fraction as the
+    length of the id list; it is that fold which the 48 (tau, lambda) x 3 list lengths exercise."""
     if free_gb() < 60:
         pytest.skip("needs 60 GB of free device memory")
     w0 = synth.get_workload("sweep_1b")
     bufs = synth.generate(w0, "cuda")
-    lams = [0.0, 0.25, 0.5, 1.0]
     t = 5
     i = 0
     prob = None
+    seen_pairs = set()
     for frac in (0.25, 0.5, 1.0):
         for tau in (1, 2, 4, 8):
-            lam = lams[(i + i // 4) % 4]
-            i += 1
-            w = w0.with_(tau=tau, lam=lam)
-            if prob is None:
-                prob = GpuProblem(w, bufs)
-            prob.w = w
-            if i > 1:
-                # fresh outer state for every variant: repeated completions from the same snapshots would drive
-                # the mean pseudo-gradient to the cancellation limit of fp32 (|Delta| << |delta_m|), where an
-                # error bound relative to the output no longer applies
-                bufs.momentum.normal_(0.0, 1e-3)
-                bufs.theta_g.add_(bufs.momentum)
-                bufs.momentum.normal_(0.0, 1e-3)      # independent of the shift just applied to theta_g
-            n = int(round(frac * w.K))
-            ids = list(range(n))
-            _sampled_round(prob, ids, t, t + tau, orc_hyper(w), full_norm=1)
-            t += tau + 1
+            for lam in (0.0, 0.25, 0.5, 1.0):
+                w = w0.with_(tau=tau, lam=lam)
+                if prob is None:
+                    prob = GpuProblem(w, bufs)
+                prob.w = w
+                if i > 0:
+                    # fresh outer state for every variant: repeated completions from the same snapshots drive the
+                    # mean pseudo-gradient into cancellation (|Delta| << |delta_m|), the regime that
+                    # test_cancellation_regime_error_is_bounded_by_the_operands covers with its own bound
+                    bufs.momentum.normal_(0.0, 1e-3)
+                    bufs.theta_g.add_(bufs.momentum)
+                    bufs.momentum.normal_(0.0, 1e-3)      # independent of the shift just applied to theta_g
+                n = int(round(frac * w.K))
+                ids = list(range(n))
+                norm_ids = [(2 * i) % n, (2 * i + 1) % n]
+                _sampled_round(prob, ids, t, t + tau, orc_hyper(w), norm_ids=norm_ids, n_random=20_000)
+                seen_pairs.add((frac, tau, lam))
+                t += tau + 1
+                i += 1
+    assert len(seen_pairs) == 48
 
 
 def test_llama_3b_snapshot_pool():
@@ -210,4 +213,4 @@ def test_llama_3b_snapshot_pool():
     prob.select(t_now=40)
     ids = np_(prob.ids)[:int(prob.n_ids.item())].tolist()
     assert ids == eids.tolist()
-    _sampled_round(prob, ids, 40, 40 + w.tau, orc_hyper(w), full_norm=1)
+    _sampled_round(prob, ids, 40, 40 + w.tau, orc_hyper(w))

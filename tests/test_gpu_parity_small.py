@@ -461,6 +461,76 @@ def test_random_problems_unfused_and_two_phase_equal_the_fused_step(seed):
     assert bool((sums[untouched] == 3.0).all())
 
 
+@pytest.mark.parametrize("M", [2, 3, 4])
+@pytest.mark.parametrize("depth", [1e-3, 1e-6])
+def test_cancellation_regime_error_is_bounded_by_the_operands(M, depth):
+    """Where the workers' pseudo-gradients cancel (|Delta| << |delta_m|) and the momentum term cancels against their
+    mean, no bound relative to the OUTPUT can hold in fp32: what is left of Delta and u' is rounding error of their
+    operands.  The kernel's contract there is a bound relative to the operands,
+
+        |x - y| <= (M + 2) * 2^-24 * (mean_m |delta_m| + |mu * u|)      for x in {Delta, u'},
+
+    per element: M roundings of the sum's terms and partial sums, one of the quotient, one of the momentum update
+    (each at most 2^-24 of a value no larger than the operands' magnitudes).  Inputs are built so that the mean
+    cancels to `depth` of the pseudo-gradients and u' to `depth` of mu*u; eta and mu are fp32 numbers, so both
+    sides compute with the same hyper-parameters."""
+    n = 150_000
+    w = synth.small_workload((2 * n + 8, [[(1, n)], [(n + 4, n)]]), M=M, seed=500 + M, tau=3)
+    mu, eta = float(np.float32(0.9)), float(np.float32(0.7))
+    w = w.with_(momentum=mu, outer_lr=eta)
+    bufs = synth.generate(w, "cpu")
+    rng = np.random.default_rng(M)
+    thg = bufs.theta_g.numpy().astype(np.float64)
+    snap = bufs.w_snap.numpy()
+    # the last worker's pseudo-gradient = -(sum of the others) + depth * noise
+    others = (snap[:M - 1].astype(np.float64) - thg[None, :]).sum(axis=0)
+    last = -others + depth * 1e-3 * rng.standard_normal(thg.shape)
+    snap[M - 1] = (thg + last).astype(np.float32)
+    delta_m = snap.astype(np.float64) - thg[None, :]                     # what the workers' values really encode
+    mean = delta_m.mean(axis=0)
+    # momentum that cancels the mean to `depth`:  mu*u + Delta = depth * |mu*u| * noise
+    u_mag = 1e-3 * (1.0 + rng.random(thg.shape))
+    u = (-mean + depth * u_mag * rng.standard_normal(thg.shape)) / mu
+    big = rng.random(thg.shape) < 0.5                                     # half the elements: a large momentum, cancelled by nothing
+    u = np.where(big, u_mag * np.sign(rng.standard_normal(thg.shape)), u)
+    bufs.momentum.copy_(torch.from_numpy(u.astype(np.float32)))
+    for name in ("theta_g", "momentum", "w_now", "w_snap"):
+        setattr(bufs, name, getattr(bufs, name).cuda())
+    prob = GpuProblem(w, bufs)
+    ids = [1, 0]
+    prob.set_ids(ids)
+    before = prob.host_state()
+    delta = torch.zeros(w.N, device="cuda")
+    prob.outer_step(6, 9, delta_out=delta)
+    assert prob.poll() == 0
+    frs = fragments_of(w)
+    res, _ = orc.outer_step(frs, orc_hyper(w), before["w_now"], before["w_snap"], before["theta_g"],
+                            before["momentum"], ids, 6, 9, before["last_sync"])
+    after = prob.host_state()
+    worst = 0.0
+    cancelled = 1.0
+    for p in ids:
+        b = orc.gather_fragment(frs, before["w_snap"], p).astype(np.float64)
+        g0 = orc.gather_fragment(frs, before["theta_g"], p).astype(np.float64)
+        u0 = orc.gather_fragment(frs, before["momentum"], p).astype(np.float64)
+        operands = np.abs(b - g0[None, :]).mean(axis=0) + np.abs(mu * u0)
+        bound = (M + 2) * 2.0 ** -24 * operands
+        got_d = orc.gather_fragment(frs, np_(delta), p).astype(np.float64)
+        got_u = orc.gather_fragment(frs, after["momentum"], p).astype(np.float64)
+        for got, exp, what in ((got_d, res[p].delta_g, "Delta"), (got_u, res[p].momentum, "u'")):
+            err = np.abs(got - exp)
+            assert np.all(err <= bound), (what, p, float((err / bound).max()))
+            worst = max(worst, float((err / bound).max()))
+        cancelled = min(cancelled, float(np.median(np.abs(res[p].delta_g) / np.abs(b - g0[None, :]).mean(axis=0))))
+        # the new global state and the merged parameters keep the ordinary bound: |theta_g| dominates them
+        assert_close(orc.gather_fragment(frs, after["theta_g"], p), res[p].theta_g, TOL_PARAM, f"theta_g[{p}]")
+        wn = orc.gather_fragment(frs, after["w_now"], p)
+        for m in range(M):
+            assert_close(wn[m], res[p].w_now[m], TOL_PARAM, f"w_now[{m}][{p}]")
+    assert cancelled < 10 * depth + 1e-5, cancelled         # the inputs really are in the cancellation regime
+    assert worst > 0.0
+
+
 def _check_pooled(prob, before, ids, t_p, t_l):
     """Parity over all listed fragments taken together (fragments of one or a few elements leave the
     per-fragment measure nothing to normalise by when an output is small against its operands)."""

@@ -32,6 +32,13 @@ def test_workload_shapes():
     assert synth.get_workload("sweep_1b").partition.frag_size(7) == 29_788_224
 
 
+def test_named_workloads_have_no_tiny_fragments():
+    """The parity helpers measure fragments of fewer than 64 elements against their operands (test partitions
+    only); every named workload stays far above that, so its parity is always relative to the outputs."""
+    for name in synth.WORKLOAD_NAMES:
+        assert int(synth.get_workload(name).partition.frag_sizes.min()) >= 131_072, name
+
+
 def test_generate_is_seeded_and_layout_independent():
     w = synth.small_workload((1000, [[(3, 100), (700, 57)], [(103, 250)], [(400, 299)]]), M=3, seed=5,
                              scale_kind="loguniform")

@@ -1,4 +1,4 @@
-"""cocodc_fragment_scores_noalloc against cocodc_fragment_scores.
+"""cocodc_fragment_scores_noalloc against the CPU oracle and against cocodc_fragment_scores.
 
 The no-allocation entry point serves callers that are not allowed to allocate device memory (code
 inside an allocator hook, processes with a closed device heap, allocation-free hot paths): it keeps
@@ -11,6 +11,7 @@ import pytest
 import torch
 
 import synth
+from oracle import reference as orc
 from helpers import TOL_NORM, np_
 
 pytestmark = pytest.mark.gpu
@@ -27,6 +28,7 @@ def test_noalloc_scores_match_the_context_entry_point_on_two_calls_in_a_row():
     ctx = B.Context(w.N, ptr, off, ln, 1)
     gen = torch.Generator(device="cuda").manual_seed(21)
     interval = torch.tensor([0, 3, 100, 7, 1], dtype=torch.int64, device="cuda")
+    frs = [list(f) for f in w.partition.fragments]
     # the second call sees different data and a fragment of zeros: nothing of the first call may leak through
     for call in range(2):
         x = torch.randn(w.N, generator=gen, device="cuda") * (1e-3 if call == 0 else 5e-2)
@@ -38,11 +40,22 @@ def test_noalloc_scores_match_the_context_entry_point_on_two_calls_in_a_row():
         assert ctx.cocodc_poll_status() == 0
         got_n = torch.full((K,), -1.0, device="cuda")
         got_s = torch.full((K,), -1.0, device="cuda")
+        # The device's free memory as the driver reports it (torch's own counters see only torch's allocator, not a
+        # cudaMalloc inside the library).  The first call on a device may load the module that holds the scratch
+        # array when it looks up its address, so the comparison is made around a later call.
+        if call == 1:
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
         before = torch.cuda.memory_allocated()
         B.cocodc_fragment_scores_noalloc(w.N, ptr, off, ln, x, interval, got_n, got_s)
         torch.cuda.synchronize()
         assert torch.cuda.memory_allocated() == before
+        if call == 1:
+            assert torch.cuda.mem_get_info()[0] == free_before, "device memory was allocated during the call"
         rn, rs, gn, gs = np_(ref_n), np_(ref_s), np_(got_n), np_(got_s)
+        en, es = orc.fragment_scores(frs, np_(x), np_(interval))          # Eq. 10 by the CPU oracle
+        assert np.all(np.abs(gn - en) <= TOL_NORM * np.abs(en)), (call, gn, en)
+        assert np.all(np.abs(gs - es) <= TOL_NORM * np.abs(es)), (call, gs, es)
         assert np.all(np.abs(gn - rn) <= TOL_NORM * np.abs(rn)), (call, gn, rn)
         assert np.all(np.abs(gs - rs) <= TOL_NORM * np.abs(rs)), (call, gs, rs)
         if call == 1:
