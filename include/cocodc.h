@@ -27,7 +27,7 @@
  *     (a copy of the fragment table, a few KB of launch scratch, a status word),
  *     allocated by cocodc_create and released by cocodc_destroy.
  *   - Device entry points are asynchronous on the given stream and allocate
- *     nothing.  Their return value reports host-side validation and launch
+ *     nothing, neither device nor host memory.  Their return value reports host-side validation and launch
  *     errors; conditions found on the device (a non-finite norm, an invalid id
  *     list, a NaN score) are recorded in the context's status word, read with
  *     cocodc_poll_status.  Nothing aborts, traps or prints.
@@ -38,6 +38,11 @@
  *     billion-parameter models.
  *   - A context serialises its own launches on one stream at a time: calls that
  *     share a context must not overlap on the GPU.
+ *   - Step numbers (t_now, t_p, t_l, last_sync[p]) are non-negative and last_sync[p] <= t_now, t_p:
+ *     differences of step numbers are formed in 64-bit integers and must not overflow.
+ *   - Every wait inside a kernel is bounded.  A launch whose wait ran out records COCODC_ERR_TIMEOUT
+ *     and returns early; its outputs, and those of later launches on the stream, are undefined until
+ *     the caller has read the status (cocodc_poll_status synchronises and resets the context).
  */
 #ifndef COCODC_H
 #define COCODC_H
@@ -90,6 +95,8 @@ typedef enum { COCODC_BUDGET_COUNT = 0, COCODC_BUDGET_PARAMS = 1, COCODC_BUDGET_
 #define COCODC_STAGE_MERGE 2u   /* S4-S5: update w_now */
 #define COCODC_STAGE_SCORE 4u   /* S6: norms, scores, last_sync of the processed fragments */
 #define COCODC_STAGE_ALL   7u
+#define COCODC_STAGE_SUMSQ 8u   /* S6 up to the sums only: sumsq_out[p] = sum of Delta^2 over fragment p (Eq. 10 before the
+                                   square root), for callers that add the sums of several devices before forming scores */
 
 /*
  * Fragment partition (Section 2.1: the model is cut into K disjoint fragments).
@@ -147,12 +154,43 @@ cocodc_status cocodc_sync_budget(int32_t K, int64_t H, double gamma, double Tc, 
  * scores[p] = norms[p] / max(1, interval[p]) for all K fragments.
  *   delta_g  dev fp32[N]   the received mean pseudo-gradients
  *   interval dev int64[K]  I_p = t_p - t_{p,b}; NULL means 1
- *   norms, scores dev fp32[K], written
+ *   norms, scores dev fp32[K], written (both NULL: only sumsq_out is wanted)
+ *   sumsq_out dev fp64[K] or NULL: the sums of squares before the square root
  * Sums of squares are accumulated in double in a fixed order (run-to-run
  * reproducible).  A non-finite norm sets COCODC_ERR_NONFINITE in the status word.
+ * One kernel launch: the last warp to finish forms the norms.
  */
 cocodc_status cocodc_fragment_scores(cocodc_ctx* ctx, const float* delta_g, const int64_t* interval,
-                                     float* norms, float* scores, void* stream);
+                                     float* norms, float* scores, double* sumsq_out, void* stream);
+
+/*
+ * The rest of Eq. 10 from sums of squares that already exist: when every device holds a slice of each
+ * fragment (all workers of an element range), a fragment's norm spans devices; each device takes its sums
+ * from cocodc_outer_step (COCODC_STAGE_SUMSQ) or cocodc_fragment_scores (sumsq_out), the caller adds them
+ * over the devices (an all-reduce of K doubles), and this call forms norms and scores from the totals:
+ *   norms[p] = sqrt(sumsq[p]),  scores[p] = norms[p] / max(1, I_p)
+ *   sumsq dev fp64[K], indexed by fragment id
+ *   completion (ids, n_ids given; interval NULL): for the listed fragments I_p = t_p - last_sync[p], then
+ *       last_sync[p] = t_l (and a bound in-flight mask is cleared, see cocodc_bind_in_flight)
+ *   stand-alone (ids, n_ids NULL): all K fragments, I_p = interval[p] (1 without intervals); t_p, t_l and
+ *       last_sync are not used
+ * A non-finite norm sets COCODC_ERR_NONFINITE, an id outside [0, K) INVALID_ARG, in the status word.
+ */
+cocodc_status cocodc_scores_from_sumsq(cocodc_ctx* ctx, const double* sumsq, const int32_t* ids, const int32_t* n_ids,
+                                       const int64_t* interval, int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                       float* norms, float* scores, void* stream);
+
+/*
+ * Algorithm 2's bookkeeping of the fragments whose synchronisation is in flight (a fragment chosen at t_p
+ * cannot be chosen again before it completes at t_p + tau).  in_flight is a dev uint8[K] array owned by the
+ * caller, zero-initialised by it; once bound to the context,
+ *   cocodc_select_fragments(_at)  treats in_flight[p] != 0 as not eligible and sets in_flight[p] = 1 for
+ *                                 every fragment it selects,
+ *   every completion that writes scores (cocodc_outer_step and its variants with COCODC_STAGE_SCORE,
+ *   cocodc_scores_from_sumsq with an id list) sets in_flight[p] = 0 for the fragments it lists.
+ * NULL unbinds.  The host-buffer entry points do not use it.
+ */
+cocodc_status cocodc_bind_in_flight(cocodc_ctx* ctx, uint8_t* in_flight);
 
 /*
  * S7 (Algorithm 2, Eq. 11, extended to a budget).  Priority order: eligible
@@ -203,7 +241,10 @@ cocodc_status cocodc_select_fragments(cocodc_ctx* ctx, const float* scores, cons
  * and theta_g[i] = G, momentum[i] = u', delta_g_out[i] = Delta (if not NULL).
  * With STAGE_SCORE, for each listed p: norms[p] = ||Delta||_2 over the fragment,
  * scores[p] = norms[p] / max(1, t_p - last_sync[p]), then last_sync[p] = t_l.
- * Fragments not listed are not touched.
+ * With STAGE_SUMSQ (or STAGE_SCORE and sumsq_out not NULL): sumsq_out[p] = sum of Delta^2 over the fragment.
+ * Fragments not listed are not touched.  The whole call is one kernel launch (the id list is expanded by
+ * the kernel itself and the norms are formed by its last warp) for fragment tables of up to 128 segments;
+ * larger tables take one more small launch.
  *
  *   w_now   dev fp32, worker m's element i at w_now[m*now_stride + i]   (theta^m_{.,t_l}, in/out)
  *   w_snap  dev fp32, theta^m_{p,t_p}: at w_snap[m*snap_stride + i] if snap_offset is NULL,
@@ -213,6 +254,7 @@ cocodc_status cocodc_select_fragments(cocodc_ctx* ctx, const float* scores, cons
  *   theta_g, momentum dev fp32[N] in/out; delta_g_out dev fp32[N] or NULL
  *   ids dev int32[<=K] distinct fragment ids; n_ids dev int32[1]
  *   last_sync dev int64[K]; norms, scores dev fp32[K] (needed with STAGE_SCORE)
+ *   sumsq_out dev fp64[K] (needed with STAGE_SUMSQ), or NULL
  * Errors: INVALID_ARG, ALIGNMENT, ALIAS (buffers overlapping other than w_snap == w_now), CUDA.
  * Device-side: an id outside [0,K) or listed twice, a listed fragment without a place in the pool
  * (snap_offset[p] < 0) or whose packed snapshot would not fit inside one row (snap_offset[p] + n_p >
@@ -224,7 +266,7 @@ cocodc_status cocodc_outer_step(cocodc_ctx* ctx, const cocodc_hyper* hyper,
                                 float* theta_g, float* momentum, float* delta_g_out,
                                 const int32_t* ids, const int32_t* n_ids,
                                 int64_t t_p, int64_t t_l, int64_t* last_sync,
-                                float* norms, float* scores, uint32_t stages, void* stream);
+                                float* norms, float* scores, double* sumsq_out, uint32_t stages, void* stream);
 
 /*
  * cocodc_select_fragments and cocodc_outer_step with their step numbers read from DEVICE memory at run time
@@ -244,7 +286,7 @@ cocodc_status cocodc_outer_step_at(cocodc_ctx* ctx, const cocodc_hyper* hyper,
                                    float* theta_g, float* momentum, float* delta_g_out,
                                    const int32_t* ids, const int32_t* n_ids,
                                    const int64_t* t_p, const int64_t* t_l, int64_t* last_sync,
-                                   float* norms, float* scores, uint32_t stages, void* stream);
+                                   float* norms, float* scores, double* sumsq_out, uint32_t stages, void* stream);
 
 /*
  * Worker-per-device deployment (Section 2.1: every worker all-reduces its pseudo-gradient).  When a
@@ -288,6 +330,8 @@ cocodc_status cocodc_outer_step_received(cocodc_ctx* ctx, const cocodc_hyper* hy
  * be overwritten until every device has finished it (a barrier on the host, or stream events, before and
  * after).  delta_g_out may be NULL or one of the listed buffers of THIS device (replaced by Delta in place).
  * With n_sums == 1 this is cocodc_outer_step_received.
+ * Reads from another device's memory have not been exercised on hardware: every test so far passed buffers of
+ * the calling device.
  */
 #define COCODC_MAX_SUMS 8
 cocodc_status cocodc_outer_step_received_peers(cocodc_ctx* ctx, const cocodc_hyper* hyper, int32_t M_total,
@@ -388,16 +432,19 @@ cocodc_status cocodc_fragment_scores_noalloc(const cocodc_partition* partition, 
 
 /*
  * Waits for the stream, then returns and clears the device status word
- * (COCODC_OK if nothing was recorded since the last poll).
+ * (COCODC_OK if nothing was recorded since the last poll).  After an error the context's launch
+ * scratch is reset, so the next call starts clean.
  */
 cocodc_status cocodc_poll_status(cocodc_ctx* ctx, void* stream);
 
 /*
  * Failure-detection self-test.  The staged kernels wait on shared-memory barriers for their bulk
  * copies; every such wait gives up after a fixed number of polls, records COCODC_ERR_TIMEOUT in the
- * status word and lets the kernel return.  This call runs that wait on a barrier nothing will
- * complete, with `polls` (1 .. 4194304) as the limit: afterwards cocodc_poll_status returns
- * COCODC_ERR_TIMEOUT and the context is as usable as before.  It cannot hang: the loop is bounded.
+ * status word and lets the kernel return (a producer first waits, again with a limit, for the copies
+ * it has already started, so that they do not land in shared memory that has moved on to another block).
+ * This call runs that wait on a barrier nothing will complete, with `polls` (1 .. 4194304) as the limit:
+ * afterwards cocodc_poll_status returns COCODC_ERR_TIMEOUT and the context is as usable as before.  It
+ * cannot hang: the loop is bounded.
  */
 cocodc_status cocodc_selftest_bounded_wait(cocodc_ctx* ctx, int32_t polls, void* stream);
 

@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_NONFINITE, ERR_TIMEOUT, ERR_C
 COMP_NONE, COMP_TAYLOR = 0, 1
 SIGN_FORWARD, SIGN_PRINTED, SIGN_DESCENT = 0, 1, 2
 BUDGET_COUNT, BUDGET_PARAMS, BUDGET_PARAMS_EXACT = 0, 1, 2
-STAGE_OUTER, STAGE_MERGE, STAGE_SCORE, STAGE_ALL = 1, 2, 4, 7
+STAGE_OUTER, STAGE_MERGE, STAGE_SCORE, STAGE_ALL, STAGE_SUMSQ = 1, 2, 4, 7, 8
 
 EXPORTS = (
     "cocodc_create", "cocodc_destroy", "cocodc_sync_budget", "cocodc_fragment_scores",
@@ -29,6 +29,7 @@ EXPORTS = (
     "cocodc_fragment_scores_noalloc", "cocodc_selftest_bounded_wait",
     "cocodc_pseudo_gradient_sum", "cocodc_outer_step_received",
     "cocodc_select_fragments_at", "cocodc_outer_step_at", "cocodc_outer_step_received_peers",
+    "cocodc_scores_from_sumsq", "cocodc_bind_in_flight",
 )
 NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
@@ -82,10 +83,12 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(_Partition), i32, i32]
     lib.cocodc_destroy.argtypes = [vp]
     lib.cocodc_sync_budget.argtypes = [i32, i64, f64, f64, f64, ctypes.POINTER(i64), ctypes.POINTER(i64)]
-    lib.cocodc_fragment_scores.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.cocodc_fragment_scores.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.cocodc_scores_from_sumsq.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp]
+    lib.cocodc_bind_in_flight.argtypes = [vp, vp]
     lib.cocodc_select_fragments.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp]
     lib.cocodc_outer_step.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, vp,
-                                      i64, i64, vp, vp, vp, u32, vp]
+                                      i64, i64, vp, vp, vp, vp, u32, vp]
     lib.cocodc_outer_step_host.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, i32,
                                            i64, i64, vp, vp, vp, i32, vp, ctypes.c_uint64, vp]
     lib.cocodc_snapshot_host.argtypes = [vp, vp, vp, i64, i64, vp, i32, vp, i32, vp]
@@ -95,7 +98,7 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_selftest_bounded_wait.argtypes = [vp, i32, vp]
     lib.cocodc_select_fragments_at.argtypes = [vp, vp, vp, vp, vp, i64, i32, i64, vp, vp, vp, vp, vp]
     lib.cocodc_outer_step_at.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, vp,
-                                         vp, vp, vp, vp, vp, u32, vp]
+                                         vp, vp, vp, vp, vp, vp, u32, vp]
     lib.cocodc_pseudo_gradient_sum.argtypes = [vp, vp, i64, vp, vp, i32, vp, vp, vp, vp]
     lib.cocodc_outer_step_received.argtypes = [vp, ctypes.POINTER(_Hyper), i32, vp, vp, i64, i64, vp, vp, vp, vp,
                                                vp, vp, vp, i64, i64, vp, vp, vp, vp]
@@ -195,9 +198,21 @@ class Context:
     def launch_count(self) -> int:
         return int(_lib.cocodc_launch_count(self._h))
 
-    def cocodc_fragment_scores(self, delta_g, interval, norms, scores, stream=None) -> None:
+    def cocodc_fragment_scores(self, delta_g, interval, norms, scores, sumsq_out=None, stream=None) -> None:
         _check(_lib.cocodc_fragment_scores(self._h, _p(delta_g), _p(interval), _p(norms), _p(scores),
-                                           _stream(stream)), "cocodc_fragment_scores")
+                                           _p(sumsq_out), _stream(stream)), "cocodc_fragment_scores")
+
+    def cocodc_scores_from_sumsq(self, sumsq, ids, n_ids, interval, t_p: int, t_l: int, last_sync, norms, scores,
+                                 stream=None) -> None:
+        """Eq. 10 from fp64 sums of squares [K]: completion mode with an id list, stand-alone (all K) without."""
+        _check(_lib.cocodc_scores_from_sumsq(self._h, _p(sumsq), _p(ids), _p(n_ids), _p(interval), int(t_p),
+                                             int(t_l), _p(last_sync), _p(norms), _p(scores), _stream(stream)),
+               "cocodc_scores_from_sumsq")
+
+    def cocodc_bind_in_flight(self, in_flight) -> None:
+        """Bind (or, with None, unbind) the caller's device uint8[K] mask of fragments in flight."""
+        self._in_flight = in_flight          # keeps the tensor alive while the context points at it
+        _check(_lib.cocodc_bind_in_flight(self._h, _p(in_flight)), "cocodc_bind_in_flight")
 
     def cocodc_select_fragments(self, scores, last_sync, ineligible, t_now: int, H: int, budget_kind: int,
                                 budget: int, mask, ids, n_sel, pool_offset=None, stream=None) -> None:
@@ -207,12 +222,13 @@ class Context:
 
     def cocodc_outer_step(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                           theta_g, momentum, delta_g_out, ids, n_ids, t_p: int, t_l: int, last_sync,
-                          norms, scores, stages: int = STAGE_ALL, stream=None) -> None:
+                          norms, scores, stages: int = STAGE_ALL, stream=None, sumsq_out=None) -> None:
         h = hyper._c()
         _check(_lib.cocodc_outer_step(self._h, ctypes.byref(h), _p(w_now), _p(w_snap), int(now_stride),
                                       int(snap_stride), _p(snap_offset), _p(theta_g), _p(momentum),
                                       _p(delta_g_out), _p(ids), _p(n_ids), int(t_p), int(t_l), _p(last_sync),
-                                      _p(norms), _p(scores), int(stages), _stream(stream)), "cocodc_outer_step")
+                                      _p(norms), _p(scores), _p(sumsq_out), int(stages), _stream(stream)),
+               "cocodc_outer_step")
 
     def cocodc_outer_step_host(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                                theta_g, momentum, delta_g_out, ids, n_ids: int, t_p: int, t_l: int,
@@ -237,13 +253,14 @@ class Context:
 
     def cocodc_outer_step_at(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                              theta_g, momentum, delta_g_out, ids, n_ids, t_p, t_l, last_sync,
-                             norms, scores, stages: int = STAGE_ALL, stream=None) -> None:
+                             norms, scores, stages: int = STAGE_ALL, stream=None, sumsq_out=None) -> None:
         """As cocodc_outer_step with t_p and t_l device int64[1] tensors."""
         h = hyper._c()
         _check(_lib.cocodc_outer_step_at(self._h, ctypes.byref(h), _p(w_now), _p(w_snap), int(now_stride),
                                          int(snap_stride), _p(snap_offset), _p(theta_g), _p(momentum),
                                          _p(delta_g_out), _p(ids), _p(n_ids), _p(t_p), _p(t_l), _p(last_sync),
-                                         _p(norms), _p(scores), int(stages), _stream(stream)), "cocodc_outer_step_at")
+                                         _p(norms), _p(scores), _p(sumsq_out), int(stages), _stream(stream)),
+               "cocodc_outer_step_at")
 
     def cocodc_pseudo_gradient_sum(self, w_snap, snap_stride: int, snap_offset, theta_g, M: int, sum_out,
                                    ids, n_ids, stream=None) -> None:

@@ -39,6 +39,10 @@ struct cocodc_ctx {
   PlanHeader* d_hdr = nullptr;
   double* d_partial = nullptr;
   int* d_status = nullptr;
+  int* d_ticket = nullptr;                  // arrival counter of the in-kernel score epilogue (zero between launches)
+  unsigned char* in_flight = nullptr;       // caller's in-flight mask (cocodc_bind_in_flight), or nullptr
+  FragTable table{};                        // the fragment table as a kernel argument, when it is small enough
+  bool inline_plan = false;                 // the streaming kernels expand the id list themselves (no k_plan launch)
   long long launches = 0;
   std::vector<std::pair<const void*, int>> occupancy;  // kernel -> resident CTAs per SM
   std::vector<std::pair<const void*, unsigned>> smem_opted_in;   // kernels opted in to large shared memory, with the size
@@ -100,7 +104,7 @@ cocodc_status launch_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_id
 // shared memory, on how many CTAs, over tiles of how many lanes.  Every variant has eight accumulating
 // warps, so the finalize kernel does not depend on the choice; the plan is built for the variant's tile.
 struct Variant {
-  void (*kernel)(const OuterArgs);
+  void (*kernel)(const OuterArgs, const FragTable);
   int threads;
   unsigned smem;
   bool one_cta_per_sm;   // staged kernel: persistent, one CTA per SM; otherwise sized by occupancy
@@ -128,7 +132,7 @@ Variant staged_variant() {
 // More than 48 KB of dynamic shared memory needs a one-time opt-in per kernel and device (the
 // caller has made the context's device current).
 void opt_in_shared_memory(cocodc_ctx* c, const void* kernel, unsigned bytes) {
-  if (bytes <= 40u * 1024u) return;   // static shared memory counts towards the 48 KB a kernel gets without opting in
+  if (bytes <= 32u * 1024u) return;   // static shared memory (about 9 KB: the plan) counts towards the 48 KB a kernel gets without opting in
   for (auto& k : c->smem_opted_in) {
     if (k.first != kernel) continue;
     if (k.second >= bytes) return;
@@ -205,19 +209,40 @@ int variant_grid(cocodc_ctx* c, const Variant& v) {
   return v.one_cta_per_sm ? c->sm_count : grid_for(c, reinterpret_cast<const void*>(v.kernel));
 }
 
-// plan + streaming kernel for a device-resident id list
+// What a launch is to work on, as the kernels take it; with a fragment table too large to be a kernel argument
+// the plan is first written to global memory by k_plan.
+cocodc_status prepare_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_ids, const int64_t* snap_offset,
+                           long long snap_row_len, int lanes_per_tile, cudaStream_t st, PlanRequest* rq,
+                           const SegPlan** gplan, const PlanHeader** ghdr) {
+  rq->ids = ids;
+  rq->n_ids = n_ids;
+  rq->snap_offset = reinterpret_cast<const long long*>(snap_offset);
+  rq->snap_row_len = snap_row_len;
+  rq->lanes_per_tile = lanes_per_tile;
+  rq->err_invalid = (int)COCODC_ERR_INVALID_ARG;
+  if (c->inline_plan) {
+    *gplan = nullptr;
+    *ghdr = nullptr;
+    return COCODC_OK;
+  }
+  *gplan = c->d_plan;
+  *ghdr = c->d_hdr;
+  return launch_plan(c, ids, n_ids, snap_offset, snap_row_len, lanes_per_tile, st);
+}
+
+// (plan +) streaming kernel for a device-resident id list
 cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool same, const int32_t* ids,
-                           const int32_t* n_ids, const int64_t* snap_offset, cudaStream_t st, int* grid_out) {
+                           const int32_t* n_ids, const int64_t* snap_offset, cudaStream_t st) {
   const Variant v = pick_variant(A.M, mode, same, A.n_recv);
   const int grid = variant_grid(c, v);
   opt_in_shared_memory(c, reinterpret_cast<const void*>(v.kernel), v.smem);
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, A.snap_stride, v.lanes_per_tile, st);
-  if (s != COCODC_OK) return s;
   OuterArgs args = A;
+  cocodc_status s = prepare_plan(c, ids, n_ids, snap_offset, A.snap_stride, v.lanes_per_tile, st, &args.rq,
+                                 &args.plan, &args.hdr);
+  if (s != COCODC_OK) return s;
   args.ring_slots = v.ring_slots;
-  v.kernel<<<grid, v.threads, v.smem, st>>>(args);
+  v.kernel<<<grid, v.threads, v.smem, st>>>(args, c->table);
   c->launches++;
-  *grid_out = grid;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
@@ -356,6 +381,7 @@ cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, 
   ok = ok && cudaMalloc(&c->d_hdr, sizeof(PlanHeader)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_partial, sizeof(double) * partial_elems) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_ticket, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_frag_sumsq, sizeof(double) * K) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_k_ids, sizeof(int) * K) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_k_last, sizeof(long long) * K) == cudaSuccess;
@@ -383,7 +409,15 @@ cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, 
     ok = ok && cudaMemcpy(c->d_frag_first_off, first_off.data(), sizeof(long long) * K, cudaMemcpyHostToDevice) == cudaSuccess;
   }
   ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_ticket, 0, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMemset(c->d_hdr, 0, sizeof(PlanHeader)) == cudaSuccess;
+  c->inline_plan = (S <= kInlineSegs);
+  if (c->inline_plan) {
+    c->table.K = K;
+    c->table.n_seg = S;
+    for (int p = 0; p <= K; ++p) c->table.seg_ptr[p] = part->frag_seg_ptr[p];
+    for (int sg = 0; sg < S; ++sg) { c->table.off[sg] = off[sg]; c->table.len[sg] = len[sg]; }
+  }
   if (!ok) { cudaGetLastError(); cocodc_destroy(c); return COCODC_ERR_CUDA; }
   *ctx_out = c;
   return COCODC_OK;
@@ -401,6 +435,7 @@ cocodc_status cocodc_destroy(cocodc_ctx* c) {
   cudaFree(c->d_hdr);
   cudaFree(c->d_partial);
   cudaFree(c->d_status);
+  cudaFree(c->d_ticket);
   cudaFree(c->d_frag_sumsq);
   cudaFree(c->d_k_ids);
   cudaFree(c->d_k_last);
@@ -427,28 +462,60 @@ cocodc_status cocodc_poll_status(cocodc_ctx* c, void* stream) {
   if (cudaMemcpyAsync(&word, c->d_status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return COCODC_ERR_CUDA;
   if (cudaMemsetAsync(c->d_status, 0, sizeof(int), st) != cudaSuccess) return COCODC_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return COCODC_ERR_CUDA;
+  // a launch that gave up on a bounded wait leaves the arrival counter of its score epilogue behind
+  if (word != 0 && cudaMemsetAsync(c->d_ticket, 0, sizeof(int), st) != cudaSuccess) return COCODC_ERR_CUDA;
   return static_cast<cocodc_status>(word);
 }
 
 cocodc_status cocodc_fragment_scores(cocodc_ctx* c, const float* delta_g, const int64_t* interval,
-                                     float* norms, float* scores, void* stream) {
-  if (!c || !delta_g || !norms || !scores) return COCODC_ERR_INVALID_ARG;
+                                     float* norms, float* scores, double* sumsq_out, void* stream) {
+  if (!c || !delta_g) return COCODC_ERR_INVALID_ARG;
+  if ((norms == nullptr) != (scores == nullptr) || (!norms && !sumsq_out)) return COCODC_ERR_INVALID_ARG;
   if (!aligned16(delta_g)) return COCODC_ERR_ALIGNMENT;
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   constexpr int U = 4;
   auto kernel = k_sumsq<U>;
   const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
-  cocodc_status s = launch_plan(c, nullptr, nullptr, nullptr, 0, kThreads * U, st);
+  PlanRequest rq{};
+  const SegPlan* gplan = nullptr;
+  const PlanHeader* ghdr = nullptr;
+  cocodc_status s = prepare_plan(c, nullptr, nullptr, nullptr, 0, kThreads * U, st, &rq, &gplan, &ghdr);
   if (s != COCODC_OK) return s;
-  kernel<<<grid, kThreads, 0, st>>>(delta_g, c->d_plan, c->d_hdr, c->d_partial);
-  c->launches++;
-  k_finalize_scores<<<c->K, kFinalizeThreads, 0, st>>>(
-      c->d_hdr, nullptr, c->d_partial, grid * (kThreads / 32), 1, 0, 0, nullptr, nullptr,
-      reinterpret_cast<const long long*>(interval), nullptr, norms, scores, c->d_status,
-      (int)COCODC_ERR_NONFINITE);
+  Finalize fin{};
+  fin.ticket = c->d_ticket;
+  fin.mode = 1;
+  fin.write_scores = norms ? 1 : 0;
+  fin.interval = reinterpret_cast<const long long*>(interval);
+  fin.norms = norms;
+  fin.scores = scores;
+  fin.sumsq_out = sumsq_out;
+  fin.err_nonfinite = (int)COCODC_ERR_NONFINITE;
+  kernel<<<grid, kThreads, 0, st>>>(delta_g, gplan, ghdr, rq, fin, c->d_partial, c->d_status, c->table);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+cocodc_status cocodc_scores_from_sumsq(cocodc_ctx* c, const double* sumsq, const int32_t* ids, const int32_t* n_ids,
+                                       const int64_t* interval, int64_t t_p, int64_t t_l, int64_t* last_sync,
+                                       float* norms, float* scores, void* stream) {
+  if (!c || !sumsq || !norms || !scores) return COCODC_ERR_INVALID_ARG;
+  const bool completion = (ids != nullptr);
+  if (completion && (!n_ids || !last_sync || interval || t_l < t_p)) return COCODC_ERR_INVALID_ARG;
+  if (!completion && n_ids) return COCODC_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  k_scores_from_sumsq<<<1, kFinalizeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      sumsq, 0, ids, n_ids, 0, c->K, completion ? 0 : 1, reinterpret_cast<const long long*>(interval), t_p, t_l,
+      reinterpret_cast<long long*>(last_sync), norms, scores, completion ? c->in_flight : nullptr, c->d_status,
+      (int)COCODC_ERR_NONFINITE, (int)COCODC_ERR_INVALID_ARG);
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+cocodc_status cocodc_bind_in_flight(cocodc_ctx* c, uint8_t* in_flight) {
+  if (!c) return COCODC_ERR_INVALID_ARG;
+  c->in_flight = in_flight;
+  return COCODC_OK;
 }
 
 }  // extern "C"
@@ -468,7 +535,7 @@ cocodc_status select_impl(cocodc_ctx* c, const float* scores, const int64_t* las
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   k_select<<<1, kSelectThreads, 0, st>>>(c->K, scores, reinterpret_cast<const long long*>(last_sync), ineligible,
                                          c->d_frag_size, c->d_frag_first_off, t_now, reinterpret_cast<const long long*>(t_now_dev), H, budget_kind, budget, mask, ids, n_sel,
-                                         reinterpret_cast<long long*>(pool_offset), c->d_status, (int)COCODC_ERR_NONFINITE,
+                                         reinterpret_cast<long long*>(pool_offset), c->in_flight, c->d_status, (int)COCODC_ERR_NONFINITE,
                                          (int)COCODC_ERR_INVALID_ARG);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
@@ -482,7 +549,7 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
                               float* theta_g, float* momentum, float* delta_g_out,
                               const int32_t* ids, const int32_t* n_ids,
                               int64_t t_p, int64_t t_l, int64_t* last_sync,
-                              float* norms, float* scores, uint32_t stages, void* stream,
+                              float* norms, float* scores, double* sumsq_out, uint32_t stages, void* stream,
                               const float* const* delta_sums, int32_t n_sums, int32_t M_total,
                               const int64_t* t_p_dev = nullptr, const int64_t* t_l_dev = nullptr) {
   cocodc_status s = check_hyper(c, h);
@@ -493,9 +560,11 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
     if (!delta_sums[r]) return COCODC_ERR_INVALID_ARG;
     if (!aligned16(delta_sums[r])) return COCODC_ERR_ALIGNMENT;
   }
-  if (!(stages & COCODC_STAGE_OUTER) || (stages & ~COCODC_STAGE_ALL)) return COCODC_ERR_INVALID_ARG;
+  if (!(stages & COCODC_STAGE_OUTER) || (stages & ~(COCODC_STAGE_ALL | COCODC_STAGE_SUMSQ))) return COCODC_ERR_INVALID_ARG;
   const bool do_merge = (stages & COCODC_STAGE_MERGE) != 0;
   const bool do_score = (stages & COCODC_STAGE_SCORE) != 0;
+  const bool do_sums = do_score || (stages & COCODC_STAGE_SUMSQ) != 0;
+  if ((stages & COCODC_STAGE_SUMSQ) && !sumsq_out) return COCODC_ERR_INVALID_ARG;
   if (!w_snap || !theta_g || !momentum || !ids || !n_ids) return COCODC_ERR_INVALID_ARG;
   if (do_merge && !w_now) return COCODC_ERR_INVALID_ARG;
   if (do_score && (!last_sync || !norms || !scores)) return COCODC_ERR_INVALID_ARG;
@@ -512,23 +581,24 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
   // aliasing: every output range must be disjoint from every other buffer
   {
     const int M = h->M;
-    std::vector<Range> r;
-    r.push_back(range_of(theta_g, N));
-    r.push_back(range_of(momentum, N));
-    if (delta_g_out) r.push_back(range_of(delta_g_out, N));
-    if (do_merge) r.push_back(range_of(w_now, (long long)(M - 1) * now_stride + N));
-    for (size_t i = 0; i < r.size(); ++i)
-      for (size_t j = i + 1; j < r.size(); ++j)
+    Range r[4];
+    int nr = 0;
+    r[nr++] = range_of(theta_g, N);
+    r[nr++] = range_of(momentum, N);
+    if (delta_g_out) r[nr++] = range_of(delta_g_out, N);
+    if (do_merge) r[nr++] = range_of(w_now, (long long)(M - 1) * now_stride + N);
+    for (int i = 0; i < nr; ++i)
+      for (int j = i + 1; j < nr; ++j)
         if (overlap(r[i], r[j])) return COCODC_ERR_ALIAS;
     if (!same) {
       const Range rs = range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N));
-      for (const Range& x : r) if (overlap(rs, x)) return COCODC_ERR_ALIAS;
+      for (int i = 0; i < nr; ++i) if (overlap(rs, r[i])) return COCODC_ERR_ALIAS;
     }
     // delta_g_out may be the same buffer as one of the sums (updated in place), nothing else may
     for (int q = 0; q < n_sums; ++q) {
       const Range rd = range_of(delta_sums[q], N);
-      for (const Range& x : r)
-        if (overlap(rd, x) && !(delta_g_out == delta_sums[q] && x.lo == rd.lo)) return COCODC_ERR_ALIAS;
+      for (int i = 0; i < nr; ++i)
+        if (overlap(rd, r[i]) && !(delta_g_out == delta_sums[q] && r[i].lo == rd.lo)) return COCODC_ERR_ALIAS;
     }
   }
   DeviceGuard guard(c->device);
@@ -543,9 +613,23 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
   A.delta_out = delta_g_out;
   for (int r = 0; r < n_sums; ++r) A.delta_in[r] = delta_sums[r];
   A.n_recv = n_sums;
-  A.plan = c->d_plan;
-  A.hdr = c->d_hdr;
-  A.partial = do_score ? c->d_partial : nullptr;
+  A.partial = do_sums ? c->d_partial : nullptr;
+  if (do_sums) {   // Eq. 10 is formed by the last warp of the same launch
+    A.fin.ticket = c->d_ticket;
+    A.fin.mode = 0;
+    A.fin.write_scores = do_score ? 1 : 0;
+    A.fin.ids = ids;
+    A.fin.t_p = t_p;
+    A.fin.t_l = t_l;
+    A.fin.t_p_dev = reinterpret_cast<const long long*>(t_p_dev);
+    A.fin.t_l_dev = reinterpret_cast<const long long*>(t_l_dev);
+    A.fin.last_sync = reinterpret_cast<long long*>(last_sync);
+    A.fin.norms = norms;
+    A.fin.scores = scores;
+    A.fin.sumsq_out = sumsq_out;
+    A.fin.in_flight = do_score ? c->in_flight : nullptr;
+    A.fin.err_nonfinite = (int)COCODC_ERR_NONFINITE;
+  }
   fold_coefficients(h, same, &A);
   if (received) {   // Eq. 1 divides the received sum by the number of workers that contributed to it
     A.Mf = (float)M_total;
@@ -553,19 +637,8 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
     A.M_pow2 = ((M_total & (M_total - 1)) == 0) ? 1 : 0;
   }
   set_status_sink(c, &A);
-  int grid = 0;
   const int mode = received ? MODE_FUSED_RECV : (do_merge ? MODE_FUSED : MODE_OUTER_ONLY);
-  s = launch_outer(c, A, mode, same, ids, n_ids, snap_offset, st, &grid);
-  if (s != COCODC_OK) return s;
-  if (do_score) {
-    k_finalize_scores<<<c->K, kFinalizeThreads, 0, st>>>(
-        c->d_hdr, ids, c->d_partial, grid * (kThreads / 32), 0, t_p, t_l,
-        reinterpret_cast<const long long*>(t_p_dev), reinterpret_cast<const long long*>(t_l_dev), nullptr,
-        reinterpret_cast<long long*>(last_sync), norms, scores, c->d_status, (int)COCODC_ERR_NONFINITE);
-    c->launches++;
-    if (cudaGetLastError() != cudaSuccess) return COCODC_ERR_CUDA;
-  }
-  return COCODC_OK;
+  return launch_outer(c, A, mode, same, ids, n_ids, snap_offset, st);
 }
 
 }  // namespace
@@ -578,9 +651,9 @@ cocodc_status cocodc_outer_step(cocodc_ctx* c, const cocodc_hyper* h,
                                 float* theta_g, float* momentum, float* delta_g_out,
                                 const int32_t* ids, const int32_t* n_ids,
                                 int64_t t_p, int64_t t_l, int64_t* last_sync,
-                                float* norms, float* scores, uint32_t stages, void* stream) {
+                                float* norms, float* scores, double* sumsq_out, uint32_t stages, void* stream) {
   return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
-                         ids, n_ids, t_p, t_l, last_sync, norms, scores, stages, stream, nullptr, 0, 0);
+                         ids, n_ids, t_p, t_l, last_sync, norms, scores, sumsq_out, stages, stream, nullptr, 0, 0);
 }
 
 cocodc_status cocodc_outer_step_received(cocodc_ctx* c, const cocodc_hyper* h, int32_t M_total,
@@ -592,7 +665,8 @@ cocodc_status cocodc_outer_step_received(cocodc_ctx* c, const cocodc_hyper* h, i
                                          float* norms, float* scores, void* stream) {
   if (!delta_sum) return COCODC_ERR_INVALID_ARG;
   return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
-                         ids, n_ids, t_p, t_l, last_sync, norms, scores, COCODC_STAGE_ALL, stream, &delta_sum, 1, M_total);
+                         ids, n_ids, t_p, t_l, last_sync, norms, scores, nullptr, COCODC_STAGE_ALL, stream, &delta_sum, 1,
+                         M_total);
 }
 
 cocodc_status cocodc_outer_step_received_peers(cocodc_ctx* c, const cocodc_hyper* h, int32_t M_total,
@@ -605,8 +679,8 @@ cocodc_status cocodc_outer_step_received_peers(cocodc_ctx* c, const cocodc_hyper
                                                float* norms, float* scores, void* stream) {
   if (!delta_sums || n_sums < 1) return COCODC_ERR_INVALID_ARG;
   return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
-                         ids, n_ids, t_p, t_l, last_sync, norms, scores, COCODC_STAGE_ALL, stream, delta_sums, n_sums,
-                         M_total);
+                         ids, n_ids, t_p, t_l, last_sync, norms, scores, nullptr, COCODC_STAGE_ALL, stream, delta_sums,
+                         n_sums, M_total);
 }
 
 cocodc_status cocodc_select_fragments(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
@@ -634,10 +708,11 @@ cocodc_status cocodc_outer_step_at(cocodc_ctx* c, const cocodc_hyper* h,
                                    float* theta_g, float* momentum, float* delta_g_out,
                                    const int32_t* ids, const int32_t* n_ids,
                                    const int64_t* t_p, const int64_t* t_l, int64_t* last_sync,
-                                   float* norms, float* scores, uint32_t stages, void* stream) {
+                                   float* norms, float* scores, double* sumsq_out, uint32_t stages, void* stream) {
   if (!t_p || !t_l) return COCODC_ERR_INVALID_ARG;
   return outer_step_impl(c, h, w_now, w_snap, now_stride, snap_stride, snap_offset, theta_g, momentum, delta_g_out,
-                         ids, n_ids, 0, 0, last_sync, norms, scores, stages, stream, nullptr, 0, 0, t_p, t_l);
+                         ids, n_ids, 0, 0, last_sync, norms, scores, sumsq_out, stages, stream, nullptr, 0, 0, t_p,
+                         t_l);
 }
 
 cocodc_status cocodc_pseudo_gradient_sum(cocodc_ctx* c, const float* w_snap, int64_t snap_stride,
@@ -658,11 +733,10 @@ cocodc_status cocodc_pseudo_gradient_sum(cocodc_ctx* c, const float* w_snap, int
   A.w_snap = w_snap; A.snap_stride = snap_stride; A.now_stride = N;
   A.theta_g = const_cast<float*>(theta_g);   // read only in this mode
   A.delta_out = sum_out;
-  A.plan = c->d_plan; A.hdr = c->d_hdr; A.partial = nullptr;
+  A.partial = nullptr;
   A.status = c->d_status; A.err_timeout = COCODC_ERR_TIMEOUT;
   A.M = M;
-  int grid = 0;
-  return launch_outer(c, A, MODE_PSEUDO_SUM, false, ids, n_ids, snap_offset, st, &grid);
+  return launch_outer(c, A, MODE_PSEUDO_SUM, false, ids, n_ids, snap_offset, st);
 }
 
 cocodc_status cocodc_merge(cocodc_ctx* c, const cocodc_hyper* h,
@@ -693,12 +767,9 @@ cocodc_status cocodc_merge(cocodc_ctx* c, const cocodc_hyper* h,
   A.now_stride = now_stride;
   A.snap_stride = snap_stride;
   A.theta_g = const_cast<float*>(theta_g_new);  // read only in this mode
-  A.plan = c->d_plan;
-  A.hdr = c->d_hdr;
   fold_coefficients(h, same, &A);
   set_status_sink(c, &A);
-  int grid = 0;
-  return launch_outer(c, A, MODE_MERGE_ONLY, same, ids, n_ids, snap_offset, st, &grid);
+  return launch_outer(c, A, MODE_MERGE_ONLY, same, ids, n_ids, snap_offset, st);
 }
 
 cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
@@ -715,10 +786,13 @@ cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   opt_in_shared_memory(c, reinterpret_cast<const void*>(k_snapshot_tma), kSnapSmemBytes);
-  cocodc_status s = launch_plan(c, ids, n_ids, snap_offset, snap_stride, kThreads * kSnapU, st);
+  PlanRequest rq{};
+  const SegPlan* gplan = nullptr;
+  const PlanHeader* ghdr = nullptr;
+  cocodc_status s = prepare_plan(c, ids, n_ids, snap_offset, snap_stride, kThreads * kSnapU, st, &rq, &gplan, &ghdr);
   if (s != COCODC_OK) return s;
-  k_snapshot_tma<<<c->sm_count, kThreads, kSnapSmemBytes, st>>>(w_now, w_snap, now_stride, snap_stride, M, c->d_plan,
-                                                                c->d_hdr, c->d_status, (int)COCODC_ERR_TIMEOUT);
+  k_snapshot_tma<<<c->sm_count, kThreads, kSnapSmemBytes, st>>>(w_now, w_snap, now_stride, snap_stride, M, gplan, ghdr,
+                                                                rq, c->d_status, (int)COCODC_ERR_TIMEOUT, c->table);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
@@ -744,7 +818,7 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
   if (!aligned16(workspace)) return COCODC_ERR_ALIGNMENT;
   if (snap_on_device && (!aligned16(w_snap) || (snap_stride & 3))) return COCODC_ERR_ALIGNMENT;
   {
-    std::vector<char> seen(K, 0);
+    char seen[kMaxK] = {};
     for (int j = 0; j < n_ids; ++j) {
       const int p = ids[j];
       if (p < 0 || p >= K || seen[p]) return COCODC_ERR_INVALID_ARG;
@@ -752,17 +826,18 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
         return COCODC_ERR_INVALID_ARG;   // no place, or not inside one row of the pool
       seen[p] = 1;
     }
-    std::vector<Range> r;
-    r.push_back(range_of(theta_g, N));
-    r.push_back(range_of(momentum, N));
-    if (delta_g_out) r.push_back(range_of(delta_g_out, N));
-    r.push_back(range_of(w_now, (long long)(M - 1) * now_stride + N));
-    for (size_t i = 0; i < r.size(); ++i)
-      for (size_t j = i + 1; j < r.size(); ++j)
+    Range r[4];
+    int nr = 0;
+    r[nr++] = range_of(theta_g, N);
+    r[nr++] = range_of(momentum, N);
+    if (delta_g_out) r[nr++] = range_of(delta_g_out, N);
+    r[nr++] = range_of(w_now, (long long)(M - 1) * now_stride + N);
+    for (int i = 0; i < nr; ++i)
+      for (int j = i + 1; j < nr; ++j)
         if (overlap(r[i], r[j])) return COCODC_ERR_ALIAS;
     if (!same && !snap_on_device) {
       const Range rs = range_of(w_snap, (long long)(M - 1) * snap_stride + (snap_offset ? snap_stride : N));
-      for (const Range& x : r) if (overlap(rs, x)) return COCODC_ERR_ALIAS;
+      for (int i = 0; i < nr; ++i) if (overlap(rs, r[i])) return COCODC_ERR_ALIAS;
     }
   }
   // staging slots: [snap M][now M][theta_g][momentum][delta] chunks of C elements each
@@ -833,7 +908,7 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
         A.delta_out = delta_g_out ? d_delta : nullptr;
         A.ring_slots = v.ring_slots;
         k_plan_chunk<<<1, 1, 0, st>>>(cnt, snap_on_device ? sbase + lo : 0, v.lanes_per_tile, c->d_plan, c->d_hdr);
-        v.kernel<<<grid, v.threads, v.smem, st>>>(A);
+        v.kernel<<<grid, v.threads, v.smem, st>>>(A, c->table);
         k_accumulate_chunk<<<1, kFinalizeThreads, 0, st>>>(c->d_partial, entries, c->d_frag_sumsq + j);
         c->launches += 3;
         CK(cudaEventRecord(c->ev_comp[slot], st));
@@ -852,9 +927,10 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
     }
   }
   if (ok && n_ids > 0) {
-    k_finalize_from_sums<<<1, kFinalizeThreads, 0, st>>>(c->d_frag_sumsq, c->d_k_ids, n_ids, t_p, t_l, c->d_k_last,
-                                                         c->d_k_norms, c->d_k_scores, c->d_status,
-                                                         (int)COCODC_ERR_NONFINITE);
+    k_scores_from_sumsq<<<1, kFinalizeThreads, 0, st>>>(c->d_frag_sumsq, 1, c->d_k_ids, nullptr, n_ids, K, 0, nullptr,
+                                                        t_p, t_l, c->d_k_last, c->d_k_norms, c->d_k_scores, nullptr,
+                                                        c->d_status, (int)COCODC_ERR_NONFINITE,
+                                                        (int)COCODC_ERR_INVALID_ARG);
     c->launches++;
   }
   CK(cudaMemcpyAsync(last_sync, c->d_k_last, sizeof(long long) * K, cudaMemcpyDeviceToHost, st));

@@ -38,8 +38,10 @@ struct OuterArgs {
   float* delta_out;         // optional
   const float* delta_in[kMaxRecv];   // MODE_FUSED_RECV: sums of pseudo-gradients, one buffer per contributing device
   int n_recv;               // how many of them (added in this order, so every device that lists them alike gets the same bits)
-  const SegPlan* plan;
-  const PlanHeader* hdr;
+  const SegPlan* plan;      // plan in global memory (written by k_plan / k_plan_chunk), or nullptr: every CTA
+  const PlanHeader* hdr;    //   expands `rq` itself in its prologue
+  PlanRequest rq;
+  Finalize fin;             // what the last warp does with the sums of squares (fin.ticket == nullptr: nothing)
   double* partial;          // nullptr: no score accumulation
   int* status;              // device status word
   int err_timeout;          // code recorded when a bounded wait runs out
@@ -270,7 +272,7 @@ struct Lane {
 // A full lane whose recorded values sit at a place that is not 16-byte compatible.  Kept out of line: inlined
 // into the staged kernels it cost their main loop 1.5 % of bandwidth (6.71 -> 6.61 TB/s on the 1B shape).
 template <int M, int MODE, bool SAME>
-__device__ __noinline__ double shifted_lane(const OuterArgs A, long long e, long long snap_e) {   // A by value: its address must not escape the caller
+__device__ __noinline__ double shifted_lane(const OuterArgs& A, long long e, long long snap_e) {
   Lane<M, MODE, SAME> L;
   double sumsq = 0.0;       // this lane's contribution to the sum of squares
   L.load_shifted(A, e, snap_e);
@@ -311,6 +313,18 @@ __device__ __forceinline__ void ragged_lane(const OuterArgs& A, const SegPlan& s
   if (mode_updates_global(MODE)) acc += (double)sq;
 }
 
+// A whole ragged tile of one thread (U lanes, kThreads lanes apart), out of line: these tiles are the exception
+// (segment edges, pool places that are not 16-byte compatible), and kept inline their code sat in the middle of
+// the staged kernels' main loop.  The segment entry travels by value so that the caller's copy stays in
+// registers.  Returns the thread's contribution to the sum of squares.
+template <int M, int MODE, bool SAME, int U>
+__device__ __noinline__ double ragged_tile(const OuterArgs& A, const SegPlan sp, long long e_first) {
+  double acc = 0.0;
+#pragma unroll
+  for (int v = 0; v < U; ++v) ragged_lane<M, MODE, SAME>(A, sp, e_first + 4LL * (v * kThreads), acc);
+  return acc;
+}
+
 // Walks the tiles of one CTA (tile = blockIdx.x + i*gridDim.x) and keeps the segment they fall in.
 struct TileWalker {
   const SegPlan* plan;
@@ -343,25 +357,34 @@ struct TileWalker {
 // the second pass over the recorded values hits in cache).
 template <int MODE, bool SAME>
 __global__ void __launch_bounds__(kThreads)
-k_outer_generic(const OuterArgs A) {
-  const PlanHeader h = *A.hdr;
+k_outer_generic(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTable T) {
+  __shared__ InlinePlan ip;
+  const PlanView pv = acquire_plan(ip, T, A.rq, A.plan, A.hdr, A.status);
+  const PlanHeader h = pv.hdr;
   SlotAccumulator sa(kThreads / 32);
-  TileWalker tw(A.plan, h.n_seg);
+  TileWalker tw(pv.seg, h.n_seg);
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
     if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
     ragged_lane<0, MODE, SAME>(A, tw.sp, tw.tile_start(tile) + 4LL * threadIdx.x, sa.acc);
   }
-  if (A.partial) sa.finish(h.n_ids, A.partial);
+  if (A.partial) {
+    sa.finish(h.n_ids, A.partial);
+    finalize_epilogue_cta(ip, A.fin, h, A.partial, kThreads / 32, A.status);
+  }
 }
 
 // ---------------------------------------------------------------------------
 // S6 stand-alone: sums of squares of an N-sized vector over the planned tiles.
 // ---------------------------------------------------------------------------
 template <int U>
-__global__ void __launch_bounds__(kThreads)
-k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ plan,
-        const PlanHeader* __restrict__ hdr, double* __restrict__ partial) {
-  const PlanHeader h = *hdr;
+__global__ void __launch_bounds__(kThreads, 8)     // 8 CTAs per SM: the loop needs few registers, the prologue may spill
+k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ gplan, const PlanHeader* __restrict__ ghdr,
+        const __grid_constant__ PlanRequest rq, const __grid_constant__ Finalize fin,
+        double* __restrict__ partial, int* __restrict__ status, const __grid_constant__ FragTable T) {
+  __shared__ InlinePlan ip;
+  const PlanView pv = acquire_plan(ip, T, rq, gplan, ghdr, status);
+  const PlanHeader h = pv.hdr;
+  const SegPlan* plan = pv.seg;
   constexpr int LPT = kThreads * U;
   SlotAccumulator sa(kThreads / 32);
   int seg = 0, seg_loaded = -1;
@@ -395,6 +418,7 @@ k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ plan,
     }
   }
   sa.finish(h.n_ids, partial);
+  finalize_epilogue_cta(ip, fin, h, partial, kThreads / 32, status);
 }
 
 }  // namespace cocodc

@@ -49,7 +49,7 @@ __host__ __device__ constexpr int ring_chunks_for(int mode, int M) {
 
 template <int MODE, bool SAME>
 __global__ void __launch_bounds__(kRingThreads, 1)
-k_outer_ring(const OuterArgs A) {
+k_outer_ring(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTable T) {
   static_assert(SAME ? (MODE == MODE_FUSED || MODE == MODE_MERGE_ONLY) : true, "zero delay needs the merge");
   constexpr bool kUpdates = mode_updates_global(MODE);
   constexpr bool kMerges = mode_merges(MODE);
@@ -64,12 +64,14 @@ k_outer_ring(const OuterArgs A) {
   __shared__ __align__(8) unsigned long long full_bar[kRingMaxChunks];
   __shared__ __align__(8) unsigned long long empty_bar[kRingMaxChunks];
   __shared__ volatile int s_fail;
+  __shared__ InlinePlan ip;
   const int tid = threadIdx.x;
   const int M = A.M;
   const unsigned R = (unsigned)A.ring_slots;            // chunks in the ring
   const int n_recv = kRecv ? A.n_recv : 0;
   const int n_head = 1 + (kUpdates ? 1 : 0) + n_recv;   // streams of the head
-  const PlanHeader h = *A.hdr;
+  const PlanView pv = acquire_plan(ip, T, A.rq, A.plan, A.hdr, A.status);
+  const PlanHeader h = pv.hdr;
   if (tid == 0) {
     for (unsigned s = 0; s < R; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
@@ -86,7 +88,7 @@ k_outer_ring(const OuterArgs A) {
   if (tid >= kThreads) {
     if ((tid & 31) != 0) return;
     const unsigned me = (unsigned)(tid - kThreads) >> 5;
-    TileWalker tw(A.plan, h.n_seg);
+    TileWalker tw(pv.seg, h.n_seg);
     unsigned s = 0, lap = 0;   // next chunk of the ring, and how often the ring has been filled
     unsigned turn = 0;         // whose chunk the next one is
     bool ok = true;
@@ -157,7 +159,7 @@ k_outer_ring(const OuterArgs A) {
 
   // ------------------------------------------------------------------ consumers
   SlotAccumulator sa(kThreads / 32);
-  TileWalker tw(A.plan, h.n_seg);
+  TileWalker tw(pv.seg, h.n_seg);
   unsigned cs = 0, cphase = 0;   // next chunk to take and the phase of its "full" barrier
   bool failed = false;
   // waits for the next chunk; the verdict is the warp's
@@ -292,7 +294,10 @@ k_outer_ring(const OuterArgs A) {
     }
   }
   if (failed) return;     // warp-uniform by construction
-  if (A.partial) sa.finish(h.n_ids, A.partial);
+  if (A.partial) {
+    sa.finish(h.n_ids, A.partial);
+    finalize_epilogue(ip, A.fin, h, A.partial, kThreads / 32, A.status);
+  }
 }
 
 }  // namespace cocodc

@@ -25,11 +25,8 @@
 
 namespace cocodc {
 
-// Producer warps of k_outer_tma (one issuing thread each).  One thread starts a 4 KB copy every few hundred
-// cycles; from seven workers on (16 and more copies per tile) a second one shares the streams (measured: +0.5 %
-// at M = 7, +1.6 % at M = 8, nothing at M = 4 and 6, -1 % at M = 5).
-__host__ __device__ constexpr int tma_producers(int M) { return M >= 7 ? 2 : 1; }
-__host__ __device__ constexpr int tma_threads(int M) { return kThreads + 32 * tma_producers(M); }
+// k_outer_tma runs eight consumer warps and one producer warp, whose lanes each issue one stream's copies.
+__host__ __device__ constexpr int tma_threads(int /*M*/) { return kThreads + 32; }
 constexpr int kTmaThreads = kThreads + 32;      // kernels with a single producer warp
 constexpr unsigned kTileBytes = kTileElems * sizeof(float);   // one stream's share of a stage
 constexpr int kWaitLimit = 1 << 22;                           // polls of a barrier before giving up
@@ -134,11 +131,12 @@ struct StageLayout {
   static_assert(SAME ? (MODE == MODE_FUSED || MODE == MODE_MERGE_ONLY) : true,
                 "zero-delay mode needs the merge and local pseudo-gradients");
   static_assert(U == 1 || MODE != MODE_FUSED_RECV, "the received-sum mode sizes its stages at run time for U = 1");
+  static_assert(kLoaded + (MODE == MODE_FUSED_RECV ? kMaxRecv : 0) <= 32, "one lane of the producer warp per stream");
 };
 
 template <int M, int MODE, bool SAME, int U = 1>
 __global__ void __launch_bounds__(tma_threads(M), 1)
-k_outer_tma(const OuterArgs A) {
+k_outer_tma(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTable T) {
   using L = StageLayout<M, MODE, SAME, U>;
   constexpr int kSlot = U * kTileElems;                         // elements of one stream in a stage
   constexpr unsigned kSlotBytes = U * kTileBytes;
@@ -151,9 +149,11 @@ k_outer_tma(const OuterArgs A) {
   __shared__ __align__(8) unsigned long long full_bar[kMaxStages];
   __shared__ __align__(8) unsigned long long empty_bar[kMaxStages];
   __shared__ volatile int s_fail;
+  __shared__ InlinePlan ip;
 
   const int tid = threadIdx.x;
-  const PlanHeader h = *A.hdr;
+  const PlanView pv = acquire_plan(ip, T, A.rq, A.plan, A.hdr, A.status);
+  const PlanHeader h = pv.hdr;
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
@@ -164,48 +164,52 @@ k_outer_tma(const OuterArgs A) {
   }
   __syncthreads();
 
-  // ------------------------------------------------------------------ producer(s)
-  // With two producers the streams of a stage are dealt out in turn; both wait for the stage to be free,
-  // the first arms the barrier with the whole byte count (a copy of the other that completes before that only
-  // runs the count negative for a moment: the phase cannot end before the arming arrival).
+  // ------------------------------------------------------------------ producer warp
+  // Lane l of the producer warp owns stream l of the stage (slot order: recorded values, current values, global
+  // state, momentum, received sums): it keeps that stream's base pointer in registers and issues the stream's
+  // one bulk copy per tile.  The lanes' copies leave with one warp instruction instead of one instruction
+  // sequence per stream (a single issuing thread needed a few hundred cycles per copy, and with only two or
+  // three stages the time from "stage free" to "last copy issued" sits on the pipeline's critical path).  Lane 0
+  // arms the barrier with the whole byte count; a copy that completes before the arming arrival only runs the
+  // transaction count negative for a moment, the phase cannot end before that arrival.
   if (tid >= kThreads) {
-    if ((tid & 31) != 0) return;
-    constexpr int P = tma_producers(M);
-    const int me = (tid - kThreads) >> 5;
-    int turn = 0;
-    auto mine = [&]() -> bool {
-      if (P == 1) return true;
-      const bool yes = (turn == me);
-      turn = (turn + 1 == P) ? 0 : turn + 1;
-      return yes;
-    };
-    TileWalker tw(A.plan, h.n_seg, kSlot);
+    const int lane = tid & 31;
+    const bool has_stream = lane < loaded;
+    const bool from_snap = lane < L::nS;
+    const float* base = nullptr;
+    if (has_stream) {
+      if (lane < L::nS) base = A.w_snap + (long long)lane * A.snap_stride;
+      else if (lane < L::nS + L::nN) base = A.w_now + (long long)(lane - L::nS) * A.now_stride;
+      else if (lane == L::kGlobal) base = A.theta_g;
+      else if (L::nU && lane == L::kMomentum) base = A.momentum;
+      else base = A.delta_in[lane - L::kDeltaIn];
+    }
+    TileWalker tw(pv.seg, h.n_seg, kSlot);
     int k = 0;   // staged tiles issued so far
+    // Leaving early (a wait ran out here or in a consumer): the copies already issued may still be landing in
+    // this CTA's shared memory, which must not be handed to another CTA before they have; wait for the stages
+    // armed last, again with a limit.
+    auto drain = [&]() {
+      for (int i = (k > S ? k - S : 0); i < k; ++i) mbar_wait_bounded(smem_u32(&full_bar[i % S]), (i / S) & 1);
+    };
     for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
       tw.seek(tile);
       const long long e0 = tw.tile_start(tile);
       if (!tw.interior(e0)) continue;
       const int s = k % S;
-      if (k >= S && !mbar_wait_bounded(smem_u32(&empty_bar[s]), ((k / S) - 1) & 1)) {
-        record_status(A.status, A.err_timeout);
+      const bool free_now = (k < S) || mbar_wait_bounded(smem_u32(&empty_bar[s]), ((k / S) - 1) & 1);
+      if (!__all_sync(0xffffffffu, free_now && !s_fail)) {      // one verdict for the warp
+        if (!free_now) record_status(A.status, A.err_timeout);
         s_fail = 1;
+        drain();
         return;
       }
-      if (s_fail) return;
       const unsigned bar = smem_u32(&full_bar[s]);
-      float* st = stages + (size_t)s * loaded * kSlot;
-      const long long snap_e0 = e0 + (tw.sp.snap_off - tw.sp.off);
-      if (me == 0) mbar_expect_tx(bar, loaded * kSlotBytes);
-#pragma unroll
-      for (int m = 0; m < L::nS; ++m)
-        if (mine()) bulk_load(smem_u32(st + (L::kSnap + m) * kSlot), A.w_snap + m * A.snap_stride + snap_e0, kSlotBytes, bar);
-#pragma unroll
-      for (int m = 0; m < L::nN; ++m)
-        if (mine()) bulk_load(smem_u32(st + (L::kNow + m) * kSlot), A.w_now + m * A.now_stride + e0, kSlotBytes, bar);
-      if (mine()) bulk_load(smem_u32(st + L::kGlobal * kSlot), A.theta_g + e0, kSlotBytes, bar);
-      if (L::nU && mine()) bulk_load(smem_u32(st + L::kMomentum * kSlot), A.momentum + e0, kSlotBytes, bar);
-      for (int r = 0; r < n_recv; ++r)
-        if (mine()) bulk_load(smem_u32(st + (L::kDeltaIn + r) * kSlot), A.delta_in[r] + e0, kSlotBytes, bar);
+      if (lane == 0) mbar_expect_tx(bar, loaded * kSlotBytes);
+      if (has_stream) {
+        const long long e_src = from_snap ? e0 + (tw.sp.snap_off - tw.sp.off) : e0;
+        bulk_load(smem_u32(stages + ((size_t)s * loaded + lane) * kSlot), base + e_src, kSlotBytes, bar);
+      }
       ++k;
     }
     return;
@@ -213,15 +217,14 @@ k_outer_tma(const OuterArgs A) {
 
   // ------------------------------------------------------------------ consumers
   SlotAccumulator sa(kThreads / 32);
-  TileWalker tw(A.plan, h.n_seg, kSlot);
+  TileWalker tw(pv.seg, h.n_seg, kSlot);
   int k = 0;           // staged tiles consumed so far
   bool failed = false;
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
     if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
     const long long e0 = tw.tile_start(tile);
     if (!tw.interior(e0)) {
-#pragma unroll
-      for (int v = 0; v < U; ++v) ragged_lane<M, MODE, SAME>(A, tw.sp, e0 + 4LL * (v * kThreads + tid), sa.acc);
+      sa.acc += ragged_tile<M, MODE, SAME, U>(A, tw.sp, e0 + 4LL * tid);
       continue;
     }
     const int s = k % S;
@@ -268,7 +271,10 @@ k_outer_tma(const OuterArgs A) {
     ++k;
   }
   if (failed) return;     // warp-uniform by construction
-  if (A.partial) sa.finish(h.n_ids, A.partial);
+  if (A.partial) {
+    sa.finish(h.n_ids, A.partial);
+    finalize_epilogue(ip, A.fin, h, A.partial, kThreads / 32, A.status);
+  }
 }
 
 }  // namespace cocodc
@@ -297,13 +303,17 @@ template <int N> __device__ __forceinline__ void bulk_wait_read_n() {
 
 __global__ void __launch_bounds__(kThreads, 1)
 k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long long now_stride,
-               long long snap_stride, int M, const SegPlan* __restrict__ plan,
-               const PlanHeader* __restrict__ hdr, int* __restrict__ status, int err_timeout) {
+               long long snap_stride, int M, const SegPlan* __restrict__ gplan,
+               const PlanHeader* __restrict__ ghdr, const __grid_constant__ PlanRequest rq,
+               int* __restrict__ status, int err_timeout, const __grid_constant__ FragTable T) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   float* const stages = reinterpret_cast<float*>(smem_raw);
   __shared__ __align__(8) unsigned long long full_bar[kSnapStages];
   __shared__ float* dst_of_stage[kSnapStages];
-  const PlanHeader h = *hdr;
+  __shared__ InlinePlan ip;
+  const PlanView pv = acquire_plan(ip, T, rq, gplan, ghdr, status);
+  const PlanHeader h = pv.hdr;
+  const SegPlan* plan = pv.seg;
   const int tid = threadIdx.x;
   if (tid == 0) {
     for (int s = 0; s < kSnapStages; ++s) mbar_init(smem_u32(&full_bar[s]), 1);
@@ -459,7 +469,7 @@ struct InplaceLayout {
 
 template <int M>
 __global__ void __launch_bounds__(kInplaceThreads, 1)
-k_outer_inplace(const OuterArgs A) {
+k_outer_inplace(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTable T) {
   using IL = InplaceLayout<M>;
   using L = typename IL::L;
   constexpr int S = IL::kStages;
@@ -469,8 +479,10 @@ k_outer_inplace(const OuterArgs A) {
   __shared__ __align__(8) unsigned long long done_bar[S];
   __shared__ __align__(8) unsigned long long empty_bar[S];
   __shared__ volatile int s_fail;
+  __shared__ InlinePlan ip;
   const int tid = threadIdx.x;
-  const PlanHeader h = *A.hdr;
+  const PlanView pv = acquire_plan(ip, T, A.rq, A.plan, A.hdr, A.status);
+  const PlanHeader h = pv.hdr;
   if (tid == 0) {
     for (int s = 0; s < S; ++s) {
       mbar_init(smem_u32(&full_bar[s]), 1);
@@ -484,7 +496,7 @@ k_outer_inplace(const OuterArgs A) {
 
   // ------------------------------------------------------------------ loader
   if (tid == kThreads) {
-    TileWalker tw(A.plan, h.n_seg);
+    TileWalker tw(pv.seg, h.n_seg);
     int k = 0;   // staged tiles issued so far
     for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
       tw.seek(tile);
@@ -494,6 +506,8 @@ k_outer_inplace(const OuterArgs A) {
       if (k >= S && (s_fail || !mbar_wait_bounded(smem_u32(&empty_bar[s]), ((k / S) - 1) & 1))) {
         record_status(A.status, A.err_timeout);
         s_fail = 1;
+        // the loads already issued must land before this CTA's shared memory can go to another one
+        for (int i = (k > S ? k - S : 0); i < k; ++i) mbar_wait_bounded(smem_u32(&full_bar[i % S]), (i / S) & 1);
         return;
       }
       const unsigned bar = smem_u32(&full_bar[s]);
@@ -510,7 +524,7 @@ k_outer_inplace(const OuterArgs A) {
   }
   // ------------------------------------------------------------------ storer
   if (tid == kThreads + 32) {
-    TileWalker tw(A.plan, h.n_seg);
+    TileWalker tw(pv.seg, h.n_seg);
     const unsigned long long policy = l2_evict_first_policy();
     int k = 0;   // staged tiles stored so far
     for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
@@ -541,14 +555,14 @@ k_outer_inplace(const OuterArgs A) {
 
   // ------------------------------------------------------------------ consumers
   SlotAccumulator sa(kThreads / 32);
-  TileWalker tw(A.plan, h.n_seg);
+  TileWalker tw(pv.seg, h.n_seg);
   int k = 0;
   bool failed = false;
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
     if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
     const long long e0 = tw.tile_start(tile);
     if (!tw.interior(e0)) {
-      ragged_lane<M, MODE_FUSED, true>(A, tw.sp, e0 + 4LL * tid, sa.acc);
+      sa.acc += ragged_tile<M, MODE_FUSED, true, 1>(A, tw.sp, e0 + 4LL * tid);
       continue;
     }
     const int s = k % S;
@@ -577,7 +591,10 @@ k_outer_inplace(const OuterArgs A) {
     ++k;
   }
   if (failed) return;     // warp-uniform by construction
-  if (A.partial) sa.finish(h.n_ids, A.partial);
+  if (A.partial) {
+    sa.finish(h.n_ids, A.partial);
+    finalize_epilogue(ip, A.fin, h, A.partial, kThreads / 32, A.status);
+  }
 }
 
 // ---------------------------------------------------------------------------------------------

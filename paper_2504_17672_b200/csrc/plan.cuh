@@ -1,10 +1,19 @@
 // Launch plan: which tiles of which segments one call processes.
 //
 // A call works on a list of fragment ids that lives in device memory (it is
-// usually written by the selection kernel, and the host never reads it).  A
-// one-block kernel expands that list into a table of segments with a running
-// tile count; the streaming kernels then map a tile index to (segment, lane
-// range) without any host round-trip.
+// usually written by the selection kernel, and the host never reads it).  The
+// list is expanded into a table of segments with a running tile count, from
+// which the streaming kernels map a tile index to (segment, lane range) without
+// any host round-trip.  Two ways to get that table:
+//   - fragment tables of up to kInlineSegs segments travel as a kernel argument
+//     (FragTable) and every CTA of the streaming kernel expands the id list
+//     itself, into shared memory, in its prologue (acquire_plan): one launch
+//     per call, and the only dependent global loads are n_ids -> ids[j] ->
+//     snap_offset[ids[j]];
+//   - larger tables stay in device memory and a one-block kernel (k_plan)
+//     writes the plan to global memory before the streaming kernel runs.
+// The per-fragment norms and scores are likewise formed by the streaming kernel
+// itself: the last warp to finish adds up the partial sums (finalize_epilogue).
 //
 // Geometry.  Every segment [off, off+len) is covered by 16-byte "lanes" of four
 // elements that start at abase = off rounded down to a multiple of 4, so lane
@@ -34,6 +43,45 @@ struct PlanHeader {
   int n_seg;
   int n_ids;
   int pad;
+};
+
+// Fragment table small enough to be a kernel argument (CSR over segments, as cocodc_partition).
+constexpr int kInlineSegs = 128;
+struct FragTable {
+  int K;
+  int n_seg;
+  int seg_ptr[kInlineSegs + 1];
+  int pad;
+  long long off[kInlineSegs];
+  long long len[kInlineSegs];
+};
+
+// What a launch is to work on.
+struct PlanRequest {
+  const int* ids;                // device id list; nullptr: all K fragments in index order
+  const int* n_ids;              // device, its length
+  const long long* snap_offset;  // device [K] places in a packed snapshot pool, or nullptr
+  long long snap_row_len;        // elements of one row of that pool
+  int lanes_per_tile;
+  int err_invalid;               // status code for a bad id list
+};
+
+// What the last warp of a launch does with the fragments' sums of squares (Eq. 10).
+struct Finalize {
+  int* ticket;                   // device counter, zero between launches; nullptr: no epilogue
+  int mode;                      // 0 completion: I_p = t_p - last_sync[p], last_sync[p] = t_l; 1 stand-alone: I_p = interval[p] or 1
+  int write_scores;              // 0: only sumsq_out is written
+  const int* ids;                // the id list (nullptr: fragment j is list position j)
+  long long t_p, t_l;
+  const long long* t_p_dev;      // step numbers kept in device memory take precedence (graph replay)
+  const long long* t_l_dev;
+  const long long* interval;
+  long long* last_sync;
+  float* norms;
+  float* scores;
+  double* sumsq_out;             // [K] per-fragment sums of squares before the square root, or nullptr
+  unsigned char* in_flight;      // [K] cleared for completed fragments, or nullptr
+  int err_nonfinite;
 };
 
 // Status word helper: keep the first error recorded since the last poll.
@@ -151,6 +199,22 @@ __device__ __forceinline__ double warp_sum(double v) {
   return v;
 }
 
+// Arrival counters of the epilogues.  An acq_rel read-modify-write orders the arriving thread's earlier writes
+// (and, through the warp or CTA barrier before it, those of the threads it speaks for) before the count, and
+// the count before the reads of whoever arrives last; this is cheaper than a sequentially consistent fence
+// (what __threadfence() compiles to) on each side of a relaxed atomic.
+__device__ __forceinline__ int arrive_cta(int* shared_counter) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.shared::cta.add.u32 %0, [%1], 1;"
+               : "=r"(old) : "r"((unsigned)__cvta_generic_to_shared(shared_counter)) : "memory");
+  return old;
+}
+__device__ __forceinline__ int arrive_gpu(int* global_counter) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(global_counter) : "memory");
+  return old;
+}
+
 struct SlotAccumulator {
   double acc = 0.0;
   int slot = 0;
@@ -180,47 +244,292 @@ struct SlotAccumulator {
 
 constexpr int kFinalizeThreads = 256;
 
-// One block per listed fragment: sum its partials in a fixed order, take the
-// square root, form the score of Eq. 10 and (for a completion) stamp last_sync.
-//   mode 0: completion - I_p = max(1, t_p - last_sync[p]); last_sync[p] = t_l
-//   mode 1: stand-alone scoring - I_p = max(1, interval[p]) or 1; last_sync untouched
-static __global__ void __launch_bounds__(kFinalizeThreads)
-k_finalize_scores(const PlanHeader* __restrict__ hdr, const int* __restrict__ ids,
-                  const double* __restrict__ partial, int entries_per_slot,
-                  int mode, long long t_p, long long t_l, const long long* __restrict__ t_p_dev,
-                  const long long* __restrict__ t_l_dev, const long long* __restrict__ interval,
-                  long long* __restrict__ last_sync, float* __restrict__ norms,
-                  float* __restrict__ scores, int* __restrict__ status, int err_nonfinite) {
-  __shared__ double red[kFinalizeThreads];
-  const int j = blockIdx.x;
-  if (j >= hdr->n_ids) return;
-  const double* src = partial + (size_t)j * entries_per_slot;
-  double s = 0.0;
-  for (int i = threadIdx.x; i < entries_per_slot; i += kFinalizeThreads) s += src[i];
-  red[threadIdx.x] = s;
-  __syncthreads();
-#pragma unroll
-  for (int w = kFinalizeThreads / 2; w > 0; w >>= 1) {
-    if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+// ---------------------------------------------------------------------------
+// The plan in shared memory, built by every CTA in its prologue.
+// ---------------------------------------------------------------------------
+struct InlinePlan {
+  SegPlan seg[kInlineSegs];
+  PlanHeader hdr;
+  long long tiles[kInlineSegs];   // tiles of list position j, then its first tile
+  int frag[kInlineSegs];          // fragment id of list position j
+  int cnt[kInlineSegs];           // segments of position j, then its first table entry
+  int seen[kInlineSegs];
+  int bad;
+  int done_warps;                 // accumulating warps of this CTA that have written their partial sums
+};
+
+struct PlanView {
+  const SegPlan* seg;
+  PlanHeader hdr;
+};
+
+__device__ __forceinline__ long long tiles_of_segment(long long off, long long len, int lanes_per_tile) {
+  const long long lanes = (off - (off & ~3LL) + len + 3) >> 2;
+  return (lanes + lanes_per_tile - 1) / lanes_per_tile;
+}
+
+// Called by EVERY thread of the CTA before the roles split.  (Out of line, like the epilogue: prologue and
+// epilogue run once per CTA, and the streaming loops between them are sensitive to what is compiled around them.)  With a plan in global memory (gplan != nullptr,
+// written by k_plan or k_plan_chunk earlier on the stream) it only returns that; otherwise the CTA expands the
+// id list itself.  Every CTA reaches the same verdict on a bad list (an id out of range or listed twice, a
+// listed fragment without a place in the pool or not inside one row of it): nothing is processed and CTA 0
+// records the error.
+static __device__ __noinline__ PlanView acquire_plan(InlinePlan& ip, const FragTable& T, const PlanRequest& rq,
+                                                 const SegPlan* gplan, const PlanHeader* ghdr, int* status) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  PlanView pv;
+  if (gplan != nullptr) {
+    if (tid == 0) ip.done_warps = 0;
     __syncthreads();
+    pv.seg = gplan;
+    pv.hdr = *ghdr;
+    return pv;
   }
-  if (threadIdx.x != 0) return;
-  const int p = (ids == nullptr) ? j : ids[j];
-  const double norm = sqrt(red[0]);
+  const int K = T.K;
+  int n = (rq.ids == nullptr) ? K : *rq.n_ids;
+  if (tid == 0) { ip.bad = (n < 0 || n > K) ? 1 : 0; ip.done_warps = 0; }
+  for (int i = tid; i < K; i += nt) ip.seen[i] = 0;
+  __syncthreads();
+  if (n < 0 || n > K) n = 0;
+  const int lpt = rq.lanes_per_tile;
+  for (int j = tid; j < n; j += nt) {
+    const int p = (rq.ids == nullptr) ? j : rq.ids[j];
+    bool ok = (p >= 0 && p < K);
+    if (ok && rq.ids != nullptr && atomicAdd(&ip.seen[p], 1) != 0) ok = false;
+    if (ok && rq.snap_offset != nullptr && rq.snap_offset[p] < 0) ok = false;   // no place in the snapshot pool
+    long long t = 0;
+    int c = 0;
+    if (ok) {
+      for (int sg = T.seg_ptr[p]; sg < T.seg_ptr[p + 1]; ++sg) t += tiles_of_segment(T.off[sg], T.len[sg], lpt);
+      c = T.seg_ptr[p + 1] - T.seg_ptr[p];
+    } else {
+      ip.bad = 1;
+    }
+    ip.frag[j] = ok ? p : 0;
+    ip.cnt[j] = c;
+    ip.tiles[j] = t;
+  }
+  __syncthreads();
+  // running segment and tile counts over the list: warp 0, four positions per lane
+  if (tid < 32) {
+    int c[4];
+    long long tl[4];
+    int csum = 0;
+    long long tsum = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int j = 4 * tid + q;
+      c[q] = (j < n) ? ip.cnt[j] : 0;
+      tl[q] = (j < n) ? ip.tiles[j] : 0;
+      csum += c[q];
+      tsum += tl[q];
+    }
+    int cinc = csum;
+    long long tinc = tsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int cv = __shfl_up_sync(0xffffffffu, cinc, o);
+      const long long tv = __shfl_up_sync(0xffffffffu, tinc, o);
+      if (tid >= o) { cinc += cv; tinc += tv; }
+    }
+    int cbase = cinc - csum;
+    long long tbase = tinc - tsum;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int j = 4 * tid + q;
+      if (j < n) { ip.cnt[j] = cbase; ip.tiles[j] = tbase; }
+      cbase += c[q];
+      tbase += tl[q];
+    }
+    if (tid == 31) {
+      if (cinc > kInlineSegs || tinc > 0x3fffffffLL) ip.bad = 1;   // tile + gridDim.x must not wrap
+      ip.hdr.total_tiles = (int)tinc;
+      ip.hdr.n_seg = cinc;
+      ip.hdr.n_ids = n;
+      ip.hdr.pad = 0;
+    }
+  }
+  __syncthreads();
+  if (!ip.bad) {
+    for (int j = tid; j < n; j += nt) {
+      const int p = ip.frag[j];
+      int ns = ip.cnt[j];
+      long long tiles = ip.tiles[j];
+      long long pos = 0;   // elements of the fragment placed so far (packed snapshot layout)
+      for (int sg = T.seg_ptr[p]; sg < T.seg_ptr[p + 1]; ++sg) {
+        SegPlan sp;
+        sp.off = T.off[sg];
+        sp.len = T.len[sg];
+        sp.snap_off = (rq.snap_offset != nullptr) ? rq.snap_offset[p] + pos : sp.off;
+        sp.abase = sp.off & ~3LL;
+        sp.first_tile = (int)tiles;
+        sp.slot = j;
+        sp.frag = p;
+        sp.vec_ok = (((sp.snap_off - sp.off) & 3LL) == 0) ? 1 : 0;
+        // a packed snapshot must lie inside one row of the pool the caller described
+        if (rq.snap_offset != nullptr && sp.snap_off + sp.len > rq.snap_row_len) ip.bad = 1;
+        ip.seg[ns++] = sp;
+        tiles += tiles_of_segment(sp.off, sp.len, lpt);
+        pos += sp.len;
+      }
+    }
+  }
+  __syncthreads();
+  pv.seg = ip.seg;
+  if (ip.bad) {
+    pv.hdr.total_tiles = 0; pv.hdr.n_seg = 0; pv.hdr.n_ids = 0; pv.hdr.pad = 0;
+    if (tid == 0 && blockIdx.x == 0) record_status(status, rq.err_invalid);
+  } else {
+    pv.hdr = ip.hdr;
+  }
+  return pv;
+}
+
+// ---------------------------------------------------------------------------
+// Norms and scores from the partial sums, inside the launch that produced them.
+//
+// Called by every accumulating warp (all 32 lanes) after SlotAccumulator::finish.  The last warp of a CTA to
+// arrive adds that CTA's per-warp entries, slot by slot, into the first of them; the last CTA of the launch to
+// get there (a ticket counter in global memory) adds the CTAs' entries of every slot in a fixed order, takes
+// the square root, forms Eq. 10's score and stamps last_sync.  Which warp does the adding varies from run to
+// run, the order of the additions does not, so the rounded result is the same every run.  The ticket counter
+// is left at zero for the next launch.  A warp that gave up on a bounded wait never arrives: the launch then
+// writes no norms (the status word says why) and the counter is reset by the next status poll.
+// ---------------------------------------------------------------------------
+
+__device__ __forceinline__ void write_fragment_score(const Finalize& F, int j, double total, long long t_p,
+                                                     long long t_l, int* status);
+
+static __device__ __noinline__ void finalize_epilogue(InlinePlan& ip, const Finalize& F, const PlanHeader& h,
+                                                  double* __restrict__ partial, int warps, int* status) {
+  if (F.ticket == nullptr) return;
+  const int lane = threadIdx.x & 31;
+  const int grid = gridDim.x, cta = blockIdx.x;
+  int t = 0;
+  __syncwarp();
+  if (lane == 0) t = arrive_cta(&ip.done_warps);
+  t = __shfl_sync(0xffffffffu, t, 0);
+  if (t != warps - 1) return;
+  // (loads first, additions after: the additions keep their order, the loads overlap)
+  for (int j = lane; j < h.n_ids; j += 32) {
+    double* e = partial + ((size_t)j * grid + cta) * warps;
+    double v = 0.0;
+    for (int w0 = 0; w0 < warps; w0 += 8) {
+      double x[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) x[q] = (w0 + q < warps) ? __ldcg(e + w0 + q) : 0.0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) if (w0 + q < warps) v += x[q];
+    }
+    __stcg(e, v);
+  }
+  __syncwarp();
+  if (lane == 0) t = arrive_gpu(F.ticket);
+  t = __shfl_sync(0xffffffffu, t, 0);
+  if (t != grid - 1) return;
+  long long t_p = F.t_p, t_l = F.t_l;
+  if (F.t_p_dev) t_p = *F.t_p_dev;
+  if (F.t_l_dev) t_l = *F.t_l_dev;
+  // Four slots at a time, so that their loads are in flight together.  Per slot: lane l adds the entries of
+  // CTAs l, l + 32, ... in that order, then the lanes' sums meet in the shuffle tree.
+  constexpr int kBatch = 4;
+  for (int j0 = 0; j0 < h.n_ids; j0 += kBatch) {
+    double s[kBatch];
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q) s[q] = 0.0;
+    for (int i0 = lane; i0 < grid; i0 += 32 * 4) {
+      double x[kBatch][4];
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int i = i0 + 32 * r;
+          x[q][r] = (j0 + q < h.n_ids && i < grid) ? __ldcg(partial + ((size_t)(j0 + q) * grid + i) * warps) : 0.0;
+        }
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q)
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+          if (j0 + q < h.n_ids && i0 + 32 * r < grid) s[q] += x[q][r];
+    }
+#pragma unroll
+    for (int q = 0; q < kBatch; ++q) {
+      const int j = j0 + q;
+      if (j >= h.n_ids) break;
+      const double total = warp_sum(s[q]);
+      if (lane == 0) write_fragment_score(F, j, total, t_p, t_l, status);
+    }
+  }
+  __syncwarp();
+  if (lane == 0) *F.ticket = 0;
+}
+
+// Last steps of Eq. 10 for one slot, by lane 0 of the warp that holds the slot's total.
+__device__ __forceinline__ void write_fragment_score(const Finalize& F, int j, double total, long long t_p,
+                                                     long long t_l, int* status) {
+  const int p = (F.ids == nullptr) ? j : F.ids[j];
+  if (F.sumsq_out) F.sumsq_out[p] = total;
+  if (!F.write_scores) return;
+  const double norm = sqrt(total);
   long long I = 1;
-  if (mode == 0) {
-    // step numbers kept in device memory (graph replay) take precedence over the launch arguments
-    if (t_p_dev) t_p = *t_p_dev;
-    if (t_l_dev) t_l = *t_l_dev;
-    I = t_p - last_sync[p];
-    last_sync[p] = t_l;
-  } else if (interval != nullptr) {
-    I = interval[p];
+  if (F.mode == 0) {
+    I = t_p - F.last_sync[p];
+    F.last_sync[p] = t_l;
+    if (F.in_flight) F.in_flight[p] = 0;
+  } else if (F.interval != nullptr) {
+    I = F.interval[p];
   }
   if (I < 1) I = 1;
-  norms[p] = (float)norm;
-  scores[p] = (float)(norm / (double)I);
-  if (!isfinite(norm)) record_status(status, err_nonfinite);
+  F.norms[p] = (float)norm;
+  F.scores[p] = (float)(norm / (double)I);
+  if (!isfinite(norm)) record_status(status, F.err_nonfinite);
+}
+
+// The same epilogue for kernels in which every thread of the CTA is an accumulating thread that reaches the
+// end of the kernel (no producer warps, no abandoned waits), so the CTA can meet at a barrier: the CTA's
+// entries are added by its threads side by side, and in the last CTA of the launch every warp takes slots.
+// The order of the additions is the one finalize_epilogue uses, hence the same bits.
+static __device__ __noinline__ void finalize_epilogue_cta(InlinePlan& ip, const Finalize& F, const PlanHeader& h,
+                                                      double* __restrict__ partial, int warps, int* status) {
+  if (F.ticket == nullptr) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int grid = gridDim.x, cta = blockIdx.x;
+  __syncthreads();     // every warp's entries are written
+  for (int j = tid; j < h.n_ids; j += blockDim.x) {
+    double* e = partial + ((size_t)j * grid + cta) * warps;
+    double v = 0.0;
+    for (int w0 = 0; w0 < warps; w0 += 8) {
+      double x[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) x[q] = (w0 + q < warps) ? __ldcg(e + w0 + q) : 0.0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) if (w0 + q < warps) v += x[q];
+    }
+    __stcg(e, v);
+  }
+  __syncthreads();
+  if (tid == 0) ip.done_warps = (arrive_gpu(F.ticket) == grid - 1) ? 1 : 0;
+  __syncthreads();
+  if (!ip.done_warps) return;
+  long long t_p = F.t_p, t_l = F.t_l;
+  if (F.t_p_dev) t_p = *F.t_p_dev;
+  if (F.t_l_dev) t_l = *F.t_l_dev;
+  for (int j = warp; j < h.n_ids; j += warps) {
+    double s = 0.0;
+    for (int i0 = lane; i0 < grid; i0 += 32 * 8) {
+      double x[8];
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        const int i = i0 + 32 * r;
+        x[r] = (i < grid) ? __ldcg(partial + ((size_t)j * grid + i) * warps) : 0.0;
+      }
+#pragma unroll
+      for (int r = 0; r < 8; ++r) if (i0 + 32 * r < grid) s += x[r];
+    }
+    const double total = warp_sum(s);
+    if (lane == 0) write_fragment_score(F, j, total, t_p, t_l, status);
+  }
+  if (tid == 0) *F.ticket = 0;
 }
 
 // ---------------------------------------------------------------------------
@@ -254,16 +563,35 @@ k_accumulate_chunk(const double* __restrict__ partial, int entries, double* __re
   if (threadIdx.x == 0) *total += red[0];
 }
 
-static __global__ void k_finalize_from_sums(const double* __restrict__ sums, const int* __restrict__ ids, int n,
-                                     long long t_p, long long t_l, long long* __restrict__ last_sync,
-                                     float* __restrict__ norms, float* __restrict__ scores,
-                                     int* __restrict__ status, int err_nonfinite) {
+// Eq. 10 from per-fragment sums of squares that already exist (added up chunk by chunk by the host-buffer entry
+// point, or all-reduced over the devices that each hold a slice of every fragment).
+//   completion (interval_mode == 0): fragments ids[0 .. n), sums indexed as `by_position` says,
+//       I_p = max(1, t_p - last_sync[p]), last_sync[p] = t_l, in_flight[p] = 0
+//   stand-alone (interval_mode == 1): all K fragments, I_p = max(1, interval[p]) (1 without intervals)
+static __global__ void k_scores_from_sumsq(const double* __restrict__ sums, int by_position, const int* __restrict__ ids,
+                                    const int* __restrict__ n_ids_dev, int n_host, int K, int interval_mode,
+                                    const long long* __restrict__ interval, long long t_p, long long t_l,
+                                    long long* __restrict__ last_sync, float* __restrict__ norms,
+                                    float* __restrict__ scores, unsigned char* __restrict__ in_flight,
+                                    int* __restrict__ status, int err_nonfinite, int err_invalid) {
+  int n = interval_mode ? K : (n_ids_dev ? *n_ids_dev : n_host);
+  if (n < 0 || n > K) {
+    if (threadIdx.x == 0) record_status(status, err_invalid);
+    return;
+  }
   for (int j = threadIdx.x; j < n; j += blockDim.x) {
-    const int p = ids[j];
-    const double norm = sqrt(sums[j]);
-    long long I = t_p - last_sync[p];
+    const int p = interval_mode ? j : ids[j];
+    if (p < 0 || p >= K) { record_status(status, err_invalid); continue; }
+    const double norm = sqrt(sums[by_position ? j : p]);
+    long long I = 1;
+    if (interval_mode) {
+      if (interval != nullptr) I = interval[p];
+    } else {
+      I = t_p - last_sync[p];
+      last_sync[p] = t_l;
+      if (in_flight) in_flight[p] = 0;
+    }
     if (I < 1) I = 1;
-    last_sync[p] = t_l;
     norms[p] = (float)norm;
     scores[p] = (float)(norm / (double)I);
     if (!isfinite(norm)) record_status(status, err_nonfinite);

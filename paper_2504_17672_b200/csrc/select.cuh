@@ -19,7 +19,8 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
          const long long* __restrict__ frag_first_off,
          long long t_now, const long long* __restrict__ t_now_dev, long long H, int budget_kind, long long budget,
          unsigned char* __restrict__ mask, int* __restrict__ ids, int* __restrict__ n_sel,
-         long long* __restrict__ pool_offset, int* __restrict__ status, int err_nonfinite, int err_too_many) {
+         long long* __restrict__ pool_offset, unsigned char* __restrict__ in_flight,
+         int* __restrict__ status, int err_nonfinite, int err_too_many) {
   __shared__ float s_score[kMaxK];
   __shared__ unsigned char s_class[kMaxK];  // 0 = ineligible, 1 = ordinary, 2 = overdue
   __shared__ int s_order[kMaxK];
@@ -33,7 +34,9 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   __syncthreads();
   if (p < K) {
     const float r = scores[p];
-    const bool elig = (ineligible == nullptr) || (ineligible[p] == 0);
+    // a fragment whose synchronisation is in flight cannot be chosen again before it completes
+    const bool elig = ((ineligible == nullptr) || (ineligible[p] == 0)) &&
+                      ((in_flight == nullptr) || (in_flight[p] == 0));
     const bool overdue = (t_now - last_sync[p]) >= H;   // Algorithm 2's staleness test
     s_score[p] = r;
     s_fsize[p] = frag_size[p];
@@ -97,6 +100,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
       const long long cost = (budget_kind == 0) ? 1 : s_fsize[f];
       if (j == 0 || cost <= remaining) {   // the head of the order is always taken
         mask[f] = 1;
+        if (in_flight) in_flight[f] = 1;
         ids[n++] = f;
         remaining -= cost;
         if (pool_offset) place(f, pool_pos);
@@ -111,7 +115,10 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     return;
   }
   if (n_free > kExactMaxFree) {      // too many candidates to enumerate: report it, select nothing
-    if (p < K) { mask[p] = 0; ids[p] = -1; if (pool_offset) pool_offset[p] = -1; }
+    if (p < K) {
+      if (in_flight && mask[p]) in_flight[p] = 0;   // taken back: marked by the walk above in this call
+      mask[p] = 0; ids[p] = -1; if (pool_offset) pool_offset[p] = -1;
+    }
     if (p == 0) { *n_sel = 0; record_status(status, err_too_many); }
     return;
   }
@@ -165,6 +172,7 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
     if (!((chosen >> j) & 1u)) continue;
     const int f = s_order[s_free_begin + j];
     mask[f] = 1;
+    if (in_flight) in_flight[f] = 1;
     ids[n++] = f;
     if (pool_offset) place(f, pool_pos);
   }

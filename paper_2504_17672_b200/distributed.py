@@ -71,16 +71,14 @@ def complete_fragments_peers(ctx, hyper, M_total: int, rank: int, sum_bufs: Sequ
     barrier()
 
 
-def combine_sharded_norms(norms_local: torch.Tensor, interval: torch.Tensor = None, group=None):
-    """Parameter-range sharding: every rank holds a slice of each fragment (all workers of that slice), so
-    the element-wise steps need no exchange and only Eq. 10's norm spans ranks.  Given the norms each rank
-    computed over its own slices, returns (norms, scores) of the whole fragments, identical on every rank:
-    one all-reduce of K doubles (the sums of squares), then R_p = norm_p / max(1, I_p)."""
-    sq = norms_local.double() ** 2
-    dist.all_reduce(sq, op=dist.ReduceOp.SUM, group=group)
-    norms = sq.sqrt()
-    if interval is None:
-        scores = norms.clone()
-    else:
-        scores = norms / interval.clamp(min=1).double()
-    return norms.float(), scores.float()
+def scores_from_sharded_sumsq(ctx, sumsq: torch.Tensor, ids_dev, n_ids_dev, t_p: int, t_l: int, last_sync, norms,
+                              scores, group=None) -> None:
+    """Parameter-range sharding: every rank holds a slice of each fragment (all workers of that slice), so the
+    element-wise steps need no exchange and only Eq. 10's norm spans ranks.
+
+    `sumsq` (device fp64 [K]) holds this rank's sums of squares of the listed fragments, as cocodc_outer_step
+    wrote them with STAGE_SUMSQ.  One all-reduce of those K doubles, then the library forms norms and scores from
+    the totals and stamps last_sync - the same values on every rank, so the replicated selection that follows
+    picks the same fragments everywhere."""
+    dist.all_reduce(sumsq, op=dist.ReduceOp.SUM, group=group)
+    ctx.cocodc_scores_from_sumsq(sumsq, ids_dev, n_ids_dev, None, t_p, t_l, last_sync, norms, scores)

@@ -7,8 +7,9 @@
   * every h steps (Eq. 8-9) a new synchronisation is initiated: `cocodc_select_fragments` (Algorithm 2,
     fragments still in flight are ineligible) and `cocodc_snapshot` of the chosen fragments.
 
-All schedule state (scores, last_sync, id lists, masks, pool offsets) lives on the device; the driver
-only marshals arguments and keeps track of which slot was initiated when.  Several synchronisations can
+All schedule state (scores, last_sync, id lists, masks, pool offsets, the in-flight mask) lives on the device
+and is updated by the library's kernels; the driver only marshals arguments and keeps track of which slot was
+initiated when.  Several synchronisations can
 be in flight at once (tau > h); each has its own slot: id list, mask and snapshot pool.
 """
 
@@ -59,7 +60,9 @@ class RoundDriver:
         self.scores = torch.full((K,), float("inf"), dtype=torch.float32, device=dev)   # never synced: +inf
         self.norms = torch.zeros(K, dtype=torch.float32, device=dev)
         self.last_sync = torch.zeros(K, dtype=torch.int64, device=dev)
-        self.ineligible = torch.zeros(K, dtype=torch.uint8, device=dev)
+        # Algorithm 2's in-flight bookkeeping: the selection kernel marks what it admits, the completion clears it
+        self.in_flight = torch.zeros(K, dtype=torch.uint8, device=dev)
+        ctx.cocodc_bind_in_flight(self.in_flight)
         self.initiated = 0
         self.completed = 0
         # optional callable(kind, phase, slot, t) with kind in {"complete", "initiate"} and phase in
@@ -77,19 +80,17 @@ class RoundDriver:
         self.ctx.cocodc_outer_step(self.hyper, self.w_now, slot.pool, self.w_now.stride(0), slot.pool.stride(0),
                                    slot.pool_off, self.theta_g, self.momentum, None, slot.ids, slot.n_ids,
                                    slot.t_p, t_l, self.last_sync, self.norms, self.scores)
-        self.ineligible.sub_(slot.mask)          # its fragments may be chosen again
         self._notify("complete", "after", slot, t_l)
         slot.t_p = -1
         self.completed += 1
 
     def _initiate(self, slot: _Slot, t_p: int) -> None:
         self._notify("initiate", "before", slot, t_p)
-        self.ctx.cocodc_select_fragments(self.scores, self.last_sync, self.ineligible, t_p, self.hyper.H,
+        self.ctx.cocodc_select_fragments(self.scores, self.last_sync, None, t_p, self.hyper.H,
                                          self.budget_kind, self.budget, slot.mask, slot.ids, slot.n_ids,
                                          slot.pool_off)
         self.ctx.cocodc_snapshot(self.w_now, slot.pool, self.w_now.stride(0), slot.pool.stride(0), slot.pool_off,
                                  self.hyper.M, slot.ids, slot.n_ids)
-        self.ineligible.add_(slot.mask)          # in flight until it completes
         slot.t_p = t_p
         self.initiated += 1
         self._notify("initiate", "after", slot, t_p)

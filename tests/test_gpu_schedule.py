@@ -41,7 +41,7 @@ def test_round_driver_in_the_papers_setting():
     def state():
         return dict(w_now=np_(bufs.w_now).copy(), theta_g=np_(bufs.theta_g).copy(), momentum=np_(bufs.momentum).copy(),
                     scores=np_(drv.scores).copy(), last_sync=np_(drv.last_sync).copy(),
-                    ineligible=np_(drv.ineligible).copy(), norms=np_(drv.norms).copy())
+                    in_flight=np_(drv.in_flight).copy(), norms=np_(drv.norms).copy())
 
     def observer(kind, phase, slot, t):
         if phase == "before":
@@ -56,11 +56,11 @@ def test_round_driver_in_the_papers_setting():
         assert ctx.cocodc_poll_status() == 0
         if kind == "initiate":
             mask, ids, n = orc.select_fragments(pre["scores"], pre["last_sync"], w.partition.frag_sizes, t, w.H,
-                                                orc.BUDGET_COUNT, 1, pre["ineligible"])
+                                                orc.BUDGET_COUNT, 1, pre["in_flight"])
             got = np_(slot.ids)[:int(slot.n_ids.item())].tolist()
             assert got == ids.tolist() and np.array_equal(np_(slot.mask), mask)
-            assert not any(pre["ineligible"][p] for p in got)          # never a fragment that is in flight
-            assert np.array_equal(post["ineligible"], pre["ineligible"] + mask)
+            assert not any(pre["in_flight"][p] for p in got)           # never a fragment that is in flight
+            assert np.array_equal(post["in_flight"], pre["in_flight"] + mask)   # marked by the selection kernel itself
             po = np_(slot.pool_off)
             exp_pool = orc.snapshot(frs, pre["w_now"], got, w.M, po, np_(slot.pool))
             assert np.array_equal(np_(slot.pool), exp_pool)             # S0 recorded exactly the chosen fragments
@@ -80,6 +80,10 @@ def test_round_driver_in_the_papers_setting():
                     assert_close(wn[m], r.w_now[m], TOL_PARAM, f"w_now[{m}]")
                 assert abs(post["scores"][p] - r.score) <= TOL_NORM * r.score
             assert np.array_equal(post["last_sync"], new_last)
+            done = np.zeros(w.K, dtype=np.uint8)
+            done[ids] = 1
+            assert all(pre["in_flight"][p] == 1 for p in ids)
+            assert np.array_equal(post["in_flight"], pre["in_flight"] - done)   # cleared by the completion's last warp
             log["completed"].append((t, ids))
 
     drv.observer = observer

@@ -302,3 +302,81 @@ def test_selected_pool_places_keep_the_native_alignment():
         assert prob.poll() == 0
         check_step_against_oracle(prob, before, ids, 10, 13, orc_hyper(w))
         prob.last_sync.zero_()
+
+
+def test_sums_of_squares_of_two_slices_give_the_whole_fragments_scores():
+    """Parameter-range sharding on one GPU: two contexts each own one half of every fragment (all workers of that
+    element range) over the same buffers.  Each completes its halves with COCODC_STAGE_SUMSQ, which stops Eq. 10
+    at the per-fragment sums of squares; the two fp64 vectors are added (the all-reduce of a real deployment) and
+    cocodc_scores_from_sumsq forms norms, scores and last_sync of the whole fragments from the totals.  Elements,
+    norms and scores are compared with the oracle run on the whole fragments."""
+    from paper_2504_17672_b200 import binding as B
+    from helpers import check_step_against_oracle, orc_hyper
+    frs = [[(4, 30_001)], [(30_009, 12_000), (60_000, 5_003)], [(42_012, 17_777)]]
+    w = synth.small_workload((70_000, frs), M=3, seed=41, scale_kind="loguniform", tau=3)
+    prob = GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3))
+    halves = ([], [])
+    for f in frs:
+        lo_half, hi_half = [], []
+        for off, ln in f:
+            cut = ln // 2 + 1
+            lo_half.append((off, cut))
+            hi_half.append((off + cut, ln - cut))
+        halves[0].append(lo_half)
+        halves[1].append(hi_half)
+    ctxs = []
+    for h in halves:
+        wh = synth.small_workload((w.N, h), M=3, seed=41)
+        ptr, off, ln = wh.partition.csr()
+        ctxs.append(B.Context(w.N, ptr, off, ln, 3))
+    ids = [2, 0]
+    prob.set_ids(ids)
+    prob.last_sync.copy_(torch.tensor([1, 0, 3], device="cuda"))
+    before = prob.host_state()
+    b = prob.bufs
+    t_p, t_l = 9, 12
+    sums = [torch.full((w.K,), -1.0, dtype=torch.float64, device="cuda") for _ in ctxs]
+    for ctx, sq in zip(ctxs, sums):
+        n0 = ctx.launch_count
+        ctx.cocodc_outer_step(prob.hyper(), b.w_now, b.w_snap, b.now_stride, b.snap_stride, None, b.theta_g, b.momentum,
+                              None, prob.ids, prob.n_ids, t_p, t_l, None, None, None,
+                              stages=B.STAGE_OUTER | B.STAGE_MERGE | B.STAGE_SUMSQ, sumsq_out=sq)
+        assert ctx.launch_count - n0 == 1               # plan, streaming pass and sums in one launch
+        assert ctx.cocodc_poll_status() == 0
+    assert float(sums[0][1]) == -1.0                    # a fragment that was not listed keeps its entry
+    assert torch.equal(prob.last_sync, torch.tensor([1, 0, 3], device="cuda"))      # sums only: nothing stamped yet
+    total = sums[0] + sums[1]                           # stands in for the all-reduce over the two devices
+    prob.ctx.cocodc_scores_from_sumsq(total, prob.ids, prob.n_ids, None, t_p, t_l, prob.last_sync, prob.norms,
+                                      prob.scores)
+    assert prob.poll() == 0
+    check_step_against_oracle(prob, before, ids, t_p, t_l, orc_hyper(w))
+    # the sums themselves against the oracle's
+    res, _ = orc.outer_step(fragments_of(w), orc_hyper(w), before["w_now"], before["w_snap"], before["theta_g"],
+                            before["momentum"], ids, t_p, t_l, before["last_sync"])
+    for p in ids:
+        assert abs(float(total[p]) - res[p].sumsq) <= 2e-6 * res[p].sumsq
+    # stand-alone form: sums of squares of a vector, then scores from them with intervals
+    x = torch.randn(w.N, device="cuda", generator=torch.Generator(device="cuda").manual_seed(3)) * 1e-2
+    sq = torch.zeros(w.K, dtype=torch.float64, device="cuda")
+    n0 = prob.ctx.launch_count
+    prob.ctx.cocodc_fragment_scores(x, None, None, None, sumsq_out=sq)
+    assert prob.ctx.launch_count - n0 == 1
+    exp_sq = orc.fragment_sumsq(fragments_of(w), np_(x))
+    assert np.all(np.abs(np_(sq) - exp_sq) <= 2e-6 * exp_sq)
+    iv = torch.tensor([4, 0, 9], dtype=torch.int64, device="cuda")
+    norms = torch.zeros(w.K, device="cuda")
+    scores = torch.zeros(w.K, device="cuda")
+    prob.ctx.cocodc_scores_from_sumsq(sq, None, None, iv, 0, 0, None, norms, scores)
+    en, es = orc.fragment_scores(fragments_of(w), np_(x), np_(iv))
+    assert np.all(np.abs(np_(norms) - en) <= TOL_NORM * en) and np.all(np.abs(np_(scores) - es) <= TOL_NORM * es)
+    assert prob.poll() == 0
+    # a fragment table too large to travel as a kernel argument takes the plan kernel as well
+    big = synth.small_workload([300] * 200, M=1, seed=1)
+    ptr, off, ln = big.partition.csr()
+    cbig = B.Context(big.N, ptr, off, ln, 1)
+    xb = torch.ones(big.N, device="cuda")
+    nb = torch.zeros(200, device="cuda")
+    n0 = cbig.launch_count
+    cbig.cocodc_fragment_scores(xb, None, nb, nb.clone())
+    assert cbig.launch_count - n0 == 2 and cbig.cocodc_poll_status() == 0
+    assert np.allclose(np_(nb), np.sqrt(300.0), rtol=1e-6)

@@ -62,12 +62,19 @@ def _worker(rank, world, port, out):
         for o, l in ranges:
             exp[o:o + l] = 3.0                                    # 1 + 2 summed over the two ranks
         assert torch.equal(buf, exp)
-        # parameter-range sharding: fragment norms from per-rank slices, one all-reduce of K sums of squares
-        full = torch.arange(1, 13, dtype=torch.float32).reshape(3, 4)          # 3 fragments of 4 elements
-        mine = full[:, 2 * rank:2 * rank + 2]                                  # each rank owns half of every fragment
-        n, sc = D.combine_sharded_norms(mine.norm(dim=1), torch.tensor([0, 2, 5]))
-        assert torch.allclose(n, full.norm(dim=1), rtol=1e-6)
-        assert torch.allclose(sc, full.norm(dim=1) / torch.tensor([1.0, 2.0, 5.0]), rtol=1e-6)
+        # parameter-range sharding: every rank holds a slice of each fragment; what crosses ranks is one all-reduce
+        # of the K fp64 sums of squares, after which the library forms the scores (a recording stand-in here)
+        full = torch.arange(1, 13, dtype=torch.float64).reshape(3, 4)          # 3 fragments of 4 elements
+        mine = (full[:, 2 * rank:2 * rank + 2] ** 2).sum(dim=1)                # this rank's half of every sum
+        seen = {}
+
+        class Recorder:
+            def cocodc_scores_from_sumsq(self, sumsq, ids, n_ids, interval, t_p, t_l, last_sync, norms, scores):
+                seen.update(sumsq=sumsq.clone(), args=(ids, n_ids, interval, t_p, t_l, last_sync, norms, scores))
+
+        D.scores_from_sharded_sumsq(Recorder(), mine, "ids", "n", 7, 11, "last", "norms", "scores")
+        assert torch.equal(seen["sumsq"], (full ** 2).sum(dim=1))
+        assert seen["args"] == ("ids", "n", None, 7, 11, "last", "norms", "scores")
         out.put((rank, "ok"))
     except Exception as e:  # pragma: no cover
         out.put((rank, repr(e)))
