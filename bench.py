@@ -8,9 +8,17 @@ The metric is fragment parameters completed per second (whole job), with the ach
 the fused kernel beside it.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+                    [--deployment replicas|param_shard|worker_per_device]
 
-N > 1 is launched by torch.distributed.run, one rank per GPU; every rank owns an independent
-parameter shard of the same shape (weak scaling, no data-path collective).
+N > 1: one rank per GPU over NCCL.  Started under torch.distributed.run (RANK / WORLD_SIZE in the environment)
+the process is one of the ranks; started plainly with --gpus N it launches the N ranks itself.  Deployments:
+    replicas           every rank owns an independent parameter shard of the same shape (no data-path collective)
+    param_shard        rank r owns one element range (all workers of it) of a model N times larger: S1-S5 are
+                       local, the K per-fragment sums of squares are all-reduced as fp64 before the scores are
+                       formed, selection runs replicated and must agree on every rank (Section 3.2)
+    worker_per_device  the workers are spread over the ranks (Section 2.1, one worker per device in the paper):
+                       per-device pseudo-gradient sums, all-reduce of the listed fragments, completion from
+                       the received sum
 """
 
 from __future__ import annotations
@@ -153,9 +161,11 @@ def pool_capacity(w: synth.Workload) -> int:
 class DeviceJob:
     """Workload resident in HBM plus its schedule state, stepped through the C-ABI binding."""
 
-    def __init__(self, w: synth.Workload, device: torch.device, variant: str = "cocodc"):
+    def __init__(self, w: synth.Workload, device: torch.device, variant: str = "cocodc",
+                 deployment: str = "replicas", world: int = 1, M_total: int = 0, worker_offset: int = 0):
         from paper_2504_17672_b200 import binding as B
         self.B, self.w, self.dev, self.variant = B, w, device, variant
+        self.deployment, self.world, self.M_total = deployment, world, (M_total or w.M)
         ptr, off, ln = w.partition.csr()
         self.ctx = B.Context(w.N, ptr, off, ln, w.M, device=device.index or 0)
         K = w.K
@@ -184,18 +194,65 @@ class DeviceJob:
         ids0 = self.ids[:n].tolist()
         offs = {p: int(self.pool_off[p].item()) for p in ids0}
         self.bufs = synth.generate(w, device, snap_layout="pool", pool_ids=ids0, pool_offsets=offs,
-                                   pool_len=pool_capacity(w))
+                                   pool_len=pool_capacity(w), worker_offset=worker_offset)
         if variant == "diloco":
             self.ids.copy_(torch.arange(K, dtype=torch.int32, device=device))
             self.n_ids.fill_(K)
+        if deployment == "param_shard":
+            self.sumsq = torch.zeros(K, dtype=torch.float64, device=device)
+        if deployment == "worker_per_device":
+            self.sum_buf = torch.zeros(w.N, dtype=torch.float32, device=device)
+        self.collective_bytes = 0       # bytes this rank handed to collectives on the data path
 
     def select(self):
         w = self.w
         self.ctx.cocodc_select_fragments(self.scores, self.last_sync, None, self.t, w.H, self.kind, w.budget,
                                          self.mask, self.ids, self.n_ids, self.pool_off)
 
+    def outer_param_shard(self):
+        """This rank's element range: S1-S5 and the local sums of squares; Eq. 10 is finished after the all-reduce."""
+        B, b, w = self.B, self.bufs, self.w
+        self.ctx.cocodc_outer_step(self.hyper, b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off,
+                                   b.theta_g, b.momentum, None, self.ids, self.n_ids, self.t, self.t + w.tau,
+                                   None, None, None, stages=B.STAGE_OUTER | B.STAGE_MERGE | B.STAGE_SUMSQ,
+                                   sumsq_out=self.sumsq)
+
+    def scores_param_shard(self):
+        import torch.distributed as dist
+        w = self.w
+        if self.world > 1:
+            dist.all_reduce(self.sumsq, op=dist.ReduceOp.SUM)
+            self.collective_bytes += self.sumsq.numel() * 8
+        self.ctx.cocodc_scores_from_sumsq(self.sumsq, self.ids, self.n_ids, None, self.t, self.t + w.tau,
+                                          self.last_sync, self.norms, self.scores)
+
+    def pseudo_sum_and_exchange(self):
+        """Worker-per-device: this rank's pseudo-gradient sums, then the all-reduce of Section 2.1 over the
+        listed fragments' ranges (the id list is read back: the host slices the buffer for the collective)."""
+        from paper_2504_17672_b200 import distributed as D
+        b, w = self.bufs, self.w
+        self.ctx.cocodc_pseudo_gradient_sum(b.w_snap, b.snap_stride, self.pool_off, b.theta_g, w.M, self.sum_buf,
+                                            self.ids, self.n_ids)
+        if self.world > 1:
+            n = int(self.n_ids.item())
+            ids_h = self.ids[:n].tolist()
+            ranges = D.fragment_ranges(w.partition.fragments, ids_h)
+            D.allreduce_ranges(self.sum_buf, ranges)
+            self.collective_bytes += 4 * sum(l for _, l in ranges)
+
+    def outer_received(self):
+        b, w = self.bufs, self.w
+        self.ctx.cocodc_outer_step_received(self.hyper, self.M_total, b.w_now, b.w_snap, b.now_stride, b.snap_stride,
+                                            self.pool_off, b.theta_g, b.momentum, self.sum_buf, None, self.ids,
+                                            self.n_ids, self.t, self.t + w.tau, self.last_sync, self.norms,
+                                            self.scores)
+
     def outer(self):
         b, w = self.bufs, self.w
+        if self.deployment == "param_shard":
+            return self.outer_param_shard()
+        if self.deployment == "worker_per_device":
+            return self.outer_received()
         if self.variant == "diloco":
             self.ctx.cocodc_outer_step(self.hyper, b.w_now, b.w_now, b.now_stride, b.now_stride, None,
                                        b.theta_g, b.momentum, None, self.ids, self.n_ids, self.t, self.t,
@@ -210,13 +267,17 @@ class DeviceJob:
         self.ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off, self.w.M,
                                  self.ids, self.n_ids)
 
-    def step(self, log_ids=None, log_n=None, ev=None):
+    def step(self, log_ids=None, log_n=None, ev=None, log_next=None, log_next_n=None):
         """Complete the fragments in flight, choose the next set, record their snapshots."""
+        if self.deployment == "worker_per_device":
+            self.pseudo_sum_and_exchange()
         if ev is not None:
             ev[0].record()
         self.outer()
         if ev is not None:
             ev[1].record()
+        if self.deployment == "param_shard":
+            self.scores_param_shard()
         if log_ids is not None:
             log_ids.copy_(self.ids)
             log_n.copy_(self.n_ids)
@@ -226,12 +287,93 @@ class DeviceJob:
         self.t += self.w.tau
         self.select()
         self.snapshot()
+        if log_next is not None:         # the set whose snapshot was just taken
+            log_next.copy_(self.ids)
+            log_next_n.copy_(self.n_ids)
+
+
+def timed_device_leg(job: DeviceJob, K: int, W: int, device: torch.device, local: int, barrier):
+    """W warm-up steps, then exactly K timed steps between two barriers; CUDA events around the whole region and
+    around every completion call.  Returns the raw figures of this rank."""
+    w = job.w
+    log_ids = torch.full((K, w.K), -1, dtype=torch.int32, device=device)
+    log_n = torch.zeros((K, 1), dtype=torch.int32, device=device)
+    next_ids = torch.full((K, w.K), -1, dtype=torch.int32, device=device)
+    next_n = torch.zeros((K, 1), dtype=torch.int32, device=device)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(W):
+        job.step()
+    status = job.ctx.cocodc_poll_status()
+    if status != 0:
+        raise RuntimeError(f"device status after warm-up: {job.B.status_string(status)}")
+    barrier()
+    launches0 = job.ctx.launch_count
+    bytes0 = job.collective_bytes
+    with ClockSampler(local) as clocks:
+        t_begin.record()
+        for i in range(K):
+            job.step(log_ids[i], log_n[i], evs[i], next_ids[i], next_n[i])
+        t_end.record()
+        barrier()
+    status = job.ctx.cocodc_poll_status()
+    if status != 0:
+        raise RuntimeError(f"device status after the timed region: {job.B.status_string(status)}")
+    ids_h, n_h = log_ids.cpu().numpy(), log_n.cpu().numpy().ravel()
+    nx_h, nn_h = next_ids.cpu().numpy(), next_n.cpu().numpy().ravel()
+    return {
+        "seconds": t_begin.elapsed_time(t_end) / 1e3,
+        "per_step": [int(job.sizes[ids_h[i, :n_h[i]]].sum()) for i in range(K)],
+        "per_step_snapshot": [int(job.sizes[nx_h[i, :nn_h[i]]].sum()) for i in range(K)],
+        "outer_ms": [a.elapsed_time(b) for a, b in evs],
+        "launches": job.ctx.launch_count - launches0,
+        "collective_bytes": job.collective_bytes - bytes0,
+        "clocks": clocks.result,
+        "ids": ids_h, "n": n_h,
+    }
+
+
+def completion_bytes_per_param(M: int, variant: str, deployment: str) -> int:
+    """Algorithmic HBM bytes per fragment parameter of the call the roofline record times."""
+    if variant == "diloco":
+        return 8 * M + 16                      # zero delay: w_now is read once and written once
+    if deployment == "worker_per_device":
+        return 12 * M + 20                     # the received sum is one more stream
+    return bytes_per_param(M)
+
+
+def roofline_record(w, variant, deployment, leg, K, peak, peak_kind, traffic=None):
+    bpp = completion_bytes_per_param(w.M, variant, deployment)
+    outer_seconds = sum(leg["outer_ms"]) / 1e3
+    params = float(sum(leg["per_step"]))
+    achieved = params * bpp / outer_seconds / 1e9
+    per_launch = sorted(leg["per_step"][i] * bpp / leg["outer_ms"][i] / 1e6 for i in range(K) if leg["outer_ms"][i] > 0)
+    if w.M > 8:
+        kernel = "k_outer_ring (fused S1-S6)"
+    elif variant == "diloco":
+        kernel = f"k_outer_inplace<{w.M}> (fused S1-S6, zero delay)"
+    elif deployment == "worker_per_device":
+        kernel = f"k_outer_tma<{w.M}, received sum> (S2-S6)"
+    else:
+        kernel = f"k_outer_tma<{w.M}> (fused S1-S6)"
+    return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
+            "bytes_per_param": bpp, "ms_per_launch": outer_seconds / K * 1e3,
+            "params_per_launch": params / K,
+            "achieved_median": per_launch[len(per_launch) // 2] if per_launch else None,
+            "achieved_best": per_launch[-1] if per_launch else None,
+            "launches_timed": len(per_launch), "traffic": traffic}
 
 
 def run_ours(args):
     rank, world, local = dist_env()
     if not torch.cuda.is_available():
+        print(f"rank {rank}: no CUDA device", file=sys.stderr, flush=True)
+        if world > 1:
+            time.sleep(3.0)    # the launcher stops the other ranks when one fails: let them report first
         raise RuntimeError("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
+    if local >= torch.cuda.device_count():
+        raise RuntimeError(f"rank {rank}: local rank {local} has no GPU ({torch.cuda.device_count()} visible)")
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
     backend_ready = False
@@ -239,21 +381,19 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
         backend_ready = True
+    deployment = args.deployment or ("param_shard" if world > 1 else "replicas")
+    if args.variant != "cocodc" and deployment != "replicas":
+        raise SystemExit("--variant other than cocodc runs with --deployment replicas")
     w = synth.get_workload(args.workload)
-    if world > 1:
-        w = w.with_(seed=w.seed + 1000 * rank)   # every rank owns a different shard of the same shape
-    job = DeviceJob(w, device, args.variant)
+    M_total, worker_offset = w.M, 0
+    if deployment in ("replicas", "param_shard") and world > 1:
+        w = w.with_(seed=w.seed + 1000 * rank)   # every rank owns a different element range of the same shape
+    if deployment == "worker_per_device":
+        M_local = max(1, w.M // world)           # the workers are spread over the ranks; at least one each
+        M_total, worker_offset = M_local * world, M_local * rank
+        w = w.with_(M=M_local)
+    job = DeviceJob(w, device, args.variant, deployment, world, M_total, worker_offset)
     K, W = args.steps, args.warmup
-    log_ids = torch.full((K, w.K), -1, dtype=torch.int32, device=device)
-    log_n = torch.zeros((K, 1), dtype=torch.int32, device=device)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-
-    for _ in range(W):
-        job.step()
-    status = job.ctx.cocodc_poll_status()
-    if status != 0:
-        raise RuntimeError(f"device status after warm-up: {job.B.status_string(status)}")
 
     def barrier():
         torch.cuda.synchronize(device)
@@ -262,60 +402,77 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize(device)
 
-    barrier()
-    launches0 = job.ctx.launch_count
-    with ClockSampler(local) as clocks:
-        t_begin.record()
-        for i in range(K):
-            job.step(log_ids[i], log_n[i], evs[i])
-        t_end.record()
-        barrier()
-    launches = job.ctx.launch_count - launches0
-    status = job.ctx.cocodc_poll_status()
-    if status != 0:
-        raise RuntimeError(f"device status after the timed region: {job.B.status_string(status)}")
-    seconds = t_begin.elapsed_time(t_end) / 1e3
-    ids_h, n_h = log_ids.cpu().numpy(), log_n.cpu().numpy().ravel()
-    per_step = [int(job.sizes[ids_h[i, :n_h[i]]].sum()) for i in range(K)]
-    params_local = float(sum(per_step))
-    outer_ms = [a.elapsed_time(b) for a, b in evs]
-    outer_seconds = sum(outer_ms) / 1e3
-    total_params, max_seconds = aggregate(params_local, seconds, world, backend_ready)
+    leg = timed_device_leg(job, K, W, device, local, barrier)
+    seconds = leg["seconds"]
+    params_local = float(sum(leg["per_step"]))
+    if deployment == "worker_per_device":
+        # every rank completes the same fragments of one replicated model: the job's parameters are one rank's
+        total_params, max_seconds = params_local, aggregate(0.0, seconds, world, backend_ready)[1]
+    else:
+        total_params, max_seconds = aggregate(params_local, seconds, world, backend_ready)
+    same_selection = None
+    if backend_ready and deployment != "replicas":
+        # the decision is replicated, not communicated: every rank must have listed the same fragments
+        import torch.distributed as dist
+        mine = torch.from_numpy(np.concatenate([leg["ids"].ravel(), leg["n"]])).to(device)
+        gathered = [torch.empty_like(mine) for _ in range(world)]
+        dist.all_gather(gathered, mine)
+        same_selection = all(bool(torch.equal(g, gathered[0])) for g in gathered)
+        if not same_selection:
+            raise RuntimeError("the ranks selected different fragments")
 
     peak, peak_kind = read_peaks()
-    bpp = bytes_per_param(w.M) if args.variant != "diloco" else 8 * w.M + 16   # zero delay: one read of w_now
     snap_bpp = 8 * w.M if args.variant != "diloco" else 0
-    achieved = params_local * bpp / outer_seconds / 1e9
-    per_launch_gbs = sorted(per_step[i] * bpp / outer_ms[i] / 1e6 for i in range(K) if outer_ms[i] > 0)
-    traffic = read_traffic_note(w, params_local / K) if args.variant != "diloco" else None
+    traffic = (read_traffic_note(w, params_local / K)
+               if args.variant == "cocodc" and deployment in ("replicas", "param_shard") else None)
+    roof = roofline_record(w, args.variant, deployment, leg, K, peak, peak_kind, traffic)
+    step_bytes = params_local * roof["bytes_per_param"] + float(sum(leg["per_step_snapshot"])) * snap_bpp
+    if deployment == "worker_per_device":
+        step_bytes += params_local * (4 * w.M + 8)       # the pseudo-gradient sum's own pass
+    steps_desc = {
+        "replicas": "outer_step(S1-S6) + select(S7) + snapshot(S0)",
+        "param_shard": "outer_step(S1-S5 + sums of squares) + all-reduce of K fp64 + scores_from_sumsq(S6) + select(S7) "
+                       "+ snapshot(S0)",
+        "worker_per_device": "pseudo_gradient_sum(S1) + all-reduce of the listed fragments + outer_step_received(S2-S6) "
+                             "+ select(S7) + snapshot(S0)",
+    }
     out = {
         "metric": METRIC, "value": total_params / max_seconds, "unit": UNIT, "n_gpus": world, "steps": K,
-        "warmup": W, "ms_per_step": max_seconds / K * 1e3, "higher_is_better": True, "scaling": "weak",
+        "warmup": W, "ms_per_step": max_seconds / K * 1e3, "higher_is_better": True,
+        "scaling": "strong" if deployment == "worker_per_device" else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": w.name, "N": w.N, "K": w.K, "M": w.M, "tau": w.tau, "H": w.H,
                    "budget": f"{w.budget} {w.budget_kind}", "params_per_step": params_local / K,
-                   "variant": args.variant,
-                   "step": ("outer_step(S1-S6) + select(S7) + snapshot(S0)" if args.variant != "diloco"
+                   "variant": args.variant, "deployment": deployment,
+                   "step": (steps_desc[deployment] if args.variant != "diloco"
                             else "outer_step(S1-S6) over all fragments, blocking"), "snapshot_layout": "pool",
-                   "l2": "inputs larger than L2 (every step streams GBs)", "parallelism": f"replicas x{world}"},
-        "gpu_launches": int(launches),
-        "clocks": clocks.result,
-        "roofline": {"bound": "hbm", "kernel": (f"{'k_outer_inplace' if args.variant == 'diloco' else 'k_outer_tma'}<{w.M}> (fused S1-S6)"
-                                               if w.M <= 8 else "k_outer_ring (fused S1-S6)"), "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
-                     "frac_of_nominal_8TBs": achieved / 8000.0, "bytes_per_param": bpp,
-                     "ms_per_launch": outer_seconds / K * 1e3,
-                     "achieved_median": per_launch_gbs[len(per_launch_gbs) // 2] if per_launch_gbs else None,
-                     "achieved_best": per_launch_gbs[-1] if per_launch_gbs else None,
-                     "launches_timed": len(per_launch_gbs), "traffic": traffic},
-        "step_gbs": (params_local * (bpp + snap_bpp)) / seconds / 1e9,
+                   "l2": "inputs larger than L2 (every step streams GBs)",
+                   "parallelism": {"replicas": f"replicas x{world}",
+                                   "param_shard": f"parameter ranges x{world} (model of {world} x N parameters)",
+                                   "worker_per_device": f"{M_total} workers over {world} devices, "
+                                                        f"{w.M} per device"}[deployment]},
+        "gpu_launches": int(leg["launches"]),
+        "clocks": leg["clocks"],
+        "roofline": roof,
+        "step_gbs": step_bytes / seconds / 1e9,
     }
-    if rank == 0 and not args.no_e2e and args.variant == "cocodc":
+    if deployment != "replicas":
+        out["collective"] = {"bytes_per_step_per_rank": leg["collective_bytes"] / K,
+                             "what": ("K fp64 sums of squares" if deployment == "param_shard"
+                                      else "fp32 pseudo-gradient sums of the listed fragments"),
+                             "nvlink_bytes_per_step_per_rank": (2.0 * (world - 1) / world * leg["collective_bytes"] / K),
+                             "same_selection_on_every_rank": same_selection}
+    if rank == 0 and not args.no_e2e and args.variant == "cocodc" and deployment == "replicas":
         out["e2e"] = run_e2e(job, args)
     elif rank == 0:
         out["e2e"] = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(job, per_step[-1] if per_step else 0, args)
+        out["cpu_baseline"] = cpu_baseline(job, leg["per_step"][-1] if leg["per_step"] else 0, args)
+    if (rank == 0 and world == 1 and args.workload == DEFAULT_WORKLOAD and args.variant == "cocodc"
+            and deployment == "replicas" and not args.no_3b):
+        job.ctx.close()
+        del job
+        out["roofline_llama_3b"] = second_shape_roofline("llama_3b", args, device, local, peak, peak_kind)
     if rank == 0:
         print(json.dumps(out))
     if backend_ready:
@@ -324,48 +481,78 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def second_shape_roofline(name: str, args, device, local, peak, peak_kind):
+    """The other shape the bandwidth target names, device-resident only (no host leg: its trainer state would need
+    about 80 GB of pinned host memory): the same step on llama_3b, timed the same way."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 115 * 2 ** 30:
+        return {"workload": name, "skipped": f"needs about 105 GB of device memory, {free / 2 ** 30:.0f} GB free"}
+    w = synth.get_workload(name)
+    job = DeviceJob(w, device, "cocodc")
+    K = max(4, min(args.steps, 20))
+    leg = timed_device_leg(job, K, 3, device, local, lambda: torch.cuda.synchronize(device))
+    roof = roofline_record(w, "cocodc", "replicas", leg, K, peak, peak_kind,
+                           read_traffic_note(w, float(sum(leg["per_step"])) / K))
+    roof.update({"workload": name, "steps": K, "ms_per_step": leg["seconds"] / K * 1e3,
+                 "params_per_s": float(sum(leg["per_step"])) / leg["seconds"],
+                 "clocks": leg["clocks"], "gpu_launches": int(leg["launches"])})
+    job.ctx.close()
+    del job
+    gc.collect()
+    torch.cuda.empty_cache()
+    return roof
+
+
 def run_sweep(args):
     """Compensation sweep at the 1B shape: tau x lambda x fraction of the 32 fragments completing per call.
 
-    Timing only (parity of the same variants is a test): per variant a few launches of cocodc_outer_step over
-    the first n fragments, fused-kernel GB/s from CUDA events.  Prints one JSON line with all variants."""
+    Per variant, from one run: agreement with the CPU oracle (sampled elements of every completed fragment on a
+    checked launch: worst relative error, which must stay within 1e-6) and the fused kernel's GB/s from CUDA
+    events over a few more launches.  The oracle here is the checker of the sweep's "oracle agreement" column,
+    as in the tests; it takes no part in what is timed.  Prints one JSON line with all variants."""
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
-    from paper_2504_17672_b200 import binding as B
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import helpers                                   # the parity tests' sampled check (oracle on sampled elements)
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)
-    w = synth.get_workload("sweep_1b")
-    bufs = synth.generate(w, device)
-    ptr, off, ln = w.partition.csr()
-    ctx = B.Context(w.N, ptr, off, ln, w.M, device=0)
-    K = w.K
-    scores = torch.full((K,), float("inf"), dtype=torch.float32, device=device)
-    norms = torch.zeros(K, dtype=torch.float32, device=device)
-    last_sync = torch.zeros(K, dtype=torch.int64, device=device)
-    ids = torch.arange(K, dtype=torch.int32, device=device)
-    n_ids = torch.zeros(1, dtype=torch.int32, device=device)
-    frag = int(w.partition.frag_sizes[0])
+    w0 = synth.get_workload("sweep_1b")
+    bufs = synth.generate(w0, device)
+    prob = helpers.GpuProblem(w0, bufs, device="cuda:0")
+    ctx, B = prob.ctx, prob.B
+    K = w0.K
+    frag = int(w0.partition.frag_sizes[0])
     peak, peak_kind = read_peaks()
-    bpp = bytes_per_param(w.M)
+    bpp = bytes_per_param(w0.M)
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     variants = []
     reps = max(3, args.steps // 4)
     t = 0
     for frac in (0.25, 0.5, 1.0):
         n = int(round(frac * K))
-        n_ids.fill_(n)
+        ids = list(range(n))
+        prob.set_ids(ids)
         for tau in (1, 2, 4, 8):
             for lam in (0.0, 0.25, 0.5, 1.0):
-                hp = B.Hyper(M=w.M, H=w.H, tau=tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=lam, alpha=w.alpha)
+                w = w0.with_(tau=tau, lam=lam)
+                prob.w = w
+                hp = prob.hyper()
+                # fresh outer state per variant (repeated completions of the same snapshots cancel Delta away)
+                bufs.momentum.normal_(0.0, 1e-3)
+                bufs.theta_g.add_(bufs.momentum)
+                bufs.momentum.normal_(0.0, 1e-3)
 
                 def launch():
                     nonlocal t
                     t += tau
-                    ctx.cocodc_outer_step(hp, bufs.w_now, bufs.w_snap, bufs.now_stride, bufs.snap_stride, None,
-                                          bufs.theta_g, bufs.momentum, None, ids, n_ids, t, t + tau, last_sync,
-                                          norms, scores)
+                    prob.outer_step(t, t + tau, hyper=hp)
+                check = helpers.SampledCheck(prob, ids, seed=len(variants), n_random=20_000)
                 launch()
                 torch.cuda.synchronize(device)
+                parity_worst = check.check(t, t + tau, helpers.orc_hyper(w))    # raises beyond 1e-6
                 a.record()
                 for _ in range(reps):
                     launch()
@@ -374,12 +561,16 @@ def run_sweep(args):
                 ms = a.elapsed_time(b) / reps
                 gbs = n * frag * bpp / ms / 1e6
                 variants.append({"tau": tau, "lambda": lam, "fraction": frac, "fragments": n, "ms": ms,
-                                 "gbs": gbs, "frac_of_peak": gbs / peak})
+                                 "gbs": gbs, "frac_of_peak": gbs / peak, "parity_worst": parity_worst,
+                                 "parity_ok": bool(parity_worst <= helpers.TOL_PARAM)})
     status = ctx.cocodc_poll_status()
     g = [v["gbs"] for v in variants]
-    print(json.dumps({"metric": "outer_step_gbs_per_variant", "workload": w.name, "unit": "GB/s", "peak": peak,
+    print(json.dumps({"metric": "outer_step_gbs_per_variant", "workload": w0.name, "unit": "GB/s", "peak": peak,
                       "peak_kind": f"of {peak_kind}", "launches_per_variant": reps, "status": int(status),
-                      "min": min(g), "median": statistics.median(g), "max": max(g), "variants": variants}))
+                      "min": min(g), "median": statistics.median(g), "max": max(g),
+                      "parity_tolerance": helpers.TOL_PARAM, "parity_worst": max(v["parity_worst"] for v in variants),
+                      "parity_checked": "sampled elements of every completed fragment, first launch of each variant",
+                      "variants": variants}))
 
 
 def run_micro(args):
@@ -595,6 +786,39 @@ def read_traffic_note(w, params_per_launch: float):
 # end to end: parameters in pinned host memory, through the host-buffer entry points
 # --------------------------------------------------------------------------------------------
 
+def measure_pcie(dev, gib: float = 1.0, reps: int = 3):
+    """Rate of plain pinned copies on this machine with both directions busy at once (GB/s each way): 1 GiB host to
+    device and 1 GiB device to host on two streams, CUDA events per stream, best of `reps`."""
+    n = int(gib * 2 ** 30) // 4
+    try:
+        h_in = torch.empty(n, dtype=torch.float32, pin_memory=True)
+        h_out = torch.empty(n, dtype=torch.float32, pin_memory=True)
+    except RuntimeError:
+        return None, None
+    h_in.fill_(1.0)
+    d_in = torch.empty(n, dtype=torch.float32, device=dev)
+    d_out = torch.ones(n, dtype=torch.float32, device=dev)
+    s1, s2 = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
+    best_h2d = best_d2h = 0.0
+    for _ in range(reps + 1):
+        torch.cuda.synchronize(dev)
+        a1, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a2, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(s1):
+            a1.record()
+            d_in.copy_(h_in, non_blocking=True)
+            b1.record()
+        with torch.cuda.stream(s2):
+            a2.record()
+            h_out.copy_(d_out, non_blocking=True)
+            b2.record()
+        torch.cuda.synchronize(dev)
+        best_h2d = max(best_h2d, n * 4 / a1.elapsed_time(b1) / 1e6)
+        best_d2h = max(best_d2h, n * 4 / a2.elapsed_time(b2) / 1e6)
+    del h_in, h_out, d_in, d_out
+    return best_h2d, best_d2h
+
+
 def run_e2e(job: DeviceJob, args):
     """Same step with the trainer's state (w_now, theta_g, momentum, schedule arrays) in pinned host memory.
 
@@ -659,6 +883,14 @@ def run_e2e(job: DeviceJob, args):
            "api": "cocodc_outer_step_host + cocodc_select_fragments + cocodc_snapshot_host",
            "host_memory": "pinned", "status": int(status)}
     del host, ws
+    # what the bus of this box gives plain pinned copies, both directions busy: the ceiling of the figure above
+    pcie_h2d, pcie_d2h = measure_pcie(dev)
+    if pcie_h2d:
+        res["pcie_h2d_gbs"] = pcie_h2d
+        res["pcie_d2h_gbs"] = pcie_d2h
+        res["h2d_gbs"] = res["h2d_bytes_per_step"] / res["ms_per_step"] / 1e6
+        res["d2h_gbs"] = res["d2h_bytes_per_step"] / res["ms_per_step"] / 1e6
+        res["frac_of_pcie"] = res["h2d_gbs"] / pcie_h2d
     return res
 
 
@@ -741,6 +973,48 @@ def run_reference(args):
     }))
 
 
+def launch_ranks(n: int, argv, extra_env=None) -> int:
+    """Start n ranks of this script on this node (one per GPU) under torch.distributed.run and wait for them.
+
+    Used when the script is started plainly with --gpus n > 1; a launcher that has already set RANK / WORLD_SIZE
+    (the usual `python -m torch.distributed.run ... bench.py --gpus n`) makes every process a rank directly."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    env = dict(os.environ)
+    env.update(extra_env or {})
+    return subprocess.run(cmd, env=env).returncode
+
+
+def run_stub(args):
+    """The multi-rank skeleton of the benchmark without a GPU: process group (gloo), barrier, a timed loop of a
+    stand-in step, units summed and seconds maximised over the ranks, one JSON line from rank 0.  It exists so
+    that the launch path and the reduction can be exercised on a machine without CUDA devices."""
+    import torch.distributed as dist
+    rank, world, _ = dist_env()
+    if world > 1:
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+    x = torch.ones(1000)
+    units = 0.0
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        x = x * 1.0001
+        units += 1000.0 * (rank + 1)
+    seconds = time.perf_counter() - t0
+    total, max_seconds = aggregate(units, seconds, world, world > 1)
+    if rank == 0:
+        print(json.dumps({"metric": "stub_units_per_s", "value": total / max_seconds, "unit": "units/s",
+                          "n_gpus": world, "steps": args.steps, "units": total, "impl": "stub"}))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -748,8 +1022,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=list(synth.WORKLOAD_NAMES), default=DEFAULT_WORKLOAD)
+    ap.add_argument("--deployment", choices=["replicas", "param_shard", "worker_per_device"], default=None,
+                    help="how the path is spread over the GPUs (default: replicas on one GPU, param_shard on several)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-3b", action="store_true", help="skip the device-only roofline record on llama_3b")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="wall time spent timing the oracle")
     ap.add_argument("--cpu-sample", type=int, default=16_000_000, help="parameters in the oracle's sample")
@@ -762,11 +1039,19 @@ def main():
                          "sum for M = 1..34 workers")
     ap.add_argument("--workers-fragment", type=int, default=24 * 1024 * 1024,
                     help="parameters per fragment (of 4) in the --workers shape")
-    ap.add_argument("--sweep", action="store_true", help="time the 48 variants of the 1B compensation sweep")
+    ap.add_argument("--sweep", action="store_true",
+                    help="the 48 variants of the 1B compensation sweep: GB/s and agreement with the oracle per variant")
+    ap.add_argument("--stub-step", action="store_true",
+                    help="run the multi-rank skeleton with a CPU stand-in step over gloo (launch-path check, no GPU)")
     args = ap.parse_args()
+    if args.gpus > 1 and "RANK" not in os.environ:
+        # started plainly: become the launcher of --gpus ranks
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
-    if args.impl == "reference":
+    if args.stub_step:
+        run_stub(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.sweep:
         run_sweep(args)

@@ -88,7 +88,7 @@ def _scatter(dst_row: torch.Tensor, segments, vec: torch.Tensor) -> None:
 def generate(w: Workload, device="cpu", *, snap_layout: str = "full",
              pool_ids: Optional[Sequence[int]] = None, pool_len: Optional[int] = None,
              pool_offsets: Optional[Dict[int, int]] = None,
-             momentum_sigma: float = 0.0) -> DeviceBuffers:
+             momentum_sigma: float = 0.0, worker_offset: int = 0) -> DeviceBuffers:
     """Fill the buffers of one workload.
 
     snap_layout="full": w_snap is [M, N] laid out like w_now.
@@ -96,6 +96,8 @@ def generate(w: Workload, device="cpu", *, snap_layout: str = "full",
     get a snapshot, packed back to back (segments of a fragment concatenated)
     in the order given, each start rounded up to a multiple of 4 elements
     unless `pool_offsets` places them explicitly.
+    worker_offset: the M workers generated here are workers worker_offset .. worker_offset + M - 1 of a larger
+    job (the workers of one device when they are spread over several); the global state does not depend on it.
     """
     device = torch.device(device)
     part = w.partition
@@ -146,14 +148,14 @@ def generate(w: Workload, device="cpu", *, snap_layout: str = "full",
             _scatter(momentum, segs, _randn(n, device, _seed(w.seed, _BUF_MOM, p, 0)).mul_(momentum_sigma))
         e = _randn(n, device, _seed(w.seed, _BUF_SHARED, p, 0)).mul_(w.sigma_drift)
         for m in range(M):
-            snap = _randn(n, device, _seed(w.seed, _BUF_SNAP, p, m)).mul_(s).add_(tg)
+            snap = _randn(n, device, _seed(w.seed, _BUF_SNAP, p, m + worker_offset)).mul_(s).add_(tg)
             if p in in_pool:
                 if snap_offset is None:
                     _scatter(w_snap[m], segs, snap)
                 else:
                     o = int(snap_offset[p])
                     w_snap[m, o:o + n] = snap
-            eps = _randn(n, device, _seed(w.seed, _BUF_WORKER, p, m)).mul_(0.1 * w.sigma_drift)
+            eps = _randn(n, device, _seed(w.seed, _BUF_WORKER, p, m + worker_offset)).mul_(0.1 * w.sigma_drift)
             eps.add_(e).mul_(s / w.sigma_drift).add_(snap)
             _scatter(w_now[m], segs, eps)
             del snap, eps

@@ -136,3 +136,28 @@ def test_peer_glue_orders_sum_barrier_step_barrier():
     assert [x[0] for x in log] == ["sum", "barrier", "step", "barrier"]
     assert log[0][1] == "rank1-buffer" and log[0][2] == 2
     assert log[2][1] == bufs and log[2][2:] == (6, 4, 7)
+
+
+def _run_bench(*argv, timeout=300):
+    import subprocess
+    return subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), *argv], capture_output=True, text=True,
+                          timeout=timeout)
+
+
+def test_gpus_flag_launches_that_many_ranks():
+    """`python bench.py --gpus 2` started plainly launches two ranks itself; with the CPU stand-in step the whole
+    launch path (launcher, process group, barrier, reduction, rank 0's line) runs here over gloo."""
+    import json
+    r = _run_bench("--gpus", "2", "--stub-step", "--steps", "4")
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["units"] == 4 * 1000.0 * (1 + 2)
+
+
+def test_gpus_flag_reaches_the_device_check_in_every_rank():
+    """Without CUDA devices the real benchmark must fail loudly in BOTH ranks (no rank silently runs elsewhere)."""
+    if torch.cuda.is_available():
+        pytest.skip("this box has a GPU")
+    r = _run_bench("--gpus", "2", "--steps", "1", "--no-e2e", "--no-cpu-baseline")
+    assert r.returncode != 0
+    assert "rank 0: no CUDA device" in r.stderr and "rank 1: no CUDA device" in r.stderr
