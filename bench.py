@@ -177,8 +177,10 @@ class DeviceJob:
         self.norms = torch.zeros(K, dtype=torch.float32, device=device)
         self.last_sync = torch.zeros(K, dtype=torch.int64, device=device)
         self.mask = torch.zeros(K, dtype=torch.uint8, device=device)
-        self.ids = torch.full((K,), -1, dtype=torch.int32, device=device)
-        self.n_ids = torch.zeros(1, dtype=torch.int32, device=device)
+        # id list and its length share one buffer, so that the benchmark's per-step log is a single copy
+        self.idbuf = torch.full((K + 1,), -1, dtype=torch.int32, device=device)
+        self.ids, self.n_ids = self.idbuf[:K], self.idbuf[K:]
+        self.n_ids.zero_()
         self.pool_off = torch.full((K,), -1, dtype=torch.int64, device=device)
         self.t = w.tau
         self.hyper = B.Hyper(M=w.M, H=w.H, tau=w.tau, outer_lr=w.outer_lr, momentum=w.momentum, lam=w.lam,
@@ -267,7 +269,7 @@ class DeviceJob:
         self.ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off, self.w.M,
                                  self.ids, self.n_ids)
 
-    def step(self, log_ids=None, log_n=None, ev=None, log_next=None, log_next_n=None):
+    def step(self, log=None, ev=None):
         """Complete the fragments in flight, choose the next set, record their snapshots."""
         if self.deployment == "worker_per_device":
             self.pseudo_sum_and_exchange()
@@ -278,28 +280,21 @@ class DeviceJob:
             ev[1].record()
         if self.deployment == "param_shard":
             self.scores_param_shard()
-        if log_ids is not None:
-            log_ids.copy_(self.ids)
-            log_n.copy_(self.n_ids)
+        if log is not None:
+            log.copy_(self.idbuf)
         if self.variant == "diloco":
             self.t += self.w.H
             return
         self.t += self.w.tau
         self.select()
         self.snapshot()
-        if log_next is not None:         # the set whose snapshot was just taken
-            log_next.copy_(self.ids)
-            log_next_n.copy_(self.n_ids)
 
 
 def timed_device_leg(job: DeviceJob, K: int, W: int, device: torch.device, local: int, barrier):
     """W warm-up steps, then exactly K timed steps between two barriers; CUDA events around the whole region and
     around every completion call.  Returns the raw figures of this rank."""
     w = job.w
-    log_ids = torch.full((K, w.K), -1, dtype=torch.int32, device=device)
-    log_n = torch.zeros((K, 1), dtype=torch.int32, device=device)
-    next_ids = torch.full((K, w.K), -1, dtype=torch.int32, device=device)
-    next_n = torch.zeros((K, 1), dtype=torch.int32, device=device)
+    log = torch.full((K, w.K + 1), -1, dtype=torch.int32, device=device)     # per step: the completed ids, their count
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for _ in range(W):
@@ -313,18 +308,24 @@ def timed_device_leg(job: DeviceJob, K: int, W: int, device: torch.device, local
     with ClockSampler(local) as clocks:
         t_begin.record()
         for i in range(K):
-            job.step(log_ids[i], log_n[i], evs[i], next_ids[i], next_n[i])
+            job.step(log[i], evs[i])
         t_end.record()
         barrier()
     status = job.ctx.cocodc_poll_status()
     if status != 0:
         raise RuntimeError(f"device status after the timed region: {job.B.status_string(status)}")
-    ids_h, n_h = log_ids.cpu().numpy(), log_n.cpu().numpy().ravel()
-    nx_h, nn_h = next_ids.cpu().numpy(), next_n.cpu().numpy().ravel()
+    log_h = log.cpu().numpy()
+    ids_h, n_h = log_h[:, :w.K], log_h[:, w.K]
+    per_step = [int(job.sizes[ids_h[i, :n_h[i]]].sum()) for i in range(K)]
+    # the set whose snapshot step i takes is the set step i + 1 completes; the last one is still in the job
+    last = job.idbuf.cpu().numpy()
+    per_step_snapshot = per_step[1:] + [int(job.sizes[last[:last[w.K]]].sum())]
+    if job.variant == "diloco":
+        per_step_snapshot = [0] * K
     return {
         "seconds": t_begin.elapsed_time(t_end) / 1e3,
-        "per_step": [int(job.sizes[ids_h[i, :n_h[i]]].sum()) for i in range(K)],
-        "per_step_snapshot": [int(job.sizes[nx_h[i, :nn_h[i]]].sum()) for i in range(K)],
+        "per_step": per_step,
+        "per_step_snapshot": per_step_snapshot,
         "outer_ms": [a.elapsed_time(b) for a, b in evs],
         "launches": job.ctx.launch_count - launches0,
         "collective_bytes": job.collective_bytes - bytes0,

@@ -376,15 +376,10 @@ k_outer_generic(const __grid_constant__ OuterArgs A, const __grid_constant__ Fra
 // ---------------------------------------------------------------------------
 // S6 stand-alone: sums of squares of an N-sized vector over the planned tiles.
 // ---------------------------------------------------------------------------
+// The accumulation loop, out of line (its registers then do not depend on the prologue and epilogue around it).
 template <int U>
-__global__ void __launch_bounds__(kThreads, 8)     // 8 CTAs per SM: the loop needs few registers, the prologue may spill
-k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ gplan, const PlanHeader* __restrict__ ghdr,
-        const __grid_constant__ PlanRequest rq, const __grid_constant__ Finalize fin,
-        double* __restrict__ partial, int* __restrict__ status, const __grid_constant__ FragTable T) {
-  __shared__ InlinePlan ip;
-  const PlanView pv = acquire_plan(ip, T, rq, gplan, ghdr, status);
-  const PlanHeader h = pv.hdr;
-  const SegPlan* plan = pv.seg;
+static __device__ __noinline__ void sumsq_tiles(const float* __restrict__ x, const SegPlan* plan, const PlanHeader h,
+                                                double* __restrict__ partial) {
   constexpr int LPT = kThreads * U;
   SlotAccumulator sa(kThreads / 32);
   int seg = 0, seg_loaded = -1;
@@ -418,7 +413,17 @@ k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ gplan, const Pl
     }
   }
   sa.finish(h.n_ids, partial);
-  finalize_epilogue_cta(ip, fin, h, partial, kThreads / 32, status);
+}
+
+template <int U>
+__global__ void __launch_bounds__(kThreads)
+k_sumsq(const float* __restrict__ x, const SegPlan* __restrict__ gplan, const PlanHeader* __restrict__ ghdr,
+        const __grid_constant__ PlanRequest rq, const __grid_constant__ Finalize fin,
+        double* __restrict__ partial, int* __restrict__ status, const __grid_constant__ FragTable T) {
+  __shared__ InlinePlan ip;
+  const PlanView pv = acquire_plan(ip, T, rq, gplan, ghdr, status);
+  sumsq_tiles<U>(x, pv.seg, pv.hdr, partial);
+  finalize_epilogue_cta(ip, fin, pv.hdr, partial, kThreads / 32, status);
 }
 
 }  // namespace cocodc

@@ -134,92 +134,89 @@ struct StageLayout {
   static_assert(kLoaded + (MODE == MODE_FUSED_RECV ? kMaxRecv : 0) <= 32, "one lane of the producer warp per stream");
 };
 
-template <int M, int MODE, bool SAME, int U = 1>
-__global__ void __launch_bounds__(tma_threads(M), 1)
-k_outer_tma(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTable T) {
+// The two roles of k_outer_tma are compiled as functions of their own (out of line): what the compiler makes
+// of the streaming loops then does not depend on the prologue and epilogue code around them (measured: the
+// same loops inlined next to that code ran up to 1 % slower, depending on what exactly stood beside them).
+struct TmaShared {
+  float* stages;
+  unsigned long long* full_bar;
+  unsigned long long* empty_bar;
+  volatile int* s_fail;
+};
+
+// Lane l of the producer warp owns stream l of the stage (slot order: recorded values, current values, global
+// state, momentum, received sums): it keeps that stream's base pointer in registers and issues the stream's
+// one bulk copy per tile.  The lanes' copies leave with one warp instruction instead of one instruction
+// sequence per stream (a single issuing thread needed a few hundred cycles per copy, and with only two or
+// three stages the time from "stage free" to "last copy issued" sits on the pipeline's critical path).  Lane 0
+// arms the barrier with the whole byte count; a copy that completes before the arming arrival only runs the
+// transaction count negative for a moment, the phase cannot end before that arrival.
+template <int M, int MODE, bool SAME, int U>
+__device__ __noinline__ void tma_producer_warp(const OuterArgs& A, const SegPlan* plan, const PlanHeader h,
+                                               const TmaShared sh) {
   using L = StageLayout<M, MODE, SAME, U>;
-  constexpr int kSlot = U * kTileElems;                         // elements of one stream in a stage
+  constexpr int kSlot = U * kTileElems;
   constexpr unsigned kSlotBytes = U * kTileBytes;
   constexpr bool kRecv = (MODE == MODE_FUSED_RECV);
   const int n_recv = kRecv ? A.n_recv : 0;
-  const int loaded = L::kLoaded + n_recv;                       // streams per stage
-  const int S = kRecv ? stages_for(loaded) : L::kStages;        // a compile-time constant unless kRecv
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  float* const stages = reinterpret_cast<float*>(smem_raw);
-  __shared__ __align__(8) unsigned long long full_bar[kMaxStages];
-  __shared__ __align__(8) unsigned long long empty_bar[kMaxStages];
-  __shared__ volatile int s_fail;
-  __shared__ InlinePlan ip;
-
-  const int tid = threadIdx.x;
-  const PlanView pv = acquire_plan(ip, T, A.rq, A.plan, A.hdr, A.status);
-  const PlanHeader h = pv.hdr;
-  if (tid == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(smem_u32(&full_bar[s]), 1);
-      mbar_init(smem_u32(&empty_bar[s]), kThreads);   // every consumer thread releases its own lane
-    }
-    s_fail = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  const int loaded = L::kLoaded + n_recv;
+  const int S = kRecv ? stages_for(loaded) : L::kStages;
+  const int lane = threadIdx.x & 31;
+  const bool has_stream = lane < loaded;
+  const bool from_snap = lane < L::nS;
+  const float* base = nullptr;
+  if (has_stream) {
+    if (lane < L::nS) base = A.w_snap + (long long)lane * A.snap_stride;
+    else if (lane < L::nS + L::nN) base = A.w_now + (long long)(lane - L::nS) * A.now_stride;
+    else if (lane == L::kGlobal) base = A.theta_g;
+    else if (L::nU && lane == L::kMomentum) base = A.momentum;
+    else base = A.delta_in[lane - L::kDeltaIn];
   }
-  __syncthreads();
-
-  // ------------------------------------------------------------------ producer warp
-  // Lane l of the producer warp owns stream l of the stage (slot order: recorded values, current values, global
-  // state, momentum, received sums): it keeps that stream's base pointer in registers and issues the stream's
-  // one bulk copy per tile.  The lanes' copies leave with one warp instruction instead of one instruction
-  // sequence per stream (a single issuing thread needed a few hundred cycles per copy, and with only two or
-  // three stages the time from "stage free" to "last copy issued" sits on the pipeline's critical path).  Lane 0
-  // arms the barrier with the whole byte count; a copy that completes before the arming arrival only runs the
-  // transaction count negative for a moment, the phase cannot end before that arrival.
-  if (tid >= kThreads) {
-    const int lane = tid & 31;
-    const bool has_stream = lane < loaded;
-    const bool from_snap = lane < L::nS;
-    const float* base = nullptr;
+  TileWalker tw(plan, h.n_seg, kSlot);
+  int k = 0;   // staged tiles issued so far
+  // Leaving early (a wait ran out here or in a consumer): the copies already issued may still be landing in
+  // this CTA's shared memory, which must not be handed to another CTA before they have; wait for the stages
+  // armed last, again with a limit.
+  auto drain = [&]() {
+    for (int i = (k > S ? k - S : 0); i < k; ++i) mbar_wait_bounded(smem_u32(&sh.full_bar[i % S]), (i / S) & 1);
+  };
+  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+    tw.seek(tile);
+    const long long e0 = tw.tile_start(tile);
+    if (!tw.interior(e0)) continue;
+    const int s = k % S;
+    const bool free_now = (k < S) || mbar_wait_bounded(smem_u32(&sh.empty_bar[s]), ((k / S) - 1) & 1);
+    if (!__all_sync(0xffffffffu, free_now && !*sh.s_fail)) {      // one verdict for the warp
+      if (!free_now) record_status(A.status, A.err_timeout);
+      *sh.s_fail = 1;
+      drain();
+      return;
+    }
+    const unsigned bar = smem_u32(&sh.full_bar[s]);
+    if (lane == 0) mbar_expect_tx(bar, loaded * kSlotBytes);
     if (has_stream) {
-      if (lane < L::nS) base = A.w_snap + (long long)lane * A.snap_stride;
-      else if (lane < L::nS + L::nN) base = A.w_now + (long long)(lane - L::nS) * A.now_stride;
-      else if (lane == L::kGlobal) base = A.theta_g;
-      else if (L::nU && lane == L::kMomentum) base = A.momentum;
-      else base = A.delta_in[lane - L::kDeltaIn];
+      const long long e_src = from_snap ? e0 + (tw.sp.snap_off - tw.sp.off) : e0;
+      bulk_load(smem_u32(sh.stages + ((size_t)s * loaded + lane) * kSlot), base + e_src, kSlotBytes, bar);
     }
-    TileWalker tw(pv.seg, h.n_seg, kSlot);
-    int k = 0;   // staged tiles issued so far
-    // Leaving early (a wait ran out here or in a consumer): the copies already issued may still be landing in
-    // this CTA's shared memory, which must not be handed to another CTA before they have; wait for the stages
-    // armed last, again with a limit.
-    auto drain = [&]() {
-      for (int i = (k > S ? k - S : 0); i < k; ++i) mbar_wait_bounded(smem_u32(&full_bar[i % S]), (i / S) & 1);
-    };
-    for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
-      tw.seek(tile);
-      const long long e0 = tw.tile_start(tile);
-      if (!tw.interior(e0)) continue;
-      const int s = k % S;
-      const bool free_now = (k < S) || mbar_wait_bounded(smem_u32(&empty_bar[s]), ((k / S) - 1) & 1);
-      if (!__all_sync(0xffffffffu, free_now && !s_fail)) {      // one verdict for the warp
-        if (!free_now) record_status(A.status, A.err_timeout);
-        s_fail = 1;
-        drain();
-        return;
-      }
-      const unsigned bar = smem_u32(&full_bar[s]);
-      if (lane == 0) mbar_expect_tx(bar, loaded * kSlotBytes);
-      if (has_stream) {
-        const long long e_src = from_snap ? e0 + (tw.sp.snap_off - tw.sp.off) : e0;
-        bulk_load(smem_u32(stages + ((size_t)s * loaded + lane) * kSlot), base + e_src, kSlotBytes, bar);
-      }
-      ++k;
-    }
-    return;
+    ++k;
   }
+}
 
-  // ------------------------------------------------------------------ consumers
+// The eight consumer warps: returns false if a wait ran out (warp-uniform), after writing this warp's partial
+// sums otherwise.
+template <int M, int MODE, bool SAME, int U>
+__device__ __noinline__ bool tma_consumer_warps(const OuterArgs& A, const SegPlan* plan, const PlanHeader h,
+                                                const TmaShared sh) {
+  using L = StageLayout<M, MODE, SAME, U>;
+  constexpr int kSlot = U * kTileElems;
+  constexpr bool kRecv = (MODE == MODE_FUSED_RECV);
+  const int n_recv = kRecv ? A.n_recv : 0;
+  const int loaded = L::kLoaded + n_recv;
+  const int S = kRecv ? stages_for(loaded) : L::kStages;
+  const int tid = threadIdx.x;
   SlotAccumulator sa(kThreads / 32);
-  TileWalker tw(pv.seg, h.n_seg, kSlot);
+  TileWalker tw(plan, h.n_seg, kSlot);
   int k = 0;           // staged tiles consumed so far
-  bool failed = false;
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
     if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
     const long long e0 = tw.tile_start(tile);
@@ -230,14 +227,13 @@ k_outer_tma(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTab
     const int s = k % S;
     // the verdict is taken per warp, so that a warp never splits around the full-warp shuffles of the
     // score accumulation
-    const bool landed = !s_fail && mbar_wait_bounded(smem_u32(&full_bar[s]), (k / S) & 1);
+    const bool landed = !*sh.s_fail && mbar_wait_bounded(smem_u32(&sh.full_bar[s]), (k / S) & 1);
     if (!__all_sync(0xffffffffu, landed)) {
       record_status(A.status, A.err_timeout);
-      s_fail = 1;
-      failed = true;
-      break;
+      *sh.s_fail = 1;
+      return false;
     }
-    const float* st = stages + (size_t)s * loaded * kSlot;
+    const float* st = sh.stages + (size_t)s * loaded * kSlot;
     Lane<M, MODE, SAME> ln[U];
 #pragma unroll
     for (int v = 0; v < U; ++v) {
@@ -262,7 +258,7 @@ k_outer_tma(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTab
         }
       }
     }
-    mbar_arrive(smem_u32(&empty_bar[s]));   // this thread's lanes are in registers: its share of the stage is free
+    mbar_arrive(smem_u32(&sh.empty_bar[s]));   // this thread's lanes are in registers: its share of the stage is free
 #pragma unroll
     for (int v = 0; v < U; ++v) {
       ln[v].compute(A, sa.acc);
@@ -270,11 +266,44 @@ k_outer_tma(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTab
     }
     ++k;
   }
-  if (failed) return;     // warp-uniform by construction
-  if (A.partial) {
-    sa.finish(h.n_ids, A.partial);
-    finalize_epilogue(ip, A.fin, h, A.partial, kThreads / 32, A.status);
+  if (A.partial) sa.finish(h.n_ids, A.partial);
+  return true;
+}
+
+template <int M, int MODE, bool SAME, int U = 1>
+__global__ void __launch_bounds__(tma_threads(M), 1)
+k_outer_tma(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTable T) {
+  using L = StageLayout<M, MODE, SAME, U>;
+  constexpr bool kRecv = (MODE == MODE_FUSED_RECV);
+  const int S = kRecv ? stages_for(L::kLoaded + A.n_recv) : L::kStages;   // a compile-time constant unless kRecv
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long full_bar[kMaxStages];
+  __shared__ __align__(8) unsigned long long empty_bar[kMaxStages];
+  __shared__ volatile int s_fail;
+  __shared__ InlinePlan ip;
+
+  const int tid = threadIdx.x;
+  const PlanView pv = acquire_plan(ip, T, A.rq, A.plan, A.hdr, A.status);
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), kThreads);   // every consumer thread releases its own lane
+    }
+    s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  __syncthreads();
+  TmaShared sh;
+  sh.stages = reinterpret_cast<float*>(smem_raw);
+  sh.full_bar = full_bar;
+  sh.empty_bar = empty_bar;
+  sh.s_fail = &s_fail;
+  if (tid >= kThreads) {
+    tma_producer_warp<M, MODE, SAME, U>(A, pv.seg, pv.hdr, sh);
+    return;
+  }
+  if (!tma_consumer_warps<M, MODE, SAME, U>(A, pv.seg, pv.hdr, sh)) return;     // warp-uniform by construction
+  if (A.partial) finalize_epilogue(ip, A.fin, pv.hdr, A.partial, kThreads / 32, A.status);
 }
 
 }  // namespace cocodc
@@ -301,26 +330,25 @@ template <int N> __device__ __forceinline__ void bulk_wait_read_n() {
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
-k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long long now_stride,
-               long long snap_stride, int M, const SegPlan* __restrict__ gplan,
-               const PlanHeader* __restrict__ ghdr, const __grid_constant__ PlanRequest rq,
-               int* __restrict__ status, int err_timeout, const __grid_constant__ FragTable T) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  float* const stages = reinterpret_cast<float*>(smem_raw);
-  __shared__ __align__(8) unsigned long long full_bar[kSnapStages];
-  __shared__ float* dst_of_stage[kSnapStages];
-  __shared__ InlinePlan ip;
-  const PlanView pv = acquire_plan(ip, T, rq, gplan, ghdr, status);
-  const PlanHeader h = pv.hdr;
-  const SegPlan* plan = pv.seg;
-  const int tid = threadIdx.x;
-  if (tid == 0) {
-    for (int s = 0; s < kSnapStages; ++s) mbar_init(smem_u32(&full_bar[s]), 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  __syncthreads();
+struct SnapshotJob {
+  const float* w_now;
+  float* w_snap;
+  long long now_stride, snap_stride;
+  int M;
+  int* status;
+  int err_timeout;
+};
 
+// The copy loops of k_snapshot_tma, out of line for the same reason as the roles of k_outer_tma.
+static __device__ __noinline__ void snapshot_copy(const SnapshotJob J, const SegPlan* plan, const PlanHeader h,
+                                                  float* stages, unsigned long long* full_bar, float** dst_of_stage) {
+  const float* __restrict__ w_now = J.w_now;
+  float* __restrict__ w_snap = J.w_snap;
+  const long long now_stride = J.now_stride, snap_stride = J.snap_stride;
+  const int M = J.M;
+  int* status = J.status;
+  const int err_timeout = J.err_timeout;
+  const int tid = threadIdx.x;
   auto tile_geometry = [&](int tile, int& seg, SegPlan& sp, int& loaded, long long& e0, bool& interior) {
     while (seg + 1 < h.n_seg && tile >= plan[seg + 1].first_tile) ++seg;
     if (seg != loaded) { sp = plan[seg]; loaded = seg; }
@@ -430,6 +458,27 @@ k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long
       }
     }
   }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long long now_stride,
+               long long snap_stride, int M, const SegPlan* __restrict__ gplan,
+               const PlanHeader* __restrict__ ghdr, const __grid_constant__ PlanRequest rq,
+               int* __restrict__ status, int err_timeout, const __grid_constant__ FragTable T) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long full_bar[kSnapStages];
+  __shared__ float* dst_of_stage[kSnapStages];
+  __shared__ InlinePlan ip;
+  const PlanView pv = acquire_plan(ip, T, rq, gplan, ghdr, status);
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kSnapStages; ++s) mbar_init(smem_u32(&full_bar[s]), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  SnapshotJob J;
+  J.w_now = w_now; J.w_snap = w_snap; J.now_stride = now_stride; J.snap_stride = snap_stride; J.M = M;
+  J.status = status; J.err_timeout = err_timeout;
+  snapshot_copy(J, pv.seg, pv.hdr, reinterpret_cast<float*>(smem_raw), full_bar, dst_of_stage);
 }
 
 // ---------------------------------------------------------------------------------------------
