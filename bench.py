@@ -692,7 +692,7 @@ def run_workers(args):
     reps = max(5, args.steps // 5)
     out = []
     status = 0
-    for M in (1, 2, 3, 4, 5, 6, 7, 8, 9, 12, 16, 24, 34):
+    for M in [int(x) for x in args.workers_list.split(",")]:
         w = synth.small_workload([frag] * K, M=M, seed=7, tau=4, name=f"workers_{M}")
         b = synth.generate(w, device)
         ptr, off, ln = w.partition.csr()
@@ -1038,6 +1038,7 @@ def main():
     ap.add_argument("--workers", action="store_true",
                     help="time the fused step, its zero-delay and received-sum forms, the snapshot and the pseudo-gradient "
                          "sum for M = 1..34 workers")
+    ap.add_argument("--workers-list", default="1,2,3,4,5,6,7,8,9,12,16,24,34", help="worker counts of --workers")
     ap.add_argument("--workers-fragment", type=int, default=24 * 1024 * 1024,
                     help="parameters per fragment (of 4) in the --workers shape")
     ap.add_argument("--sweep", action="store_true",
