@@ -491,21 +491,21 @@ k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long
 //              stage, proxy fence, arrive on "done" (one arrival per consumer thread);
 //   storer   : waits on "done", bulk stores of the stage to theta_g, momentum and w_now, waits until they
 //              have read shared memory, arrives on "empty".
-// Loader and storer are two further warps whose lane l moves stream l (one thread doing both jobs measured 6.57
-// against 6.62 TB/s at M = 4).  The ring depth per worker count is measured: inplace_stages().
+// Loader and storer are single threads of two further warps (one thread doing both jobs: 6.57 against 6.62 TB/s
+// at M = 4).  The ring depth per worker count is measured: inplace_stages().
 // ---------------------------------------------------------------------------------------------
 constexpr int kInplaceThreads = kThreads + 64;
 
-// Stages of the in-place ring per worker count (a stage is M + 2 tiles of 4 KB), measured on B200 with 2 to 10
+// Stages of the in-place ring per worker count (a stage is M + 2 tiles of 4 KB), measured on B200 with 2 to 6
 // stages each (GB/s of the zero-delay step, 100 M parameters per worker; the chosen depth first):
-//   M = 1: 6 stages 5773 (5: 5731, 4: 5562, 3: 5018)    M = 5: 3 stages 6473 (4: 6090, 2: 5335)
-//   M = 2: 5 stages 6455 (6: 6457, 4: 6195, 3: 5536)    M = 6: 3 stages 6469 (4: 5998, 2: 5523)
-//   M = 3: 4 stages 6449 (5: 6065, 3: 5906)             M = 7: 3 stages 6334 (4: 5974, 2: 5689)
-//   M = 4: 3 stages 6269 (4: 6195, 5: 5909, 2: 5149)    M = 8: 3 stages 6255 (4: 5953, 2: 5888)
-// Loading, updating and storing each hold a stage, so fewer than three serialise the pipeline; beyond about
-// 80 KB the loads in flight crowd out the stores.
+//   M = 1: 6 stages 6453 (5: 6351, 4: 5943)      M = 5: 3 stages 6369 (4: 6011, 2: 5725)
+//   M = 2: 4 stages 6413 (5: 6168, 3: 5829)      M = 6: 3 stages 6224 (4: 5967, 2: 5915)
+//   M = 3: 4 stages 6282 (3: 6216, 5: 5962)      M = 7: 3 stages 6187 (2: 6080, 4: 5961)
+//   M = 4: 3 stages 6501 (4: 6120, 2: 5521)      M = 8: 2 stages 6292 (3: 6165, 4: 6023)
+// Loading, updating and storing each hold a stage, so fewer than three serialise the pipeline unless a stage is
+// large; beyond about 80 KB the loads in flight crowd out the stores.
 __host__ __device__ constexpr int inplace_stages(int M) {
-  return M == 1 ? 6 : M == 2 ? 5 : M == 3 ? 4 : 3;
+  return M == 1 ? 6 : M <= 3 ? 4 : M <= 7 ? 3 : 2;
 }
 
 template <int M>
@@ -516,105 +516,97 @@ struct InplaceLayout {
   static_assert(kSmemBytes <= 227 * 1024, "stages do not fit in shared memory");
 };
 
-struct InplaceShared {
-  float* stages;
-  unsigned long long* full_bar;
-  unsigned long long* done_bar;
-  unsigned long long* empty_bar;
-  volatile int* s_fail;
-};
-
-// Stream l of an in-place stage (slot order of StageLayout<M, MODE_FUSED, true>: current values of the M workers,
-// global state, momentum) as lane l of the loader and of the storer warp sees it.
 template <int M>
-__device__ __forceinline__ float* inplace_stream_base(const OuterArgs& A, int lane) {
-  using L = typename InplaceLayout<M>::L;
-  if (lane < M) return A.w_now + (long long)lane * A.now_stride;
-  if (lane == L::kGlobal) return A.theta_g;
-  return A.momentum;
-}
-
-// Loader warp: lane l brings in stream l of every staged tile (one warp instruction starts all M + 2 copies).
-template <int M>
-static __device__ __noinline__ void inplace_loader_warp(const OuterArgs& A, const SegPlan* plan, const PlanHeader h,
-                                                        const InplaceShared sh) {
+__global__ void __launch_bounds__(kInplaceThreads, 1)
+k_outer_inplace(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTable T) {
   using IL = InplaceLayout<M>;
   using L = typename IL::L;
   constexpr int S = IL::kStages;
-  const int lane = threadIdx.x & 31;
-  const bool has_stream = lane < L::kLoaded;
-  const float* base = has_stream ? inplace_stream_base<M>(A, lane) : nullptr;
-  TileWalker tw(plan, h.n_seg);
-  int k = 0;   // staged tiles issued so far
-  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
-    tw.seek(tile);
-    const long long e0 = tw.tile_start(tile);
-    if (!tw.interior(e0)) continue;
-    const int s = k % S;
-    const bool free_now = (k < S) || mbar_wait_bounded(smem_u32(&sh.empty_bar[s]), ((k / S) - 1) & 1);
-    if (!__all_sync(0xffffffffu, free_now && !*sh.s_fail)) {
-      if (!free_now) record_status(A.status, A.err_timeout);
-      *sh.s_fail = 1;
-      // the loads already issued must land before this CTA's shared memory can go to another one
-      for (int i = (k > S ? k - S : 0); i < k; ++i) mbar_wait_bounded(smem_u32(&sh.full_bar[i % S]), (i / S) & 1);
-      return;
-    }
-    const unsigned bar = smem_u32(&sh.full_bar[s]);
-    if (lane == 0) mbar_expect_tx(bar, L::kLoaded * kTileBytes);
-    if (has_stream)
-      bulk_load(smem_u32(sh.stages + ((size_t)s * L::kLoaded + lane) * kTileElems), base + e0, kTileBytes, bar);
-    ++k;
-  }
-}
-
-// Storer warp: once the consumers have updated a stage, lane l writes stream l back; every lane waits until its
-// own store has read shared memory, then lane 0 hands the stage back to the loader.
-template <int M>
-static __device__ __noinline__ void inplace_storer_warp(const OuterArgs& A, const SegPlan* plan, const PlanHeader h,
-                                                        const InplaceShared sh) {
-  using IL = InplaceLayout<M>;
-  using L = typename IL::L;
-  constexpr int S = IL::kStages;
-  const int lane = threadIdx.x & 31;
-  const bool has_stream = lane < L::kLoaded;
-  float* base = has_stream ? inplace_stream_base<M>(A, lane) : nullptr;
-  TileWalker tw(plan, h.n_seg);
-  const unsigned long long policy = l2_evict_first_policy();
-  int k = 0;   // staged tiles stored so far
-  for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
-    tw.seek(tile);
-    const long long e0 = tw.tile_start(tile);
-    if (!tw.interior(e0)) continue;
-    const int s = k % S;
-    const bool updated = !*sh.s_fail && mbar_wait_bounded(smem_u32(&sh.done_bar[s]), (k / S) & 1);
-    if (!__all_sync(0xffffffffu, updated)) {
-      record_status(A.status, A.err_timeout);
-      *sh.s_fail = 1;
-      break;
-    }
-    if (has_stream) {
-      bulk_store(base + e0, smem_u32(sh.stages + ((size_t)s * L::kLoaded + lane) * kTileElems), kTileBytes, policy);
-      bulk_commit();
-      bulk_wait_read_n<0>();                  // this lane's store has read the stage
-    }
-    __syncwarp();
-    if (lane == 0) mbar_arrive(smem_u32(&sh.empty_bar[s]));   // all of them have: the stage may be loaded again
-    ++k;
-  }
-  bulk_wait_all();    // shared memory must outlive the last stores (also after a failed wait)
-}
-
-// Consumer warps: update the stage in place.  Returns false if a wait ran out (warp-uniform).
-template <int M>
-static __device__ __noinline__ bool inplace_consumer_warps(const OuterArgs& A, const SegPlan* plan, const PlanHeader h,
-                                                           const InplaceShared sh) {
-  using IL = InplaceLayout<M>;
-  using L = typename IL::L;
-  constexpr int S = IL::kStages;
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  float* const stages = reinterpret_cast<float*>(smem_raw);
+  __shared__ __align__(8) unsigned long long full_bar[S];
+  __shared__ __align__(8) unsigned long long done_bar[S];
+  __shared__ __align__(8) unsigned long long empty_bar[S];
+  __shared__ volatile int s_fail;
+  __shared__ InlinePlan ip;
   const int tid = threadIdx.x;
+  const PlanView pv = acquire_plan(ip, T, A.rq, A.plan, A.hdr, A.status);
+  const PlanHeader h = pv.hdr;
+  if (tid == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&done_bar[s]), kThreads);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    s_fail = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // ------------------------------------------------------------------ loader
+  if (tid == kThreads) {
+    TileWalker tw(pv.seg, h.n_seg);
+    int k = 0;   // staged tiles issued so far
+    for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+      tw.seek(tile);
+      const long long e0 = tw.tile_start(tile);
+      if (!tw.interior(e0)) continue;
+      const int s = k % S;
+      if (k >= S && (s_fail || !mbar_wait_bounded(smem_u32(&empty_bar[s]), ((k / S) - 1) & 1))) {
+        record_status(A.status, A.err_timeout);
+        s_fail = 1;
+        // the loads already issued must land before this CTA's shared memory can go to another one
+        for (int i = (k > S ? k - S : 0); i < k; ++i) mbar_wait_bounded(smem_u32(&full_bar[i % S]), (i / S) & 1);
+        return;
+      }
+      const unsigned bar = smem_u32(&full_bar[s]);
+      float* st = stages + (size_t)s * L::kLoaded * kTileElems;
+      mbar_expect_tx(bar, L::kLoaded * kTileBytes);
+#pragma unroll
+      for (int m = 0; m < M; ++m)
+        bulk_load(smem_u32(st + (L::kNow + m) * kTileElems), A.w_now + m * A.now_stride + e0, kTileBytes, bar);
+      bulk_load(smem_u32(st + L::kGlobal * kTileElems), A.theta_g + e0, kTileBytes, bar);
+      bulk_load(smem_u32(st + L::kMomentum * kTileElems), A.momentum + e0, kTileBytes, bar);
+      ++k;
+    }
+    return;
+  }
+  // ------------------------------------------------------------------ storer
+  if (tid == kThreads + 32) {
+    TileWalker tw(pv.seg, h.n_seg);
+    const unsigned long long policy = l2_evict_first_policy();
+    int k = 0;   // staged tiles stored so far
+    for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
+      tw.seek(tile);
+      const long long e0 = tw.tile_start(tile);
+      if (!tw.interior(e0)) continue;
+      const int s = k % S;
+      if (s_fail || !mbar_wait_bounded(smem_u32(&done_bar[s]), (k / S) & 1)) {
+        record_status(A.status, A.err_timeout);
+        s_fail = 1;
+        break;
+      }
+      const float* st = stages + (size_t)s * L::kLoaded * kTileElems;
+      bulk_store(A.theta_g + e0, smem_u32(st + L::kGlobal * kTileElems), kTileBytes, policy);
+      bulk_store(A.momentum + e0, smem_u32(st + L::kMomentum * kTileElems), kTileBytes, policy);
+#pragma unroll
+      for (int m = 0; m < M; ++m)
+        bulk_store(A.w_now + m * A.now_stride + e0, smem_u32(st + (L::kNow + m) * kTileElems), kTileBytes, policy);
+      bulk_commit();
+      bulk_wait_read_n<0>();                    // the stores have read the stage: it may be loaded again
+      mbar_arrive(smem_u32(&empty_bar[s]));
+      ++k;
+    }
+    bulk_wait_all();    // shared memory must outlive the last stores (also after a failed wait)
+    return;
+  }
+  if (tid >= kThreads) return;
+
+  // ------------------------------------------------------------------ consumers
   SlotAccumulator sa(kThreads / 32);
-  TileWalker tw(plan, h.n_seg);
+  TileWalker tw(pv.seg, h.n_seg);
   int k = 0;
+  bool failed = false;
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
     if (tw.seek(tile) && A.partial) sa.advance(tw.sp.slot, A.partial);
     const long long e0 = tw.tile_start(tile);
@@ -623,13 +615,14 @@ static __device__ __noinline__ bool inplace_consumer_warps(const OuterArgs& A, c
       continue;
     }
     const int s = k % S;
-    const bool landed = !*sh.s_fail && mbar_wait_bounded(smem_u32(&sh.full_bar[s]), (k / S) & 1);
+    const bool landed = !s_fail && mbar_wait_bounded(smem_u32(&full_bar[s]), (k / S) & 1);
     if (!__all_sync(0xffffffffu, landed)) {   // per-warp verdict, as in k_outer_tma
       record_status(A.status, A.err_timeout);
-      *sh.s_fail = 1;
-      return false;
+      s_fail = 1;
+      failed = true;
+      break;
     }
-    float* st = sh.stages + (size_t)s * L::kLoaded * kTileElems;
+    float* st = stages + (size_t)s * L::kLoaded * kTileElems;
     auto slot = [&](int idx) -> float4& { return reinterpret_cast<float4*>(st + idx * kTileElems)[tid]; };
     Lane<M, MODE_FUSED, true> ln;
     ln.thg = slot(L::kGlobal);
@@ -643,44 +636,14 @@ static __device__ __noinline__ bool inplace_consumer_warps(const OuterArgs& A, c
     for (int m = 0; m < M; ++m) slot(L::kNow + m) = ln.out(m);
     if (A.delta_out) st4(A.delta_out + e0 + 4LL * tid, ln.delta);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // make the lane visible to the bulk store
-    mbar_arrive(smem_u32(&sh.done_bar[s]));
+    mbar_arrive(smem_u32(&done_bar[s]));
     ++k;
   }
-  if (A.partial) sa.finish(h.n_ids, A.partial);
-  return true;
-}
-
-template <int M>
-__global__ void __launch_bounds__(kInplaceThreads, 1)
-k_outer_inplace(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTable T) {
-  using IL = InplaceLayout<M>;
-  constexpr int S = IL::kStages;
-  static_assert(IL::L::kNow == 0 && IL::L::kLoaded == M + 2, "lane l of the loader and storer warps owns stream l");
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long full_bar[S];
-  __shared__ __align__(8) unsigned long long done_bar[S];
-  __shared__ __align__(8) unsigned long long empty_bar[S];
-  __shared__ volatile int s_fail;
-  __shared__ InlinePlan ip;
-  const int tid = threadIdx.x;
-  const PlanView pv = acquire_plan(ip, T, A.rq, A.plan, A.hdr, A.status);
-  if (tid == 0) {
-    for (int s = 0; s < S; ++s) {
-      mbar_init(smem_u32(&full_bar[s]), 1);
-      mbar_init(smem_u32(&done_bar[s]), kThreads);
-      mbar_init(smem_u32(&empty_bar[s]), 1);
-    }
-    s_fail = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  if (failed) return;     // warp-uniform by construction
+  if (A.partial) {
+    sa.finish(h.n_ids, A.partial);
+    finalize_epilogue(ip, A.fin, h, A.partial, kThreads / 32, A.status);
   }
-  __syncthreads();
-  InplaceShared sh;
-  sh.stages = reinterpret_cast<float*>(smem_raw);
-  sh.full_bar = full_bar; sh.done_bar = done_bar; sh.empty_bar = empty_bar; sh.s_fail = &s_fail;
-  if (tid >= kThreads + 32) { inplace_storer_warp<M>(A, pv.seg, pv.hdr, sh); return; }
-  if (tid >= kThreads) { inplace_loader_warp<M>(A, pv.seg, pv.hdr, sh); return; }
-  if (!inplace_consumer_warps<M>(A, pv.seg, pv.hdr, sh)) return;     // warp-uniform by construction
-  if (A.partial) finalize_epilogue(ip, A.fin, pv.hdr, A.partial, kThreads / 32, A.status);
 }
 
 // ---------------------------------------------------------------------------------------------
