@@ -586,3 +586,53 @@ def test_maximum_fragment_count():
     with pytest.raises(prob.B.CocodcError):
         ptr = np.arange(1026, dtype=np.int32)
         prob.B.Context(1025, ptr, np.arange(1025), np.ones(1025, dtype=np.int64), 1)
+
+
+@pytest.mark.parametrize("n_seg", [127, 128, 129])
+def test_fragment_tables_on_both_sides_of_the_kernel_argument_limit(n_seg):
+    """Fragment tables of up to 128 segments travel as a kernel argument and the streaming kernel expands the id list
+    itself; larger ones go through the plan kernel.  Same results on both sides of the limit: completion (all
+    fragments, then a permuted subset), snapshot, stand-alone scores, and the rejection of a bad id list."""
+    rng = np.random.default_rng(n_seg)
+    K = n_seg - 20                       # twenty fragments have two segments
+    frs, pos = [], 3
+    for p in range(K):
+        segs = []
+        for _ in range(2 if p < 20 else 1):
+            ln = int(rng.choice([5, 700, 1024, 2049, 4100]))
+            segs.append((pos, ln))
+            pos += ln + int(rng.choice([0, 1, 4]))
+        frs.append(segs)
+    w = synth.small_workload((pos + 8 - pos % 4, frs), M=3, seed=n_seg, scale_kind="loguniform", tau=2)
+    assert w.partition.n_segments == n_seg
+    prob = GpuProblem(w, synth.generate(w, "cuda", momentum_sigma=1e-3))
+    for ids in (list(range(K)), [int(p) for p in rng.permutation(K)[:K // 3]]):
+        prob.set_ids(ids)
+        before = prob.host_state()
+        n0 = prob.ctx.launch_count
+        prob.outer_step(4, 6)
+        assert prob.ctx.launch_count - n0 == (1 if n_seg <= 128 else 2)
+        assert prob.poll() == 0
+        _check_pooled(prob, before, ids, 4, 6)
+        snap_before = prob.host_state()
+        prob.snapshot()
+        assert prob.poll() == 0
+        exp = orc.snapshot(fragments_of(w), snap_before["w_now"], ids, w.M, None, snap_before["w_snap"])
+        assert np.array_equal(np_(prob.bufs.w_snap), exp)
+    x = prob.bufs.theta_g
+    norms = torch.zeros(K, device="cuda")
+    scores = torch.zeros(K, device="cuda")
+    prob.ctx.cocodc_fragment_scores(x, None, norms, scores)
+    en, _ = orc.fragment_scores(fragments_of(w), np_(x))
+    assert np.all(np.abs(np_(norms) - en) <= 1e-5 * en) and prob.poll() == 0
+    prob.ids[:2] = 7                     # listed twice
+    prob.n_ids.fill_(2)
+    before = prob.host_state()
+    prob.outer_step(8, 9)
+    assert prob.poll() == prob.B.ERR_INVALID_ARG
+    assert np.array_equal(prob.host_state()["theta_g"], before["theta_g"])
+    prob.set_ids([1, 0])                 # and the context works on afterwards
+    before = prob.host_state()
+    prob.outer_step(8, 9)
+    assert prob.poll() == 0
+    _check_pooled(prob, before, [1, 0], 8, 9)
