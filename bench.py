@@ -3,7 +3,7 @@
 
 One step = one pass of the whole path over the fragments in flight:
     cocodc_outer_step (S1-S6, fused) on the fragments whose sync completes now,
-    cocodc_select_fragments (S7) for the next set, cocodc_snapshot (S0) of that set.
+    cocodc_initiate for the next set: cocodc_select_fragments (S7) and cocodc_snapshot (S0) of that set in one launch.
 The metric is fragment parameters completed per second (whole job), with the achieved HBM rate of
 the fused kernel beside it.
 
@@ -177,9 +177,9 @@ class DeviceJob:
         self.norms = torch.zeros(K, dtype=torch.float32, device=device)
         self.last_sync = torch.zeros(K, dtype=torch.int64, device=device)
         self.mask = torch.zeros(K, dtype=torch.uint8, device=device)
-        # id list and its length share one buffer, so that the benchmark's per-step log is a single copy
-        self.idbuf = torch.full((K + 1,), -1, dtype=torch.int32, device=device)
-        self.ids, self.n_ids = self.idbuf[:K], self.idbuf[K:]
+        # id list and its length live in one row of K + 1 integers; use_row() points the job at another row, so
+        # that a benchmark can keep every step's list (selection writes straight into the next row: no copies)
+        self.use_row(torch.full((K + 1,), -1, dtype=torch.int32, device=device))
         self.n_ids.zero_()
         self.pool_off = torch.full((K,), -1, dtype=torch.int64, device=device)
         self.t = w.tau
@@ -205,6 +205,10 @@ class DeviceJob:
         if deployment == "worker_per_device":
             self.sum_buf = torch.zeros(w.N, dtype=torch.float32, device=device)
         self.collective_bytes = 0       # bytes this rank handed to collectives on the data path
+
+    def use_row(self, row: torch.Tensor):
+        self.idbuf = row
+        self.ids, self.n_ids = row[:self.w.K], row[self.w.K:]
 
     def select(self):
         w = self.w
@@ -264,12 +268,19 @@ class DeviceJob:
                                    b.theta_g, b.momentum, None, self.ids, self.n_ids, self.t, self.t + w.tau,
                                    self.last_sync, self.norms, self.scores)
 
+    def initiate(self):
+        """Algorithm 2 for the next set and the snapshot of what it picks (cocodc_initiate: one launch)."""
+        b, w = self.bufs, self.w
+        self.ctx.cocodc_initiate(self.scores, self.last_sync, None, self.t, w.H, self.kind, w.budget, self.mask,
+                                 self.ids, self.n_ids, self.pool_off, b.w_now, b.w_snap, b.now_stride, b.snap_stride,
+                                 w.M)
+
     def snapshot(self):
         b = self.bufs
         self.ctx.cocodc_snapshot(b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off, self.w.M,
                                  self.ids, self.n_ids)
 
-    def step(self, log=None, ev=None):
+    def step(self, next_row=None, ev=None):
         """Complete the fragments in flight, choose the next set, record their snapshots."""
         if self.deployment == "worker_per_device":
             self.pseudo_sum_and_exchange()
@@ -280,21 +291,21 @@ class DeviceJob:
             ev[1].record()
         if self.deployment == "param_shard":
             self.scores_param_shard()
-        if log is not None:
-            log.copy_(self.idbuf)
         if self.variant == "diloco":
             self.t += self.w.H
             return
         self.t += self.w.tau
-        self.select()
-        self.snapshot()
+        if next_row is not None:      # the next set's list goes to a fresh row; this step's row stays as its record
+            self.use_row(next_row)
+        self.initiate()
 
 
 def timed_device_leg(job: DeviceJob, K: int, W: int, device: torch.device, local: int, barrier):
     """W warm-up steps, then exactly K timed steps between two barriers; CUDA events around the whole region and
     around every completion call.  Returns the raw figures of this rank."""
     w = job.w
-    log = torch.full((K, w.K + 1), -1, dtype=torch.int32, device=device)     # per step: the completed ids, their count
+    # row i: the ids step i completes and their count (row K: the set still in flight at the end)
+    log = torch.full((K + 1, w.K + 1), -1, dtype=torch.int32, device=device)
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for _ in range(W):
@@ -302,26 +313,28 @@ def timed_device_leg(job: DeviceJob, K: int, W: int, device: torch.device, local
     status = job.ctx.cocodc_poll_status()
     if status != 0:
         raise RuntimeError(f"device status after warm-up: {job.B.status_string(status)}")
+    log[0].copy_(job.idbuf)
+    job.use_row(log[0])
     barrier()
     launches0 = job.ctx.launch_count
     bytes0 = job.collective_bytes
     with ClockSampler(local) as clocks:
         t_begin.record()
         for i in range(K):
-            job.step(log[i], evs[i])
+            job.step(log[i + 1], evs[i])
         t_end.record()
         barrier()
     status = job.ctx.cocodc_poll_status()
     if status != 0:
         raise RuntimeError(f"device status after the timed region: {job.B.status_string(status)}")
     log_h = log.cpu().numpy()
-    ids_h, n_h = log_h[:, :w.K], log_h[:, w.K]
-    per_step = [int(job.sizes[ids_h[i, :n_h[i]]].sum()) for i in range(K)]
-    # the set whose snapshot step i takes is the set step i + 1 completes; the last one is still in the job
-    last = job.idbuf.cpu().numpy()
-    per_step_snapshot = per_step[1:] + [int(job.sizes[last[:last[w.K]]].sum())]
-    if job.variant == "diloco":
-        per_step_snapshot = [0] * K
+    if job.variant == "diloco":           # one fixed list (all fragments), no selection
+        log_h[:] = log_h[0]
+    ids_h, n_h = log_h[:K, :w.K], log_h[:K, w.K]
+    sizes_of = lambda i: int(job.sizes[log_h[i, :log_h[i, w.K]]].sum())
+    per_step = [sizes_of(i) for i in range(K)]
+    # the set whose snapshot step i takes is the set step i + 1 completes
+    per_step_snapshot = [0] * K if job.variant == "diloco" else [sizes_of(i + 1) for i in range(K)]
     return {
         "seconds": t_begin.elapsed_time(t_end) / 1e3,
         "per_step": per_step,
@@ -431,11 +444,11 @@ def run_ours(args):
     if deployment == "worker_per_device":
         step_bytes += params_local * (4 * w.M + 8)       # the pseudo-gradient sum's own pass
     steps_desc = {
-        "replicas": "outer_step(S1-S6) + select(S7) + snapshot(S0)",
-        "param_shard": "outer_step(S1-S5 + sums of squares) + all-reduce of K fp64 + scores_from_sumsq(S6) + select(S7) "
-                       "+ snapshot(S0)",
+        "replicas": "outer_step(S1-S6) + initiate(S7 + S0)",
+        "param_shard": "outer_step(S1-S5 + sums of squares) + all-reduce of K fp64 + scores_from_sumsq(S6) "
+                       "+ initiate(S7 + S0)",
         "worker_per_device": "pseudo_gradient_sum(S1) + all-reduce of the listed fragments + outer_step_received(S2-S6) "
-                             "+ select(S7) + snapshot(S0)",
+                             "+ initiate(S7 + S0)",
     }
     out = {
         "metric": METRIC, "value": total_params / max_seconds, "unit": UNIT, "n_gpus": world, "steps": K,

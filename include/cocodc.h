@@ -184,8 +184,8 @@ cocodc_status cocodc_scores_from_sumsq(cocodc_ctx* ctx, const double* sumsq, con
  * Algorithm 2's bookkeeping of the fragments whose synchronisation is in flight (a fragment chosen at t_p
  * cannot be chosen again before it completes at t_p + tau).  in_flight is a dev uint8[K] array owned by the
  * caller, zero-initialised by it; once bound to the context,
- *   cocodc_select_fragments(_at)  treats in_flight[p] != 0 as not eligible and sets in_flight[p] = 1 for
- *                                 every fragment it selects,
+ *   cocodc_select_fragments(_at) and cocodc_initiate treat in_flight[p] != 0 as not eligible and set
+ *                                 in_flight[p] = 1 for every fragment they select,
  *   every completion that writes scores (cocodc_outer_step and its variants with COCODC_STAGE_SCORE,
  *   cocodc_scores_from_sumsq with an id list) sets in_flight[p] = 0 for the fragments it lists.
  * NULL unbinds.  The host-buffer entry points do not use it.
@@ -361,6 +361,23 @@ cocodc_status cocodc_merge(cocodc_ctx* ctx, const cocodc_hyper* hyper,
 cocodc_status cocodc_snapshot(cocodc_ctx* ctx, const float* w_now, float* w_snap,
                               int64_t now_stride, int64_t snap_stride, const int64_t* snap_offset,
                               int32_t M, const int32_t* ids, const int32_t* n_ids, void* stream);
+
+/*
+ * Initiation of a synchronisation at t_p in one call: Algorithm 2 (as cocodc_select_fragments, same arguments
+ * and outputs) followed by S0 for the fragments it picked (as cocodc_snapshot, with the places just written to
+ * pool_offset as the snapshot layout; pool_offset NULL keeps the native layout).  The two always happen
+ * together in the method - a fragment is chosen and its theta^m_{p,t_p} recorded - and for fragment tables of
+ * up to 128 segments and the COUNT and PARAMS budgets they are ONE kernel launch: every block of the snapshot
+ * kernel works out the (deterministic) selection for itself in its prologue.  Larger tables and
+ * COCODC_BUDGET_PARAMS_EXACT run the two kernels one after the other.  Results are bit-identical to the two
+ * separate calls.  The output arrays (mask, ids, n_sel, pool_offset) must not overlap the inputs.
+ */
+cocodc_status cocodc_initiate(cocodc_ctx* ctx, const float* scores, const int64_t* last_sync,
+                              const uint8_t* ineligible, int64_t t_now, int64_t H,
+                              int32_t budget_kind, int64_t budget,
+                              uint8_t* mask, int32_t* ids, int32_t* n_sel, int64_t* pool_offset,
+                              const float* w_now, float* w_snap, int64_t now_stride, int64_t snap_stride, int32_t M,
+                              void* stream);
 
 /*
  * S1-S6 as cocodc_outer_step (all stages), for callers whose parameters live in HOST memory.

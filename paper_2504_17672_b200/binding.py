@@ -29,7 +29,7 @@ EXPORTS = (
     "cocodc_fragment_scores_noalloc", "cocodc_selftest_bounded_wait",
     "cocodc_pseudo_gradient_sum", "cocodc_outer_step_received",
     "cocodc_select_fragments_at", "cocodc_outer_step_at", "cocodc_outer_step_received_peers",
-    "cocodc_scores_from_sumsq", "cocodc_bind_in_flight",
+    "cocodc_scores_from_sumsq", "cocodc_bind_in_flight", "cocodc_initiate",
 )
 NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
@@ -86,6 +86,7 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_fragment_scores.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.cocodc_scores_from_sumsq.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp]
     lib.cocodc_bind_in_flight.argtypes = [vp, vp]
+    lib.cocodc_initiate.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp, vp, i64, i64, i32, vp]
     lib.cocodc_select_fragments.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp]
     lib.cocodc_outer_step.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, vp,
                                       i64, i64, vp, vp, vp, vp, u32, vp]
@@ -219,6 +220,15 @@ class Context:
         _check(_lib.cocodc_select_fragments(self._h, _p(scores), _p(last_sync), _p(ineligible), int(t_now), int(H),
                                             int(budget_kind), int(budget), _p(mask), _p(ids), _p(n_sel),
                                             _p(pool_offset), _stream(stream)), "cocodc_select_fragments")
+
+    def cocodc_initiate(self, scores, last_sync, ineligible, t_now: int, H: int, budget_kind: int, budget: int,
+                        mask, ids, n_sel, pool_offset, w_now, w_snap, now_stride: int, snap_stride: int, M: int,
+                        stream=None) -> None:
+        """Algorithm 2 and the snapshot of what it picks, one launch (cocodc_select_fragments + cocodc_snapshot)."""
+        _check(_lib.cocodc_initiate(self._h, _p(scores), _p(last_sync), _p(ineligible), int(t_now), int(H),
+                                    int(budget_kind), int(budget), _p(mask), _p(ids), _p(n_sel), _p(pool_offset),
+                                    _p(w_now), _p(w_snap), int(now_stride), int(snap_stride), int(M),
+                                    _stream(stream)), "cocodc_initiate")
 
     def cocodc_outer_step(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                           theta_g, momentum, delta_g_out, ids, n_ids, t_p: int, t_l: int, last_sync,

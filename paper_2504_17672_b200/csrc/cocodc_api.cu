@@ -792,7 +792,60 @@ cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
   cocodc_status s = prepare_plan(c, ids, n_ids, snap_offset, snap_stride, kThreads * kSnapU, st, &rq, &gplan, &ghdr);
   if (s != COCODC_OK) return s;
   k_snapshot_tma<<<c->sm_count, kThreads, kSnapSmemBytes, st>>>(w_now, w_snap, now_stride, snap_stride, M, gplan, ghdr,
-                                                                rq, c->d_status, (int)COCODC_ERR_TIMEOUT, c->table);
+                                                                rq, c->d_status, (int)COCODC_ERR_TIMEOUT, c->table,
+                                                                SelectRequest{});
+  c->launches++;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
+cocodc_status cocodc_initiate(cocodc_ctx* c, const float* scores, const int64_t* last_sync, const uint8_t* ineligible,
+                              int64_t t_now, int64_t H, int32_t budget_kind, int64_t budget,
+                              uint8_t* mask, int32_t* ids, int32_t* n_sel, int64_t* pool_offset,
+                              const float* w_now, float* w_snap, int64_t now_stride, int64_t snap_stride, int32_t M,
+                              void* stream) {
+  if (!c || !scores || !last_sync || !mask || !ids || !n_sel || !w_now || !w_snap) return COCODC_ERR_INVALID_ARG;
+  if (H < 1 || budget < 0 || M < 1 || M > c->max_M) return COCODC_ERR_INVALID_ARG;
+  if (budget_kind != COCODC_BUDGET_COUNT && budget_kind != COCODC_BUDGET_PARAMS &&
+      budget_kind != COCODC_BUDGET_PARAMS_EXACT)
+    return COCODC_ERR_INVALID_ARG;
+  const long long N = c->N;
+  if (now_stride < N || snap_stride < (pool_offset ? 1 : N)) return COCODC_ERR_INVALID_ARG;
+  if (!aligned16(w_now) || !aligned16(w_snap) || (now_stride & 3) || (snap_stride & 3)) return COCODC_ERR_ALIGNMENT;
+  if (overlap(range_of(w_now, (long long)(M - 1) * now_stride + N),
+              range_of(w_snap, (long long)(M - 1) * snap_stride + (pool_offset ? snap_stride : N))))
+    return COCODC_ERR_ALIAS;
+  if (!c->inline_plan || budget_kind == COCODC_BUDGET_PARAMS_EXACT) {
+    // a table too large to be a kernel argument, or the enumerating budget: the two calls one after the other
+    cocodc_status s = cocodc_select_fragments(c, scores, last_sync, ineligible, t_now, H, budget_kind, budget, mask,
+                                              ids, n_sel, pool_offset, stream);
+    if (s != COCODC_OK) return s;
+    return cocodc_snapshot(c, w_now, w_snap, now_stride, snap_stride, pool_offset, M, ids, n_sel, stream);
+  }
+  DeviceGuard guard(c->device);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  opt_in_shared_memory(c, reinterpret_cast<const void*>(k_snapshot_tma), kSnapSmemBytes);
+  PlanRequest rq{};
+  rq.snap_row_len = snap_stride;
+  rq.lanes_per_tile = kThreads * kSnapU;
+  rq.err_invalid = (int)COCODC_ERR_INVALID_ARG;
+  SelectRequest q{};
+  q.scores = scores;
+  q.last_sync = reinterpret_cast<const long long*>(last_sync);
+  q.ineligible = ineligible;
+  q.in_flight = c->in_flight;
+  q.t_now = t_now;
+  q.H = H;
+  q.budget_kind = budget_kind;
+  q.budget = budget;
+  q.mask = mask;
+  q.ids = ids;
+  q.n_sel = n_sel;
+  q.pool_offset = reinterpret_cast<long long*>(pool_offset);
+  q.ticket = c->d_ticket;
+  q.err_nonfinite = (int)COCODC_ERR_NONFINITE;
+  k_snapshot_tma<<<c->sm_count, kThreads, kSnapSmemBytes, st>>>(w_now, w_snap, now_stride, snap_stride, M, nullptr,
+                                                                nullptr, rq, c->d_status, (int)COCODC_ERR_TIMEOUT,
+                                                                c->table, q);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }

@@ -22,6 +22,7 @@
 #pragma once
 
 #include "outer.cuh"
+#include "select.cuh"
 
 namespace cocodc {
 
@@ -464,12 +465,25 @@ __global__ void __launch_bounds__(kThreads, 1)
 k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long long now_stride,
                long long snap_stride, int M, const SegPlan* __restrict__ gplan,
                const PlanHeader* __restrict__ ghdr, const __grid_constant__ PlanRequest rq,
-               int* __restrict__ status, int err_timeout, const __grid_constant__ FragTable T) {
+               int* __restrict__ status, int err_timeout, const __grid_constant__ FragTable T,
+               const __grid_constant__ SelectRequest sel) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long full_bar[kSnapStages];
   __shared__ float* dst_of_stage[kSnapStages];
   __shared__ InlinePlan ip;
-  const PlanView pv = acquire_plan(ip, T, rq, gplan, ghdr, status);
+  __shared__ InlineSelect is;
+  PlanView pv;
+  if (sel.scores != nullptr) {
+    // initiation in one launch: Algorithm 2 first, then the snapshot of what it picked
+    select_in_cta(is, sel, T, status);
+    PlanRequest mine = rq;
+    mine.ids = is.ids;
+    mine.n_ids = &is.n;
+    mine.snap_offset = sel.pool_offset ? is.pool : nullptr;
+    pv = acquire_plan(ip, T, mine, nullptr, nullptr, status);
+  } else {
+    pv = acquire_plan(ip, T, rq, gplan, ghdr, status);
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < kSnapStages; ++s) mbar_init(smem_u32(&full_bar[s]), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

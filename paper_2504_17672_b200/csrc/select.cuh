@@ -179,4 +179,127 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
   *n_sel = n;
 }
 
+// ---------------------------------------------------------------------------------------------------
+// The same decision inside another kernel's prologue (cocodc_initiate: Algorithm 2 and the snapshot of what it
+// picks are one event, at t_p, so they are one launch).  For fragment tables that travel as a kernel argument
+// (K <= kInlineSegs) and the budgets that are walked (COUNT, PARAMS), every CTA of the snapshot kernel works out
+// the selection for itself - it is a deterministic function of the schedule state - and keeps the id list and
+// the pool places in shared memory, where the plan is then built from; CTA 0 also writes them to the caller's
+// arrays.  The in-flight marks are written by whichever CTA finishes its selection last (a ticket): no CTA
+// may see them before it has read the mask itself.
+// ---------------------------------------------------------------------------------------------------
+struct SelectRequest {
+  const float* scores;                 // nullptr: no selection in this launch
+  const long long* last_sync;
+  const unsigned char* ineligible;
+  unsigned char* in_flight;
+  long long t_now;
+  long long H;
+  int budget_kind;                     // 0 COUNT, 1 PARAMS
+  long long budget;
+  unsigned char* mask;
+  int* ids;
+  int* n_sel;
+  long long* pool_offset;              // nullptr: the snapshot keeps the native layout
+  int* ticket;                         // zero between launches
+  int err_nonfinite;
+};
+
+struct InlineSelect {
+  float score[kInlineSegs];
+  int order[kInlineSegs];
+  int ids[kInlineSegs];
+  long long fsize[kInlineSegs];
+  long long pool[kInlineSegs];         // by fragment id; -1: not selected
+  unsigned char cls[kInlineSegs];      // 0 = ineligible, 1 = ordinary, 2 = overdue
+  unsigned char falign[kInlineSegs];
+  int n;
+  int n_elig;
+  int nan;
+};
+
+// Called by every thread of the CTA (at least K threads).
+static __device__ __noinline__ void select_in_cta(InlineSelect& is, const SelectRequest& q, const FragTable& T,
+                                                  int* status) {
+  const int p = threadIdx.x;
+  const int K = T.K;
+  const bool writer = (blockIdx.x == 0);
+  if (p == 0) { is.n = 0; is.n_elig = 0; is.nan = 0; }
+  __syncthreads();
+  if (p < K) {
+    const float r = q.scores[p];
+    const bool elig = ((q.ineligible == nullptr) || (q.ineligible[p] == 0)) &&
+                      ((q.in_flight == nullptr) || (q.in_flight[p] == 0));
+    const bool overdue = (q.t_now - q.last_sync[p]) >= q.H;   // Algorithm 2's staleness test
+    long long size = 0;
+    for (int sg = T.seg_ptr[p]; sg < T.seg_ptr[p + 1]; ++sg) size += T.len[sg];
+    is.score[p] = r;
+    is.fsize[p] = size;
+    is.falign[p] = (unsigned char)(T.off[T.seg_ptr[p]] & 3);
+    is.cls[p] = elig ? (overdue ? 2 : 1) : 0;
+    is.pool[p] = -1;
+    if (r != r) is.nan = 1;
+    if (writer) {
+      q.mask[p] = 0;
+      q.ids[p] = -1;
+      if (q.pool_offset) q.pool_offset[p] = -1;
+    }
+  }
+  __syncthreads();
+  if (is.nan) {
+    if (p == 0 && writer) { *q.n_sel = 0; record_status(status, q.err_nonfinite); }
+  } else {
+    if (p < K && is.cls[p] != 0) {
+      const float r = is.score[p];
+      const int cls = is.cls[p];
+      int rank = 0;
+      for (int o = 0; o < K; ++o) {
+        const int co = is.cls[o];
+        if (co == 0 || o == p) continue;
+        bool before;
+        if (co != cls) before = co > cls;                 // overdue fragments come first
+        else if (cls == 2) before = o < p;                // among overdue: by index
+        else {
+          const float ro = is.score[o];
+          before = (ro > r) || (ro == r && o < p);        // by score, ties to the lower index
+        }
+        rank += before ? 1 : 0;
+      }
+      is.order[rank] = p;
+      atomicAdd(&is.n_elig, 1);
+    }
+    __syncthreads();
+    if (p == 0) {
+      long long remaining = q.budget, pool_pos = 0;
+      int n = 0;
+      for (int j = 0; j < is.n_elig; ++j) {
+        const int f = is.order[j];
+        const long long cost = (q.budget_kind == 0) ? 1 : is.fsize[f];
+        if (j == 0 || cost <= remaining) {                // the head of the order is always taken
+          is.ids[n++] = f;
+          remaining -= cost;
+          const long long start = pool_pos + is.falign[f];   // same placement rule as k_select
+          is.pool[f] = start;
+          pool_pos = (start + is.fsize[f] + 3) & ~3LL;
+          if (writer) {
+            q.mask[f] = 1;
+            q.ids[n - 1] = f;
+            if (q.pool_offset) q.pool_offset[f] = start;
+          }
+        }
+      }
+      is.n = n;
+      if (writer) *q.n_sel = n;
+    }
+  }
+  __syncthreads();
+  // every CTA has read the in-flight mask once the last one gets here: only then is it marked
+  if (p == 0 && q.in_flight != nullptr) {
+    if (arrive_gpu(q.ticket) == (int)gridDim.x - 1) {
+      for (int j = 0; j < is.n; ++j) q.in_flight[is.ids[j]] = 1;
+      *q.ticket = 0;
+    }
+  }
+}
+
 }  // namespace cocodc

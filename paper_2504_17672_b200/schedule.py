@@ -4,8 +4,8 @@
 
   * every synchronisation initiated at t - tau completes now: `cocodc_outer_step` on its fragment list
     (Eq. 1-2, Algorithm 1, Eq. 10);
-  * every h steps (Eq. 8-9) a new synchronisation is initiated: `cocodc_select_fragments` (Algorithm 2,
-    fragments still in flight are ineligible) and `cocodc_snapshot` of the chosen fragments.
+  * every h steps (Eq. 8-9) a new synchronisation is initiated: `cocodc_initiate` = Algorithm 2 (fragments
+    still in flight are ineligible) and the snapshot of the chosen fragments, one launch.
 
 All schedule state (scores, last_sync, id lists, masks, pool offsets, the in-flight mask) lives on the device
 and is updated by the library's kernels; the driver only marshals arguments and keeps track of which slot was
@@ -86,11 +86,9 @@ class RoundDriver:
 
     def _initiate(self, slot: _Slot, t_p: int) -> None:
         self._notify("initiate", "before", slot, t_p)
-        self.ctx.cocodc_select_fragments(self.scores, self.last_sync, None, t_p, self.hyper.H,
-                                         self.budget_kind, self.budget, slot.mask, slot.ids, slot.n_ids,
-                                         slot.pool_off)
-        self.ctx.cocodc_snapshot(self.w_now, slot.pool, self.w_now.stride(0), slot.pool.stride(0), slot.pool_off,
-                                 self.hyper.M, slot.ids, slot.n_ids)
+        self.ctx.cocodc_initiate(self.scores, self.last_sync, None, t_p, self.hyper.H, self.budget_kind, self.budget,
+                                 slot.mask, slot.ids, slot.n_ids, slot.pool_off, self.w_now, slot.pool,
+                                 self.w_now.stride(0), slot.pool.stride(0), self.hyper.M)
         slot.t_p = t_p
         self.initiated += 1
         self._notify("initiate", "after", slot, t_p)

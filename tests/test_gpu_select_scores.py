@@ -380,3 +380,99 @@ def test_sums_of_squares_of_two_slices_give_the_whole_fragments_scores():
     cbig.cocodc_fragment_scores(xb, None, nb, nb.clone())
     assert cbig.launch_count - n0 == 2 and cbig.cocodc_poll_status() == 0
     assert np.allclose(np_(nb), np.sqrt(300.0), rtol=1e-6)
+
+
+@pytest.mark.parametrize("case", range(10))
+def test_initiate_equals_selection_followed_by_snapshot(case):
+    """cocodc_initiate (Algorithm 2 and the snapshot of what it picks in one launch) against the two separate calls
+    and, through them, the oracle: bit for bit on mask, ids, count, pool places, in-flight marks and every word of
+    the snapshot pool.  Random schedule states: overdue fragments, never-synced ones, ties, ineligible and in-flight
+    fragments, both walked budgets, with and without a pool; the tenth case has a table too large for one launch."""
+    from paper_2504_17672_b200 import binding as B
+    rng = np.random.default_rng(700 + case)
+    K = 150 if case == 9 else int(rng.integers(1, 41))
+    sizes = rng.choice([3, 64, 1000, 1025, 4096, 9000, 20_001], size=K).tolist()
+    frs, pos = [], int(rng.integers(0, 4))
+    for s_ in sizes:
+        frs.append([(pos, int(s_))])
+        pos += int(s_) + int(rng.choice([0, 1, 2, 5]))
+    M = int(rng.integers(1, 4))
+    w = synth.small_workload((pos + 8 - pos % 4, frs), M=M, seed=case)
+    ptr, off, ln = w.partition.csr()
+    bufs = synth.generate(w, "cuda")
+    scores_h = rng.choice([0.5, 1.0, 1.0, 2.5, 7.0, np.inf], size=K).astype(np.float32) * rng.choice([1.0, 1.0, 3.0], size=K).astype(np.float32)
+    last_h = rng.integers(0, 160, size=K).astype(np.int64)
+    inel_h = (rng.random(K) < 0.15).astype(np.uint8)
+    flight_h = (rng.random(K) < 0.15).astype(np.uint8)
+    t_now, H = 200, 100
+    kind = int(rng.integers(0, 2))
+    budget = int(rng.integers(1, 6)) if kind == 0 else int(rng.integers(1, max(2, sum(sizes) // 2)))
+    use_pool = bool(rng.integers(0, 2)) or True if case % 3 else False
+    pool_len = (sum(sizes) + 8 * K + 1023) // 1024 * 1024
+    out = {}
+    for name in ("two_calls", "initiate"):
+        ctx = B.Context(w.N, ptr, off, ln, M)
+        scores = torch.from_numpy(scores_h).cuda()
+        last = torch.from_numpy(last_h).cuda()
+        inel = torch.from_numpy(inel_h).cuda()
+        flight = torch.from_numpy(flight_h.copy()).cuda()
+        ctx.cocodc_bind_in_flight(flight)
+        mask = torch.full((K,), 9, dtype=torch.uint8, device="cuda")
+        ids = torch.full((K,), 77, dtype=torch.int32, device="cuda")
+        n_sel = torch.full((1,), -5, dtype=torch.int32, device="cuda")
+        pool_off = torch.full((K,), 123, dtype=torch.int64, device="cuda") if use_pool else None
+        snap = (torch.full((M, pool_len), -3.0, device="cuda") if use_pool
+                else torch.full((M, w.N), -3.0, device="cuda"))
+        n0 = ctx.launch_count
+        if name == "two_calls":
+            ctx.cocodc_select_fragments(scores, last, inel, t_now, H, kind, budget, mask, ids, n_sel, pool_off)
+            ctx.cocodc_snapshot(bufs.w_now, snap, bufs.now_stride, snap.stride(0), pool_off, M, ids, n_sel)
+        else:
+            ctx.cocodc_initiate(scores, last, inel, t_now, H, kind, budget, mask, ids, n_sel, pool_off, bufs.w_now, snap,
+                                bufs.now_stride, snap.stride(0), M)
+            assert ctx.launch_count - n0 == (1 if K <= 128 else 3)      # beyond the limit: select, plan, snapshot
+        assert ctx.cocodc_poll_status() == 0
+        out[name] = dict(mask=np_(mask), ids=np_(ids), n=int(n_sel.item()), flight=np_(flight),
+                         pool_off=None if pool_off is None else np_(pool_off), snap=np_(snap))
+        ctx.close()
+    a, b = out["two_calls"], out["initiate"]
+    assert a["n"] == b["n"] and np.array_equal(a["mask"], b["mask"]) and np.array_equal(a["ids"], b["ids"])
+    assert np.array_equal(a["flight"], b["flight"])
+    if use_pool:
+        assert np.array_equal(a["pool_off"], b["pool_off"])
+    assert np.array_equal(a["snap"], b["snap"])
+    # and against the oracle
+    emask, eids, en = orc.select_fragments(scores_h, last_h, np.array(sizes), t_now, H, kind, budget,
+                                           ineligible=np.maximum(inel_h, flight_h))
+    assert b["n"] == en and b["ids"][:en].tolist() == eids.tolist() and np.array_equal(b["mask"], emask)
+    assert np.array_equal(b["flight"], np.maximum(flight_h, emask))
+    exp = orc.snapshot(fragments_of(w), np_(bufs.w_now), eids, M, b["pool_off"],
+                       np.full(b["snap"].shape, -3.0, dtype=np.float32))
+    assert np.array_equal(b["snap"], exp)
+
+
+def test_initiate_rejects_nan_scores_and_takes_the_enumerating_budget_in_two_launches():
+    from paper_2504_17672_b200 import binding as B
+    w = synth.small_workload([4096, 5000, 776], M=2, seed=4)
+    ptr, off, ln = w.partition.csr()
+    ctx = B.Context(w.N, ptr, off, ln, 2)
+    bufs = synth.generate(w, "cuda")
+    K = 3
+    scores = torch.tensor([1.0, float("nan"), 2.0], device="cuda")
+    last = torch.zeros(K, dtype=torch.int64, device="cuda")
+    mask = torch.zeros(K, dtype=torch.uint8, device="cuda")
+    ids = torch.zeros(K, dtype=torch.int32, device="cuda")
+    n_sel = torch.ones(1, dtype=torch.int32, device="cuda")
+    snap = torch.full((2, w.N), -1.0, device="cuda")
+    ctx.cocodc_initiate(scores, last, None, 5, 100, B.BUDGET_COUNT, 2, mask, ids, n_sel, None, bufs.w_now, snap,
+                        bufs.now_stride, snap.stride(0), 2)
+    assert ctx.cocodc_poll_status() == B.ERR_NONFINITE
+    assert int(n_sel.item()) == 0 and bool((snap == -1.0).all())
+    scores[1] = 0.5
+    n0 = ctx.launch_count
+    ctx.cocodc_initiate(scores, last, None, 5, 100, B.BUDGET_PARAMS_EXACT, 6000, mask, ids, n_sel, None, bufs.w_now,
+                        snap, bufs.now_stride, snap.stride(0), 2)
+    assert ctx.launch_count - n0 == 2 and ctx.cocodc_poll_status() == 0
+    _, eids, en = orc.select_fragments(np_(scores), np_(last), w.partition.frag_sizes, 5, 100,
+                                       orc.BUDGET_PARAMS_EXACT, 6000)
+    assert np_(ids)[:en].tolist() == eids.tolist()
