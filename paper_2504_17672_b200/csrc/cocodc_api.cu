@@ -102,7 +102,7 @@ cocodc_status launch_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_id
 
 // One way to run the streaming step: which kernel, with how many threads and how much dynamic
 // shared memory, on how many CTAs, over tiles of how many lanes.  Every variant has eight accumulating
-// warps, so the finalize kernel does not depend on the choice; the plan is built for the variant's tile.
+// warps, so the score epilogue does not depend on the choice; the plan is built for the variant's tile.
 struct Variant {
   void (*kernel)(const OuterArgs, const FragTable);
   int threads;

@@ -1,8 +1,8 @@
 // The fused outer-step kernel for the instantiated worker counts: the inputs of every tile are brought
 // into shared memory by the TMA unit (1-D bulk asynchronous copies); the outputs leave from registers.
 //
-// One CTA per SM: warps 0-7 compute, warp 8 holds the producer thread.  A stage is one tile
-// (1024 elements = 4 KB) of every stream the mode reads.  Per tile:
+// One CTA per SM: warps 0-7 compute, warp 8 is the producer (lane l issues the copies of stream l).  A stage is
+// one tile (1024 elements = 4 KB) of every stream the mode reads.  Per tile:
 //   producer : waits until the stage is free ("empty" barrier, one arrival per consumer thread), arms the
 //              stage's "full" barrier with the byte count, issues one bulk copy global->shared per stream;
 //   consumers: wait on "full", read their 16-byte lane of every stream from shared memory into registers,
@@ -19,6 +19,12 @@
 // others poll, and leaves; no thread waits on a barrier another thread could have abandoned.
 // Every copy is a plain one-CTA bulk copy (no cluster-wide form); only this GPU's memory is read, apart from
 // buffers of received sums that the caller may have mapped from a peer.
+//
+// Every kernel here is the whole of its C-ABI call: it expands the device-resident id list in its prologue
+// (acquire_plan) and, where scores are asked for, its last warp forms them (finalize_epilogue); the snapshot
+// kernel can also run Algorithm 2 first (select_in_cta).  The streaming loops between prologue and epilogue are
+// separate out-of-line functions: inlined next to that code they ran up to 1 % slower, by amounts that moved
+// with unrelated edits.
 #pragma once
 
 #include "outer.cuh"
@@ -28,7 +34,6 @@ namespace cocodc {
 
 // k_outer_tma runs eight consumer warps and one producer warp, whose lanes each issue one stream's copies.
 __host__ __device__ constexpr int tma_threads(int /*M*/) { return kThreads + 32; }
-constexpr int kTmaThreads = kThreads + 32;      // kernels with a single producer warp
 constexpr unsigned kTileBytes = kTileElems * sizeof(float);   // one stream's share of a stage
 constexpr int kWaitLimit = 1 << 22;                           // polls of a barrier before giving up
 constexpr int kMaxStages = 10;

@@ -189,7 +189,7 @@ k_plan(const int* __restrict__ ids, const int* __restrict__ n_ids_p, int K,
 // works on never decreases.  Every thread keeps a double accumulator for the
 // current slot; when the slot changes the warp reduces it and lane 0 writes
 // partial[(slot*gridDim.x + blockIdx.x)*warps + warp] (warps = accumulating warps per CTA).  Slots a CTA never
-// touched get an explicit zero, so the finalize kernel can sum every entry
+// touched get an explicit zero, so the score epilogue can sum every entry
 // without the buffer being cleared first.  The tile-to-CTA map is static,
 // hence the summation order - and the rounded result - is the same every run.
 // ---------------------------------------------------------------------------
