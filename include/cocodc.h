@@ -379,6 +379,15 @@ cocodc_status cocodc_initiate(cocodc_ctx* ctx, const float* scores, const int64_
                               const float* w_now, float* w_snap, int64_t now_stride, int64_t snap_stride, int32_t M,
                               void* stream);
 
+/* cocodc_initiate with t_now read from device memory (dev int64[1]) at run time, for graph replay (see
+ * cocodc_select_fragments_at). */
+cocodc_status cocodc_initiate_at(cocodc_ctx* ctx, const float* scores, const int64_t* last_sync,
+                                 const uint8_t* ineligible, const int64_t* t_now, int64_t H,
+                                 int32_t budget_kind, int64_t budget,
+                                 uint8_t* mask, int32_t* ids, int32_t* n_sel, int64_t* pool_offset,
+                                 const float* w_now, float* w_snap, int64_t now_stride, int64_t snap_stride, int32_t M,
+                                 void* stream);
+
 /*
  * S1-S6 as cocodc_outer_step (all stages), for callers whose parameters live in HOST memory.
  * Every buffer argument here is a host pointer (pinned memory makes the copies asynchronous and

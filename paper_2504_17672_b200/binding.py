@@ -29,7 +29,7 @@ EXPORTS = (
     "cocodc_fragment_scores_noalloc", "cocodc_selftest_bounded_wait",
     "cocodc_pseudo_gradient_sum", "cocodc_outer_step_received",
     "cocodc_select_fragments_at", "cocodc_outer_step_at", "cocodc_outer_step_received_peers",
-    "cocodc_scores_from_sumsq", "cocodc_bind_in_flight", "cocodc_initiate",
+    "cocodc_scores_from_sumsq", "cocodc_bind_in_flight", "cocodc_initiate", "cocodc_initiate_at",
 )
 NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
@@ -87,6 +87,7 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_scores_from_sumsq.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp]
     lib.cocodc_bind_in_flight.argtypes = [vp, vp]
     lib.cocodc_initiate.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp, vp, i64, i64, i32, vp]
+    lib.cocodc_initiate_at.argtypes = [vp, vp, vp, vp, vp, i64, i32, i64, vp, vp, vp, vp, vp, vp, i64, i64, i32, vp]
     lib.cocodc_select_fragments.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp]
     lib.cocodc_outer_step.argtypes = [vp, ctypes.POINTER(_Hyper), vp, vp, i64, i64, vp, vp, vp, vp, vp, vp,
                                       i64, i64, vp, vp, vp, vp, u32, vp]
@@ -229,6 +230,15 @@ class Context:
                                     int(budget_kind), int(budget), _p(mask), _p(ids), _p(n_sel), _p(pool_offset),
                                     _p(w_now), _p(w_snap), int(now_stride), int(snap_stride), int(M),
                                     _stream(stream)), "cocodc_initiate")
+
+    def cocodc_initiate_at(self, scores, last_sync, ineligible, t_now, H: int, budget_kind: int, budget: int,
+                           mask, ids, n_sel, pool_offset, w_now, w_snap, now_stride: int, snap_stride: int, M: int,
+                           stream=None) -> None:
+        """As cocodc_initiate with t_now a device int64[1] tensor."""
+        _check(_lib.cocodc_initiate_at(self._h, _p(scores), _p(last_sync), _p(ineligible), _p(t_now), int(H),
+                                       int(budget_kind), int(budget), _p(mask), _p(ids), _p(n_sel), _p(pool_offset),
+                                       _p(w_now), _p(w_snap), int(now_stride), int(snap_stride), int(M),
+                                       _stream(stream)), "cocodc_initiate_at")
 
     def cocodc_outer_step(self, hyper: Hyper, w_now, w_snap, now_stride: int, snap_stride: int, snap_offset,
                           theta_g, momentum, delta_g_out, ids, n_ids, t_p: int, t_l: int, last_sync,

@@ -798,11 +798,14 @@ cocodc_status cocodc_snapshot(cocodc_ctx* c, const float* w_now, float* w_snap,
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
-cocodc_status cocodc_initiate(cocodc_ctx* c, const float* scores, const int64_t* last_sync, const uint8_t* ineligible,
-                              int64_t t_now, int64_t H, int32_t budget_kind, int64_t budget,
-                              uint8_t* mask, int32_t* ids, int32_t* n_sel, int64_t* pool_offset,
-                              const float* w_now, float* w_snap, int64_t now_stride, int64_t snap_stride, int32_t M,
-                              void* stream) {
+}  // extern "C"
+
+namespace {
+cocodc_status initiate_impl(cocodc_ctx* c, const float* scores, const int64_t* last_sync, const uint8_t* ineligible,
+                            int64_t t_now, const int64_t* t_now_dev, int64_t H, int32_t budget_kind, int64_t budget,
+                            uint8_t* mask, int32_t* ids, int32_t* n_sel, int64_t* pool_offset,
+                            const float* w_now, float* w_snap, int64_t now_stride, int64_t snap_stride, int32_t M,
+                            void* stream) {
   if (!c || !scores || !last_sync || !mask || !ids || !n_sel || !w_now || !w_snap) return COCODC_ERR_INVALID_ARG;
   if (H < 1 || budget < 0 || M < 1 || M > c->max_M) return COCODC_ERR_INVALID_ARG;
   if (budget_kind != COCODC_BUDGET_COUNT && budget_kind != COCODC_BUDGET_PARAMS &&
@@ -816,8 +819,8 @@ cocodc_status cocodc_initiate(cocodc_ctx* c, const float* scores, const int64_t*
     return COCODC_ERR_ALIAS;
   if (!c->inline_plan || budget_kind == COCODC_BUDGET_PARAMS_EXACT) {
     // a table too large to be a kernel argument, or the enumerating budget: the two calls one after the other
-    cocodc_status s = cocodc_select_fragments(c, scores, last_sync, ineligible, t_now, H, budget_kind, budget, mask,
-                                              ids, n_sel, pool_offset, stream);
+    cocodc_status s = select_impl(c, scores, last_sync, ineligible, t_now, t_now_dev, H, budget_kind, budget, mask,
+                                  ids, n_sel, pool_offset, stream);
     if (s != COCODC_OK) return s;
     return cocodc_snapshot(c, w_now, w_snap, now_stride, snap_stride, pool_offset, M, ids, n_sel, stream);
   }
@@ -834,6 +837,7 @@ cocodc_status cocodc_initiate(cocodc_ctx* c, const float* scores, const int64_t*
   q.ineligible = ineligible;
   q.in_flight = c->in_flight;
   q.t_now = t_now;
+  q.t_now_dev = reinterpret_cast<const long long*>(t_now_dev);
   q.H = H;
   q.budget_kind = budget_kind;
   q.budget = budget;
@@ -848,6 +852,28 @@ cocodc_status cocodc_initiate(cocodc_ctx* c, const float* scores, const int64_t*
                                                                 c->table, q);
   c->launches++;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+}  // namespace
+
+extern "C" {
+
+cocodc_status cocodc_initiate(cocodc_ctx* c, const float* scores, const int64_t* last_sync, const uint8_t* ineligible,
+                              int64_t t_now, int64_t H, int32_t budget_kind, int64_t budget,
+                              uint8_t* mask, int32_t* ids, int32_t* n_sel, int64_t* pool_offset,
+                              const float* w_now, float* w_snap, int64_t now_stride, int64_t snap_stride, int32_t M,
+                              void* stream) {
+  return initiate_impl(c, scores, last_sync, ineligible, t_now, nullptr, H, budget_kind, budget, mask, ids, n_sel,
+                       pool_offset, w_now, w_snap, now_stride, snap_stride, M, stream);
+}
+
+cocodc_status cocodc_initiate_at(cocodc_ctx* c, const float* scores, const int64_t* last_sync,
+                                 const uint8_t* ineligible, const int64_t* t_now, int64_t H, int32_t budget_kind,
+                                 int64_t budget, uint8_t* mask, int32_t* ids, int32_t* n_sel, int64_t* pool_offset,
+                                 const float* w_now, float* w_snap, int64_t now_stride, int64_t snap_stride, int32_t M,
+                                 void* stream) {
+  if (!t_now) return COCODC_ERR_INVALID_ARG;
+  return initiate_impl(c, scores, last_sync, ineligible, 0, t_now, H, budget_kind, budget, mask, ids, n_sel,
+                       pool_offset, w_now, w_snap, now_stride, snap_stride, M, stream);
 }
 
 cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,

@@ -194,6 +194,7 @@ struct SelectRequest {
   const unsigned char* ineligible;
   unsigned char* in_flight;
   long long t_now;
+  const long long* t_now_dev;          // the step number kept in device memory takes precedence (graph replay)
   long long H;
   int budget_kind;                     // 0 COUNT, 1 PARAMS
   long long budget;
@@ -224,13 +225,14 @@ static __device__ __noinline__ void select_in_cta(InlineSelect& is, const Select
   const int p = threadIdx.x;
   const int K = T.K;
   const bool writer = (blockIdx.x == 0);
+  const long long t_now = q.t_now_dev ? *q.t_now_dev : q.t_now;
   if (p == 0) { is.n = 0; is.n_elig = 0; is.nan = 0; }
   __syncthreads();
   if (p < K) {
     const float r = q.scores[p];
     const bool elig = ((q.ineligible == nullptr) || (q.ineligible[p] == 0)) &&
                       ((q.in_flight == nullptr) || (q.in_flight[p] == 0));
-    const bool overdue = (q.t_now - q.last_sync[p]) >= q.H;   // Algorithm 2's staleness test
+    const bool overdue = (t_now - q.last_sync[p]) >= q.H;     // Algorithm 2's staleness test
     long long size = 0;
     for (int sg = T.seg_ptr[p]; sg < T.seg_ptr[p + 1]; ++sg) size += T.len[sg];
     is.score[p] = r;

@@ -261,6 +261,34 @@ def test_schedule_step_replayed_from_a_cuda_graph_equals_eager_steps():
                  (a.bufs.w_snap, g.bufs.w_snap), (a.scores, g.scores), (a.last_sync, g.last_sync), (a.ids, g.ids)):
         assert torch.equal(x, y)
 
+    # the same schedule step as two launches (completion, initiation), again from a graph
+    h = fresh()
+    clock2 = torch.tensor([10, 10 + tau], dtype=torch.int64, device="cuda")
+
+    def step2():
+        b = h.bufs
+        h.ctx.cocodc_outer_step_at(h.hyper(), b.w_now, b.w_snap, b.now_stride, b.snap_stride, h.pool_off, b.theta_g,
+                                   b.momentum, None, h.ids, h.n_ids, clock2[0:1], clock2[1:2], h.last_sync, h.norms,
+                                   h.scores)
+        h.ctx.cocodc_initiate_at(h.scores, h.last_sync, None, clock2[1:2], w.H, B.BUDGET_COUNT, w.budget, h.mask,
+                                 h.ids, h.n_ids, h.pool_off, b.w_now, b.w_snap, b.now_stride, b.snap_stride, w.M)
+        clock2.add_(tau)
+
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step2()
+    torch.cuda.current_stream().wait_stream(side)
+    graph2 = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph2):
+        step2()
+    for _ in range(4):
+        graph2.replay()
+    torch.cuda.synchronize()
+    assert h.poll() == 0
+    for x, y in ((a.bufs.w_now, h.bufs.w_now), (a.bufs.theta_g, h.bufs.theta_g), (a.bufs.momentum, h.bufs.momentum),
+                 (a.bufs.w_snap, h.bufs.w_snap), (a.scores, h.scores), (a.last_sync, h.last_sync), (a.ids, h.ids)):
+        assert torch.equal(x, y)
+
 
 def test_selected_pool_places_keep_the_native_alignment():
     """Fragments whose native offsets are not multiples of 4: the places cocodc_select_fragments hands out in
