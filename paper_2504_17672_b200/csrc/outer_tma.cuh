@@ -148,6 +148,7 @@ struct TmaShared {
   unsigned long long* full_bar;
   unsigned long long* empty_bar;
   volatile int* s_fail;
+  double* warp_part;     // where the warps' sums of squares go (shared memory for short id lists), or nullptr
 };
 
 // Lane l of the producer warp owns stream l of the stage (slot order: recorded values, current values, global
@@ -221,6 +222,7 @@ __device__ __noinline__ bool tma_consumer_warps(const OuterArgs& A, const SegPla
   const int S = kRecv ? stages_for(loaded) : L::kStages;
   const int tid = threadIdx.x;
   SlotAccumulator sa(kThreads / 32);
+  sa.cta_part = sh.warp_part;
   TileWalker tw(plan, h.n_seg, kSlot);
   int k = 0;           // staged tiles consumed so far
   for (int tile = blockIdx.x; tile < h.total_tiles; tile += gridDim.x) {
@@ -304,12 +306,15 @@ k_outer_tma(const __grid_constant__ OuterArgs A, const __grid_constant__ FragTab
   sh.full_bar = full_bar;
   sh.empty_bar = empty_bar;
   sh.s_fail = &s_fail;
+  // short id lists: the warps' sums meet in shared memory and the CTA writes one entry per slot
+  const bool in_shared = A.fin.ticket != nullptr && pv.hdr.n_ids <= kFastSlots;
+  sh.warp_part = in_shared ? ip.warp_part : nullptr;
   if (tid >= kThreads) {
     tma_producer_warp<M, MODE, SAME, U>(A, pv.seg, pv.hdr, sh);
     return;
   }
   if (!tma_consumer_warps<M, MODE, SAME, U>(A, pv.seg, pv.hdr, sh)) return;     // warp-uniform by construction
-  if (A.partial) finalize_epilogue(ip, A.fin, pv.hdr, A.partial, kThreads / 32, A.status);
+  if (A.partial) finalize_epilogue(ip, A.fin, pv.hdr, A.partial, kThreads / 32, A.status, in_shared);
 }
 
 }  // namespace cocodc

@@ -209,16 +209,27 @@ __device__ __forceinline__ int arrive_cta(int* shared_counter) {
                : "=r"(old) : "r"((unsigned)__cvta_generic_to_shared(shared_counter)) : "memory");
   return old;
 }
+// the same when both the data and its readers stay inside the CTA (shared memory)
+__device__ __forceinline__ int arrive_cta_local(int* shared_counter) {
+  int old;
+  asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;"
+               : "=r"(old) : "r"((unsigned)__cvta_generic_to_shared(shared_counter)) : "memory");
+  return old;
+}
 __device__ __forceinline__ int arrive_gpu(int* global_counter) {
   int old;
   asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(global_counter) : "memory");
   return old;
 }
 
+constexpr int kFastSlots = 32;   // id lists up to this long keep the per-warp sums of a CTA in shared memory
+
 struct SlotAccumulator {
   double acc = 0.0;
   int slot = 0;
   int warps;   // accumulating warps per CTA (warps 0 .. warps-1 must all call the methods below)
+  double* cta_part = nullptr;   // shared [kFastSlots][warps]: the warps' sums stay in the CTA (the score epilogue
+                                // adds them there and writes one entry per slot); nullptr: one global entry per warp
 
   __device__ __forceinline__ explicit SlotAccumulator(int accumulating_warps) : warps(accumulating_warps) {}
 
@@ -226,9 +237,14 @@ struct SlotAccumulator {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     double v = warp_sum(acc);
     if (lane == 0) {
-      partial[((size_t)slot * gridDim.x + blockIdx.x) * warps + warp] = v;
-      for (int s = slot + 1; s < new_slot; ++s)
-        partial[((size_t)s * gridDim.x + blockIdx.x) * warps + warp] = 0.0;
+      if (cta_part != nullptr) {
+        cta_part[slot * warps + warp] = v;
+        for (int s = slot + 1; s < new_slot; ++s) cta_part[s * warps + warp] = 0.0;
+      } else {
+        partial[((size_t)slot * gridDim.x + blockIdx.x) * warps + warp] = v;
+        for (int s = slot + 1; s < new_slot; ++s)
+          partial[((size_t)s * gridDim.x + blockIdx.x) * warps + warp] = 0.0;
+      }
     }
     acc = 0.0;
     slot = new_slot;
@@ -254,6 +270,8 @@ struct InlinePlan {
   int frag[kInlineSegs];          // fragment id of list position j
   int cnt[kInlineSegs];           // segments of position j, then its first table entry
   int seen[kInlineSegs];
+  long long place[kInlineSegs];   // pool place of every fragment (fetched beside the id list, not after it)
+  double warp_part[kFastSlots * 8];   // per-warp sums of squares of short id lists (SlotAccumulator::cta_part)
   int bad;
   int done_warps;                 // accumulating warps of this CTA that have written their partial sums
 };
@@ -286,9 +304,14 @@ static __device__ __noinline__ PlanView acquire_plan(InlinePlan& ip, const FragT
     return pv;
   }
   const int K = T.K;
+  // the pool places of all K fragments are fetched alongside the list length and the ids, so that the chain of
+  // dependent global loads is two long, not three
+  for (int i = tid; i < K; i += nt) {
+    ip.seen[i] = 0;
+    ip.place[i] = (rq.snap_offset != nullptr) ? rq.snap_offset[i] : 0;
+  }
   int n = (rq.ids == nullptr) ? K : *rq.n_ids;
   if (tid == 0) { ip.bad = (n < 0 || n > K) ? 1 : 0; ip.done_warps = 0; }
-  for (int i = tid; i < K; i += nt) ip.seen[i] = 0;
   __syncthreads();
   if (n < 0 || n > K) n = 0;
   const int lpt = rq.lanes_per_tile;
@@ -296,7 +319,7 @@ static __device__ __noinline__ PlanView acquire_plan(InlinePlan& ip, const FragT
     const int p = (rq.ids == nullptr) ? j : rq.ids[j];
     bool ok = (p >= 0 && p < K);
     if (ok && rq.ids != nullptr && atomicAdd(&ip.seen[p], 1) != 0) ok = false;
-    if (ok && rq.snap_offset != nullptr && rq.snap_offset[p] < 0) ok = false;   // no place in the snapshot pool
+    if (ok && rq.snap_offset != nullptr && ip.place[p] < 0) ok = false;   // no place in the snapshot pool
     long long t = 0;
     int c = 0;
     if (ok) {
@@ -360,7 +383,7 @@ static __device__ __noinline__ PlanView acquire_plan(InlinePlan& ip, const FragT
         SegPlan sp;
         sp.off = T.off[sg];
         sp.len = T.len[sg];
-        sp.snap_off = (rq.snap_offset != nullptr) ? rq.snap_offset[p] + pos : sp.off;
+        sp.snap_off = (rq.snap_offset != nullptr) ? ip.place[p] + pos : sp.off;
         sp.abase = sp.off & ~3LL;
         sp.first_tile = (int)tiles;
         sp.slot = j;
@@ -397,29 +420,34 @@ static __device__ __noinline__ PlanView acquire_plan(InlinePlan& ip, const FragT
 // writes no norms (the status word says why) and the counter is reset by the next status poll.
 // ---------------------------------------------------------------------------
 
-__device__ __forceinline__ void write_fragment_score(const Finalize& F, int j, double total, long long t_p,
-                                                     long long t_l, int* status);
+__device__ __forceinline__ void write_fragment_score(const Finalize& F, int p, long long last, double total,
+                                                     long long t_p, long long t_l, int* status);
 
 static __device__ __noinline__ void finalize_epilogue(InlinePlan& ip, const Finalize& F, const PlanHeader& h,
-                                                  double* __restrict__ partial, int warps, int* status) {
+                                                  double* __restrict__ partial, int warps, int* status,
+                                                  bool in_shared = false) {
   if (F.ticket == nullptr) return;
   const int lane = threadIdx.x & 31;
   const int grid = gridDim.x, cta = blockIdx.x;
   int t = 0;
   __syncwarp();
-  if (lane == 0) t = arrive_cta(&ip.done_warps);
+  if (lane == 0) t = in_shared ? arrive_cta_local(&ip.done_warps) : arrive_cta(&ip.done_warps);
   t = __shfl_sync(0xffffffffu, t, 0);
   if (t != warps - 1) return;
   // (loads first, additions after: the additions keep their order, the loads overlap)
   for (int j = lane; j < h.n_ids; j += 32) {
     double* e = partial + ((size_t)j * grid + cta) * warps;
     double v = 0.0;
-    for (int w0 = 0; w0 < warps; w0 += 8) {
-      double x[8];
+    if (in_shared) {
+      for (int w = 0; w < warps; ++w) v += ip.warp_part[j * warps + w];
+    } else {
+      for (int w0 = 0; w0 < warps; w0 += 8) {
+        double x[8];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) x[q] = (w0 + q < warps) ? __ldcg(e + w0 + q) : 0.0;
+        for (int q = 0; q < 8; ++q) x[q] = (w0 + q < warps) ? __ldcg(e + w0 + q) : 0.0;
 #pragma unroll
-      for (int q = 0; q < 8; ++q) if (w0 + q < warps) v += x[q];
+        for (int q = 0; q < 8; ++q) if (w0 + q < warps) v += x[q];
+      }
     }
     __stcg(e, v);
   }
@@ -431,25 +459,32 @@ static __device__ __noinline__ void finalize_epilogue(InlinePlan& ip, const Fina
   if (F.t_p_dev) t_p = *F.t_p_dev;
   if (F.t_l_dev) t_l = *F.t_l_dev;
   // Four slots at a time, so that their loads are in flight together.  Per slot: lane l adds the entries of
-  // CTAs l, l + 32, ... in that order, then the lanes' sums meet in the shuffle tree.
-  constexpr int kBatch = 4;
+  // CTAs l, l + 32, ... in that order, then the lanes' sums meet in the shuffle tree.  The fragment ids and their
+  // last_sync entries are fetched by lanes 0-3 beside those loads, not after the sums.
+  constexpr int kBatch = 4, kPerLane = 5;       // 32 * 5 = 160 entries per pass: one pass for a grid of 148
   for (int j0 = 0; j0 < h.n_ids; j0 += kBatch) {
+    int my_p = 0;
+    long long my_last = 0;
+    if (lane < kBatch && j0 + lane < h.n_ids) {
+      my_p = (F.ids == nullptr) ? j0 + lane : F.ids[j0 + lane];
+      if (F.write_scores && F.mode == 0) my_last = F.last_sync[my_p];
+    }
     double s[kBatch];
 #pragma unroll
     for (int q = 0; q < kBatch; ++q) s[q] = 0.0;
-    for (int i0 = lane; i0 < grid; i0 += 32 * 4) {
-      double x[kBatch][4];
+    for (int i0 = lane; i0 < grid; i0 += 32 * kPerLane) {
+      double x[kBatch][kPerLane];
 #pragma unroll
       for (int q = 0; q < kBatch; ++q)
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
+        for (int r = 0; r < kPerLane; ++r) {
           const int i = i0 + 32 * r;
           x[q][r] = (j0 + q < h.n_ids && i < grid) ? __ldcg(partial + ((size_t)(j0 + q) * grid + i) * warps) : 0.0;
         }
 #pragma unroll
       for (int q = 0; q < kBatch; ++q)
 #pragma unroll
-        for (int r = 0; r < 4; ++r)
+        for (int r = 0; r < kPerLane; ++r)
           if (j0 + q < h.n_ids && i0 + 32 * r < grid) s[q] += x[q][r];
     }
 #pragma unroll
@@ -457,23 +492,25 @@ static __device__ __noinline__ void finalize_epilogue(InlinePlan& ip, const Fina
       const int j = j0 + q;
       if (j >= h.n_ids) break;
       const double total = warp_sum(s[q]);
-      if (lane == 0) write_fragment_score(F, j, total, t_p, t_l, status);
+      const int p = __shfl_sync(0xffffffffu, my_p, q);
+      const long long last = __shfl_sync(0xffffffffu, my_last, q);
+      if (lane == 0) write_fragment_score(F, p, last, total, t_p, t_l, status);
     }
   }
   __syncwarp();
   if (lane == 0) *F.ticket = 0;
 }
 
-// Last steps of Eq. 10 for one slot, by lane 0 of the warp that holds the slot's total.
-__device__ __forceinline__ void write_fragment_score(const Finalize& F, int j, double total, long long t_p,
-                                                     long long t_l, int* status) {
-  const int p = (F.ids == nullptr) ? j : F.ids[j];
+// Last steps of Eq. 10 for fragment p (last = last_sync[p] as read before), by lane 0 of the warp that holds
+// the fragment's total.
+__device__ __forceinline__ void write_fragment_score(const Finalize& F, int p, long long last, double total,
+                                                     long long t_p, long long t_l, int* status) {
   if (F.sumsq_out) F.sumsq_out[p] = total;
   if (!F.write_scores) return;
   const double norm = sqrt(total);
   long long I = 1;
   if (F.mode == 0) {
-    I = t_p - F.last_sync[p];
+    I = t_p - last;
     F.last_sync[p] = t_l;
     if (F.in_flight) F.in_flight[p] = 0;
   } else if (F.interval != nullptr) {
@@ -527,7 +564,11 @@ static __device__ __noinline__ void finalize_epilogue_cta(InlinePlan& ip, const 
       for (int r = 0; r < 8; ++r) if (i0 + 32 * r < grid) s += x[r];
     }
     const double total = warp_sum(s);
-    if (lane == 0) write_fragment_score(F, j, total, t_p, t_l, status);
+    if (lane == 0) {
+      const int p = (F.ids == nullptr) ? j : F.ids[j];
+      const long long last = (F.write_scores && F.mode == 0) ? F.last_sync[p] : 0;
+      write_fragment_score(F, p, last, total, t_p, t_l, status);
+    }
   }
   if (tid == 0) *F.ticket = 0;
 }
