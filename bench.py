@@ -770,11 +770,16 @@ def run_workers(args):
 
 
 def kernel_source_sha() -> str:
+    """Hash of the fused kernel's sources as the compiler sees them: comments and white space do not count."""
     import hashlib
+    import re
     h = hashlib.sha256()
     for name in ("outer.cuh", "outer_tma.cuh", "plan.cuh"):
-        with open(os.path.join(ROOT, "paper_2504_17672_b200", "csrc", name), "rb") as f:
-            h.update(f.read())
+        with open(os.path.join(ROOT, "paper_2504_17672_b200", "csrc", name), "r") as f:
+            text = f.read()
+        text = re.sub(r"/\*.*?\*/", " ", text, flags=re.S)
+        text = re.sub(r"//[^\n]*", " ", text)
+        h.update(" ".join(text.split()).encode())
     return h.hexdigest()[:16]
 
 

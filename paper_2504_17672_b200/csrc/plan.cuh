@@ -412,7 +412,9 @@ static __device__ __noinline__ PlanView acquire_plan(InlinePlan& ip, const FragT
 // Norms and scores from the partial sums, inside the launch that produced them.
 //
 // Called by every accumulating warp (all 32 lanes) after SlotAccumulator::finish.  The last warp of a CTA to
-// arrive adds that CTA's per-warp entries, slot by slot, into the first of them; the last CTA of the launch to
+// arrive adds that CTA's per-warp sums, slot by slot, into the CTA's first global entry of the slot (the
+// per-warp sums come from shared memory when the id list has at most kFastSlots fragments - in_shared - and from
+// the warps' global entries otherwise; the order of the additions is the same); the last CTA of the launch to
 // get there (a ticket counter in global memory) adds the CTAs' entries of every slot in a fixed order, takes
 // the square root, forms Eq. 10's score and stamps last_sync.  Which warp does the adding varies from run to
 // run, the order of the additions does not, so the rounded result is the same every run.  The ticket counter
