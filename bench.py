@@ -162,7 +162,8 @@ class DeviceJob:
     """Workload resident in HBM plus its schedule state, stepped through the C-ABI binding."""
 
     def __init__(self, w: synth.Workload, device: torch.device, variant: str = "cocodc",
-                 deployment: str = "replicas", world: int = 1, M_total: int = 0, worker_offset: int = 0):
+                 deployment: str = "replicas", world: int = 1, M_total: int = 0, worker_offset: int = 0,
+                 shard: int = 0):
         from paper_2504_17672_b200 import binding as B
         self.B, self.w, self.dev, self.variant = B, w, device, variant
         self.deployment, self.world, self.M_total = deployment, world, (M_total or w.M)
@@ -196,7 +197,7 @@ class DeviceJob:
         ids0 = self.ids[:n].tolist()
         offs = {p: int(self.pool_off[p].item()) for p in ids0}
         self.bufs = synth.generate(w, device, snap_layout="pool", pool_ids=ids0, pool_offsets=offs,
-                                   pool_len=pool_capacity(w), worker_offset=worker_offset)
+                                   pool_len=pool_capacity(w), worker_offset=worker_offset, shard=shard)
         if variant == "diloco":
             self.ids.copy_(torch.arange(K, dtype=torch.int32, device=device))
             self.n_ids.fill_(K)
@@ -218,6 +219,7 @@ class DeviceJob:
     def outer_param_shard(self):
         """This rank's element range: S1-S5 and the local sums of squares; Eq. 10 is finished after the all-reduce."""
         B, b, w = self.B, self.bufs, self.w
+        self.sumsq.zero_()      # entries of fragments not listed now must not carry old totals into the all-reduce
         self.ctx.cocodc_outer_step(self.hyper, b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off,
                                    b.theta_g, b.momentum, None, self.ids, self.n_ids, self.t, self.t + w.tau,
                                    None, None, None, stages=B.STAGE_OUTER | B.STAGE_MERGE | B.STAGE_SUMSQ,
@@ -399,14 +401,18 @@ def run_ours(args):
     if args.variant != "cocodc" and deployment != "replicas":
         raise SystemExit("--variant other than cocodc runs with --deployment replicas")
     w = synth.get_workload(args.workload)
-    M_total, worker_offset = w.M, 0
-    if deployment in ("replicas", "param_shard") and world > 1:
-        w = w.with_(seed=w.seed + 1000 * rank)   # every rank owns a different element range of the same shape
+    M_total, worker_offset, shard = w.M, 0, 0
+    if deployment == "replicas" and world > 1:
+        w = w.with_(seed=w.seed + 1000 * rank)   # every rank owns an independent problem of the same shape
+    if deployment == "param_shard":
+        # every rank owns a different element range of the same fragments: same table, same drift scales and hence
+        # the same initial scores everywhere (the selection is replicated, not communicated), other values
+        shard = rank
     if deployment == "worker_per_device":
         M_local = max(1, w.M // world)           # the workers are spread over the ranks; at least one each
         M_total, worker_offset = M_local * world, M_local * rank
         w = w.with_(M=M_local)
-    job = DeviceJob(w, device, args.variant, deployment, world, M_total, worker_offset)
+    job = DeviceJob(w, device, args.variant, deployment, world, M_total, worker_offset, shard)
     K, W = args.steps, args.warmup
 
     def barrier():

@@ -88,7 +88,7 @@ def _scatter(dst_row: torch.Tensor, segments, vec: torch.Tensor) -> None:
 def generate(w: Workload, device="cpu", *, snap_layout: str = "full",
              pool_ids: Optional[Sequence[int]] = None, pool_len: Optional[int] = None,
              pool_offsets: Optional[Dict[int, int]] = None,
-             momentum_sigma: float = 0.0, worker_offset: int = 0) -> DeviceBuffers:
+             momentum_sigma: float = 0.0, worker_offset: int = 0, shard: int = 0) -> DeviceBuffers:
     """Fill the buffers of one workload.
 
     snap_layout="full": w_snap is [M, N] laid out like w_now.
@@ -98,20 +98,23 @@ def generate(w: Workload, device="cpu", *, snap_layout: str = "full",
     unless `pool_offsets` places them explicitly.
     worker_offset: the M workers generated here are workers worker_offset .. worker_offset + M - 1 of a larger
     job (the workers of one device when they are spread over several); the global state does not depend on it.
+    shard: which element range of a larger model this is (a model split over several devices by parameter range):
+    another shard has the same fragment table and drift scales but its own random values.
     """
     device = torch.device(device)
     part = w.partition
     N, M, K = w.N, w.M, w.K
     scales = fragment_scales(w)
+    vseed = w.seed + 1_000_003 * shard          # seed of the value streams; the scales keep the workload's own
 
     theta_g = torch.empty(N, dtype=torch.float32, device=device)
     momentum = torch.zeros(N, dtype=torch.float32, device=device)
     w_now = torch.empty((M, N), dtype=torch.float32, device=device)
     covered = sum(part.frag_size(p) for p in range(K))
     if covered != N:  # gaps between fragments (test workloads only): fill the background first
-        theta_g.copy_(_randn(N, device, _seed(w.seed, _BUF_GAP, 0, 0)) * w.sigma_global)
+        theta_g.copy_(_randn(N, device, _seed(vseed, _BUF_GAP, 0, 0)) * w.sigma_global)
         for m in range(M):
-            w_now[m].copy_(theta_g + _randn(N, device, _seed(w.seed, _BUF_GAP, 1, m)) * w.sigma_drift)
+            w_now[m].copy_(theta_g + _randn(N, device, _seed(vseed, _BUF_GAP, 1, m)) * w.sigma_drift)
 
     snap_offset = None
     if snap_layout == "full":
@@ -142,20 +145,20 @@ def generate(w: Workload, device="cpu", *, snap_layout: str = "full",
         segs = part.fragments[p]
         n = part.frag_size(p)
         s = float(scales[p])
-        tg = _randn(n, device, _seed(w.seed, _BUF_GLOBAL, p, 0)).mul_(w.sigma_global)
+        tg = _randn(n, device, _seed(vseed, _BUF_GLOBAL, p, 0)).mul_(w.sigma_global)
         _scatter(theta_g, segs, tg)
         if momentum_sigma > 0.0:
-            _scatter(momentum, segs, _randn(n, device, _seed(w.seed, _BUF_MOM, p, 0)).mul_(momentum_sigma))
-        e = _randn(n, device, _seed(w.seed, _BUF_SHARED, p, 0)).mul_(w.sigma_drift)
+            _scatter(momentum, segs, _randn(n, device, _seed(vseed, _BUF_MOM, p, 0)).mul_(momentum_sigma))
+        e = _randn(n, device, _seed(vseed, _BUF_SHARED, p, 0)).mul_(w.sigma_drift)
         for m in range(M):
-            snap = _randn(n, device, _seed(w.seed, _BUF_SNAP, p, m + worker_offset)).mul_(s).add_(tg)
+            snap = _randn(n, device, _seed(vseed, _BUF_SNAP, p, m + worker_offset)).mul_(s).add_(tg)
             if p in in_pool:
                 if snap_offset is None:
                     _scatter(w_snap[m], segs, snap)
                 else:
                     o = int(snap_offset[p])
                     w_snap[m, o:o + n] = snap
-            eps = _randn(n, device, _seed(w.seed, _BUF_WORKER, p, m + worker_offset)).mul_(0.1 * w.sigma_drift)
+            eps = _randn(n, device, _seed(vseed, _BUF_WORKER, p, m + worker_offset)).mul_(0.1 * w.sigma_drift)
             eps.add_(e).mul_(s / w.sigma_drift).add_(snap)
             _scatter(w_now[m], segs, eps)
             del snap, eps

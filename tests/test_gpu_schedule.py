@@ -126,3 +126,34 @@ def test_toy_training_converges_under_every_variant(variant, lam, tau):
     assert r.syncs >= 300 // 20
     start, final = r.losses[0][1], r.final
     assert np.isfinite(final) and final < 0.02 * start, (start, final)
+
+
+def test_two_parameter_range_shards_keep_the_same_selection():
+    """The benchmark's param_shard deployment, two ranks taken in turn on one GPU: each shard completes its element
+    range and contributes its sums of squares, the totals (added here where the all-reduce would add them) give
+    every shard the same scores and last_sync, and the replicated selection must pick the same fragments on both,
+    step after step - without any exchange of the decision itself (Section 3.2)."""
+    import bench
+    w = synth.get_workload("gpt2_small")
+    dev = torch.device("cuda", 0)
+    jobs = [bench.DeviceJob(w, dev, "cocodc", "param_shard", world=1, M_total=w.M, worker_offset=0, shard=r)
+            for r in range(2)]
+    assert not torch.equal(jobs[0].bufs.theta_g, jobs[1].bufs.theta_g)          # different element ranges
+    assert torch.equal(jobs[0].ids, jobs[1].ids) and torch.equal(jobs[0].n_ids, jobs[1].n_ids)
+    seen = []
+    for step in range(6):
+        for j in jobs:
+            j.outer_param_shard()
+        total = jobs[0].sumsq + jobs[1].sumsq
+        for j in jobs:
+            j.sumsq.copy_(total)
+            j.ctx.cocodc_scores_from_sumsq(j.sumsq, j.ids, j.n_ids, None, j.t, j.t + w.tau, j.last_sync, j.norms,
+                                           j.scores)
+            j.t += w.tau
+            j.initiate()
+            assert j.ctx.cocodc_poll_status() == 0
+        a, b = jobs
+        assert torch.equal(a.ids, b.ids) and torch.equal(a.n_ids, b.n_ids), step
+        assert torch.equal(a.scores, b.scores) and torch.equal(a.last_sync, b.last_sync), step
+        seen.append(np_(a.ids)[:int(a.n_ids.item())].tolist())
+    assert len({tuple(s) for s in seen}) > 1          # the schedule moves on
