@@ -157,3 +157,42 @@ def test_two_parameter_range_shards_keep_the_same_selection():
         assert torch.equal(a.scores, b.scores) and torch.equal(a.last_sync, b.last_sync), step
         seen.append(np_(a.ids)[:int(a.n_ids.item())].tolist())
     assert len({tuple(s) for s in seen}) > 1          # the schedule moves on
+
+
+def test_two_worker_groups_keep_the_replicated_state_identical():
+    """The benchmark's worker_per_device deployment, two ranks taken in turn on one GPU: each holds two of the four
+    workers and the whole (replicated) global state; the pseudo-gradient sums are added where the all-reduce would
+    add them, and every rank completes from the same received sum - global state, momentum, scores and the
+    selection must stay bit-identical on both ranks, and agree with the four-worker step on one device."""
+    import bench
+    w4 = synth.get_workload("gpt2_small")
+    w2 = w4.with_(M=2)
+    dev = torch.device("cuda", 0)
+    ranks = [bench.DeviceJob(w2, dev, "cocodc", "worker_per_device", world=1, M_total=4, worker_offset=2 * r)
+             for r in range(2)]
+    whole = bench.DeviceJob(w4, dev, "cocodc", "replicas")
+    assert torch.equal(ranks[0].bufs.theta_g, ranks[1].bufs.theta_g) and torch.equal(ranks[0].bufs.theta_g, whole.bufs.theta_g)
+    assert torch.equal(ranks[1].bufs.w_now[0], whole.bufs.w_now[2])               # rank 1 holds workers 2 and 3
+    for step in range(4):
+        assert torch.equal(ranks[0].ids, whole.ids)
+        for j in ranks:
+            j.pseudo_sum_and_exchange()
+        total = ranks[0].sum_buf + ranks[1].sum_buf
+        for j in ranks:
+            j.sum_buf.copy_(total)
+            j.outer_received()
+            j.t += w2.tau
+            j.initiate()
+            assert j.ctx.cocodc_poll_status() == 0
+        whole.step()
+        a, b = ranks
+        for x, y in ((a.bufs.theta_g, b.bufs.theta_g), (a.bufs.momentum, b.bufs.momentum), (a.scores, b.scores),
+                     (a.last_sync, b.last_sync), (a.ids, b.ids), (a.n_ids, b.n_ids)):
+            assert torch.equal(x, y), step
+        # against all four workers on one device: the same up to the order in which the four differences are added
+        ref = whole.bufs.theta_g
+        err = float((a.bufs.theta_g - ref).abs().max() / ref.abs().max())
+        assert err <= 1e-6, (step, err)
+        assert torch.allclose(a.scores, whole.scores, rtol=1e-5)
+        # each rank merged its own two workers: they match the four-worker job's rows
+        assert float((b.bufs.w_now - whole.bufs.w_now[2:4]).abs().max()) <= 1e-6 * float(whole.bufs.w_now.abs().max())
