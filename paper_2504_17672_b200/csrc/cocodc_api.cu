@@ -132,7 +132,7 @@ Variant staged_variant() {
 // More than 48 KB of dynamic shared memory needs a one-time opt-in per kernel and device (the
 // caller has made the context's device current).
 void opt_in_shared_memory(cocodc_ctx* c, const void* kernel, unsigned bytes) {
-  if (bytes <= 32u * 1024u) return;   // static shared memory (about 9 KB: the plan) counts towards the 48 KB a kernel gets without opting in
+  if (bytes <= 24u * 1024u) return;   // static shared memory (up to 16 KB: plan, selection state) counts towards the 48 KB a kernel gets without opting in
   for (auto& k : c->smem_opted_in) {
     if (k.first != kernel) continue;
     if (k.second >= bytes) return;
