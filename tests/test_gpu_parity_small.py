@@ -240,7 +240,46 @@ def test_host_validation_errors():
     assert code(stages=2) == B.ERR_INVALID_ARG
     assert code(ids=None) == B.ERR_INVALID_ARG
     assert code(t_p=5, t_l=4) == B.ERR_INVALID_ARG
+    assert code(stages=1 | 2 | 8) == B.ERR_INVALID_ARG               # sums asked for without a place for them
+    assert code(stages=16 | 1) == B.ERR_INVALID_ARG
     call(hyper=prob.hyper(tau=0, comp_mode=0))                        # legal: no compensation
+    assert prob.poll() == 0
+
+    # the other new calls
+    K = prob.w.K
+    sq = torch.zeros(K, dtype=torch.float64, device="cuda")
+    ctx = prob.ctx
+
+    def raises(fn, *a, **kw):
+        with pytest.raises(B.CocodcError) as e:
+            fn(*a, **kw)
+        return e.value.code
+
+    assert raises(ctx.cocodc_scores_from_sumsq, None, prob.ids, prob.n_ids, None, 1, 2, prob.last_sync, prob.norms,
+                  prob.scores) == B.ERR_INVALID_ARG
+    assert raises(ctx.cocodc_scores_from_sumsq, sq, prob.ids, None, None, 1, 2, prob.last_sync, prob.norms,
+                  prob.scores) == B.ERR_INVALID_ARG              # a list without its length
+    assert raises(ctx.cocodc_scores_from_sumsq, sq, prob.ids, prob.n_ids, None, 3, 2, prob.last_sync, prob.norms,
+                  prob.scores) == B.ERR_INVALID_ARG              # completes before it was initiated
+    assert raises(ctx.cocodc_scores_from_sumsq, sq, prob.ids, prob.n_ids, prob.last_sync, 1, 2, prob.last_sync,
+                  prob.norms, prob.scores) == B.ERR_INVALID_ARG  # intervals belong to the stand-alone form
+    assert raises(ctx.cocodc_fragment_scores, b.theta_g, None, prob.norms, None) == B.ERR_INVALID_ARG
+    assert raises(ctx.cocodc_fragment_scores, b.theta_g, None, None, None) == B.ERR_INVALID_ARG
+
+    def initiate(**kw):
+        a = dict(scores=prob.scores, last_sync=prob.last_sync, ineligible=None, t_now=5, H=100, budget_kind=0,
+                 budget=1, mask=prob.mask, ids=prob.ids, n_sel=prob.n_ids, pool_offset=None, w_now=b.w_now,
+                 w_snap=b.w_snap, now_stride=b.now_stride, snap_stride=b.snap_stride, M=2)
+        a.update(kw)
+        return raises(ctx.cocodc_initiate, **a)
+
+    assert initiate(w_snap=b.w_now) == B.ERR_ALIAS
+    assert initiate(now_stride=b.now_stride + 2) == B.ERR_ALIGNMENT
+    assert initiate(w_now=b.w_now.view(-1)[1:]) == B.ERR_ALIGNMENT
+    assert initiate(M=3) == B.ERR_INVALID_ARG
+    assert initiate(budget_kind=7) == B.ERR_INVALID_ARG
+    assert initiate(H=0) == B.ERR_INVALID_ARG
+    assert initiate(mask=None) == B.ERR_INVALID_ARG
     assert prob.poll() == 0
 
 
