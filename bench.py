@@ -367,7 +367,8 @@ def roofline_record(w, variant, deployment, leg, K, peak, peak_kind, traffic=Non
     if w.M > 8:
         kernel = "k_outer_ring (fused S1-S6)"
     elif variant == "diloco":
-        kernel = f"k_outer_inplace<{w.M}> (fused S1-S6, zero delay)"
+        name = "k_outer_inplace" if w.M in (3, 4, 5) else "k_outer_tma"   # the library's choice per worker count
+        kernel = f"{name}<{w.M}> (fused S1-S6, zero delay)"
     elif deployment == "worker_per_device":
         kernel = f"k_outer_tma<{w.M}, received sum> (S2-S6)"
     else:
