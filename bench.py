@@ -163,9 +163,11 @@ class DeviceJob:
 
     def __init__(self, w: synth.Workload, device: torch.device, variant: str = "cocodc",
                  deployment: str = "replicas", world: int = 1, M_total: int = 0, worker_offset: int = 0,
-                 shard: int = 0):
+                 shard: int = 0, defer_scores: bool = False):
         from paper_2504_17672_b200 import binding as B
         self.B, self.w, self.dev, self.variant = B, w, device, variant
+        # the completion leaves the last steps of Eq. 10 to the initiation that follows it in the same step
+        self.defer = defer_scores and deployment == "replicas" and variant != "diloco"
         self.deployment, self.world, self.M_total = deployment, world, (M_total or w.M)
         ptr, off, ln = w.partition.csr()
         self.ctx = B.Context(w.N, ptr, off, ln, w.M, device=device.index or 0)
@@ -268,7 +270,8 @@ class DeviceJob:
             return
         self.ctx.cocodc_outer_step(self.hyper, b.w_now, b.w_snap, b.now_stride, b.snap_stride, self.pool_off,
                                    b.theta_g, b.momentum, None, self.ids, self.n_ids, self.t, self.t + w.tau,
-                                   self.last_sync, self.norms, self.scores)
+                                   self.last_sync, self.norms, self.scores,
+                                   stages=self.B.STAGE_ALL | (self.B.STAGE_DEFER if self.defer else 0))
 
     def initiate(self):
         """Algorithm 2 for the next set and the snapshot of what it picks (cocodc_initiate: one launch)."""
@@ -358,7 +361,7 @@ def completion_bytes_per_param(M: int, variant: str, deployment: str) -> int:
     return bytes_per_param(M)
 
 
-def roofline_record(w, variant, deployment, leg, K, peak, peak_kind, traffic=None):
+def roofline_record(w, variant, deployment, leg, K, peak, peak_kind, traffic=None, deferred=False):
     bpp = completion_bytes_per_param(w.M, variant, deployment)
     outer_seconds = sum(leg["outer_ms"]) / 1e3
     params = float(sum(leg["per_step"]))
@@ -373,6 +376,8 @@ def roofline_record(w, variant, deployment, leg, K, peak, peak_kind, traffic=Non
         kernel = f"k_outer_tma<{w.M}, received sum> (S2-S6)"
     else:
         kernel = f"k_outer_tma<{w.M}> (fused S1-S6)"
+    if deferred:      # the launch ends with the CTAs' sums of squares; the next launch's prologue forms the scores
+        kernel = kernel.replace("S1-S6", "S1-S5 + sums of squares of S6")
     return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
             "bytes_per_param": bpp, "ms_per_launch": outer_seconds / K * 1e3,
@@ -413,7 +418,8 @@ def run_ours(args):
         M_local = max(1, w.M // world)           # the workers are spread over the ranks; at least one each
         M_total, worker_offset = M_local * world, M_local * rank
         w = w.with_(M=M_local)
-    job = DeviceJob(w, device, args.variant, deployment, world, M_total, worker_offset, shard)
+    job = DeviceJob(w, device, args.variant, deployment, world, M_total, worker_offset, shard,
+                    defer_scores=args.defer_scores)
     K, W = args.steps, args.warmup
 
     def barrier():
@@ -446,12 +452,13 @@ def run_ours(args):
     snap_bpp = 8 * w.M if args.variant != "diloco" else 0
     traffic = (read_traffic_note(w, params_local / K)
                if args.variant == "cocodc" and deployment in ("replicas", "param_shard") else None)
-    roof = roofline_record(w, args.variant, deployment, leg, K, peak, peak_kind, traffic)
+    roof = roofline_record(w, args.variant, deployment, leg, K, peak, peak_kind, traffic, deferred=job.defer)
     step_bytes = params_local * roof["bytes_per_param"] + float(sum(leg["per_step_snapshot"])) * snap_bpp
     if deployment == "worker_per_device":
         step_bytes += params_local * (4 * w.M + 8)       # the pseudo-gradient sum's own pass
     steps_desc = {
-        "replicas": "outer_step(S1-S6) + initiate(S7 + S0)",
+        "replicas": ("outer_step(S1-S6, the root and division of Eq. 10 left to the next launch) + "
+                     "initiate(those, S7 + S0)" if job.defer else "outer_step(S1-S6) + initiate(S7 + S0)"),
         "param_shard": "outer_step(S1-S5 + sums of squares) + all-reduce of K fp64 + scores_from_sumsq(S6) "
                        "+ initiate(S7 + S0)",
         "worker_per_device": "pseudo_gradient_sum(S1) + all-reduce of the listed fragments + outer_step_received(S2-S6) "
@@ -512,11 +519,11 @@ def second_shape_roofline(name: str, args, device, local, peak, peak_kind):
     if free < 115 * 2 ** 30:
         return {"workload": name, "skipped": f"needs about 105 GB of device memory, {free / 2 ** 30:.0f} GB free"}
     w = synth.get_workload(name)
-    job = DeviceJob(w, device, "cocodc")
+    job = DeviceJob(w, device, "cocodc", defer_scores=args.defer_scores)
     K = max(4, min(args.steps, 20))
     leg = timed_device_leg(job, K, 3, device, local, lambda: torch.cuda.synchronize(device))
     roof = roofline_record(w, "cocodc", "replicas", leg, K, peak, peak_kind,
-                           read_traffic_note(w, float(sum(leg["per_step"])) / K))
+                           read_traffic_note(w, float(sum(leg["per_step"])) / K), deferred=job.defer)
     roof.update({"workload": name, "steps": K, "ms_per_step": leg["seconds"] / K * 1e3,
                  "params_per_s": float(sum(leg["per_step"])) / leg["seconds"],
                  "clocks": leg["clocks"], "gpu_launches": int(leg["launches"])})
@@ -1053,6 +1060,10 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-3b", action="store_true", help="skip the device-only roofline record on llama_3b")
+    ap.add_argument("--defer-scores", action="store_true",
+                    help="leave the last steps of Eq. 10 (root, division by I_p, last_sync) to the initiation that "
+                         "follows the completion in the same step (COCODC_STAGE_DEFER) instead of forming them inside "
+                         "the completion's own launch")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="wall time spent timing the oracle")
     ap.add_argument("--cpu-sample", type=int, default=16_000_000, help="parameters in the oracle's sample")

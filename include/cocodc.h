@@ -97,6 +97,19 @@ typedef enum { COCODC_BUDGET_COUNT = 0, COCODC_BUDGET_PARAMS = 1, COCODC_BUDGET_
 #define COCODC_STAGE_ALL   7u
 #define COCODC_STAGE_SUMSQ 8u   /* S6 up to the sums only: sumsq_out[p] = sum of Delta^2 over fragment p (Eq. 10 before the
                                    square root), for callers that add the sums of several devices before forming scores */
+#define COCODC_STAGE_DEFER 16u  /* with COCODC_STAGE_SCORE (and without sumsq_out): the launch ends once every thread block
+                                   has left its sum of squares per fragment in the context's scratch; the square root, the
+                                   division by I_p, last_sync and the in-flight marks (the rest of Eq. 10 and the text after
+                                   it) are formed by the next call on the context that decides on fragments -
+                                   cocodc_initiate(_at), in the prologue of its one launch when it is given the same scores
+                                   and last_sync arrays - or, failing that, by one small launch placed before any other
+                                   call that reads or writes norms, scores, last_sync or that scratch (cocodc_outer_step
+                                   and its variants, cocodc_select_fragments(_at), cocodc_fragment_scores,
+                                   cocodc_scores_from_sumsq, cocodc_outer_step_host) or by cocodc_flush_scores.  Until
+                                   then norms, scores, last_sync and the in-flight marks keep their previous contents.
+                                   The values are bit for bit those of the undeferred stage.  Why: forming the scores
+                                   inside the completion's launch costs a grid-wide hand-off after its last tile (about
+                                   7 us whatever the launch size); the boundary to the next launch is that hand-off. */
 
 /*
  * Fragment partition (Section 2.1: the model is cut into K disjoint fragments).
@@ -191,6 +204,15 @@ cocodc_status cocodc_scores_from_sumsq(cocodc_ctx* ctx, const double* sumsq, con
  * NULL unbinds.  The host-buffer entry points do not use it.
  */
 cocodc_status cocodc_bind_in_flight(cocodc_ctx* ctx, uint8_t* in_flight);
+
+/*
+ * Forms the norms, scores, last_sync entries and in-flight marks that a completion launched with
+ * COCODC_STAGE_DEFER has left unformed (one launch of one thread block on `stream`, which must be the
+ * stream of that completion or ordered after it); does nothing when no such completion is outstanding.
+ * The arrays written are the ones that completion was given.  Errors: INVALID_ARG for a NULL context; a
+ * non-finite norm is reported through the status word (COCODC_ERR_NONFINITE) as in the undeferred stage.
+ */
+cocodc_status cocodc_flush_scores(cocodc_ctx* ctx, void* stream);
 
 /*
  * S7 (Algorithm 2, Eq. 11, extended to a budget).  Priority order: eligible

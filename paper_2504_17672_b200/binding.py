@@ -20,7 +20,7 @@ OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_ALIAS, ERR_NONFINITE, ERR_TIMEOUT, ERR_C
 COMP_NONE, COMP_TAYLOR = 0, 1
 SIGN_FORWARD, SIGN_PRINTED, SIGN_DESCENT = 0, 1, 2
 BUDGET_COUNT, BUDGET_PARAMS, BUDGET_PARAMS_EXACT = 0, 1, 2
-STAGE_OUTER, STAGE_MERGE, STAGE_SCORE, STAGE_ALL, STAGE_SUMSQ = 1, 2, 4, 7, 8
+STAGE_OUTER, STAGE_MERGE, STAGE_SCORE, STAGE_ALL, STAGE_SUMSQ, STAGE_DEFER = 1, 2, 4, 7, 8, 16
 
 EXPORTS = (
     "cocodc_create", "cocodc_destroy", "cocodc_sync_budget", "cocodc_fragment_scores",
@@ -29,7 +29,7 @@ EXPORTS = (
     "cocodc_fragment_scores_noalloc", "cocodc_selftest_bounded_wait",
     "cocodc_pseudo_gradient_sum", "cocodc_outer_step_received",
     "cocodc_select_fragments_at", "cocodc_outer_step_at", "cocodc_outer_step_received_peers",
-    "cocodc_scores_from_sumsq", "cocodc_bind_in_flight", "cocodc_initiate", "cocodc_initiate_at",
+    "cocodc_scores_from_sumsq", "cocodc_bind_in_flight", "cocodc_flush_scores", "cocodc_initiate", "cocodc_initiate_at",
 )
 NOALLOC_MAX_K, NOALLOC_MAX_SEGMENTS = 64, 64
 
@@ -86,6 +86,7 @@ def _load() -> ctypes.CDLL:
     lib.cocodc_fragment_scores.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.cocodc_scores_from_sumsq.argtypes = [vp, vp, vp, vp, vp, i64, i64, vp, vp, vp, vp]
     lib.cocodc_bind_in_flight.argtypes = [vp, vp]
+    lib.cocodc_flush_scores.argtypes = [vp, vp]
     lib.cocodc_initiate.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp, vp, i64, i64, i32, vp]
     lib.cocodc_initiate_at.argtypes = [vp, vp, vp, vp, vp, i64, i32, i64, vp, vp, vp, vp, vp, vp, i64, i64, i32, vp]
     lib.cocodc_select_fragments.argtypes = [vp, vp, vp, vp, i64, i64, i32, i64, vp, vp, vp, vp, vp]
@@ -215,6 +216,10 @@ class Context:
         """Bind (or, with None, unbind) the caller's device uint8[K] mask of fragments in flight."""
         self._in_flight = in_flight          # keeps the tensor alive while the context points at it
         _check(_lib.cocodc_bind_in_flight(self._h, _p(in_flight)), "cocodc_bind_in_flight")
+
+    def cocodc_flush_scores(self, stream=None) -> None:
+        """Form the scores a completion launched with STAGE_DEFER left unformed (no-op when there is none)."""
+        _check(_lib.cocodc_flush_scores(self._h, _stream(stream)), "cocodc_flush_scores")
 
     def cocodc_select_fragments(self, scores, last_sync, ineligible, t_now: int, H: int, budget_kind: int,
                                 budget: int, mask, ids, n_sel, pool_offset=None, stream=None) -> None:

@@ -41,6 +41,13 @@ struct cocodc_ctx {
   int* d_status = nullptr;
   int* d_ticket = nullptr;                  // arrival counter of the in-kernel score epilogue (zero between launches)
   unsigned char* in_flight = nullptr;       // caller's in-flight mask (cocodc_bind_in_flight), or nullptr
+  // a completion launched with COCODC_STAGE_DEFER whose scores no call has formed yet (host view of d_pending->n)
+  PendingScores* d_pending = nullptr;
+  bool pending = false;
+  float* pend_norms = nullptr;
+  float* pend_scores = nullptr;
+  long long* pend_last = nullptr;
+  int pend_grid = 0;                         // CTAs of the deferred completion's launch
   FragTable table{};                        // the fragment table as a kernel argument, when it is small enough
   bool inline_plan = false;                 // the streaming kernels expand the id list themselves (no k_plan launch)
   long long launches = 0;
@@ -100,6 +107,17 @@ cocodc_status launch_plan(cocodc_ctx* c, const int32_t* ids, const int32_t* n_id
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
+// Scores that a deferred completion left unformed are formed now (one small launch), before a call that reads or
+// writes the schedule arrays, or the scratch the CTAs' sums sit in, without being the selection that consumes them.
+cocodc_status flush_pending(cocodc_ctx* c, cudaStream_t st) {
+  if (!c->pending) return COCODC_OK;
+  k_flush_pending<<<1, 256, 0, st>>>(c->d_pending, c->d_partial, c->K, c->pend_norms, c->pend_scores, c->pend_last,
+                                     c->in_flight, c->d_status, (int)COCODC_ERR_NONFINITE);
+  c->launches++;
+  c->pending = false;
+  return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
+}
+
 // One way to run the streaming step: which kernel, with how many threads and how much dynamic
 // shared memory, on how many CTAs, over tiles of how many lanes.  Every variant has eight accumulating
 // warps, so the score epilogue does not depend on the choice; the plan is built for the variant's tile.
@@ -132,7 +150,7 @@ Variant staged_variant() {
 // More than 48 KB of dynamic shared memory needs a one-time opt-in per kernel and device (the
 // caller has made the context's device current).
 void opt_in_shared_memory(cocodc_ctx* c, const void* kernel, unsigned bytes) {
-  if (bytes <= 24u * 1024u) return;   // static shared memory (up to 16 KB: plan, selection state) counts towards the 48 KB a kernel gets without opting in
+  if (bytes <= 24u * 1024u) return;   // static shared memory (up to 18 KB: plan, selection state) counts towards the 48 KB a kernel gets without opting in
   for (auto& k : c->smem_opted_in) {
     if (k.first != kernel) continue;
     if (k.second >= bytes) return;
@@ -241,6 +259,7 @@ cocodc_status launch_outer(cocodc_ctx* c, const OuterArgs& A, int mode, bool sam
   args.ring_slots = v.ring_slots;
   v.kernel<<<grid, v.threads, v.smem, st>>>(args, c->table);
   c->launches++;
+  if (A.fin.defer) c->pend_grid = grid;
   return cudaGetLastError() == cudaSuccess ? COCODC_OK : COCODC_ERR_CUDA;
 }
 
@@ -380,6 +399,7 @@ cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, 
   ok = ok && cudaMalloc(&c->d_partial, sizeof(double) * partial_elems) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_status, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_ticket, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->d_pending, sizeof(PendingScores)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_frag_sumsq, sizeof(double) * K) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_k_ids, sizeof(int) * K) == cudaSuccess;
   ok = ok && cudaMalloc(&c->d_k_last, sizeof(long long) * K) == cudaSuccess;
@@ -408,6 +428,7 @@ cocodc_status cocodc_create(cocodc_ctx** ctx_out, const cocodc_partition* part, 
   }
   ok = ok && cudaMemset(c->d_status, 0, sizeof(int)) == cudaSuccess;
   ok = ok && cudaMemset(c->d_ticket, 0, sizeof(int)) == cudaSuccess;
+  ok = ok && cudaMemset(c->d_pending, 0, sizeof(PendingScores)) == cudaSuccess;
   ok = ok && cudaMemset(c->d_hdr, 0, sizeof(PlanHeader)) == cudaSuccess;
   c->inline_plan = (S <= kInlineSegs);
   if (c->inline_plan) {
@@ -434,6 +455,7 @@ cocodc_status cocodc_destroy(cocodc_ctx* c) {
   cudaFree(c->d_partial);
   cudaFree(c->d_status);
   cudaFree(c->d_ticket);
+  cudaFree(c->d_pending);
   cudaFree(c->d_frag_sumsq);
   cudaFree(c->d_k_ids);
   cudaFree(c->d_k_last);
@@ -462,6 +484,11 @@ cocodc_status cocodc_poll_status(cocodc_ctx* c, void* stream) {
   if (cudaStreamSynchronize(st) != cudaSuccess) return COCODC_ERR_CUDA;
   // a launch that gave up on a bounded wait leaves the arrival counter of its score epilogue behind
   if (word != 0 && cudaMemsetAsync(c->d_ticket, 0, sizeof(int), st) != cudaSuccess) return COCODC_ERR_CUDA;
+  // ... and a deferred completion that failed leaves nothing worth forming
+  if (word != 0 && c->pending) {
+    if (cudaMemsetAsync(c->d_pending, 0, sizeof(int), st) != cudaSuccess) return COCODC_ERR_CUDA;
+    c->pending = false;
+  }
   return static_cast<cocodc_status>(word);
 }
 
@@ -472,6 +499,7 @@ cocodc_status cocodc_fragment_scores(cocodc_ctx* c, const float* delta_g, const 
   if (!aligned16(delta_g)) return COCODC_ERR_ALIGNMENT;
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (flush_pending(c, st) != COCODC_OK) return COCODC_ERR_CUDA;
   constexpr int U = 4;
   auto kernel = k_sumsq<U>;
   const int grid = grid_for(c, reinterpret_cast<const void*>(kernel));
@@ -502,6 +530,7 @@ cocodc_status cocodc_scores_from_sumsq(cocodc_ctx* c, const double* sumsq, const
   if (completion && (!n_ids || !last_sync || interval || t_l < t_p)) return COCODC_ERR_INVALID_ARG;
   if (!completion && n_ids) return COCODC_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
+  if (flush_pending(c, static_cast<cudaStream_t>(stream)) != COCODC_OK) return COCODC_ERR_CUDA;
   k_scores_from_sumsq<<<1, kFinalizeThreads, 0, static_cast<cudaStream_t>(stream)>>>(
       sumsq, 0, ids, n_ids, 0, c->K, completion ? 0 : 1, reinterpret_cast<const long long*>(interval), t_p, t_l,
       reinterpret_cast<long long*>(last_sync), norms, scores, completion ? c->in_flight : nullptr, c->d_status,
@@ -514,6 +543,12 @@ cocodc_status cocodc_bind_in_flight(cocodc_ctx* c, uint8_t* in_flight) {
   if (!c) return COCODC_ERR_INVALID_ARG;
   c->in_flight = in_flight;
   return COCODC_OK;
+}
+
+cocodc_status cocodc_flush_scores(cocodc_ctx* c, void* stream) {
+  if (!c) return COCODC_ERR_INVALID_ARG;
+  DeviceGuard guard(c->device);
+  return flush_pending(c, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"
@@ -531,6 +566,7 @@ cocodc_status select_impl(cocodc_ctx* c, const float* scores, const int64_t* las
     return COCODC_ERR_INVALID_ARG;
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (flush_pending(c, st) != COCODC_OK) return COCODC_ERR_CUDA;
   k_select<<<1, kSelectThreads, 0, st>>>(c->K, scores, reinterpret_cast<const long long*>(last_sync), ineligible,
                                          c->d_frag_size, c->d_frag_first_off, t_now, reinterpret_cast<const long long*>(t_now_dev), H, budget_kind, budget, mask, ids, n_sel,
                                          reinterpret_cast<long long*>(pool_offset), c->in_flight, c->d_status, (int)COCODC_ERR_NONFINITE,
@@ -558,9 +594,13 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
     if (!delta_sums[r]) return COCODC_ERR_INVALID_ARG;
     if (!aligned16(delta_sums[r])) return COCODC_ERR_ALIGNMENT;
   }
-  if (!(stages & COCODC_STAGE_OUTER) || (stages & ~(COCODC_STAGE_ALL | COCODC_STAGE_SUMSQ))) return COCODC_ERR_INVALID_ARG;
+  if (!(stages & COCODC_STAGE_OUTER) || (stages & ~(COCODC_STAGE_ALL | COCODC_STAGE_SUMSQ | COCODC_STAGE_DEFER)))
+    return COCODC_ERR_INVALID_ARG;
   const bool do_merge = (stages & COCODC_STAGE_MERGE) != 0;
   const bool do_score = (stages & COCODC_STAGE_SCORE) != 0;
+  const bool defer = (stages & COCODC_STAGE_DEFER) != 0;
+  // deferring is a way of running the SCORE stage; the sums of squares themselves are then not handed out
+  if (defer && (!do_score || (stages & COCODC_STAGE_SUMSQ) || sumsq_out)) return COCODC_ERR_INVALID_ARG;
   const bool do_sums = do_score || (stages & COCODC_STAGE_SUMSQ) != 0;
   if ((stages & COCODC_STAGE_SUMSQ) && !sumsq_out) return COCODC_ERR_INVALID_ARG;
   if (!w_snap || !theta_g || !momentum || !ids || !n_ids) return COCODC_ERR_INVALID_ARG;
@@ -601,6 +641,7 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
   }
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (flush_pending(c, st) != COCODC_OK) return COCODC_ERR_CUDA;
   OuterArgs A{};
   A.w_now = w_now;
   A.w_snap = w_snap;
@@ -627,6 +668,7 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
     A.fin.sumsq_out = sumsq_out;
     A.fin.in_flight = do_score ? c->in_flight : nullptr;
     A.fin.err_nonfinite = (int)COCODC_ERR_NONFINITE;
+    A.fin.defer = defer ? c->d_pending : nullptr;
   }
   fold_coefficients(h, same, &A);
   if (received) {   // Eq. 1 divides the received sum by the number of workers that contributed to it
@@ -636,7 +678,14 @@ cocodc_status outer_step_impl(cocodc_ctx* c, const cocodc_hyper* h,
   }
   set_status_sink(c, &A);
   const int mode = received ? MODE_FUSED_RECV : (do_merge ? MODE_FUSED : MODE_OUTER_ONLY);
-  return launch_outer(c, A, mode, same, ids, n_ids, snap_offset, st);
+  s = launch_outer(c, A, mode, same, ids, n_ids, snap_offset, st);
+  if (s == COCODC_OK && defer) {
+    c->pending = true;
+    c->pend_norms = norms;
+    c->pend_scores = scores;
+    c->pend_last = reinterpret_cast<long long*>(last_sync);
+  }
+  return s;
 }
 
 }  // namespace
@@ -817,6 +866,7 @@ cocodc_status initiate_impl(cocodc_ctx* c, const float* scores, const int64_t* l
     return COCODC_ERR_ALIAS;
   if (!c->inline_plan || budget_kind == COCODC_BUDGET_PARAMS_EXACT) {
     // a table too large to be a kernel argument, or the enumerating budget: the two calls one after the other
+    // (select_impl forms the scores of a deferred completion first)
     cocodc_status s = select_impl(c, scores, last_sync, ineligible, t_now, t_now_dev, H, budget_kind, budget, mask,
                                   ids, n_sel, pool_offset, stream);
     if (s != COCODC_OK) return s;
@@ -824,6 +874,11 @@ cocodc_status initiate_impl(cocodc_ctx* c, const float* scores, const int64_t* l
   }
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // A deferred completion is consumed by this launch if it was given the arrays this selection reads; otherwise
+  // its scores are formed first, where it said.
+  if (c->pending && (c->pend_scores != scores || c->pend_last != reinterpret_cast<const long long*>(last_sync)) &&
+      flush_pending(c, st) != COCODC_OK)
+    return COCODC_ERR_CUDA;
   opt_in_shared_memory(c, reinterpret_cast<const void*>(k_snapshot_tma), kSnapSmemBytes);
   PlanRequest rq{};
   rq.snap_row_len = snap_stride;
@@ -845,6 +900,16 @@ cocodc_status initiate_impl(cocodc_ctx* c, const float* scores, const int64_t* l
   q.pool_offset = reinterpret_cast<long long*>(pool_offset);
   q.ticket = c->d_ticket;
   q.err_nonfinite = (int)COCODC_ERR_NONFINITE;
+  if (c->pending) {
+    q.pending = c->d_pending;
+    q.partial = c->d_partial;
+    q.norms = c->pend_norms;
+    q.scores_out = c->pend_scores;
+    q.last_sync_out = c->pend_last;
+    q.pend_grid = c->pend_grid;
+    q.pend_warps = kThreads / 32;
+    c->pending = false;
+  }
   k_snapshot_tma<<<c->sm_count, kThreads, kSnapSmemBytes, st>>>(w_now, w_snap, now_stride, snap_stride, M, nullptr,
                                                                 nullptr, rq, c->d_status, (int)COCODC_ERR_TIMEOUT,
                                                                 c->table, q);
@@ -926,6 +991,7 @@ cocodc_status cocodc_outer_step_host(cocodc_ctx* c, const cocodc_hyper* h,
 
   DeviceGuard guard(c->device);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (flush_pending(c, st) != COCODC_OK) return COCODC_ERR_CUDA;
   const Variant v = pick_variant(M, MODE_FUSED, same);
   const int grid = variant_grid(c, v);
   opt_in_shared_memory(c, reinterpret_cast<const void*>(v.kernel), v.smem);

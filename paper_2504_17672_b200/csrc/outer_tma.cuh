@@ -503,6 +503,9 @@ k_snapshot_tma(const float* __restrict__ w_now, float* __restrict__ w_snap, long
   J.w_now = w_now; J.w_snap = w_snap; J.now_stride = now_stride; J.snap_stride = snap_stride; J.M = M;
   J.status = status; J.err_timeout = err_timeout;
   snapshot_copy(J, pv.seg, pv.hdr, reinterpret_cast<float*>(smem_raw), full_bar, dst_of_stage);
+  // the selection's writes to the schedule state, from a copy warp that is done (the DMA thread still has the
+  // whole copy ahead of it, so the counter's round trip costs nothing)
+  if (sel.scores != nullptr && threadIdx.x == 32) select_commit(is, sel, status);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -66,6 +66,19 @@ struct PlanRequest {
   int err_invalid;               // status code for a bad id list
 };
 
+// A completion whose scores are left to the next selection (COCODC_STAGE_DEFER): the launch ends with every CTA's
+// sum of squares per list position in `partial` and this record in device memory; the launch that next decides
+// which fragments to synchronise adds the CTAs' sums up in its prologue, where the boundary between the two
+// launches has already done the grid-wide hand-off that the ticket counter otherwise provides.
+constexpr int kMaxK = 1024;
+struct PendingScores {
+  int n;                         // list positions waiting; 0: nothing pending
+  int grid, warps;               // shape of `partial` as the completion wrote it: [n][grid][warps], first entry per CTA
+  int pad;
+  long long t_p, t_l;            // step numbers of the completion
+  int ids[kMaxK];                // fragment of list position j
+};
+
 // What the last warp of a launch does with the fragments' sums of squares (Eq. 10).
 struct Finalize {
   int* ticket;                   // device counter, zero between launches; nullptr: no epilogue
@@ -82,6 +95,7 @@ struct Finalize {
   double* sumsq_out;             // [K] per-fragment sums of squares before the square root, or nullptr
   unsigned char* in_flight;      // [K] cleared for completed fragments, or nullptr
   int err_nonfinite;
+  PendingScores* defer;          // non-null: stop after the CTAs' sums and leave this record (mode 0 only)
 };
 
 // Status word helper: keep the first error recorded since the last poll.
@@ -90,7 +104,6 @@ __device__ __forceinline__ void record_status(int* status, int code) {
 }
 
 constexpr int kPlanThreads = 256;
-constexpr int kMaxK = 1024;
 
 // ids == nullptr means "all K fragments in index order" (stand-alone scoring).
 static __global__ void __launch_bounds__(kPlanThreads)
@@ -425,6 +438,38 @@ static __device__ __noinline__ PlanView acquire_plan(InlinePlan& ip, const FragT
 __device__ __forceinline__ void write_fragment_score(const Finalize& F, int p, long long last, double total,
                                                      long long t_p, long long t_l, int* status);
 
+// Deferred completion: CTA 0 leaves the record from which the next selection forms the scores (called by one warp).
+__device__ __forceinline__ void leave_pending_record(const Finalize& F, const PlanHeader& h, int warps) {
+  const int lane = threadIdx.x & 31;
+  PendingScores* P = F.defer;
+  for (int j = lane; j < h.n_ids; j += 32) P->ids[j] = (F.ids == nullptr) ? j : F.ids[j];
+  if (lane == 0) {
+    P->t_p = F.t_p_dev ? *F.t_p_dev : F.t_p;
+    P->t_l = F.t_l_dev ? *F.t_l_dev : F.t_l;
+    P->grid = (int)gridDim.x;
+    P->warps = warps;
+    P->n = h.n_ids;
+  }
+}
+
+// Sum over the CTAs' entries of list position j, by one warp: lane l adds the entries of CTAs l, l + 32, ... in that
+// order, then the lanes' sums meet in the shuffle tree - the order finalize_epilogue uses, hence the same bits.
+__device__ __forceinline__ double pending_slot_total(const double* __restrict__ partial, int j, int grid, int warps) {
+  const int lane = threadIdx.x & 31;
+  double s = 0.0;
+  for (int i0 = lane; i0 < grid; i0 += 32 * 8) {
+    double x[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+      const int i = i0 + 32 * r;
+      x[r] = (i < grid) ? __ldcg(partial + ((size_t)j * grid + i) * warps) : 0.0;
+    }
+#pragma unroll
+    for (int r = 0; r < 8; ++r) if (i0 + 32 * r < grid) s += x[r];
+  }
+  return warp_sum(s);
+}
+
 static __device__ __noinline__ void finalize_epilogue(InlinePlan& ip, const Finalize& F, const PlanHeader& h,
                                                   double* __restrict__ partial, int warps, int* status,
                                                   bool in_shared = false) {
@@ -454,6 +499,10 @@ static __device__ __noinline__ void finalize_epilogue(InlinePlan& ip, const Fina
     __stcg(e, v);
   }
   __syncwarp();
+  if (F.defer) {                 // the next selection adds the CTAs' entries up
+    if (cta == 0) leave_pending_record(F, h, warps);
+    return;
+  }
   if (lane == 0) t = arrive_gpu(F.ticket);
   t = __shfl_sync(0xffffffffu, t, 0);
   if (t != grid - 1) return;
@@ -545,6 +594,10 @@ static __device__ __noinline__ void finalize_epilogue_cta(InlinePlan& ip, const 
       for (int q = 0; q < 8; ++q) if (w0 + q < warps) v += x[q];
     }
     __stcg(e, v);
+  }
+  if (F.defer) {
+    if (cta == 0 && warp == 0) leave_pending_record(F, h, warps);
+    return;
   }
   __syncthreads();
   if (tid == 0) ip.done_warps = (arrive_gpu(F.ticket) == grid - 1) ? 1 : 0;

@@ -185,8 +185,8 @@ k_select(int K, const float* __restrict__ scores, const long long* __restrict__ 
 // (K <= kInlineSegs) and the budgets that are walked (COUNT, PARAMS), every CTA of the snapshot kernel works out
 // the selection for itself - it is a deterministic function of the schedule state - and keeps the id list and
 // the pool places in shared memory, where the plan is then built from; CTA 0 also writes them to the caller's
-// arrays.  The in-flight marks are written by whichever CTA finishes its selection last (a ticket): no CTA
-// may see them before it has read the mask itself.
+// arrays.  The in-flight marks are written by whichever CTA finishes its selection last (a ticket, select_commit):
+// no CTA may see them before it has read the mask itself.
 // ---------------------------------------------------------------------------------------------------
 struct SelectRequest {
   const float* scores;                 // nullptr: no selection in this launch
@@ -204,6 +204,14 @@ struct SelectRequest {
   long long* pool_offset;              // nullptr: the snapshot keeps the native layout
   int* ticket;                         // zero between launches
   int err_nonfinite;
+  // A completion whose scores were left to this selection (PendingScores): the record, the CTAs' sums it describes,
+  // and the arrays the completion was given (scores and last_sync above are the same arrays, read-only there).
+  PendingScores* pending;              // nullptr: nothing can be pending
+  const double* partial;
+  int pend_grid, pend_warps;           // shape of `partial` as the host remembers it (the record has the last word)
+  float* norms;
+  float* scores_out;
+  long long* last_sync_out;
 };
 
 struct InlineSelect {
@@ -214,10 +222,66 @@ struct InlineSelect {
   long long pool[kInlineSegs];         // by fragment id; -1: not selected
   unsigned char cls[kInlineSegs];      // 0 = ineligible, 1 = ordinary, 2 = overdue
   unsigned char falign[kInlineSegs];
+  long long last[kInlineSegs];         // last_sync as this selection sees it (pending completions applied)
+  unsigned char infl[kInlineSegs];     // the in-flight marks likewise
+  int pend_id[kInlineSegs];            // pending list position -> fragment
+  float pend_norm[kInlineSegs];
   int n;
   int n_elig;
   int nan;
+  int bad_norm;
+  int n_pend;
 };
+
+// Eq. 10 for the fragments of a pending completion, into the selection's shared-memory view of the schedule state.
+// One warp per list position adds the CTAs' sums; the arithmetic after the sum is write_fragment_score's.  The
+// loads are issued in two parts so that they cost no round trip of their own: fetch() runs before the barrier at
+// which the schedule arrays arrive and already adds up list position `warp` with the shape the host remembers of
+// the completion's launch; apply() runs after it, uses that sum when the record confirms the shape, and takes any
+// further positions (lists longer than the CTA has warps) with plain loads.
+struct PendingFetch {
+  int n, grid, warps, frag;      // the record's fields; frag = ids[warp]
+  long long t_p, t_l;
+  double total;                  // sum of list position `warp`, formed with the host's shape
+};
+
+__device__ __forceinline__ PendingFetch fetch_pending_scores(const PendingScores* P, const double* __restrict__ partial,
+                                                             int K, int host_grid, int host_warps) {
+  PendingFetch f{};
+  if (P == nullptr) return f;
+  const int warp = threadIdx.x >> 5;
+  f.n = P->n; f.grid = P->grid; f.warps = P->warps; f.t_p = P->t_p; f.t_l = P->t_l;
+  if (warp < K) {
+    f.frag = P->ids[warp];
+    f.total = pending_slot_total(partial, warp, host_grid, host_warps);
+  }
+  if (f.n < 0 || f.n > K) f.n = 0;   // (cannot happen: the completion's list was validated)
+  return f;
+}
+
+__device__ __forceinline__ void apply_pending_scores(const PendingFetch& pf, const PendingScores* P,
+                                                     const double* __restrict__ partial, int host_grid, int host_warps,
+                                                     float* score, long long* last, unsigned char* infl,
+                                                     int* pend_id, float* pend_norm, int* bad_norm) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const bool shape_ok = (pf.grid == host_grid && pf.warps == host_warps);
+  for (int j = warp; j < pf.n; j += nw) {
+    const bool fetched = (j == warp) && shape_ok;
+    const int f = fetched ? pf.frag : P->ids[j];
+    const double total = fetched ? pf.total : pending_slot_total(partial, j, pf.grid, pf.warps);
+    if (lane == 0) {
+      const double norm = sqrt(total);
+      long long I = pf.t_p - last[f];
+      if (I < 1) I = 1;
+      pend_id[j] = f;
+      pend_norm[j] = (float)norm;
+      score[f] = (float)(norm / (double)I);
+      last[f] = pf.t_l;
+      infl[f] = 0;
+      if (!isfinite(norm)) *bad_norm = 1;
+    }
+  }
+}
 
 // Called by every thread of the CTA (at least K threads).
 static __device__ __noinline__ void select_in_cta(InlineSelect& is, const SelectRequest& q, const FragTable& T,
@@ -226,16 +290,26 @@ static __device__ __noinline__ void select_in_cta(InlineSelect& is, const Select
   const int K = T.K;
   const bool writer = (blockIdx.x == 0);
   const long long t_now = q.t_now_dev ? *q.t_now_dev : q.t_now;
-  if (p == 0) { is.n = 0; is.n_elig = 0; is.nan = 0; }
-  __syncthreads();
+  if (p == 0) { is.n = 0; is.n_elig = 0; is.nan = 0; is.bad_norm = 0; }
   if (p < K) {
-    const float r = q.scores[p];
-    const bool elig = ((q.ineligible == nullptr) || (q.ineligible[p] == 0)) &&
-                      ((q.in_flight == nullptr) || (q.in_flight[p] == 0));
-    const bool overdue = (t_now - q.last_sync[p]) >= q.H;     // Algorithm 2's staleness test
+    is.score[p] = q.scores[p];
+    is.last[p] = q.last_sync[p];
+    is.infl[p] = (q.in_flight != nullptr) ? q.in_flight[p] : (unsigned char)0;
+  }
+  const PendingFetch pf = fetch_pending_scores(q.pending, q.partial, K, q.pend_grid, q.pend_warps);
+  const int n_pend = pf.n;
+  __syncthreads();
+  if (n_pend > 0) {   // a completion left its scores to this selection: form them first (the same on every CTA)
+    apply_pending_scores(pf, q.pending, q.partial, q.pend_grid, q.pend_warps, is.score, is.last, is.infl, is.pend_id,
+                         is.pend_norm, &is.bad_norm);
+    __syncthreads();
+  }
+  if (p < K) {
+    const float r = is.score[p];
+    const bool elig = ((q.ineligible == nullptr) || (q.ineligible[p] == 0)) && (is.infl[p] == 0);
+    const bool overdue = (t_now - is.last[p]) >= q.H;         // Algorithm 2's staleness test
     long long size = 0;
     for (int sg = T.seg_ptr[p]; sg < T.seg_ptr[p + 1]; ++sg) size += T.len[sg];
-    is.score[p] = r;
     is.fsize[p] = size;
     is.falign[p] = (unsigned char)(T.off[T.seg_ptr[p]] & 3);
     is.cls[p] = elig ? (overdue ? 2 : 1) : 0;
@@ -294,14 +368,61 @@ static __device__ __noinline__ void select_in_cta(InlineSelect& is, const Select
       if (writer) *q.n_sel = n;
     }
   }
+  if (p == 0) is.n_pend = n_pend;
   __syncthreads();
-  // every CTA has read the in-flight mask once the last one gets here: only then is it marked
-  if (p == 0 && q.in_flight != nullptr) {
-    if (arrive_gpu(q.ticket) == (int)gridDim.x - 1) {
-      for (int j = 0; j < is.n; ++j) q.in_flight[is.ids[j]] = 1;
-      *q.ticket = 0;
+}
+
+// What a selection writes to the schedule state, by one thread per CTA once its CTA has finished select_in_cta
+// and at a point where waiting for the counter's answer delays nothing (the snapshot kernel calls it from a copy
+// warp that has run out of work, long before the DMA thread is done).  Every CTA has read the schedule state
+// once the last one gets here: only then is it written - the pending completion's norms, scores, last_sync and
+// cleared in-flight marks first, then the marks of what was selected.
+__device__ __forceinline__ void select_commit(InlineSelect& is, const SelectRequest& q, int* status) {
+  const int n_pend = is.n_pend;
+  if (q.in_flight == nullptr && n_pend == 0) return;
+  if (arrive_gpu(q.ticket) != (int)gridDim.x - 1) return;
+  for (int j = 0; j < n_pend; ++j) {
+    const int f = is.pend_id[j];
+    q.norms[f] = is.pend_norm[j];
+    q.scores_out[f] = is.score[f];
+    q.last_sync_out[f] = is.last[f];
+    if (q.in_flight != nullptr) q.in_flight[f] = 0;
+  }
+  if (n_pend > 0) {
+    q.pending->n = 0;
+    if (is.bad_norm) record_status(status, q.err_nonfinite);
+  }
+  if (q.in_flight != nullptr)
+    for (int j = 0; j < is.n; ++j) q.in_flight[is.ids[j]] = 1;
+  *q.ticket = 0;
+}
+
+// The same for a pending completion that no selection is about to consume (one block).
+static __global__ void __launch_bounds__(256)
+k_flush_pending(PendingScores* P, const double* __restrict__ partial, int K, float* __restrict__ norms,
+                float* __restrict__ scores, long long* __restrict__ last_sync, unsigned char* __restrict__ in_flight,
+                int* __restrict__ status, int err_nonfinite) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  const int n_pend = P->n;
+  if (n_pend <= 0 || n_pend > K) return;
+  const int grid = P->grid, warps = P->warps;
+  const long long t_p = P->t_p, t_l = P->t_l;
+  for (int j = warp; j < n_pend; j += nw) {
+    const int f = P->ids[j];
+    const double total = pending_slot_total(partial, j, grid, warps);
+    if (lane == 0) {
+      const double norm = sqrt(total);
+      long long I = t_p - last_sync[f];
+      if (I < 1) I = 1;
+      norms[f] = (float)norm;
+      scores[f] = (float)(norm / (double)I);
+      last_sync[f] = t_l;
+      if (in_flight != nullptr) in_flight[f] = 0;
+      if (!isfinite(norm)) record_status(status, err_nonfinite);
     }
   }
+  __syncthreads();
+  if (threadIdx.x == 0) P->n = 0;
 }
 
 }  // namespace cocodc
