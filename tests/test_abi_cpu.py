@@ -125,6 +125,7 @@ def test_null_context_is_rejected(B):
     assert lib.cocodc_fragment_scores(None, None, None, None, None, None, None) == B.ERR_INVALID_ARG
     assert lib.cocodc_scores_from_sumsq(None, None, None, None, None, 0, 0, None, None, None, None) == B.ERR_INVALID_ARG
     assert lib.cocodc_bind_in_flight(None, None) == B.ERR_INVALID_ARG
+    assert lib.cocodc_flush_scores(None, None) == B.ERR_INVALID_ARG
     assert lib.cocodc_destroy(None) == B.OK
     assert lib.cocodc_launch_count(None) == 0
 
