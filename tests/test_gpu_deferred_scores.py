@@ -292,3 +292,26 @@ def test_deferring_is_refused_where_it_has_no_meaning():
     prob.ctx.cocodc_flush_scores()
     assert prob.poll() == 0
     assert float(prob.norms[0].item()) > 0.0
+
+
+def test_a_status_poll_that_reports_an_error_drops_the_outstanding_completion():
+    """After an error the outputs of the launches before the poll are undefined; the scores a deferred completion left
+    unformed are then not formed later either (the error here is the self-test's bounded wait running out)."""
+    prob = make(4, seed=2)
+    prob.set_ids([1, 3])
+    prob.outer_step(4, 8, stages=DEFER)
+    was = schedule_state(prob)
+    prob.ctx.cocodc_selftest_bounded_wait(2000)
+    assert prob.poll() == prob.B.ERR_TIMEOUT
+    n0 = prob.ctx.launch_count
+    prob.ctx.cocodc_flush_scores()
+    assert prob.ctx.launch_count == n0
+    torch.cuda.synchronize()
+    for x, y in zip(was, schedule_state(prob)):
+        assert np.array_equal(x, y)
+    # the context is usable as before
+    before = prob.host_state()
+    prob.outer_step(8, 12, stages=DEFER)
+    prob.ctx.cocodc_flush_scores()
+    assert prob.poll() == 0
+    check_step_against_oracle(prob, before, [1, 3], 8, 12, orc_hyper(prob.w))
