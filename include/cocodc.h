@@ -481,7 +481,9 @@ cocodc_status cocodc_fragment_scores_noalloc(const cocodc_partition* partition, 
 /*
  * Waits for the stream, then returns and clears the device status word
  * (COCODC_OK if nothing was recorded since the last poll).  After an error the context's launch
- * scratch is reset, so the next call starts clean.
+ * scratch is reset, so the next call starts clean; a completion launched with COCODC_STAGE_DEFER whose
+ * scores have not been formed by then is dropped with it (its outputs are undefined after the error, as
+ * those of every launch before the poll).
  */
 cocodc_status cocodc_poll_status(cocodc_ctx* ctx, void* stream);
 
